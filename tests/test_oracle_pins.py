@@ -1,0 +1,503 @@
+"""Pins of the CPU oracle against what the paper (arXiv 2407.04480) and the mathematics fix.
+
+None of these tests touches the CUDA library.  Each names the statement it checks.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import loco_definition as defn
+from oracle import loco_oracle as orc
+from oracle.loco_oracle import OracleConfig
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+RNG = np.random.default_rng(20240704)
+
+
+def qrange(p):
+    return -(2 ** (p - 1)), 2 ** (p - 1) - 1
+
+
+def run_steps(cfg, grads, k0=1):
+    """Run consecutive send steps k0, k0+1, ... on one worker; return the per-step traces and final state."""
+    n = grads[0].size
+    state = orc.new_state(cfg, n)
+    comm = orc.new_comm(cfg, n)
+    traces = []
+    for i, g in enumerate(grads):
+        (_, _), tr = orc.send_step(cfg, g, state, comm, k0 + i, trace=True)
+        traces.append(tr)
+    return traces, state, comm
+
+
+# ------------------------------------------------------------------ Eq. 1: the compressor
+
+@pytest.mark.parametrize("p", [2, 4, 8])
+def test_code_range(p):
+    """Text under Eq. 1: codes lie in [-2^(p-1), 2^(p-1)-1]."""
+    x = np.concatenate([RNG.normal(0, 1, 4096), [1e30, -1e30, np.inf, -np.inf, 0.0]]).astype(np.float32)
+    q = orc.compressor(x, 3.0, p)
+    lo, hi = qrange(p)
+    assert q.min() == lo and q.max() == hi
+    assert np.all((q >= lo) & (q <= hi))
+
+
+@pytest.mark.parametrize("p", [2, 4, 8])
+@pytest.mark.parametrize("s", [4.0, 2.0 ** 11, 2.0 ** 19, 6.0 * 2 ** 11, 1000.0])
+def test_half_step_bound_and_saturation(p, s):
+    """Lemma "round": |x - C(x)| <= 1/(2s) inside the range; outside, C(x) is the end of the range
+    and the error is |x| minus that end."""
+    lo, hi = qrange(p)
+    x = (RNG.normal(0, 1.0, 20000) * (hi + 2) / s / 2).astype(np.float32)
+    q = orc.compressor(x, s, p).astype(np.float64)
+    Cx = q / s
+    x64 = x.astype(np.float64)
+    # x*s is rounded once to fp32 before the nearest-integer step: allow that half-ulp in the bound
+    slack = np.abs(x64) * 2.0 ** -24 + 1e-300
+    inside = (x64 * s >= lo - 0.5) & (x64 * s <= hi + 0.5)
+    assert np.all(np.abs(x64 - Cx)[inside] <= 0.5 / s + slack[inside])
+    above, below = x64 * s > hi + 0.5, x64 * s < lo - 0.5
+    assert above.any() and below.any()
+    assert np.all(q[above] == hi) and np.all(q[below] == lo)
+    assert np.allclose((x64 - Cx)[above], x64[above] - hi / s, rtol=0, atol=1e-12)
+    assert np.allclose((Cx - x64)[below], lo / s - x64[below], rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("p", [2, 4, 8])
+def test_brute_force_nearest_code(p):
+    """Eq. 1's text: the nearest integer within the range.  Brute force over all 2^p codes; a tie
+    between two integers goes to the even one."""
+    s = 2.0 ** 7
+    lo, hi = qrange(p)
+    codes = np.arange(lo, hi + 1, dtype=np.float64)
+    ties = (np.arange(lo - 2, hi + 2) + 0.5) / s
+    x = np.concatenate([RNG.uniform(lo - 3, hi + 3, 5000) / s, ties, codes / s]).astype(np.float32)
+    q = orc.compressor(x, s, p)
+    y = x.astype(np.float64) * s                      # exact: s is a power of two
+    dist = np.abs(y[:, None] - codes[None, :])
+    best = dist.min(axis=1)
+    for yi, qi, row, b in zip(y, q, dist, best):
+        cands = codes[row == b]
+        if len(cands) == 1:
+            assert qi == cands[0]
+        else:                                         # exact tie inside the range
+            assert qi in cands and qi % 2 == 0, (yi, qi, cands)
+
+
+@pytest.mark.parametrize("p,s", [(4, 2.0 ** 19), (8, 6 * 2.0 ** 19), (4, 37.5), (2, 2.0 ** 17)])
+def test_matches_pytorch_default_rounding(p, s):
+    """Eq. 1's text calls it the default quantisation in PyTorch: round, then clamp."""
+    lo, hi = qrange(p)
+    x = (RNG.normal(0, 1, 50000) * 6.0 / s).astype(np.float32)
+    x[:200] = ((np.arange(200) - 100) + 0.5) / np.float32(s)
+    want = torch.clamp(torch.round(torch.from_numpy(x) * torch.tensor(s, dtype=torch.float32)), lo, hi)
+    assert np.array_equal(orc.compressor(x, s, p), want.numpy().astype(np.int32))
+
+
+@pytest.mark.parametrize("p", [2, 4, 8])
+def test_idempotent_on_the_grid(p):
+    """C(C(x)) = C(x): a value already on the grid is reproduced (follows from Eq. 1)."""
+    s = 2.0 ** 10
+    x = (RNG.normal(0, 1, 4096) * 4 / s).astype(np.float32)
+    q1 = orc.compressor(x, s, p)
+    c1 = orc.decompressor(q1, s)
+    q2 = orc.compressor(c1, s, p)
+    assert np.array_equal(q1, q2)
+    assert np.array_equal(orc.decompressor(q2, s), c1)
+
+
+def test_round_trip_all_codes():
+    """comp(dec(q)) = q for every code, for power-of-two and other scales."""
+    for p in (2, 4, 8):
+        lo, hi = qrange(p)
+        q = np.arange(lo, hi + 1, dtype=np.int32)
+        for s in (2.0 ** 19, 2.0 ** 17, 6 * 2.0 ** 19, 3.0, 1e-3):
+            assert np.array_equal(orc.compressor(orc.decompressor(q, s), s, p), q)
+
+
+def test_decompressor_is_division():
+    """Eq. 1, second line: float(q) / s (IEEE division, not a rounded reciprocal)."""
+    q = np.arange(-128, 128, dtype=np.int32)
+    for s in (6 * 2.0 ** 19, 3.0, 7.0):
+        want = (q.astype(np.float32) / np.float32(s)).astype(np.float32)
+        assert np.array_equal(orc.decompressor(q, s), want)
+
+
+# ------------------------------------------------------------------ Algorithm 1: worked example
+
+def load_golden(name):
+    rec = {}
+    for line in open(os.path.join(GOLDEN, name)):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        k, *v = line.split()
+        rec[k] = v
+    return rec
+
+
+def test_hand_worked_example():
+    """tests/golden/alg1_worked_example.txt: two iterations of Algorithm 1 worked by hand."""
+    G = load_golden("alg1_worked_example.txt")
+    f = lambda k: np.array([float(v) for v in G[k]], dtype=np.float32)
+    cfg = OracleConfig(bits=int(G["p"][0]), s=float(G["s"][0]), s_e=float(G["s_e"][0]),
+                       beta=float(G["beta"][0]), reset_period=0, state_fmt=orc.STATE_INT8)
+    n = 6
+    state, comm = orc.new_state(cfg, n), orc.new_comm(cfg, n)
+    comms = []
+    for k, tag in ((1, "1"), (2, "2")):
+        (flags, sat), tr = orc.send_step(cfg, f("g" + tag), state, comm, k, trace=True)
+        nxt = str(k + 1)
+        assert flags == 0 and sat == int(G["sat" + tag][0])
+        assert np.array_equal(tr["h"], f("h" + tag))
+        assert np.array_equal(tr["q"], f("q" + tag).astype(np.int32))
+        assert np.array_equal(tr["d"], f("d" + tag))
+        assert np.array_equal(tr["e_new"], f("et" + nxt))
+        assert np.array_equal(state[:n].view(np.int8), f("e" + nxt).astype(np.int8))
+        comms.append(comm.copy())
+    assert [int(b) for b in comms[0][:3]] == [int(v, 16) for v in G["packed1"]]
+    assert np.array_equal(orc.reduce(cfg, n, comms), f("mean"))
+
+
+# ------------------------------------------------------------------ Algorithm 1: invariants
+
+def dyadic(n, bits, scale):
+    """Values m * scale with |m| < 2^bits: sums and products by powers of two stay exact in fp32."""
+    return (RNG.integers(-(2 ** bits), 2 ** bits, n) * scale).astype(np.float32)
+
+
+@pytest.mark.parametrize("fmt", [orc.STATE_INT8, orc.STATE_FP32, orc.STATE_FP32_Q8COMP])
+def test_identity_compression_keeps_zero_error(fmt):
+    """If every g*s is an integer inside the range, compression loses nothing: d = g and e~ stays 0."""
+    s = 2.0 ** 9
+    cfg = OracleConfig(bits=4, s=s, s_e=4 * s, beta=0.3, reset_period=0, state_fmt=fmt)
+    grads = [(RNG.integers(-8, 8, 257) / s).astype(np.float32) for _ in range(5)]
+    traces, state, _ = run_steps(cfg, grads)
+    for g, tr in zip(grads, traces):
+        assert np.array_equal(tr["d"], g) and not tr["e_new"].any()
+    assert not state.any()
+
+
+def test_beta_one_is_classic_error_feedback():
+    """Eq. 4 versus Eq. 5: with beta = 1 the new error is h - d of this iteration alone, so the
+    sum of what was sent equals the sum of the gradients minus the last error."""
+    s = 2.0 ** 6
+    cfg = OracleConfig(bits=4, s=s, s_e=4 * s, beta=1.0, reset_period=0, state_fmt=orc.STATE_FP32)
+    grads = [dyadic(64, 6, 2.0 ** -10) for _ in range(6)]
+    traces, state, _ = run_steps(cfg, grads)
+    for tr in traces:
+        assert np.array_equal(tr["e_new"], tr["h"] - tr["d"])
+    sent = np.sum([t["d"].astype(np.float64) for t in traces], axis=0)
+    want = np.sum([g.astype(np.float64) for g in grads], axis=0) - state.view(np.float32)[:64]
+    assert np.array_equal(sent, want)
+
+
+@pytest.mark.parametrize("variant", ["state_none", "beta_zero"])
+def test_no_feedback_is_plain_quantisation(variant):
+    """Ablation row without error feedback: the output is compressor(g) and nothing carries over."""
+    s = 2.0 ** 11
+    cfg = OracleConfig(bits=4, s=s, s_e=4 * s, beta=0.0, reset_period=0,
+                       state_fmt=orc.STATE_NONE if variant == "state_none" else orc.STATE_INT8)
+    grads = [(RNG.normal(0, 1e-3, 300)).astype(np.float32) for _ in range(3)]
+    traces, state, _ = run_steps(cfg, grads)
+    for g, tr in zip(grads, traces):
+        assert np.array_equal(tr["q"], orc.compressor(g, s, 4))
+    assert not state.any()
+
+
+@pytest.mark.parametrize("beta", [0.5, 0.25, 0.75])
+def test_closed_form_unrolling(beta):
+    """Eq. 5 unrolled from e~_0 = 0 without reset: e~_K = beta * sum_i (1-beta)^(K-i) * delta_i."""
+    s = 2.0 ** 8
+    cfg = OracleConfig(bits=4, s=s, s_e=4 * s, beta=beta, reset_period=0, state_fmt=orc.STATE_FP32)
+    K = 4
+    grads = [(RNG.normal(0, 2e-2, 8)).astype(np.float32) for _ in range(K)]
+    traces, state, _ = run_steps(cfg, grads)
+    deltas = [t["delta"].astype(np.float64) for t in traces]
+    want = beta * sum((1 - beta) ** (K - 1 - i) * deltas[i] for i in range(K))
+    got = state.view(np.float32)[:8].astype(np.float64)
+    assert np.allclose(got, want, rtol=1e-6, atol=1e-12)
+    assert np.abs(want).max() > 0
+
+
+@pytest.mark.parametrize("fmt,beta", [(orc.STATE_FP32, 0.5), (orc.STATE_FP32, 0.1),
+                                      (orc.STATE_FP32_Q8COMP, 0.5), (orc.STATE_FP32_Q8COMP, 0.25),
+                                      (orc.STATE_INT8, 0.5), (orc.STATE_INT8, 1.0)])
+def test_lemma_1_identity(fmt, beta):
+    """Lemma 1, per element and worker:
+         d_k = g_k + (e~_k - e~_{k+1})/beta + e^_k - e~_k,   e^_k = dec(comp(e~_k; s_e, 8); s_e).
+    With fp32 storage used as it is, e^ = e~.  With only the 8-bit state stored, e~_k is its image
+    e^_k, which leaves d_k - g_k = (e^_k - e~_{k+1})/beta."""
+    s = 2.0 ** 9
+    s_e = 4 * s
+    cfg = OracleConfig(bits=4, s=s, s_e=s_e, beta=beta, reset_period=0, state_fmt=fmt)
+    n, K = 96, 6
+    grads = [(RNG.normal(0, 6e-3, n)).astype(np.float32) for _ in range(K)]
+    state = orc.new_state(cfg, n)
+    comm = orc.new_comm(cfg, n)
+    seen_nonzero = False
+    for k, g in enumerate(grads, start=1):
+        before = state.copy()
+        (_, _), tr = orc.send_step(cfg, g, state, comm, k, trace=True)
+        g64, d64 = g.astype(np.float64), tr["d"].astype(np.float64)
+        e_next = tr["e_new"].astype(np.float64)
+        if fmt == orc.STATE_INT8:
+            e_hat = before[:n].view(np.int8).astype(np.float64) / s_e
+            e_prev = e_hat
+        else:
+            e_prev = before.view(np.float32)[:n].astype(np.float64)
+            e_hat = e_prev if fmt == orc.STATE_FP32 else defn.decompressor(defn.compressor(e_prev, s_e, 8), s_e)
+        want = g64 + (e_prev - e_next) / beta + e_hat - e_prev
+        assert np.allclose(d64, want, rtol=0, atol=4e-7 / beta * 6e-3 + 1e-9)
+        seen_nonzero |= bool(np.abs(e_hat).max() > 0)
+    assert seen_nonzero
+
+
+def test_lemma_1_identity_detects_swapped_beta():
+    """The identity above is sharp enough to catch Eq. 5 written with beta and 1-beta exchanged
+    (the mistake is planted in a copy of the double-precision definition, not in any product code)."""
+    s, s_e, beta = 2.0 ** 9, 2.0 ** 11, 0.25
+    g = RNG.normal(0, 6e-3, 64)
+    e_prev = RNG.normal(0, 1e-3, 64)
+    q, d, h, e_next, _, _ = defn.loco_step(g, e_prev, None, 1, s=s, s_e=s_e, beta=beta, T_c=0, state="fp32")
+    assert np.allclose(d, g + (e_prev - e_next) / beta, rtol=0, atol=1e-12)
+    wrong_next = beta * e_prev + (1 - beta) * (h - d)
+    assert not np.allclose(d, g + (e_prev - wrong_next) / beta, rtol=0, atol=1e-6)
+
+
+def test_errors_do_not_accumulate():
+    """Proof of Lemma 2 (and Eq. 6): with fp32 storage the sum telescopes exactly,
+         sum_{i<=K} (d_i - g_i) = (e~_0 - e~_K)/beta;
+    with the 8-bit state each iteration adds at most one half step 1/(2 s_e) of the state grid."""
+    s, beta, n, K = 2.0 ** 9, 0.5, 128, 40
+    s_e = 4 * s
+    grads = [(RNG.normal(0, 5e-3, n)).astype(np.float32) for _ in range(K)]
+    gsum = np.sum([g.astype(np.float64) for g in grads], axis=0)
+    # fp32 state: exact telescoping
+    cfg = OracleConfig(bits=4, s=s, s_e=s_e, beta=beta, reset_period=0, state_fmt=orc.STATE_FP32)
+    traces, state, _ = run_steps(cfg, grads)
+    dsum = np.sum([t["d"].astype(np.float64) for t in traces], axis=0)
+    assert np.allclose(dsum - gsum, -state.view(np.float32)[:n].astype(np.float64) / beta, rtol=0, atol=1e-7)
+    # 8-bit state: bounded drift
+    cfg8 = OracleConfig(bits=4, s=s, s_e=s_e, beta=beta, reset_period=0, state_fmt=orc.STATE_INT8)
+    traces8, _, _ = run_steps(cfg8, grads)
+    dsum8 = np.sum([t["d"].astype(np.float64) for t in traces8], axis=0)
+    last = traces8[-1]["e_new"].astype(np.float64)
+    assert np.all(np.abs(dsum8 - gsum) <= np.abs(last) / beta + K * 0.5 / s_e / beta + 1e-9)
+    # and a plain quantiser without feedback drifts further than that on at least one element
+    plain = np.sum([orc.decompressor(orc.compressor(g, s, 4), s).astype(np.float64) for g in grads], axis=0)
+    assert np.abs(plain - gsum).max() > np.abs(dsum - gsum).max()
+
+
+def test_error_bound_after_reset():
+    """Lemma "err_bound", first case: the first error after a reset is at most beta/(2s) wherever
+    h stayed inside the range, and beta*(|h| - end of range) where it saturated."""
+    s, beta = 2.0 ** 9, 0.5
+    cfg = OracleConfig(bits=4, s=s, s_e=4 * s, beta=beta, reset_period=4, state_fmt=orc.STATE_FP32)
+    n = 512
+    grads = [(RNG.normal(0, 8e-3, n)).astype(np.float32) for _ in range(6)]
+    state, comm = orc.new_state(cfg, n), orc.new_comm(cfg, n)
+    for k, g in enumerate(grads):
+        (_, _), tr = orc.send_step(cfg, g, state, comm, k, trace=True)
+        if k % 4 == 1:                                   # first iteration after the reset at k % T_c == 0
+            h = tr["h"].astype(np.float64)
+            assert np.array_equal(tr["h"], g)            # compensation was zero
+            inside = (h * s >= -8.5) & (h * s <= 7.5)
+            e = np.abs(tr["e_new"].astype(np.float64))
+            assert np.all(e[inside] <= beta / (2 * s) + 1e-12)
+            assert (~inside).any()
+            bound = np.where(h > 0, 7 / s, 8 / s)
+            assert np.allclose(e[~inside], beta * (np.abs(h[~inside]) - bound[~inside]), rtol=1e-6, atol=1e-12)
+
+
+@pytest.mark.parametrize("fmt", [orc.STATE_INT8, orc.STATE_FP32, orc.STATE_FP32_Q8COMP])
+def test_reset_rule(fmt):
+    """Eq. 7 / Algorithm 1: e_{k+1} = 0 exactly when k % T_c == 0 (the caller's 0-based k); the codes
+    of that iteration are still compensated with e_k."""
+    s = 2.0 ** 9
+    cfg = OracleConfig(bits=4, s=s, s_e=4 * s, beta=0.5, reset_period=3, state_fmt=fmt)
+    n = 200
+    state, comm = orc.new_state(cfg, n), orc.new_comm(cfg, n)
+    for k in range(8):
+        g = RNG.normal(0, 6e-3, n).astype(np.float32)
+        before_nonzero = bool(state.any())
+        (_, _), tr = orc.send_step(cfg, g, state, comm, k, trace=True)
+        if k % 3 == 0:
+            assert not state.any()
+            if before_nonzero:
+                assert np.abs(tr["c"]).max() > 0 and np.array_equal(tr["h"], g + tr["c"])
+        else:
+            assert state.any()
+    cfg0 = OracleConfig(bits=4, s=s, s_e=4 * s, beta=0.5, reset_period=0, state_fmt=fmt)
+    state = orc.new_state(cfg0, n)
+    orc.send_step(cfg0, RNG.normal(0, 6e-3, n).astype(np.float32), state, comm, 0)
+    assert state.any()                                   # T_c = 0: never reset
+
+
+def test_int8_state_matches_definition_on_exact_inputs():
+    """On dyadic inputs every fp32 operation is exact, so the fp32 oracle must reproduce the
+    double-precision definition bit for bit (codes, state codes, d)."""
+    s, s_e, beta = 2.0 ** 6, 2.0 ** 8, 0.5
+    cfg = OracleConfig(bits=4, s=s, s_e=s_e, beta=beta, reset_period=5, state_fmt=orc.STATE_INT8)
+    n = 300
+    state, comm = orc.new_state(cfg, n), orc.new_comm(cfg, n)
+    e_code = np.zeros(n)
+    for k in range(12):
+        g = dyadic(n, 7, 2.0 ** -10)
+        (_, _), tr = orc.send_step(cfg, g, state, comm, k, trace=True)
+        q, d, h, e_next, _, e_code = defn.loco_step(g, None, e_code, k, s=s, s_e=s_e, beta=beta, T_c=5)
+        assert np.array_equal(tr["q"], q) and np.array_equal(tr["d"], d) and np.array_equal(tr["h"], h)
+        assert np.array_equal(tr["e_new"], e_next)
+        assert np.array_equal(state[:n].view(np.int8), e_code)
+
+
+# ------------------------------------------------------------------ Eq. 8: the average
+
+def make_comms(cfg, n, N, sigma=2e-3):
+    comms, ds = [], []
+    for w in range(N):
+        g = RNG.normal(0, sigma, n).astype(np.float32)
+        if cfg.grad_dtype == orc.BF16:
+            g = orc.f32_to_bf16_bits(g)
+        state, comm = orc.new_state(cfg, n), orc.new_comm(cfg, n)
+        (_, _), tr = orc.send_step(cfg, g, state, comm, 1, trace=True)
+        comms.append(comm)
+        ds.append(tr["d"])
+    return comms, ds
+
+
+@pytest.mark.parametrize("N", [1, 2, 3, 8, 16])
+@pytest.mark.parametrize("mode", [orc.SCALE_FIXED, orc.SCALE_BLOCK_ABSMAX])
+def test_average_is_the_mean(N, mode):
+    """Eq. 8: (1/N) * sum_n dec(h~^n), computed after dequantisation in high precision."""
+    n = 1000
+    cfg = OracleConfig(bits=4, scale_mode=mode, block_size=64, s=2.0 ** 10, s_e=2.0 ** 12, num_partitions=1,
+                       reset_period=0)
+    comms, ds = make_comms(cfg, n, N)
+    got = orc.reduce(cfg, n, comms).astype(np.float64)
+    want = defn.average(ds)
+    assert np.allclose(got, want, rtol=1e-6, atol=1e-9)
+    same = orc.reduce(cfg, n, [comms[0]] * N)
+    assert np.allclose(same, ds[0], rtol=1e-6, atol=0)      # N identical workers give d back
+    if mode == orc.SCALE_FIXED and N in (1, 2, 8, 16):
+        assert np.array_equal(same, ds[0])                   # exactly: few-bit codes, 1/N a power of two
+
+
+def test_average_all_code_pairs():
+    """Brute force for N = 2: every pair of 4-bit codes averages to (a + b) / (2 s)."""
+    s = 2.0 ** 5
+    cfg = OracleConfig(bits=4, s=s, s_e=4 * s, state_fmt=orc.STATE_NONE, reset_period=0)
+    pairs = np.array(list(itertools.product(range(-8, 8), repeat=2)), dtype=np.float32)
+    n = len(pairs)
+    comms = []
+    for col in (0, 1):
+        comm = orc.new_comm(cfg, n)
+        orc.send_step(cfg, (pairs[:, col] / np.float32(s)).astype(np.float32), orc.new_state(cfg, n), comm, 1)
+        comms.append(comm)
+    got = orc.reduce(cfg, n, comms)
+    assert np.array_equal(got, (pairs[:, 0] + pairs[:, 1]) / (2 * s))
+
+
+def test_partitions_cover_the_vector():
+    """Sec. 3.3: the vector is cut into N parts; reducing part j of every worker gives part j of the
+    full average, and the parts together give all of it."""
+    n, P = 5000, 4
+    cfg = OracleConfig(bits=4, s=2.0 ** 10, s_e=2.0 ** 12, num_partitions=P, reset_period=0, out_dtype=orc.BF16)
+    comms, ds = make_comms(cfg, n, 3)
+    whole = orc.reduce(cfg, n, comms)
+    parts = [orc.reduce(cfg, n, comms, first=j, count=1) for j in range(P)]
+    assert sum(p.size for p in parts) == n and np.array_equal(np.concatenate(parts), whole)
+    cfg1 = OracleConfig(bits=4, s=2.0 ** 10, s_e=2.0 ** 12, num_partitions=1, reset_period=0, out_dtype=orc.BF16)
+    flat = []
+    for d in ds:                                              # same codes, unpartitioned layout
+        comm = orc.new_comm(cfg1, n)
+        orc.send_step(OracleConfig(**{**cfg1.__dict__, "state_fmt": orc.STATE_NONE}), d, orc.new_state(cfg1, n), comm, 1)
+        flat.append(comm)
+    assert np.array_equal(orc.reduce(cfg1, n, flat), whole)
+    want = orc.f32_to_bf16_bits(defn.average(ds).astype(np.float32))
+    assert np.mean(whole == want) > 0.99                      # bf16 output is the rounded mean
+
+
+# ------------------------------------------------------------------ storage
+
+def test_storage_sizes():
+    """Table 1's text: the error state costs one byte per parameter, the gradient 4 bits on the wire."""
+    n = 25_000_000
+    cfg = OracleConfig(bits=4, num_partitions=8)
+    assert n <= orc.state_bytes(cfg, n) < n + 256
+    assert n // 2 <= orc.packed_bytes(cfg, n) <= n // 2 + 8 * (128 + 128)
+    assert orc.state_bytes(OracleConfig(state_fmt=orc.STATE_NONE), n) == 0
+    assert orc.state_bytes(OracleConfig(state_fmt=orc.STATE_FP32), n) == 4 * n
+    blk = OracleConfig(bits=4, scale_mode=orc.SCALE_BLOCK_ABSMAX, block_size=256, num_partitions=8)
+    assert orc.packed_bytes(blk, n) >= n // 2 + 4 * (n // 256)
+    for cfg_ in (cfg, blk):
+        assert sum(orc.partition_elems(cfg_, n, j) for j in range(8)) == n
+        assert orc.partition_bytes(cfg_, n) % 128 == 0 and orc.partition_capacity(cfg_, n) % 256 == 0
+    assert orc.packed_bytes(cfg, 0) == 0 and orc.state_bytes(cfg, 0) == 0
+
+
+@pytest.mark.parametrize("p", [2, 4, 8])
+def test_packing_all_byte_values(p):
+    """Brute force over all 256 byte values: unpack then pack reproduces the byte, fields are two's
+    complement, element i sits at bit (i mod 8/p)*p of byte i*p/8 (little end first)."""
+    per = 8 // p
+    lo, hi = qrange(p)
+    for b in range(256):
+        q = orc.unpack_codes(np.array([b], np.uint8), per, p)
+        assert np.all((q >= lo) & (q <= hi))
+        assert orc.pack_codes(q, p)[0] == b
+        for i in range(per):
+            field = (b >> (i * p)) & (2 ** p - 1)
+            assert q[i] == (field - 2 ** p if field >= 2 ** (p - 1) else field)
+
+
+def test_packing_all_code_tuples_of_a_tiny_block():
+    """Brute force: all 16^3 code triples survive pack / unpack through the partitioned layout."""
+    cfg = OracleConfig(bits=4, s=1.0, s_e=4.0, state_fmt=orc.STATE_NONE, reset_period=0, num_partitions=1)
+    triples = np.array(list(itertools.product(range(-8, 8), repeat=3)), dtype=np.float32).ravel()
+    comm = orc.new_comm(cfg, triples.size, fill=0xAA)
+    orc.send_step(cfg, triples, orc.new_state(cfg, triples.size), comm, 1)
+    codes, _ = orc.comm_views(cfg, triples.size, comm)[0]
+    assert np.array_equal(orc.unpack_codes(codes, triples.size, 4), triples.astype(np.int32))
+    assert not codes[(triples.size + 1) // 2:].any()          # padding elements carry code 0
+
+
+# ------------------------------------------------------------------ block-scaled extension, non-finite
+
+def test_block_absmax_properties():
+    """Extension without counterpart in the paper: per block, scale = amax/qmax, the largest element
+    maps to +-qmax, an all-zero block has scale 0 and codes 0, and Lemma 1's identity still holds."""
+    n, B = 1000, 64
+    cfg = OracleConfig(bits=4, scale_mode=orc.SCALE_BLOCK_ABSMAX, block_size=B, beta=0.5, reset_period=0,
+                       state_fmt=orc.STATE_FP32)
+    g = RNG.normal(0, 1e-3, n).astype(np.float32)
+    g[128:192] = 0
+    state, comm = orc.new_state(cfg, n), orc.new_comm(cfg, n)
+    (_, sat), tr = orc.send_step(cfg, g, state, comm, 1, trace=True)
+    codes, scales = orc.comm_views(cfg, n, comm)[0]
+    assert sat == 0 and scales[2] == 0 and not tr["q"][128:192].any()
+    for b in range((n + B - 1) // B):
+        blk = slice(b * B, min((b + 1) * B, n))
+        amax = np.abs(g[blk]).max()
+        assert scales[b] == np.float32(amax) / np.float32(7)
+        if amax > 0:
+            assert np.abs(tr["q"][blk]).max() == 7 and tr["q"][blk].min() >= -7
+            assert np.all(np.abs(tr["delta"][blk]) <= scales[b] / 2 * (1 + 1e-6))
+    e_next = state.view(np.float32)[:n].astype(np.float64)
+    assert np.allclose(tr["d"].astype(np.float64), g - e_next / 0.5, rtol=0, atol=1e-9)
+
+
+def test_non_finite_inputs():
+    """Reading for inputs the paper's boundedness assumption excludes: NaN -> code 0, +-Inf -> the end
+    of the range, the element's error is taken as 0, and a flag is raised."""
+    cfg = OracleConfig(bits=4, s=2.0 ** 10, s_e=2.0 ** 12, beta=0.5, reset_period=0, state_fmt=orc.STATE_FP32)
+    g = np.array([np.nan, np.inf, -np.inf, 1e-3, 3e38], dtype=np.float32)
+    state, comm = orc.new_state(cfg, 5), orc.new_comm(cfg, 5)
+    (flags, sat), tr = orc.send_step(cfg, g, state, comm, 1, trace=True)
+    assert flags & orc.FLAG_NONFINITE
+    assert list(tr["q"]) == [0, 7, -8, 1, 7] and sat == 1
+    e = state.view(np.float32)[:5]
+    assert e[0] == 0 and e[1] == 0 and e[2] == 0 and np.isfinite(e).all()
