@@ -1,0 +1,172 @@
+/*
+ * loco.h -- C ABI of the B200 (sm_100a) LoCo hot-path library.
+ *
+ * LoCo (Low-bit Communication Adaptor, arXiv 2407.04480) sends gradients between
+ * data-parallel workers as low-bit integer codes and feeds the compression error
+ * back into the next iteration.  This library implements the two elementwise passes
+ * every worker runs per gradient bucket and iteration:
+ *
+ *   send    (Algorithm 1, steps 1-2; Eq. 1-7): compensate the fresh gradient with the
+ *           stored error, quantise, form the new moving-average error, store it in the
+ *           8-bit state, pack the codes into the communication buffer;
+ *   receive (Algorithm 1, step 3; Eq. 8): unpack N workers' buffers, dequantise,
+ *           average in fp32, write the fp32/bf16 gradient for the optimizer.
+ *
+ * Conventions for every call
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  All device
+ *     buffers are owned by the caller and must be 16-byte aligned and must not
+ *     overlap.  The library never frees or reallocates them.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Kernel launches are asynchronous on it; nothing synchronises unless stated.
+ *   - Every function that returns int returns LOCO_OK (0) or a negative loco_status_t.
+ *     Nothing aborts, traps or throws.  On error no kernel has been launched.
+ *   - Element counts are 64-bit; a flat buffer may exceed 2^32 elements.
+ *
+ * Layout of the communication buffer ("wire layout", little-endian)
+ *   The bucket's n elements are cut into P = num_partitions consecutive parts of
+ *   Lp = loco_partition_capacity() elements (the N parts of Sec. 3.3; the last parts
+ *   may be short or empty).  Part j occupies bytes [j*stride, (j+1)*stride),
+ *   stride = loco_partition_bytes():
+ *       [ codes: Lp*p/8 bytes ][ scales: (Lp/B) fp32, BLOCK_ABSMAX only ][ pad to 128 B ]
+ *   Element o of a part is the p-bit two's-complement field at bit (o mod 8/p)*p of
+ *   byte o*p/8 (4-bit: even element in the low nibble).  Elements past n carry code 0,
+ *   blocks entirely past n carry scale 0.  Pad bytes are never written.
+ *   Lp = ceil(n/P) rounded up to a multiple of max(256, B).
+ *
+ * Layout of the error state
+ *   STATE_INT8  : n int8 codes e (1 byte per element, as Table 1's text counts);
+ *                 BLOCK_ABSMAX adds ceil(n/B) fp32 scales at byte offset roundup(n, 256).
+ *   STATE_FP32 / STATE_FP32_Q8COMP : n fp32 values of the uncompressed error.
+ *   STATE_NONE  : nothing.
+ */
+#ifndef LOCO_B200_H
+#define LOCO_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LOCO_OK = 0,
+    LOCO_ERR_ARG = -1,          /* null pointer, value out of range, bad configuration       */
+    LOCO_ERR_ALIGN = -2,        /* a device pointer is not 16-byte aligned                   */
+    LOCO_ERR_SIZE = -3,         /* a buffer is smaller than the layout requires               */
+    LOCO_ERR_CUDA = -4,         /* the CUDA runtime reported an error (no device, launch...)  */
+    LOCO_ERR_UNSUPPORTED = -5   /* valid request that this build does not implement           */
+} loco_status_t;
+
+typedef enum { LOCO_F32 = 0, LOCO_BF16 = 1 } loco_dtype_t;
+
+typedef enum {
+    LOCO_SCALE_FIXED = 0,        /* Eq. 1: one global s (and s_e); only codes travel            */
+    LOCO_SCALE_BLOCK_ABSMAX = 1  /* extension, not in the paper: fp32 scale amax/qmax per B      */
+} loco_scale_mode_t;
+
+typedef enum {
+    LOCO_STATE_INT8 = 0,         /* the paper's 8-bit error e_k (Eq. 7); Eq. 5 uses dec(e_k)     */
+    LOCO_STATE_FP32 = 1,         /* uncompressed error, the ablation without error compression   */
+    LOCO_STATE_NONE = 2,         /* no error feedback: plain quantisation                        */
+    LOCO_STATE_FP32_Q8COMP = 3   /* keep e~ in fp32, compensate with dec(comp(e~; s_e, 8); s_e),
+                                    the form Lemma 1 is stated for; FIXED scale only            */
+} loco_state_fmt_t;
+
+/* Bits of the status word returned by loco_last_status(). */
+#define LOCO_FLAG_NONFINITE 1u   /* some compensated gradient was NaN or +-Inf */
+
+/* Algorithm 1's inputs (s, s_e, T_c, beta), Eq. 1's p, and the storage choices. */
+typedef struct {
+    int32_t bits;            /* p of Eq. 1 for the gradient codes: 2, 4 or 8 (the paper uses 4)   */
+    int32_t scale_mode;      /* loco_scale_mode_t                                                 */
+    int32_t block_size;      /* B, BLOCK_ABSMAX only: power of two in [32, 4096]                  */
+    float   s;               /* Eq. 1 / Eq. 3 scale, FIXED only (> 0, finite)                     */
+    float   s_e;             /* Eq. 2 / Eq. 7 scale of the 8-bit error, FIXED only                */
+    float   beta;            /* Eq. 5, in [0, 1]: weight of the NEW compression error             */
+    int32_t reset_period;    /* T_c of Eq. 7: state := 0 after iteration k when k % T_c == 0;
+                                0 = never                                                        */
+    int32_t state_fmt;       /* loco_state_fmt_t                                                  */
+    int32_t grad_dtype;      /* loco_dtype_t of the gradient handed to the send pass              */
+    int32_t out_dtype;       /* loco_dtype_t of the averaged gradient the receive pass writes     */
+    int32_t num_partitions;  /* P >= 1: parts of the all-to-all layout (Sec. 3.3)                 */
+    int32_t collect_stats;   /* non-zero: count saturated gradient codes (second case of the
+                                rounding lemma) during send; costs a few instructions/element   */
+} loco_config_t;
+
+/* Per-bucket, per-worker handle: a host object holding the configuration, the bucket
+ * length, the caller's state pointer and a 16-byte device status word. */
+typedef struct loco_state loco_state_t;
+
+/* ---- sizes (pure host arithmetic; 0 on a bad configuration or n == 0) ------------------ */
+uint64_t loco_state_bytes(const loco_config_t *cfg, uint64_t n);        /* error state            */
+uint64_t loco_packed_bytes(const loco_config_t *cfg, uint64_t n);       /* whole comm buffer      */
+uint64_t loco_partition_bytes(const loco_config_t *cfg, uint64_t n);    /* stride of one part     */
+uint64_t loco_partition_capacity(const loco_config_t *cfg, uint64_t n); /* Lp, padded elements    */
+uint64_t loco_partition_elems(const loco_config_t *cfg, uint64_t n, int32_t j); /* valid elements */
+
+/* LOCO_OK if the configuration is one this library accepts, else the error it would give. */
+int loco_config_check(const loco_config_t *cfg);
+
+/*
+ * Create the handle for one bucket of n elements whose error state lives in the caller's
+ * device buffer d_state (>= loco_state_bytes(); may be NULL for STATE_NONE) and zero-fill
+ * that buffer asynchronously on `stream`: the error starts at zero (Eq. 5's initialisation).
+ * Allocates the host handle and 16 bytes of device memory; the only allocating call.
+ * Errors: ARG (null out/cfg, bad cfg), ALIGN, SIZE (d_state_bytes too small), CUDA.
+ */
+int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n,
+                    void *d_state, uint64_t d_state_bytes, void *stream);
+
+/* Zero the error state (the explicit reset of Algorithm 1) and the status word; asynchronous. */
+int loco_state_reset(loco_state_t *st, void *stream);
+
+/* Free the handle and its status word.  The caller's buffers are untouched. */
+int loco_state_destroy(loco_state_t *st);
+
+/*
+ * Send pass for iteration `step_k` (the paper's 0-based k) -- Algorithm 1 steps 1-2:
+ *     h = g + dec(e_k; s_e);  q = comp(h; s, p);  d = dec(q; s);
+ *     e~_{k+1} = (1-beta) e~_k + beta (h - d);   e_{k+1} = 0 if k % T_c == 0 else comp(e~_{k+1}; s_e, 8)
+ * in one fused pass: reads d_grad (n elements of grad_dtype) and the state, writes the
+ * state in place and every code (and scale) byte of d_comm (>= loco_packed_bytes()).
+ * d_grad is not modified.  One launch, no allocation, no synchronisation.
+ * Errors: ARG (null, step_k < 0), ALIGN, CUDA.
+ */
+int loco_compensate_quantize_pack(loco_state_t *st, const void *d_grad, void *d_comm,
+                                  int64_t step_k, void *stream);
+
+/*
+ * Receive pass -- Eq. 8: for `partition_count` consecutive parts starting at
+ * `first_partition`, average the dequantised codes of `num_workers` workers (summed in
+ * worker order in fp32, divided by N) and write out_dtype values to d_out.
+ *   d_packed   HOST array of num_workers DEVICE pointers; d_packed[w] points at part
+ *              `first_partition` inside worker w's communication buffer (the next parts
+ *              follow at +loco_partition_bytes() each), 16-byte aligned.
+ *   n          length of the whole bucket (fixes Lp and the valid length of each part).
+ *   d_out      receives the valid elements of those parts contiguously, i.e. bucket
+ *              elements [first*Lp, min((first+count)*Lp, n)).
+ * 1 <= num_workers <= 64.  One launch, no allocation, no synchronisation.
+ * Errors: ARG, ALIGN, UNSUPPORTED (num_workers > 64), CUDA.
+ */
+int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_packed,
+                               int32_t num_workers, uint64_t n, int32_t first_partition,
+                               int32_t partition_count, void *d_out, void *stream);
+
+/*
+ * Read the status word accumulated by the send passes of this handle since init/reset.
+ * SYNCHRONISES `stream` (the one the passes ran on).  n_saturated counts gradient codes
+ * whose nearest integer fell outside the p-bit range; it stays 0 unless collect_stats.
+ * Either output pointer may be NULL.
+ */
+int loco_last_status(loco_state_t *st, uint32_t *flags, uint64_t *n_saturated, void *stream);
+
+/* Human-readable name of a loco_status_t. */
+const char *loco_status_string(int status);
+
+/* Number of kernels this library has launched in the calling process (for accounting). */
+uint64_t loco_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOCO_B200_H */

@@ -1,0 +1,414 @@
+// C ABI of the LoCo hot-path library: argument checks, layout arithmetic, kernel dispatch.
+// See include/loco.h for the contract of every entry point.
+#include "../../include/loco.h"
+
+#include <atomic>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "loco_kernels.cuh"
+
+namespace {
+
+using namespace loco;
+
+std::atomic<uint64_t> g_launches{0};
+
+inline uint64_t round_up(uint64_t x, uint64_t m) { return (x + m - 1) / m * m; }
+inline bool is_pow2(uint64_t x) { return x && !(x & (x - 1)); }
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int ilog2(uint32_t x) { int l = 0; while ((1u << l) < x) ++l; return l; }
+
+int check_config(const loco_config_t *c) {
+    if (!c) return LOCO_ERR_ARG;
+    if (c->bits != 2 && c->bits != 4 && c->bits != 8) return LOCO_ERR_ARG;
+    if (c->scale_mode != LOCO_SCALE_FIXED && c->scale_mode != LOCO_SCALE_BLOCK_ABSMAX) return LOCO_ERR_ARG;
+    if (c->state_fmt < LOCO_STATE_INT8 || c->state_fmt > LOCO_STATE_FP32_Q8COMP) return LOCO_ERR_ARG;
+    if (c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX) {
+        const int b = c->block_size;
+        if (b < 32 || b > 4096 || !is_pow2(static_cast<uint64_t>(b))) return LOCO_ERR_ARG;
+        if (c->state_fmt == LOCO_STATE_FP32_Q8COMP) return LOCO_ERR_ARG;
+    } else {
+        if (!(c->s > 0.0f) || !std::isfinite(c->s)) return LOCO_ERR_ARG;
+        if (c->state_fmt == LOCO_STATE_INT8 || c->state_fmt == LOCO_STATE_FP32_Q8COMP)
+            if (!(c->s_e > 0.0f) || !std::isfinite(c->s_e)) return LOCO_ERR_ARG;
+    }
+    if (c->state_fmt != LOCO_STATE_NONE && !(c->beta >= 0.0f && c->beta <= 1.0f)) return LOCO_ERR_ARG;
+    if (c->reset_period < 0) return LOCO_ERR_ARG;
+    if (c->grad_dtype != LOCO_F32 && c->grad_dtype != LOCO_BF16) return LOCO_ERR_ARG;
+    if (c->out_dtype != LOCO_F32 && c->out_dtype != LOCO_BF16) return LOCO_ERR_ARG;
+    if (c->num_partitions < 1 || c->num_partitions > 65535) return LOCO_ERR_ARG;
+    if (c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX && c->block_size > 256) return LOCO_ERR_UNSUPPORTED;
+    return LOCO_OK;
+}
+
+// Layout arithmetic accepts every well-formed configuration, also those the kernels do not cover.
+bool layout_ok(const loco_config_t *c) {
+    const int rc = check_config(c);
+    return rc == LOCO_OK || rc == LOCO_ERR_UNSUPPORTED;
+}
+
+struct Layout {
+    uint64_t lp, code_bytes, scale_bytes, stride;
+};
+
+Layout make_layout(const loco_config_t *c, uint64_t n) {
+    Layout L{0, 0, 0, 0};
+    if (n == 0) return L;
+    uint64_t unit = kRow;
+    if (c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX && static_cast<uint64_t>(c->block_size) > unit)
+        unit = static_cast<uint64_t>(c->block_size);
+    const uint64_t per = (n + static_cast<uint64_t>(c->num_partitions) - 1) / static_cast<uint64_t>(c->num_partitions);
+    L.lp = round_up(per, unit);
+    L.code_bytes = L.lp * static_cast<uint64_t>(c->bits) / 8;
+    L.scale_bytes = c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX ? (L.lp / static_cast<uint64_t>(c->block_size)) * 4 : 0;
+    L.stride = round_up(L.code_bytes + L.scale_bytes, 128);
+    return L;
+}
+
+uint64_t state_bytes(const loco_config_t *c, uint64_t n) {
+    if (n == 0) return 0;
+    switch (c->state_fmt) {
+    case LOCO_STATE_NONE: return 0;
+    case LOCO_STATE_INT8: {
+        uint64_t b = round_up(n, 256);
+        if (c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX)
+            b += round_up(((n + static_cast<uint64_t>(c->block_size) - 1) / static_cast<uint64_t>(c->block_size)) * 4, 256);
+        return b;
+    }
+    default: return round_up(n * 4, 256);
+    }
+}
+
+// Does multiplying by 1/scale reproduce the IEEE division by `scale` for every integer in [lo, hi]?
+bool reciprocal_exact(float scale, int lo, int hi) {
+    const volatile float inv = 1.0f / scale;
+    for (int q = lo; q <= hi; ++q) {
+        const volatile float a = static_cast<float>(q) * inv;
+        const volatile float b = static_cast<float>(q) / scale;
+        float fa = a, fb = b;
+        if (std::memcmp(&fa, &fb, 4) != 0) return false;
+    }
+    return true;
+}
+
+int kernel_mode(const loco_config_t *c, bool need_se) {
+    if (c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX) return MODE_BLOCK;
+    const int lo = -(1 << (c->bits - 1)), hi = (1 << (c->bits - 1)) - 1;
+    bool ok = reciprocal_exact(c->s, lo, hi);
+    if (need_se && (c->state_fmt == LOCO_STATE_INT8 || c->state_fmt == LOCO_STATE_FP32_Q8COMP))
+        ok = ok && reciprocal_exact(c->s_e, -128, 127);
+    return ok ? MODE_FIXED_RCP : MODE_FIXED_DIV;
+}
+
+int num_sms() {
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
+        sms = v;
+    }
+    return sms;
+}
+
+// ---- send dispatch -----------------------------------------------------------------------
+
+using SendFn = void (*)(const SendParams);
+
+template <int GRAD, int STATE, int BITS>
+SendFn pick_send_mode(int mode) {
+    switch (mode) {
+    case MODE_FIXED_RCP: return loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED_RCP>;
+    case MODE_FIXED_DIV: return loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED_DIV>;
+    default: return loco_send_kernel<GRAD, STATE, BITS, MODE_BLOCK>;
+    }
+}
+template <int GRAD, int STATE>
+SendFn pick_send_bits(int bits, int mode) {
+    switch (bits) {
+    case 2: return pick_send_mode<GRAD, STATE, 2>(mode);
+    case 4: return pick_send_mode<GRAD, STATE, 4>(mode);
+    default: return pick_send_mode<GRAD, STATE, 8>(mode);
+    }
+}
+template <int GRAD>
+SendFn pick_send_state(int state, int bits, int mode) {
+    switch (state) {
+    case LOCO_STATE_INT8: return pick_send_bits<GRAD, ST_INT8>(bits, mode);
+    case LOCO_STATE_FP32: return pick_send_bits<GRAD, ST_FP32>(bits, mode);
+    case LOCO_STATE_NONE: return pick_send_bits<GRAD, ST_NONE>(bits, mode);
+    default:
+        // Q8COMP exists for the global scales only (checked in check_config)
+        if (mode == MODE_BLOCK) return nullptr;
+        return pick_send_bits<GRAD, ST_Q8COMP>(bits, mode);
+    }
+}
+SendFn pick_send(const loco_config_t *c, int mode) {
+    return c->grad_dtype == LOCO_BF16 ? pick_send_state<GRAD_BF16>(c->state_fmt, c->bits, mode)
+                                      : pick_send_state<GRAD_F32>(c->state_fmt, c->bits, mode);
+}
+
+// ---- reduce dispatch ---------------------------------------------------------------------
+
+using ReduceFn = void (*)(const ReduceParams);
+
+template <int OUT, int BITS>
+ReduceFn pick_reduce_mode(int mode) {
+    switch (mode) {
+    case MODE_FIXED_RCP: return loco_reduce_kernel<OUT, BITS, MODE_FIXED_RCP>;
+    case MODE_FIXED_DIV: return loco_reduce_kernel<OUT, BITS, MODE_FIXED_DIV>;
+    default: return loco_reduce_kernel<OUT, BITS, MODE_BLOCK>;
+    }
+}
+template <int OUT>
+ReduceFn pick_reduce_bits(int bits, int mode) {
+    switch (bits) {
+    case 2: return pick_reduce_mode<OUT, 2>(mode);
+    case 4: return pick_reduce_mode<OUT, 4>(mode);
+    default: return pick_reduce_mode<OUT, 8>(mode);
+    }
+}
+ReduceFn pick_reduce(const loco_config_t *c, int mode) {
+    return c->out_dtype == LOCO_BF16 ? pick_reduce_bits<GRAD_BF16>(c->bits, mode)
+                                     : pick_reduce_bits<GRAD_F32>(c->bits, mode);
+}
+
+unsigned grid_x_for(uint64_t rows_per_partition, int partitions, int ctas_per_sm) {
+    const uint64_t want = (rows_per_partition + kWarps - 1) / kWarps;             // one row per warp
+    uint64_t budget = static_cast<uint64_t>(num_sms()) * static_cast<uint64_t>(ctas_per_sm);
+    uint64_t per_part = (budget + static_cast<uint64_t>(partitions) - 1) / static_cast<uint64_t>(partitions);
+    if (per_part < 1) per_part = 1;
+    uint64_t gx = want < per_part ? want : per_part;
+    if (gx < 1) gx = 1;
+    return static_cast<unsigned>(gx);
+}
+
+}  // namespace
+
+struct loco_state {
+    loco_config_t cfg;
+    uint64_t n;
+    void *d_state;
+    uint64_t state_bytes;
+    unsigned long long *d_status;   // 2 words on the device
+    int device;
+    int mode;
+    SendFn send_fn;
+    int send_ctas_per_sm;
+    Layout layout;
+};
+
+extern "C" {
+
+const char *loco_status_string(int status) {
+    switch (status) {
+    case LOCO_OK: return "LOCO_OK";
+    case LOCO_ERR_ARG: return "LOCO_ERR_ARG";
+    case LOCO_ERR_ALIGN: return "LOCO_ERR_ALIGN";
+    case LOCO_ERR_SIZE: return "LOCO_ERR_SIZE";
+    case LOCO_ERR_CUDA: return "LOCO_ERR_CUDA";
+    case LOCO_ERR_UNSUPPORTED: return "LOCO_ERR_UNSUPPORTED";
+    default: return "LOCO_ERR_UNKNOWN";
+    }
+}
+
+uint64_t loco_launch_count(void) { return g_launches.load(); }
+
+int loco_config_check(const loco_config_t *cfg) { return check_config(cfg); }
+
+uint64_t loco_state_bytes(const loco_config_t *cfg, uint64_t n) {
+    return layout_ok(cfg) ? state_bytes(cfg, n) : 0;
+}
+uint64_t loco_partition_capacity(const loco_config_t *cfg, uint64_t n) {
+    return layout_ok(cfg) ? make_layout(cfg, n).lp : 0;
+}
+uint64_t loco_partition_bytes(const loco_config_t *cfg, uint64_t n) {
+    return layout_ok(cfg) ? make_layout(cfg, n).stride : 0;
+}
+uint64_t loco_packed_bytes(const loco_config_t *cfg, uint64_t n) {
+    return layout_ok(cfg) ? make_layout(cfg, n).stride * static_cast<uint64_t>(cfg->num_partitions) : 0;
+}
+uint64_t loco_partition_elems(const loco_config_t *cfg, uint64_t n, int32_t j) {
+    if (!layout_ok(cfg) || j < 0 || j >= cfg->num_partitions) return 0;
+    const uint64_t lp = make_layout(cfg, n).lp;
+    const uint64_t lo = static_cast<uint64_t>(j) * lp;
+    if (lp == 0 || lo >= n) return 0;
+    return (n - lo < lp) ? n - lo : lp;
+}
+
+int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, void *d_state,
+                    uint64_t d_state_bytes, void *stream) {
+    if (!out) return LOCO_ERR_ARG;
+    *out = nullptr;
+    const int rc = check_config(cfg);
+    if (rc != LOCO_OK) return rc;
+    const uint64_t need = state_bytes(cfg, n);
+    if (need > 0) {
+        if (!d_state) return LOCO_ERR_ARG;
+        if (!aligned16(d_state)) return LOCO_ERR_ALIGN;
+        if (d_state_bytes < need) return LOCO_ERR_SIZE;
+    }
+    loco_state *st = new (std::nothrow) loco_state;
+    if (!st) return LOCO_ERR_ARG;
+    st->cfg = *cfg;
+    st->n = n;
+    st->d_state = d_state;
+    st->state_bytes = need;
+    st->d_status = nullptr;
+    st->layout = make_layout(cfg, n);
+    st->mode = kernel_mode(cfg, true);
+    st->send_fn = pick_send(cfg, st->mode);
+    st->send_ctas_per_sm = 1;
+    if (!st->send_fn) { delete st; return LOCO_ERR_UNSUPPORTED; }
+    if (cudaGetDevice(&st->device) != cudaSuccess) { delete st; return LOCO_ERR_CUDA; }
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, st->send_fn, kThreads, 0) != cudaSuccess || occ < 1) {
+        cudaGetLastError();
+        delete st;
+        return LOCO_ERR_CUDA;
+    }
+    st->send_ctas_per_sm = occ;
+    if (cudaMalloc(reinterpret_cast<void **>(&st->d_status), 16) != cudaSuccess) {
+        cudaGetLastError();
+        delete st;
+        return LOCO_ERR_CUDA;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(st->d_status, 0, 16, s);
+    if (e == cudaSuccess && need > 0) e = cudaMemsetAsync(d_state, 0, need, s);   // e~_0 = 0
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(st->d_status);
+        delete st;
+        return LOCO_ERR_CUDA;
+    }
+    *out = st;
+    return LOCO_OK;
+}
+
+int loco_state_reset(loco_state_t *st, void *stream) {
+    if (!st) return LOCO_ERR_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(st->d_status, 0, 16, s);
+    if (e == cudaSuccess && st->state_bytes > 0) e = cudaMemsetAsync(st->d_state, 0, st->state_bytes, s);
+    if (e != cudaSuccess) { cudaGetLastError(); return LOCO_ERR_CUDA; }
+    return LOCO_OK;
+}
+
+int loco_state_destroy(loco_state_t *st) {
+    if (!st) return LOCO_ERR_ARG;
+    int rc = LOCO_OK;
+    if (st->d_status && cudaFree(st->d_status) != cudaSuccess) { cudaGetLastError(); rc = LOCO_ERR_CUDA; }
+    delete st;
+    return rc;
+}
+
+int loco_compensate_quantize_pack(loco_state_t *st, const void *d_grad, void *d_comm, int64_t step_k,
+                                  void *stream) {
+    if (!st || step_k < 0) return LOCO_ERR_ARG;
+    if (st->n == 0) return LOCO_OK;
+    if (!d_grad || !d_comm) return LOCO_ERR_ARG;
+    if (!aligned16(d_grad) || !aligned16(d_comm)) return LOCO_ERR_ALIGN;
+    const loco_config_t &c = st->cfg;
+    SendParams P;
+    std::memset(&P, 0, sizeof(P));
+    P.grad = d_grad;
+    P.state = st->d_state;
+    P.comm = static_cast<uint8_t *>(d_comm);
+    P.n = st->n;
+    P.lp = st->layout.lp;
+    P.stride = st->layout.stride;
+    P.code_bytes = st->layout.code_bytes;
+    P.state_scale_off = round_up(st->n, 256);
+    P.s = c.s;
+    P.inv_s = 1.0f / c.s;
+    P.s_e = c.s_e;
+    P.inv_se = 1.0f / c.s_e;
+    P.beta = c.beta;
+    {
+        const volatile float omb = 1.0f - c.beta;    // (1 - beta), rounded once to fp32
+        P.omb = omb;
+    }
+    P.block_log2 = c.scale_mode == LOCO_SCALE_BLOCK_ABSMAX ? ilog2(static_cast<uint32_t>(c.block_size)) : 0;
+    P.reset = (c.reset_period > 0 && (step_k % static_cast<int64_t>(c.reset_period)) == 0) ? 1 : 0;
+    P.collect_stats = c.collect_stats ? 1 : 0;
+    P.status = st->d_status;
+    const uint64_t rows = P.lp / kRow;
+    dim3 grid(grid_x_for(rows, c.num_partitions, st->send_ctas_per_sm), static_cast<unsigned>(c.num_partitions), 1);
+    st->send_fn<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(P);
+    if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return LOCO_OK;
+}
+
+int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_packed, int32_t num_workers,
+                               uint64_t n, int32_t first_partition, int32_t partition_count, void *d_out,
+                               void *stream) {
+    const int rc = check_config(cfg);
+    if (rc != LOCO_OK) return rc;
+    if (num_workers < 1 || first_partition < 0 || partition_count < 0 ||
+        first_partition + partition_count > cfg->num_partitions) return LOCO_ERR_ARG;
+    if (num_workers > 64) return LOCO_ERR_UNSUPPORTED;
+    if (n == 0 || partition_count == 0) return LOCO_OK;
+    const Layout L = make_layout(cfg, n);
+    if (static_cast<uint64_t>(first_partition) * L.lp >= n) return LOCO_OK;      // nothing valid there
+    if (!d_packed || !d_out) return LOCO_ERR_ARG;
+    if (!aligned16(d_out)) return LOCO_ERR_ALIGN;
+    ReduceParams P;
+    std::memset(&P, 0, sizeof(P));
+    for (int w = 0; w < num_workers; ++w) {
+        if (!d_packed[w]) return LOCO_ERR_ARG;
+        if (!aligned16(d_packed[w])) return LOCO_ERR_ALIGN;
+        P.parts[w] = static_cast<const uint8_t *>(d_packed[w]);
+    }
+    P.out = d_out;
+    P.n = n;
+    P.lp = L.lp;
+    P.stride = L.stride;
+    P.code_bytes = L.code_bytes;
+    P.first = static_cast<unsigned long long>(first_partition);
+    P.num_workers = num_workers;
+    P.block_log2 = cfg->scale_mode == LOCO_SCALE_BLOCK_ABSMAX ? ilog2(static_cast<uint32_t>(cfg->block_size)) : 0;
+    P.s = cfg->s;
+    P.inv_s = 1.0f / cfg->s;
+    P.n_workers_f = static_cast<float>(num_workers);
+    P.inv_n = 1.0f / static_cast<float>(num_workers);
+    P.inv_n_exact = is_pow2(static_cast<uint64_t>(num_workers)) ? 1 : 0;
+    const int mode = kernel_mode(cfg, false);
+    ReduceFn fn = pick_reduce(cfg, mode);
+    static int occ_cache[2][3][3] = {};
+    int &occ = occ_cache[cfg->out_dtype == LOCO_BF16][cfg->bits == 2 ? 0 : (cfg->bits == 4 ? 1 : 2)][mode];
+    if (occ == 0) {
+        int v = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, fn, kThreads, 0) != cudaSuccess || v < 1) {
+            cudaGetLastError();
+            return LOCO_ERR_CUDA;
+        }
+        occ = v;
+    }
+    const uint64_t rows = L.lp / kRow;
+    dim3 grid(grid_x_for(rows, partition_count, occ), static_cast<unsigned>(partition_count), 1);
+    fn<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(P);
+    if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return LOCO_OK;
+}
+
+int loco_last_status(loco_state_t *st, uint32_t *flags, uint64_t *n_saturated, void *stream) {
+    if (!st) return LOCO_ERR_ARG;
+    unsigned long long host[2] = {0, 0};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(host, st->d_status, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return LOCO_ERR_CUDA;
+    }
+    if (flags) *flags = static_cast<uint32_t>(host[0]);
+    if (n_saturated) *n_saturated = host[1];
+    return LOCO_OK;
+}
+
+}  // extern "C"
