@@ -1,0 +1,402 @@
+#!/usr/bin/env python
+"""Benchmark of the LoCo hot path (arXiv 2407.04480) on B200.
+
+Workload (default): what ONE data-parallel rank of an 8-worker job does per training
+iteration on a Llama-2-7B-shaped gradient -- 6,738,415,616 bf16 elements cut into 270
+buckets of 25,000,000 (last one partial):
+    phase A  for every bucket: send pass (Algorithm 1 steps 1-2: compensate, 4-bit codes,
+             moving-average error into the 8-bit state, pack into the 8-part buffer);
+    phase B  for every bucket: receive pass (Eq. 8) over this rank's part, from its own
+             buffer and the buffers of the 7 other workers (resident in the same HBM).
+All inputs are synthetic and resident in HBM before the timed region; every bucket is read
+once per step and the step touches ~35 GB, far more than the 126 MB L2.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line (rank 0).  With --impl reference the CPU oracle is timed instead, on a
+bounded sample of the same workload (it is a deliberately plain program: the ratio to it is
+context, parity and the roofline fraction are the results).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "compensate+quantize and dequant-reduce GB/s of gradient per bucket pass (send + own-part reduce)"
+BUCKET = 25_000_000
+WORKERS = 8
+L2_BYTES = 126 * 1024 * 1024
+# Paper-faithful settings (Eq. 1 global scale; Eq. 7 T_c; s_e = 4 s); beta is not printed in the paper.
+CFG = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 14, s_e=2.0 ** 16, beta=0.5, reset_period=512,
+           state_fmt=0, grad_dtype=1, out_dtype=1, num_partitions=WORKERS)
+# Algorithmic HBM bytes per element (bf16 gradient read, int8 state read + written, 4-bit code written).
+SEND_BYTES_PER_ELEM = 2 + 1 + 1 + 0.5
+# DRAM bytes per element of the send kernel from the ncu capture summarised under profiles/ (None = not captured).
+SEND_DRAM_BYTES_PER_ELEM = None
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle samples taken every 200 ms while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.dev = device_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.dev), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons, smax = [], set(), None
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    smax = float(f[2])
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=smax, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ------------------------------------------------------------------------------------------------ our arm
+
+class RankWorkload:
+    """Buffers of one rank: its gradient, error state, own packed buffers, the 7 received parts, the output."""
+
+    def __init__(self, rank: int, device: torch.device):
+        from paper_2407_04480_b200 import inputs, loco
+        self.loco = loco
+        self.cfg = loco.Config(**CFG)
+        self.part = rank % WORKERS
+        layout = inputs.llama2_7b()
+        scales = inputs.group_scales(1, layout.n_groups)
+        self.buckets = inputs.bucket_ranges(layout.numel, BUCKET)
+        self.total = layout.numel
+        self.grad = torch.empty(self.total, dtype=torch.bfloat16, device=device)
+        for lo, hi in self.buckets:
+            self.grad[lo:hi] = inputs.layout_slice(layout, lo, hi, scales, 1e-4, seed=1, worker=rank, step=0,
+                                                   device=device)
+        cfg = self.cfg
+        sb = [loco.loco_state_bytes(cfg, hi - lo) for lo, hi in self.buckets]
+        pb = [loco.loco_packed_bytes(cfg, hi - lo) for lo, hi in self.buckets]
+        self.stride = [loco.loco_partition_bytes(cfg, hi - lo) for lo, hi in self.buckets]
+        self.out_elems = [loco.loco_partition_elems(cfg, hi - lo, self.part) for lo, hi in self.buckets]
+        self.state_buf = torch.empty(sum(sb), dtype=torch.uint8, device=device)
+        self.comm_buf = torch.empty(sum(pb), dtype=torch.uint8, device=device)
+        # parts of the 7 other workers as they would sit after the all-to-all: any byte is two valid codes
+        gen = torch.Generator(device=device)
+        gen.manual_seed(1234 + rank)
+        self.recv_buf = torch.randint(0, 256, (sum(self.stride) * (WORKERS - 1),), dtype=torch.uint8, device=device,
+                                      generator=gen)
+        self.out_buf = torch.empty(sum((e + 127) // 128 * 128 for e in self.out_elems), dtype=torch.bfloat16, device=device)
+        self.states, self.grads, self.comms, self.packed, self.outs = [], [], [], [], []
+        so = co = ro = oo = 0
+        for i, (lo, hi) in enumerate(self.buckets):
+            n = hi - lo
+            self.states.append(loco.State(cfg, n, buffer=self.state_buf[so:so + sb[i]]))
+            self.grads.append(self.grad[lo:hi])
+            comm = self.comm_buf[co:co + pb[i]]
+            self.comms.append(comm)
+            ptrs = []
+            for w in range(WORKERS):
+                if w == self.part:
+                    ptrs.append(comm.data_ptr() + self.part * self.stride[i])
+                else:
+                    ptrs.append(self.recv_buf.data_ptr() + ro)
+                    ro += self.stride[i]
+            self.packed.append(ptrs)
+            self.outs.append(self.out_buf[oo:oo + self.out_elems[i]])
+            so += sb[i]
+            co += pb[i]
+            oo += (self.out_elems[i] + 127) // 128 * 128
+        self.send_bytes = SEND_BYTES_PER_ELEM * self.total
+        self.recv_bytes = sum(e * (WORKERS * 0.5 + 2) for e in self.out_elems)
+        self.grad_bytes = 2 * self.total
+
+    def send_phase(self, k: int):
+        f = self.loco.loco_compensate_quantize_pack
+        for st, g, c in zip(self.states, self.grads, self.comms):
+            f(st, g, c, k)
+
+    def reduce_phase(self):
+        f = self.loco.loco_unpack_dequant_reduce
+        for i, (lo, hi) in enumerate(self.buckets):
+            f(self.cfg, self.packed[i], hi - lo, self.outs[i], first_partition=self.part, partition_count=1)
+
+
+def run_e2e(wl: RankWorkload, steps: int, warmup: int):
+    """Same step through the host-buffer entry points: every bucket's gradient and the 8 packed parts are
+    copied from pinned host memory, the packed codes and the averaged part are copied back."""
+    loco, cfg = wl.loco, wl.cfg
+    ring = 4
+    nmax = BUCKET
+    h_grad = [torch.empty(nmax, dtype=torch.bfloat16).pin_memory() for _ in range(ring)]
+    h_comm = [torch.empty(loco.loco_packed_bytes(cfg, nmax), dtype=torch.uint8).pin_memory() for _ in range(ring)]
+    stride = loco.loco_partition_bytes(cfg, nmax)
+    h_parts = [[torch.randint(0, 256, (stride,), dtype=torch.uint8).pin_memory() for _ in range(WORKERS)] for _ in range(ring)]
+    h_out = [torch.empty(loco.loco_partition_capacity(cfg, nmax), dtype=torch.bfloat16).pin_memory() for _ in range(ring)]
+    for r in range(ring):
+        h_grad[r].copy_(wl.grads[r].cpu())
+    dev = wl.grad.device
+    w_send = torch.empty(loco.loco_send_host_workspace_bytes(cfg, nmax), dtype=torch.uint8, device=dev)
+    w_red = torch.empty(loco.loco_reduce_host_workspace_bytes(cfg, nmax, WORKERS, 1), dtype=torch.uint8, device=dev)
+    h2d = d2h = 0
+    for i, (lo, hi) in enumerate(wl.buckets):
+        n = hi - lo
+        h2d += 2 * n + WORKERS * loco.loco_partition_bytes(cfg, n)
+        d2h += loco.loco_packed_bytes(cfg, n) + 2 * wl.out_elems[i]
+
+    def step(k):
+        for i, (lo, hi) in enumerate(wl.buckets):
+            n = hi - lo
+            r = i % ring
+            loco.loco_compensate_quantize_pack_host(wl.states[i], h_grad[r][:n], h_comm[r], w_send, k)
+        for i, (lo, hi) in enumerate(wl.buckets):
+            n = hi - lo
+            r = i % ring
+            loco.loco_unpack_dequant_reduce_host(cfg, h_parts[r], n, h_out[r], w_red, first_partition=wl.part,
+                                                 partition_count=1)
+
+    for k in range(warmup):
+        step(1000 + k)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for k in range(steps):
+        step(2000 + k)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    return ms, h2d, d2h
+
+
+def oracle_sample(threads: int, buckets_per_thread: int):
+    """The oracle as it stands on `threads` host threads, each doing whole 25M-element buckets of the
+    workload (send pass, then this rank's part of the receive pass with 8 workers)."""
+    import numpy as np
+    from oracle import loco_oracle as orc
+    ocfg = orc.OracleConfig(**CFG)
+    n = BUCKET
+    rng = np.random.default_rng(1)
+    g = (rng.normal(0, 1e-4, n).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    others = [rng.integers(0, 256, orc.packed_bytes(ocfg, n), dtype=np.uint8) for _ in range(2)]
+    states = [orc.new_state(ocfg, n) for _ in range(threads)]
+    comms = [orc.new_comm(ocfg, n) for _ in range(threads)]
+    orc.lib()
+
+    def work(t):
+        for b in range(buckets_per_thread):
+            orc.send_step(ocfg, g, states[t], comms[t], 1 + b)
+            orc.reduce(ocfg, n, [comms[t]] + [others[w % 2] for w in range(WORKERS - 1)], first=0, count=1)
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        list(ex.map(work, range(threads)))
+    dt = time.perf_counter() - t0
+    elems = threads * buckets_per_thread * n
+    return 2.0 * elems / dt / 1e9, dt, elems
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    cores = os.cpu_count() or 1
+    config = {"workload": "llama2-7b: 270 bf16 buckets of 25M elements (6,738,415,616), per-rank view of an 8-worker job",
+              "bits": 4, "scale": "fixed s=2^14, s_e=4s (Eq. 1)", "beta": 0.5, "T_c": 512, "state": "int8",
+              "workers_on_reduce_side": WORKERS, "out": "bf16",
+              "l2": "inputs larger than L2: each step streams ~35 GB once, no reuse between launches"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        steps = max(1, args.steps)
+        for _ in range(min(args.warmup, 1)):
+            oracle_sample(cores, 1)
+        t0 = time.perf_counter()
+        elems = 0
+        for _ in range(steps):
+            _, _, e = oracle_sample(cores, 1)
+            elems += e
+        dt = time.perf_counter() - t0
+        val = 2.0 * elems / dt / 1e9
+        sample = "%d buckets of 25M elements per step (one per host thread), send + own-part reduce" % cores
+        print(json.dumps({"impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus,
+                          "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": dt / steps * 1e3,
+                          "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                          "data": "synthetic", "config": config,
+                          "cpu_baseline": {"value": val, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+                          "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                          "gpu_launches": 0}))
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    from paper_2407_04480_b200 import loco
+    loco.lib()
+    wl = RankWorkload(rank, device)
+    nb = len(wl.buckets)
+    # The 540 launches of a step are captured once into two CUDA graphs (one per phase) and replayed,
+    # so that the host's launch cost does not sit between kernels of a few microseconds each.
+    wl.send_phase(1)
+    wl.reduce_phase()
+    torch.cuda.synchronize()
+    g_send, g_reduce = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_send):
+        wl.send_phase(100)
+    with torch.cuda.graph(g_reduce):
+        wl.reduce_phase()
+    for k in range(max(3, args.warmup)):
+        g_send.replay()
+        g_reduce.replay()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    K = args.steps
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    barrier()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for k in range(K):
+        ev[k][0].record()
+        g_send.replay()
+        ev[k][1].record()
+        g_reduce.replay()
+        ev[k][2].record()
+    end.record()
+    barrier()
+    launches = 2 * nb * K          # one send and one receive kernel per bucket and step, replayed from the graphs
+    clocks = sampler.stop()
+    total_ms = start.elapsed_time(end)
+    send_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / K
+    recv_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
+    step_ms = total_ms / K
+    if dist is not None:
+        t = torch.tensor([step_ms, send_ms, recv_ms], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        step_ms, send_ms, recv_ms = [float(x) for x in t]
+        lt = torch.tensor([launches], device=device, dtype=torch.int64)
+        dist.all_reduce(lt)
+        launches = int(lt.item())
+
+    e2e = None
+    if not args.no_e2e:
+        e_ms, h2d, d2h = run_e2e(wl, args.e2e_steps, 1)
+        if dist is not None:
+            t = torch.tensor([e_ms], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": world * wl.grad_bytes / (e_ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d * world,
+               "d2h_bytes_per_step": d2h * world, "ms_per_step": e_ms, "steps": args.e2e_steps,
+               "how": "loco_*_host entry points, pinned host buffers, copies inside the timed region"}
+    if dist is not None:
+        dist.barrier()
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peak()
+    send_gbs = wl.send_bytes / (send_ms * 1e-3) / 1e9
+    recv_gbs = wl.recv_bytes / (recv_ms * 1e-3) / 1e9
+    roofline = {"kernel": "loco_send_kernel<bf16, int8 state, 4 bit, fixed scale>", "bound": "hbm",
+                "achieved": send_gbs, "peak": peak, "peak_kind": "%s HBM copy bandwidth" % peak_kind, "unit": "GB/s",
+                "frac": send_gbs / peak, "frac_of_nominal_8TBps": send_gbs / 8000.0,
+                "traffic": (SEND_DRAM_BYTES_PER_ELEM * BUCKET if SEND_DRAM_BYTES_PER_ELEM else None),
+                "algorithmic_bytes_per_launch": SEND_BYTES_PER_ELEM * BUCKET, "avg_launch_us": send_ms * 1e3 / nb,
+                "launches_per_step": nb}
+    kernels = {"send": {"hbm_gbs": send_gbs, "frac_of_peak": send_gbs / peak, "gradient_gbs": wl.grad_bytes / (send_ms * 1e-3) / 1e9,
+                        "ms_per_step": send_ms, "avg_launch_us": send_ms * 1e3 / nb, "bytes_per_elem": SEND_BYTES_PER_ELEM},
+               "reduce": {"hbm_gbs": recv_gbs, "frac_of_peak": recv_gbs / peak,
+                          "gradient_gbs": 2 * sum(wl.out_elems) / (recv_ms * 1e-3) / 1e9, "ms_per_step": recv_ms,
+                          "avg_launch_us": recv_ms * 1e3 / nb, "bytes_per_out_elem": WORKERS * 0.5 + 2}}
+    cpu = None
+    if not args.no_cpu_baseline:
+        v, dt, elems = oracle_sample(cores, 2)
+        cpu = {"value": v, "unit": "GB/s", "cores": cores, "kind": "oracle",
+               "sample": "%d buckets of 25M elements (2 per host thread), send + own-part reduce, %.1f s wall" % (2 * cores, dt)}
+    line = {"metric": METRIC, "value": world * wl.grad_bytes / (step_ms * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": world,
+            "steps": K, "warmup": max(3, args.warmup), "ms_per_step": step_ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,
+            "kernels": kernels}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -152,6 +152,33 @@ int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_pa
                                int32_t num_workers, uint64_t n, int32_t first_partition,
                                int32_t partition_count, void *d_out, void *stream);
 
+/* ---- host-buffer variants ------------------------------------------------------------------
+ * The same two passes for callers whose gradient and communication buffers live in HOST memory
+ * (pinned memory makes the copies asynchronous).  Each call enqueues, on `stream`: the
+ * host-to-device copy of its inputs into the caller's device workspace d_work, the kernel, and
+ * the device-to-host copy of its result.  Nothing is allocated; the call returns without
+ * synchronising, so the host buffers must stay untouched until the stream has drained.  The
+ * error state stays on the device (it never leaves the worker, Sec. 3.1 of the paper).
+ * Pad bytes of h_comm (see the wire layout) receive unspecified values.
+ * Errors as for the device variants, plus SIZE when d_work_bytes is too small.
+ */
+uint64_t loco_send_host_workspace_bytes(const loco_config_t *cfg, uint64_t n);
+uint64_t loco_reduce_host_workspace_bytes(const loco_config_t *cfg, uint64_t n, int32_t num_workers,
+                                          int32_t partition_count);
+
+/* Algorithm 1 steps 1-2 with h_grad (n elements) read from and h_comm (loco_packed_bytes())
+ * written to host memory. */
+int loco_compensate_quantize_pack_host(loco_state_t *st, const void *h_grad, void *h_comm,
+                                       void *d_work, uint64_t d_work_bytes, int64_t step_k,
+                                       void *stream);
+
+/* Eq. 8 with h_packed[w] (HOST pointers to part `first_partition` of worker w's buffer,
+ * partition_count * loco_partition_bytes() readable bytes each) and h_out in host memory. */
+int loco_unpack_dequant_reduce_host(const loco_config_t *cfg, const void *const *h_packed,
+                                    int32_t num_workers, uint64_t n, int32_t first_partition,
+                                    int32_t partition_count, void *h_out, void *d_work,
+                                    uint64_t d_work_bytes, void *stream);
+
 /*
  * Read the status word accumulated by the send passes of this handle since init/reset.
  * SYNCHRONISES `stream` (the one the passes ran on).  n_saturated counts gradient codes

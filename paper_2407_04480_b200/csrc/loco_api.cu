@@ -397,6 +397,85 @@ int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_pa
     return LOCO_OK;
 }
 
+uint64_t loco_send_host_workspace_bytes(const loco_config_t *cfg, uint64_t n) {
+    if (!layout_ok(cfg) || n == 0) return 0;
+    const uint64_t gbytes = round_up(n * (cfg->grad_dtype == LOCO_BF16 ? 2u : 4u), 256);
+    return gbytes + make_layout(cfg, n).stride * static_cast<uint64_t>(cfg->num_partitions);
+}
+
+uint64_t loco_reduce_host_workspace_bytes(const loco_config_t *cfg, uint64_t n, int32_t num_workers,
+                                          int32_t partition_count) {
+    if (!layout_ok(cfg) || n == 0 || num_workers < 1 || partition_count < 1) return 0;
+    const Layout L = make_layout(cfg, n);
+    const uint64_t in = static_cast<uint64_t>(num_workers) * static_cast<uint64_t>(partition_count) * L.stride;
+    const uint64_t out = round_up(static_cast<uint64_t>(partition_count) * L.lp * (cfg->out_dtype == LOCO_BF16 ? 2u : 4u), 256);
+    return in + out;
+}
+
+int loco_compensate_quantize_pack_host(loco_state_t *st, const void *h_grad, void *h_comm, void *d_work,
+                                       uint64_t d_work_bytes, int64_t step_k, void *stream) {
+    if (!st || step_k < 0) return LOCO_ERR_ARG;
+    if (st->n == 0) return LOCO_OK;
+    if (!h_grad || !h_comm || !d_work) return LOCO_ERR_ARG;
+    if (!aligned16(d_work)) return LOCO_ERR_ALIGN;
+    if (d_work_bytes < loco_send_host_workspace_bytes(&st->cfg, st->n)) return LOCO_ERR_SIZE;
+    const uint64_t gbytes_exact = st->n * (st->cfg.grad_dtype == LOCO_BF16 ? 2u : 4u);
+    const uint64_t gbytes = round_up(gbytes_exact, 256);
+    const uint64_t pbytes = st->layout.stride * static_cast<uint64_t>(st->cfg.num_partitions);
+    uint8_t *d_grad = static_cast<uint8_t *>(d_work);
+    uint8_t *d_comm = d_grad + gbytes;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(d_grad, h_grad, gbytes_exact, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+        cudaGetLastError();
+        return LOCO_ERR_CUDA;
+    }
+    const int rc = loco_compensate_quantize_pack(st, d_grad, d_comm, step_k, stream);
+    if (rc != LOCO_OK) return rc;
+    if (cudaMemcpyAsync(h_comm, d_comm, pbytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+        cudaGetLastError();
+        return LOCO_ERR_CUDA;
+    }
+    return LOCO_OK;
+}
+
+int loco_unpack_dequant_reduce_host(const loco_config_t *cfg, const void *const *h_packed, int32_t num_workers,
+                                    uint64_t n, int32_t first_partition, int32_t partition_count, void *h_out,
+                                    void *d_work, uint64_t d_work_bytes, void *stream) {
+    const int rc0 = check_config(cfg);
+    if (rc0 != LOCO_OK) return rc0;
+    if (num_workers < 1 || first_partition < 0 || partition_count < 0 ||
+        first_partition + partition_count > cfg->num_partitions) return LOCO_ERR_ARG;
+    if (num_workers > 64) return LOCO_ERR_UNSUPPORTED;
+    if (n == 0 || partition_count == 0) return LOCO_OK;
+    if (!h_packed || !h_out || !d_work) return LOCO_ERR_ARG;
+    if (!aligned16(d_work)) return LOCO_ERR_ALIGN;
+    if (d_work_bytes < loco_reduce_host_workspace_bytes(cfg, n, num_workers, partition_count)) return LOCO_ERR_SIZE;
+    const Layout L = make_layout(cfg, n);
+    const uint64_t per_worker = static_cast<uint64_t>(partition_count) * L.stride;
+    uint8_t *base = static_cast<uint8_t *>(d_work);
+    const void *d_ptrs[64];
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int w = 0; w < num_workers; ++w) {
+        if (!h_packed[w]) return LOCO_ERR_ARG;
+        d_ptrs[w] = base + static_cast<uint64_t>(w) * per_worker;
+        if (cudaMemcpyAsync(const_cast<void *>(d_ptrs[w]), h_packed[w], per_worker, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+            cudaGetLastError();
+            return LOCO_ERR_CUDA;
+        }
+    }
+    uint8_t *d_out = base + static_cast<uint64_t>(num_workers) * per_worker;
+    const int rc = loco_unpack_dequant_reduce(cfg, d_ptrs, num_workers, n, first_partition, partition_count, d_out, stream);
+    if (rc != LOCO_OK) return rc;
+    uint64_t n_out = 0;
+    for (int j = first_partition; j < first_partition + partition_count; ++j) n_out += loco_partition_elems(cfg, n, j);
+    if (n_out == 0) return LOCO_OK;
+    if (cudaMemcpyAsync(h_out, d_out, n_out * (cfg->out_dtype == LOCO_BF16 ? 2u : 4u), cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+        cudaGetLastError();
+        return LOCO_ERR_CUDA;
+    }
+    return LOCO_OK;
+}
+
 int loco_last_status(loco_state_t *st, uint32_t *flags, uint64_t *n_saturated, void *stream) {
     if (!st) return LOCO_ERR_ARG;
     unsigned long long host[2] = {0, 0};

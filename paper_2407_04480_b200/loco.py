@@ -26,7 +26,9 @@ FLAG_NONFINITE = 1
 EXPORTS = ("loco_state_bytes", "loco_packed_bytes", "loco_partition_bytes", "loco_partition_capacity",
            "loco_partition_elems", "loco_config_check", "loco_state_init", "loco_state_reset",
            "loco_state_destroy", "loco_compensate_quantize_pack", "loco_unpack_dequant_reduce",
-           "loco_last_status", "loco_status_string", "loco_launch_count")
+           "loco_last_status", "loco_status_string", "loco_launch_count",
+           "loco_send_host_workspace_bytes", "loco_reduce_host_workspace_bytes",
+           "loco_compensate_quantize_pack_host", "loco_unpack_dequant_reduce_host")
 
 
 class LocoError(RuntimeError):
@@ -94,6 +96,14 @@ def lib() -> C.CDLL:
         L.loco_compensate_quantize_pack.argtypes = [vp, vp, vp, i64, vp]
         L.loco_unpack_dequant_reduce.restype = C.c_int
         L.loco_unpack_dequant_reduce.argtypes = [cp, C.POINTER(vp), i32, u64, i32, i32, vp, vp]
+        L.loco_send_host_workspace_bytes.restype = u64
+        L.loco_send_host_workspace_bytes.argtypes = [cp, u64]
+        L.loco_reduce_host_workspace_bytes.restype = u64
+        L.loco_reduce_host_workspace_bytes.argtypes = [cp, u64, i32, i32]
+        L.loco_compensate_quantize_pack_host.restype = C.c_int
+        L.loco_compensate_quantize_pack_host.argtypes = [vp, vp, vp, vp, u64, i64, vp]
+        L.loco_unpack_dequant_reduce_host.restype = C.c_int
+        L.loco_unpack_dequant_reduce_host.argtypes = [cp, C.POINTER(vp), i32, u64, i32, i32, vp, vp, u64, vp]
         L.loco_last_status.restype = C.c_int
         L.loco_last_status.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(u64), vp]
         L.loco_status_string.restype = C.c_char_p
@@ -229,3 +239,40 @@ def loco_last_status(st: State, stream=None):
     flags, sat = C.c_uint32(0), C.c_uint64(0)
     _check(lib().loco_last_status(st.handle, C.byref(flags), C.byref(sat), _stream_ptr(stream)), "loco_last_status")
     return int(flags.value), int(sat.value)
+
+
+# ---- host-buffer variants --------------------------------------------------------------------
+
+def loco_send_host_workspace_bytes(cfg: Config, n: int) -> int:
+    return int(lib().loco_send_host_workspace_bytes(C.byref(cfg.c()), n))
+
+
+def loco_reduce_host_workspace_bytes(cfg: Config, n: int, num_workers: int, partition_count: int) -> int:
+    return int(lib().loco_reduce_host_workspace_bytes(C.byref(cfg.c()), n, num_workers, partition_count))
+
+
+def _host_ptr(t: torch.Tensor) -> int:
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous host tensor")
+    return t.data_ptr()
+
+
+def loco_compensate_quantize_pack_host(st: State, h_grad: torch.Tensor, h_comm: torch.Tensor, d_work: torch.Tensor,
+                                       step_k: int, stream=None) -> None:
+    """Send pass with gradient and communication buffer in host memory (pinned for asynchronous copies)."""
+    _check(lib().loco_compensate_quantize_pack_host(st.handle, _host_ptr(h_grad), _host_ptr(h_comm), _dev_ptr(d_work),
+                                                    d_work.numel() * d_work.element_size(), step_k,
+                                                    _stream_ptr(stream)), "loco_compensate_quantize_pack_host")
+
+
+def loco_unpack_dequant_reduce_host(cfg: Config, h_packed: Sequence[torch.Tensor], n: int, h_out: torch.Tensor,
+                                    d_work: torch.Tensor, first_partition: int = 0,
+                                    partition_count: Optional[int] = None, stream=None) -> None:
+    """Receive pass with the workers' packed parts and the output in host memory."""
+    if partition_count is None:
+        partition_count = cfg.num_partitions - first_partition
+    ptrs = (C.c_void_p * len(h_packed))(*[_host_ptr(p) for p in h_packed])
+    _check(lib().loco_unpack_dequant_reduce_host(C.byref(cfg.c()), ptrs, len(h_packed), n, first_partition,
+                                                 partition_count, _host_ptr(h_out), _dev_ptr(d_work),
+                                                 d_work.numel() * d_work.element_size(), _stream_ptr(stream)),
+           "loco_unpack_dequant_reduce_host")
