@@ -115,7 +115,7 @@ class ClockSampler:
 class RankWorkload:
     """Buffers of one rank: its gradient, error state, own packed buffers, the 7 received parts, the output."""
 
-    def __init__(self, rank: int, device: torch.device):
+    def __init__(self, rank: int, device: torch.device, max_buckets: int = 0):
         from paper_2407_04480_b200 import inputs, loco
         self.loco = loco
         self.cfg = loco.Config(**CFG)
@@ -123,7 +123,9 @@ class RankWorkload:
         layout = inputs.llama2_7b()
         scales = inputs.group_scales(1, layout.n_groups)
         self.buckets = inputs.bucket_ranges(layout.numel, BUCKET)
-        self.total = layout.numel
+        if max_buckets > 0:
+            self.buckets = self.buckets[:max_buckets]
+        self.total = self.buckets[-1][1]
         self.grad = torch.empty(self.total, dtype=torch.bfloat16, device=device)
         for lo, hi in self.buckets:
             self.grad[lo:hi] = inputs.layout_slice(layout, lo, hi, scales, 1e-4, seed=1, worker=rank, step=0,
@@ -258,6 +260,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--buckets", type=int, default=0,
+                    help="profiling aid: only the first K buckets of the workload (0 = all 270); not a bench line")
+    ap.add_argument("--no-graph", action="store_true", help="profiling aid: launch every kernel directly")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -307,18 +312,25 @@ def main():
 
     from paper_2407_04480_b200 import loco
     loco.lib()
-    wl = RankWorkload(rank, device)
+    wl = RankWorkload(rank, device, args.buckets)
     nb = len(wl.buckets)
+    if args.buckets > 0:
+        config["workload"] += " -- REDUCED to the first %d buckets (profiling aid, not the bench workload)" % nb
     # The 540 launches of a step are captured once into two CUDA graphs (one per phase) and replayed,
     # so that the host's launch cost does not sit between kernels of a few microseconds each.
     wl.send_phase(1)
     wl.reduce_phase()
     torch.cuda.synchronize()
-    g_send, g_reduce = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
-    with torch.cuda.graph(g_send):
-        wl.send_phase(100)
-    with torch.cuda.graph(g_reduce):
-        wl.reduce_phase()
+    if args.no_graph:
+        class _Direct:
+            def __init__(self, fn): self.replay = fn
+        g_send, g_reduce = _Direct(lambda: wl.send_phase(100)), _Direct(wl.reduce_phase)
+    else:
+        g_send, g_reduce = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_send):
+            wl.send_phase(100)
+        with torch.cuda.graph(g_reduce):
+            wl.reduce_phase()
     for k in range(max(3, args.warmup)):
         g_send.replay()
         g_reduce.replay()

@@ -255,3 +255,49 @@ def test_state_reset_and_checkpoint_resume():
     loco.loco_state_reset(a)
     torch.cuda.synchronize()
     assert not a.buffer.any()
+
+
+# ---------------------------------------------------------------- host-buffer entry points
+
+@pytest.mark.parametrize("mode", [loco.SCALE_FIXED, loco.SCALE_BLOCK_ABSMAX])
+def test_host_buffer_variants(mode):
+    """The *_host entry points (gradient, packed parts and result in pinned host memory, staged through a
+    caller-provided device workspace) give the oracle's bytes."""
+    n, P, N = 300_001, 4, 3
+    gcfg, ocfg = both_configs(bits=4, scale_mode=mode, block_size=128, s=2.0 ** 12, s_e=2.0 ** 14, beta=0.5,
+                              reset_period=0, state_fmt=loco.STATE_INT8, grad_dtype=loco.BF16, out_dtype=loco.BF16,
+                              num_partitions=P)
+    stride = loco.loco_partition_bytes(gcfg, n)
+    w_send = torch.empty(loco.loco_send_host_workspace_bytes(gcfg, n), dtype=torch.uint8, device="cuda")
+    h_comms, o_comms = [], []
+    for w in range(N):
+        st = loco.State(gcfg, n)
+        ostate, ocomm = orc.new_state(ocfg, n), orc.new_comm(ocfg, n)
+        h_comm = torch.zeros(loco.loco_packed_bytes(gcfg, n), dtype=torch.uint8).pin_memory()
+        for k in range(2):
+            g = inputs.gaussian(n, 1e-3, seed=31, worker=w, step=k, dtype=torch.bfloat16)
+            h_grad = g.pin_memory()
+            loco.loco_compensate_quantize_pack_host(st, h_grad, h_comm, w_send, k + 1)
+            torch.cuda.synchronize()
+            orc.send_step(ocfg, grad_bits(g), ostate, ocomm, k + 1)
+        for (gc, gs), (oc, os_) in zip(orc.comm_views(ocfg, n, h_comm.numpy()), orc.comm_views(ocfg, n, ocomm)):
+            assert np.array_equal(gc, oc)
+            if gs is not None:
+                assert np.array_equal(gs.view(np.uint32), os_.view(np.uint32))
+        assert np.array_equal(orc.state_views(ocfg, n, st.buffer.cpu().numpy())[0], orc.state_views(ocfg, n, ostate)[0])
+        h_comms.append(h_comm)
+        o_comms.append(ocomm)
+    first, count = 1, 2
+    w_red = torch.empty(loco.loco_reduce_host_workspace_bytes(gcfg, n, N, count), dtype=torch.uint8, device="cuda")
+    n_out = sum(loco.loco_partition_elems(gcfg, n, j) for j in range(first, first + count))
+    h_out = torch.zeros(n_out, dtype=torch.bfloat16).pin_memory()
+    loco.loco_unpack_dequant_reduce_host(gcfg, [c[first * stride:] for c in h_comms], n, h_out, w_red,
+                                         first_partition=first, partition_count=count)
+    torch.cuda.synchronize()
+    want = orc.reduce(ocfg, n, o_comms, first=first, count=count)
+    assert_reduced_equal(h_out.view(torch.int16).numpy().view(np.uint16), want, True)
+    # a workspace one byte short is refused before anything is enqueued
+    with pytest.raises(loco.LocoError) as ei:
+        loco.loco_unpack_dequant_reduce_host(gcfg, [c[first * stride:] for c in h_comms], n, h_out, w_red[:-1],
+                                             first_partition=first, partition_count=count)
+    assert ei.value.code == loco.ERR_SIZE
