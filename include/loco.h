@@ -180,6 +180,42 @@ int loco_unpack_dequant_reduce_host(const loco_config_t *cfg, const void *const 
                                     uint64_t d_work_bytes, void *stream);
 
 /*
+ * Receive pass for host buffers that needs no device memory from the caller and allocates none.
+ * (No counterpart in the paper: this is a convenience of the library, not a step of the method.)
+ *
+ * Who needs it: code that has host buffers to reduce but no way to obtain device memory at the
+ * point of the call -- a communication hook running while the training framework's caching
+ * allocator already owns all of the GPU's free memory (a raw cudaMalloc then fails although the
+ * framework "has" memory), a plug-in loaded into a process whose memory budget is fixed at
+ * start-up, or a latency-critical loop in which cudaMalloc/cudaFree are banned because they
+ * synchronise the whole device.  loco_unpack_dequant_reduce_host asks such a caller for a
+ * workspace it cannot provide; this variant brings its own.
+ *
+ * Same arguments, result and errors as loco_unpack_dequant_reduce_host without d_work: the staging
+ * area is a fixed array of LOCO_NOALLOC_SCRATCH_BYTES that is part of the library image, so every
+ * GPU on which the library is used holds that much memory from the moment the library's device
+ * code is loaded there until the process exits.  The call performs only asynchronous copies and one
+ * kernel launch on `stream`; it calls no cudaMalloc, cudaFree or any other allocating routine.
+ *   - Limit: loco_reduce_host_workspace_bytes(cfg, n, num_workers, partition_count) must not
+ *     exceed LOCO_NOALLOC_SCRATCH_BYTES; a larger request returns LOCO_ERR_SIZE and enqueues
+ *     nothing (e.g. 8 workers, 4-bit codes, bf16 output: up to about 690,000 elements per call).
+ *     Reduce a longer part in several calls, one partition range at a time.
+ *   - The first call on each device looks up the array's device address (a host-side query, done
+ *     once per device with that device current).  Make that first call outside any stream
+ *     capture; later calls only enqueue work.
+ *   - All calls on one device share the one array and it keeps whatever the previous call left
+ *     in it.  Nothing in it has to start at zero: every byte the kernel reads is first overwritten
+ *     by this call's own host-to-device copies.  For the same reason two calls whose work overlaps
+ *     on the GPU (different streams, or a second process thread) race on the array and corrupt
+ *     each other's result: keep all calls on one device in one stream, or order them with events.
+ *   - h_packed / h_out must stay untouched until `stream` has drained, as for the _host variant.
+ */
+#define LOCO_NOALLOC_SCRATCH_BYTES (4u * 1024u * 1024u)
+int loco_unpack_dequant_reduce_host_noalloc(const loco_config_t *cfg, const void *const *h_packed,
+                                            int32_t num_workers, uint64_t n, int32_t first_partition,
+                                            int32_t partition_count, void *h_out, void *stream);
+
+/*
  * Read the status word accumulated by the send passes of this handle since init/reset.
  * SYNCHRONISES `stream` (the one the passes ran on).  n_saturated counts gradient codes
  * whose nearest integer fell outside the p-bit range; it stays 0 unless collect_stats.

@@ -6,6 +6,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "loco_kernels.cuh"
@@ -474,6 +475,57 @@ int loco_unpack_dequant_reduce_host(const loco_config_t *cfg, const void *const 
         return LOCO_ERR_CUDA;
     }
     return LOCO_OK;
+}
+
+// ---- receive pass for host buffers with a built-in staging area -------------------------------
+
+}  // extern "C"
+
+namespace {
+
+// Staging area of loco_unpack_dequant_reduce_host_noalloc: part of the library image, present on
+// every device that loads it, never allocated or freed.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[LOCO_NOALLOC_SCRATCH_BYTES];
+
+// Device address of g_noalloc_scratch on the current device.  In host code the array's name only
+// identifies the symbol to the runtime; it is not an address a copy or a kernel could use, so the
+// address is asked for once per device (with that device current) and remembered.
+int noalloc_scratch_address(void **out) {
+    constexpr int kCached = 64;
+    static std::mutex mu;
+    static void *cached[kCached] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) { cudaGetLastError(); return LOCO_ERR_CUDA; }
+    std::lock_guard<std::mutex> lock(mu);
+    if (dev < kCached && cached[dev]) { *out = cached[dev]; return LOCO_OK; }
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) { cudaGetLastError(); return LOCO_ERR_CUDA; }
+    if (dev < kCached) cached[dev] = p;
+    *out = p;
+    return LOCO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int loco_unpack_dequant_reduce_host_noalloc(const loco_config_t *cfg, const void *const *h_packed,
+                                            int32_t num_workers, uint64_t n, int32_t first_partition,
+                                            int32_t partition_count, void *h_out, void *stream) {
+    const int rc0 = check_config(cfg);
+    if (rc0 != LOCO_OK) return rc0;
+    if (num_workers < 1 || first_partition < 0 || partition_count < 0 ||
+        first_partition + partition_count > cfg->num_partitions) return LOCO_ERR_ARG;
+    if (num_workers > 64) return LOCO_ERR_UNSUPPORTED;
+    if (n == 0 || partition_count == 0) return LOCO_OK;
+    // the request must fit the fixed array: refuse it before anything is enqueued
+    if (loco_reduce_host_workspace_bytes(cfg, n, num_workers, partition_count) > LOCO_NOALLOC_SCRATCH_BYTES)
+        return LOCO_ERR_SIZE;
+    void *d_scratch = nullptr;
+    const int rc1 = noalloc_scratch_address(&d_scratch);
+    if (rc1 != LOCO_OK) return rc1;
+    return loco_unpack_dequant_reduce_host(cfg, h_packed, num_workers, n, first_partition, partition_count, h_out,
+                                           d_scratch, LOCO_NOALLOC_SCRATCH_BYTES, stream);
 }
 
 int loco_last_status(loco_state_t *st, uint32_t *flags, uint64_t *n_saturated, void *stream) {

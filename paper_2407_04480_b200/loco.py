@@ -28,7 +28,9 @@ EXPORTS = ("loco_state_bytes", "loco_packed_bytes", "loco_partition_bytes", "loc
            "loco_state_destroy", "loco_compensate_quantize_pack", "loco_unpack_dequant_reduce",
            "loco_last_status", "loco_status_string", "loco_launch_count",
            "loco_send_host_workspace_bytes", "loco_reduce_host_workspace_bytes",
-           "loco_compensate_quantize_pack_host", "loco_unpack_dequant_reduce_host")
+           "loco_compensate_quantize_pack_host", "loco_unpack_dequant_reduce_host",
+           "loco_unpack_dequant_reduce_host_noalloc")
+NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
 class LocoError(RuntimeError):
@@ -104,6 +106,8 @@ def lib() -> C.CDLL:
         L.loco_compensate_quantize_pack_host.argtypes = [vp, vp, vp, vp, u64, i64, vp]
         L.loco_unpack_dequant_reduce_host.restype = C.c_int
         L.loco_unpack_dequant_reduce_host.argtypes = [cp, C.POINTER(vp), i32, u64, i32, i32, vp, vp, u64, vp]
+        L.loco_unpack_dequant_reduce_host_noalloc.restype = C.c_int
+        L.loco_unpack_dequant_reduce_host_noalloc.argtypes = [cp, C.POINTER(vp), i32, u64, i32, i32, vp, vp]
         L.loco_last_status.restype = C.c_int
         L.loco_last_status.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(u64), vp]
         L.loco_status_string.restype = C.c_char_p
@@ -276,3 +280,18 @@ def loco_unpack_dequant_reduce_host(cfg: Config, h_packed: Sequence[torch.Tensor
                                                  partition_count, _host_ptr(h_out), _dev_ptr(d_work),
                                                  d_work.numel() * d_work.element_size(), _stream_ptr(stream)),
            "loco_unpack_dequant_reduce_host")
+
+
+def loco_unpack_dequant_reduce_host_noalloc(cfg: Config, h_packed: Sequence[torch.Tensor], n: int, h_out: torch.Tensor,
+                                            first_partition: int = 0, partition_count: Optional[int] = None,
+                                            stream=None) -> None:
+    """Receive pass on host buffers for callers that cannot hand over device memory (the framework's allocator
+    holds it all, or allocation is banned where the call is made): the library stages through its own fixed
+    array of NOALLOC_SCRATCH_BYTES instead of a workspace.  Larger requests raise LocoError(ERR_SIZE).  Calls on
+    one device share that array, so keep them on one stream; make the first call outside stream capture."""
+    if partition_count is None:
+        partition_count = cfg.num_partitions - first_partition
+    ptrs = (C.c_void_p * len(h_packed))(*[_host_ptr(p) for p in h_packed])
+    _check(lib().loco_unpack_dequant_reduce_host_noalloc(C.byref(cfg.c()), ptrs, len(h_packed), n, first_partition,
+                                                         partition_count, _host_ptr(h_out), _stream_ptr(stream)),
+           "loco_unpack_dequant_reduce_host_noalloc")
