@@ -83,25 +83,61 @@ uint64_t state_bytes(const loco_config_t *c, uint64_t n) {
     }
 }
 
-// Does multiplying by 1/scale reproduce the IEEE division by `scale` for every integer in [lo, hi]?
+inline bool same_bits(float a, float b) { return std::memcmp(&a, &b, 4) == 0; }
+
+// The kernels replace Eq. 1's division  code / scale  by cheaper sequences, but only when the sequence
+// gives the bits of the IEEE division for EVERY code it can meet; these routines run that check.
+// `bias` is what the kernel adds to the code inside the magic float: m = kMagic + bias + code.
+struct DecChoice { int mode; float a, b, inv; };
+
+DecChoice choose_dec(float scale, int lo, int hi, int bias) {
+    DecChoice c{DEC_DIVIDE, 0.0f, 0.0f, 0.0f};
+    const volatile float vinv = 1.0f / scale;
+    const float inv = vinv;
+    c.inv = inv;
+    if (!std::isfinite(inv) || inv == 0.0f) return c;
+    const float base = kMagic + static_cast<float>(bias);           // exact: an integer below 2^24
+    const volatile float vb = -base * inv;
+    const float a = inv, b = vb;
+    bool fma_ok = std::isfinite(b), nr_ok = true;
+    for (int q = lo; q <= hi; ++q) {
+        const volatile float vwant = static_cast<float>(q) / scale;
+        const float want = vwant;
+        const float m = base + static_cast<float>(q);                // exact
+        if (fma_ok && !same_bits(std::fmaf(m, a, b), want)) fma_ok = false;
+        if (nr_ok) {
+            const float cq = m - base;                               // exact
+            const volatile float vq0 = cq * inv;
+            const float q0 = vq0;
+            const float rem = std::fmaf(-q0, scale, cq);
+            if (!same_bits(std::fmaf(rem, inv, q0), want)) nr_ok = false;
+        }
+    }
+    if (fma_ok) { c.mode = DEC_FMA; c.a = a; c.b = b; }
+    else if (nr_ok) c.mode = DEC_NEWTON;
+    return c;
+}
+
+// Does multiplying by fl(1/scale) reproduce the division by `scale` for every integer in [lo, hi]?
 bool reciprocal_exact(float scale, int lo, int hi) {
     const volatile float inv = 1.0f / scale;
     for (int q = lo; q <= hi; ++q) {
         const volatile float a = static_cast<float>(q) * inv;
         const volatile float b = static_cast<float>(q) / scale;
-        float fa = a, fb = b;
-        if (std::memcmp(&fa, &fb, 4) != 0) return false;
+        if (!same_bits(a, b)) return false;
     }
     return true;
 }
 
-int kernel_mode(const loco_config_t *c, bool need_se) {
-    if (c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX) return MODE_BLOCK;
-    const int lo = -(1 << (c->bits - 1)), hi = (1 << (c->bits - 1)) - 1;
-    bool ok = reciprocal_exact(c->s, lo, hi);
-    if (need_se && (c->state_fmt == LOCO_STATE_INT8 || c->state_fmt == LOCO_STATE_FP32_Q8COMP))
-        ok = ok && reciprocal_exact(c->s_e, -128, 127);
-    return ok ? MODE_FIXED_RCP : MODE_FIXED_DIV;
+bool is_pow2_float(float x) {
+    uint32_t u;
+    std::memcpy(&u, &x, 4);
+    const uint32_t expo = (u >> 23) & 0xffu;
+    return (u >> 31) == 0 && (u & 0x7fffffu) == 0 && expo >= 27 && expo <= 227;    // 2^-100 .. 2^100
+}
+
+int kernel_mode(const loco_config_t *c) {
+    return c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX ? MODE_BLOCK : MODE_FIXED;
 }
 
 int num_sms() {
@@ -120,36 +156,32 @@ int num_sms() {
 using SendFn = void (*)(const SendParams);
 
 template <int GRAD, int STATE, int BITS>
-SendFn pick_send_mode(int mode) {
-    switch (mode) {
-    case MODE_FIXED_RCP: return loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED_RCP>;
-    case MODE_FIXED_DIV: return loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED_DIV>;
-    default: return loco_send_kernel<GRAD, STATE, BITS, MODE_BLOCK>;
-    }
+SendFn pick_send_mode(int mode, bool lean) {
+    if (mode == MODE_FIXED)
+        return lean ? loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, true> : loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, false>;
+    if (STATE == ST_Q8COMP) return nullptr;                     // Q8COMP exists for the global scales only
+    return loco_send_kernel<GRAD, (STATE == ST_Q8COMP ? ST_FP32 : STATE), BITS, MODE_BLOCK, true>;
 }
 template <int GRAD, int STATE>
-SendFn pick_send_bits(int bits, int mode) {
+SendFn pick_send_bits(int bits, int mode, bool lean) {
     switch (bits) {
-    case 2: return pick_send_mode<GRAD, STATE, 2>(mode);
-    case 4: return pick_send_mode<GRAD, STATE, 4>(mode);
-    default: return pick_send_mode<GRAD, STATE, 8>(mode);
+    case 2: return pick_send_mode<GRAD, STATE, 2>(mode, lean);
+    case 4: return pick_send_mode<GRAD, STATE, 4>(mode, lean);
+    default: return pick_send_mode<GRAD, STATE, 8>(mode, lean);
     }
 }
 template <int GRAD>
-SendFn pick_send_state(int state, int bits, int mode) {
+SendFn pick_send_state(int state, int bits, int mode, bool lean) {
     switch (state) {
-    case LOCO_STATE_INT8: return pick_send_bits<GRAD, ST_INT8>(bits, mode);
-    case LOCO_STATE_FP32: return pick_send_bits<GRAD, ST_FP32>(bits, mode);
-    case LOCO_STATE_NONE: return pick_send_bits<GRAD, ST_NONE>(bits, mode);
-    default:
-        // Q8COMP exists for the global scales only (checked in check_config)
-        if (mode == MODE_BLOCK) return nullptr;
-        return pick_send_bits<GRAD, ST_Q8COMP>(bits, mode);
+    case LOCO_STATE_INT8: return pick_send_bits<GRAD, ST_INT8>(bits, mode, lean);
+    case LOCO_STATE_FP32: return pick_send_bits<GRAD, ST_FP32>(bits, mode, lean);
+    case LOCO_STATE_NONE: return pick_send_bits<GRAD, ST_NONE>(bits, mode, lean);
+    default: return pick_send_bits<GRAD, ST_Q8COMP>(bits, mode, lean);
     }
 }
-SendFn pick_send(const loco_config_t *c, int mode) {
-    return c->grad_dtype == LOCO_BF16 ? pick_send_state<GRAD_BF16>(c->state_fmt, c->bits, mode)
-                                      : pick_send_state<GRAD_F32>(c->state_fmt, c->bits, mode);
+SendFn pick_send(const loco_config_t *c, int mode, bool lean) {
+    return c->grad_dtype == LOCO_BF16 ? pick_send_state<GRAD_BF16>(c->state_fmt, c->bits, mode, lean)
+                                      : pick_send_state<GRAD_F32>(c->state_fmt, c->bits, mode, lean);
 }
 
 // ---- reduce dispatch ---------------------------------------------------------------------
@@ -158,11 +190,8 @@ using ReduceFn = void (*)(const ReduceParams);
 
 template <int OUT, int BITS>
 ReduceFn pick_reduce_mode(int mode) {
-    switch (mode) {
-    case MODE_FIXED_RCP: return loco_reduce_kernel<OUT, BITS, MODE_FIXED_RCP>;
-    case MODE_FIXED_DIV: return loco_reduce_kernel<OUT, BITS, MODE_FIXED_DIV>;
-    default: return loco_reduce_kernel<OUT, BITS, MODE_BLOCK>;
-    }
+    if (mode == MODE_FIXED) return loco_reduce_kernel<OUT, BITS, MODE_FIXED>;
+    return loco_reduce_kernel<OUT, BITS, MODE_BLOCK>;
 }
 template <int OUT>
 ReduceFn pick_reduce_bits(int bits, int mode) {
@@ -180,7 +209,8 @@ ReduceFn pick_reduce(const loco_config_t *c, int mode) {
 unsigned grid_x_for(uint64_t rows_per_partition, int partitions, int ctas_per_sm) {
     const uint64_t want = (rows_per_partition + kWarps - 1) / kWarps;             // one row per warp
     uint64_t budget = static_cast<uint64_t>(num_sms()) * static_cast<uint64_t>(ctas_per_sm);
-    uint64_t per_part = (budget + static_cast<uint64_t>(partitions) - 1) / static_cast<uint64_t>(partitions);
+    // all CTAs of a launch must be resident together: a CTA that has to wait for a free slot would run alone
+    uint64_t per_part = budget / static_cast<uint64_t>(partitions);
     if (per_part < 1) per_part = 1;
     uint64_t gx = want < per_part ? want : per_part;
     if (gx < 1) gx = 1;
@@ -200,6 +230,8 @@ struct loco_state {
     SendFn send_fn;
     int send_ctas_per_sm;
     Layout layout;
+    DecChoice dq, de;               // how the kernels evaluate dec(q; s) and dec(e; s_e)
+    int fast;                       // the fast routine may be used
 };
 
 extern "C" {
@@ -260,8 +292,22 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
     st->state_bytes = need;
     st->d_status = nullptr;
     st->layout = make_layout(cfg, n);
-    st->mode = kernel_mode(cfg, true);
-    st->send_fn = pick_send(cfg, st->mode);
+    st->mode = kernel_mode(cfg);
+    st->dq = DecChoice{DEC_FMA, 0.0f, 0.0f, 0.0f};
+    st->de = st->dq;
+    st->fast = 1;
+    if (st->mode == MODE_FIXED) {
+        const int half = 1 << (cfg->bits - 1);
+        st->dq = choose_dec(cfg->s, -half, half - 1, half);
+        if (cfg->state_fmt == LOCO_STATE_INT8 || cfg->state_fmt == LOCO_STATE_FP32_Q8COMP)
+            st->de = choose_dec(cfg->s_e, -128, 127, 128);
+        st->fast = (st->dq.mode != DEC_DIVIDE && st->de.mode != DEC_DIVIDE) ? 1 : 0;
+    }
+    {
+        const bool lean = st->mode == MODE_BLOCK ||
+                          (st->dq.mode == DEC_FMA && st->de.mode == DEC_FMA && !cfg->collect_stats);
+        st->send_fn = pick_send(cfg, st->mode, lean);
+    }
     st->send_ctas_per_sm = 1;
     if (!st->send_fn) { delete st; return LOCO_ERR_UNSUPPORTED; }
     if (cudaGetDevice(&st->device) != cudaSuccess) { delete st; return LOCO_ERR_CUDA; }
@@ -325,9 +371,12 @@ int loco_compensate_quantize_pack(loco_state_t *st, const void *d_grad, void *d_
     P.code_bytes = st->layout.code_bytes;
     P.state_scale_off = round_up(st->n, 256);
     P.s = c.s;
-    P.inv_s = 1.0f / c.s;
     P.s_e = c.s_e;
-    P.inv_se = 1.0f / c.s_e;
+    P.inv_s = st->dq.inv;
+    P.inv_se = st->de.inv;
+    P.dq_a = st->dq.a; P.dq_b = st->dq.b; P.dq_mode = st->dq.mode;
+    P.de_a = st->de.a; P.de_b = st->de.b; P.de_mode = st->de.mode;
+    P.fast = st->fast;
     P.beta = c.beta;
     {
         const volatile float omb = 1.0f - c.beta;    // (1 - beta), rounded once to fp32
@@ -374,13 +423,47 @@ int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_pa
     P.num_workers = num_workers;
     P.block_log2 = cfg->scale_mode == LOCO_SCALE_BLOCK_ABSMAX ? ilog2(static_cast<uint32_t>(cfg->block_size)) : 0;
     P.s = cfg->s;
-    P.inv_s = 1.0f / cfg->s;
     P.n_workers_f = static_cast<float>(num_workers);
-    P.inv_n = 1.0f / static_cast<float>(num_workers);
-    P.inv_n_exact = is_pow2(static_cast<uint64_t>(num_workers)) ? 1 : 0;
-    const int mode = kernel_mode(cfg, false);
+    {
+        const volatile float inv_n = 1.0f / static_cast<float>(num_workers);
+        P.inv_n = inv_n;
+    }
+    const int mode = kernel_mode(cfg);
+    const bool n_pow2 = is_pow2(static_cast<uint64_t>(num_workers));
+    P.div_mode = n_pow2 ? 0 : 2;          // a multiply by 1/N is the division only for powers of two
+    P.gen_mul = 0.0f;
+    P.int_path = 0;
+    if (mode == MODE_FIXED) {
+        const int half = 1 << (cfg->bits - 1);
+        if (reciprocal_exact(cfg->s, -half, half - 1)) {
+            const volatile float inv = 1.0f / cfg->s;
+            P.gen_mul = inv;
+        }
+        // Integer path: with s a power of two every partial sum of Eq. 8 is exact in fp32, so the codes can be
+        // added as integers.  The lane sums are bounded by (2^p - 1) * N, which 8- and 16-bit lanes hold for N <= 16.
+        if (cfg->bits != 2 && num_workers <= 16 && is_pow2_float(cfg->s)) {
+            P.int_path = 1;
+            const float inv_s = 1.0f / cfg->s;                                    // exact
+            float ra = inv_s;
+            if (n_pow2) ra = inv_s * P.inv_n;                                     // exact: both powers of two
+            P.ra = ra;
+            P.rb = -(kMagic + static_cast<float>(half * num_workers)) * ra;       // exact: integer < 2^24 times 2^k
+            if (!n_pow2) {
+                // acc takes the values t / s, t in [-half N, (half-1) N]: check the short division on all of them
+                bool nr_ok = true;
+                for (int t = -half * num_workers; t <= (half - 1) * num_workers && nr_ok; ++t) {
+                    const float acc = static_cast<float>(t) * inv_s;
+                    const volatile float want = acc / P.n_workers_f;
+                    const volatile float q0 = acc * P.inv_n;
+                    const float rem = std::fmaf(-q0, P.n_workers_f, acc);
+                    nr_ok = same_bits(std::fmaf(rem, P.inv_n, q0), want);
+                }
+                P.div_mode = nr_ok ? 1 : 2;
+            }
+        }
+    }
     ReduceFn fn = pick_reduce(cfg, mode);
-    static int occ_cache[2][3][3] = {};
+    static int occ_cache[2][3][2] = {};
     int &occ = occ_cache[cfg->out_dtype == LOCO_BF16][cfg->bits == 2 ? 0 : (cfg->bits == 4 ? 1 : 2)][mode];
     if (occ == 0) {
         int v = 0;

@@ -1,14 +1,25 @@
 // LoCo send / receive kernels for sm_100a.
 //
-// Both passes are elementwise streams over HBM (no contraction, no tensor cores).
-// Work unit: a "row" of 256 consecutive elements handled by one warp, 8 consecutive
-// elements per lane, so that the widest stream (the gradient) moves as one 128-bit
-// access per lane and every warp-wide access covers one contiguous span of memory.
-// A warp takes ROWS rows per trip and issues all their loads before the arithmetic.
+// Both passes are elementwise streams over HBM (no contraction, no tensor cores).  At HBM speed the
+// send pass has about 25 issue slots per element, and the logic / min-max / convert instructions
+// share one pipe that accepts a warp instruction only every second clock, so the instruction mix is
+// part of the design:
+//   * integers enter and leave fp32 through the mantissa of a "magic" float (1.5 * 2^23 + k) instead of
+//     through I2F / F2I, except for the 8-bit error codes, which use the one F2I per element that the
+//     slow conversion pipe can absorb followed by a saturating two-at-a-time byte pack;
+//   * the division of Eq. 1's decompressor is replaced by one fused multiply-add, or by a three-step
+//     Newton-Raphson sequence, only after the host has checked that the replacement reproduces the IEEE
+//     division bit for bit on every code it can meet; otherwise the division is kept;
+//   * codes are packed by a Horner chain of integer multiply-adds (they run on the fp32 pipe);
+//   * non-finite inputs are detected with one fused multiply-add per element (h * 0 accumulates NaN)
+//     and the rare rows that contain one are redone by a plain, careful routine.
+// Work unit: a "row" of 256 consecutive elements handled by one warp, 8 consecutive elements per
+// lane, so that every warp-wide access covers one contiguous span.  A warp loads several rows before
+// it starts computing, which keeps enough bytes in flight to cover the HBM latency.
 //
-// Rounding discipline: every floating-point step of Algorithm 1 is one IEEE fp32
-// operation rounded to nearest even, written with the __f*_rn intrinsics so that the
-// compiler can never contract a multiply and an add into an FMA.
+// Rounding discipline: every floating-point step of Algorithm 1 is one IEEE fp32 operation rounded to
+// nearest even, written with intrinsics, so that nothing is contracted into an FMA by the compiler; an
+// FMA is used only where it is proven (on the host, exhaustively) to give the same bits.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -17,18 +28,21 @@ namespace loco {
 
 enum : int { GRAD_F32 = 0, GRAD_BF16 = 1 };
 enum : int { ST_INT8 = 0, ST_FP32 = 1, ST_NONE = 2, ST_Q8COMP = 3 };
-// MODE_FIXED_RCP: global scales whose reciprocals reproduce Eq. 1's division bit for bit
-// on every possible code (checked on the host); MODE_FIXED_DIV: IEEE division;
-// MODE_BLOCK: per-block absmax scales.
-enum : int { MODE_FIXED_RCP = 0, MODE_FIXED_DIV = 1, MODE_BLOCK = 2 };
+enum : int { MODE_FIXED = 0, MODE_BLOCK = 1 };
+// How dec(code; scale) = code / scale is evaluated on the fast path.
+enum : int { DEC_FMA = 0,      // one fused multiply-add on the magic-biased code
+             DEC_NEWTON = 1,   // q0 = c * r; rem = fma(-q0, scale, c); q0 + rem * r
+             DEC_DIVIDE = 2 }; // neither was proven: every row takes the careful routine (IEEE division)
 
 constexpr int kRow = 256;          // elements per warp row
 constexpr int kLaneElems = 8;      // elements per lane per row
 constexpr int kThreads = 256;      // threads per CTA
 constexpr int kWarps = kThreads / 32;
-constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it rounds to an integer, ties to even
+constexpr float kMagic = 12582912.0f;       // 1.5 * 2^23: adding it rounds to an integer, ties to even
+constexpr unsigned kMagicBits = 0x4B400000u;
 constexpr float kFltMax = 3.402823466e+38f;
 constexpr unsigned kFlagNonFinite = 1u;
+constexpr unsigned kFull = 0xffffffffu;
 
 struct SendParams {
     const void *grad;
@@ -39,7 +53,12 @@ struct SendParams {
     unsigned long long stride;       // bytes per partition
     unsigned long long code_bytes;   // bytes of the code area of a partition
     unsigned long long state_scale_off;   // byte offset of the state scales (BLOCK + INT8)
-    float s, inv_s, s_e, inv_se, beta, omb;
+    float s, s_e, beta, omb;
+    float inv_s, inv_se;             // fl(1/s), fl(1/s_e) for the Newton-Raphson form
+    float dq_a, dq_b;                // DEC_FMA: dec(q; s)   = fma(kMagic + 2^(p-1) + q, dq_a, dq_b)
+    float de_a, de_b;                // DEC_FMA: dec(e; s_e) = fma(kMagic + 128 + e,     de_a, de_b)
+    int dq_mode, de_mode;            // DEC_* chosen by the host for s and for s_e
+    int fast;                        // 0: every row takes the careful routine
     int block_log2;                  // log2(B), BLOCK mode
     int reset;                       // k % T_c == 0
     int collect_stats;
@@ -53,8 +72,12 @@ struct ReduceParams {
     unsigned long long first;        // first partition
     int num_workers;
     int block_log2;
-    float s, inv_s, n_workers_f, inv_n;
-    int inv_n_exact;                 // multiplying by inv_n equals dividing by N for all sums
+    float s;
+    float n_workers_f, inv_n;
+    int int_path;                    // codes may be summed as integers (power-of-two s, N <= 16)
+    float ra, rb;                    // int path: sum/s (and /N when exact) = fma(kMagic + S, ra, rb)
+    int div_mode;                    // division by N: 0 folded into ra/rb or a multiply, 1 Newton-Raphson, 2 IEEE
+    float gen_mul;                   // generic FIXED path: multiplier that reproduces q/s, 0 if division is needed
 };
 
 // ------------------------------------------------------------------------------------------
@@ -63,6 +86,7 @@ struct ReduceParams {
 template <int BITS> struct QRange {
     static constexpr float lo = -float(1 << (BITS - 1));
     static constexpr float hi = float((1 << (BITS - 1)) - 1);
+    static constexpr float off = float(1 << (BITS - 1));
 };
 
 // Nearest integer (ties to even) of y clamped to [lo, hi]; `bits` receives a word whose low
@@ -77,26 +101,18 @@ __device__ __forceinline__ float round_clamp(float y, float lo, float hi, unsign
 
 __device__ __forceinline__ float warp_group_max(float v, int lanes) {
     // max over aligned groups of `lanes` lanes (power of two, <= 32)
-    for (int o = 1; o < lanes; o <<= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    for (int o = 1; o < lanes; o <<= 1) v = fmaxf(v, __shfl_xor_sync(kFull, v, o));
     return v;
 }
 
-template <int GRAD>
-__device__ __forceinline__ void load_grad8(const void *grad, unsigned long long i, float (&g)[8]) {
-    if (GRAD == GRAD_BF16) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(static_cast<const uint16_t *>(grad) + i));
-        const unsigned w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            g[2 * j] = __uint_as_float(w[j] << 16);
-            g[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
-        }
-    } else {
-        const float4 a = __ldg(reinterpret_cast<const float4 *>(static_cast<const float *>(grad) + i));
-        const float4 b = __ldg(reinterpret_cast<const float4 *>(static_cast<const float *>(grad) + i) + 1);
-        g[0] = a.x; g[1] = a.y; g[2] = a.z; g[3] = a.w;
-        g[4] = b.x; g[5] = b.y; g[6] = b.z; g[7] = b.w;
-    }
+// code / scale on the fast path, from the magic-biased float m = kMagic + bias + code.
+__device__ __forceinline__ float dec_fast(float m, float bias_magic, int mode, float a, float b, float scale,
+                                          float inv) {
+    if (mode == DEC_FMA) return __fmaf_rn(m, a, b);
+    const float c = __fadd_rn(m, -bias_magic);          // the code itself, exact
+    const float q0 = __fmul_rn(c, inv);
+    const float rem = __fmaf_rn(-q0, scale, c);
+    return __fmaf_rn(rem, inv, q0);
 }
 
 template <int GRAD>
@@ -110,12 +126,33 @@ __device__ __forceinline__ float byte_to_float(unsigned w, int b) {
     return __int2float_rn(static_cast<int>(static_cast<signed char>((w >> (8 * b)) & 0xffu)));
 }
 
+// d = sat8(a) | sat8(b) << 8 | c << 16 (signed saturation of two 32-bit integers to bytes)
+__device__ __forceinline__ unsigned pack_sat_s8(int a, int b, unsigned c) {
+    unsigned d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(b), "r"(a), "r"(c));
+    return d;
+}
+
+__device__ __forceinline__ unsigned pack4_bytes(unsigned a, unsigned b, unsigned c, unsigned d) {
+    // low bytes of a, b, c, d -> one word, a lowest
+    return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
+}
+
+// Streaming accesses: every byte of both passes is touched exactly once.
+__device__ __forceinline__ uint4 ld_stream16(const void *p) { return __ldcs(static_cast<const uint4 *>(p)); }
+__device__ __forceinline__ uint2 ld_stream8(const void *p) { return __ldcs(static_cast<const uint2 *>(p)); }
+__device__ __forceinline__ unsigned ld_stream4(const void *p) { return __ldcs(static_cast<const unsigned *>(p)); }
+__device__ __forceinline__ void st_stream16(void *p, uint4 v) { __stcs(static_cast<uint4 *>(p), v); }
+__device__ __forceinline__ void st_stream8(void *p, uint2 v) { __stcs(static_cast<uint2 *>(p), v); }
+__device__ __forceinline__ void st_stream4(void *p, unsigned v) { __stcs(static_cast<unsigned *>(p), v); }
+
 // ------------------------------------------------------------------------------------------
-// send: Algorithm 1 steps 1-2 on 8 elements held by one lane.
+// send, careful routine: Algorithm 1 steps 1-2 on 8 elements held by one lane, every operation written
+// out as the paper states it (IEEE division for the decompressor), any value accepted.
 //
 //  g      gradient values (already fp32)
 //  prev   e~_k as Eq. 5 sees it;  c  what is added to g (dec(e_k), e~_k, or dec(comp(e~_k)))
-//  valid  number of leading elements that exist (8 on the fast path)
+//  valid  number of leading elements that exist
 //  Outputs: code bits (low byte of each word = code), e_new = e~_{k+1}, scale of the block.
 template <int STATE, int BITS, int MODE>
 __device__ __forceinline__ void send_core(const SendParams &P, const float (&g)[8], const float (&c)[8],
@@ -148,8 +185,7 @@ __device__ __forceinline__ void send_core(const SendParams &P, const float (&g)[
         if (!fin[j]) y = hq;                                // +-Inf saturates whatever the scale
         const float r = round_clamp(y, lo, hi, code[j]);    // round_p-bit
         float d;                                            // step 2: dec(q; s)
-        if (MODE == MODE_FIXED_RCP) d = __fmul_rn(r, P.inv_s);
-        else if (MODE == MODE_FIXED_DIV) d = __fdiv_rn(r, P.s);
+        if (MODE == MODE_FIXED) d = __fdiv_rn(r, P.s);
         else d = __fmul_rn(r, scale);
         const float delta = fin[j] ? __fsub_rn(h[j], d) : 0.0f;
         e_new[j] = __fadd_rn(__fmul_rn(P.omb, prev[j]), __fmul_rn(P.beta, delta));   // Eq. 5
@@ -161,7 +197,7 @@ __device__ __forceinline__ void send_core(const SendParams &P, const float (&g)[
     }
 }
 
-// Eq. 7 for 8 elements in the int8 format: codes of e~_{k+1} (or zeros at a reset).
+// Eq. 7 for 8 elements in the int8 format: codes of e~_{k+1}.
 template <int MODE>
 __device__ __forceinline__ void state_compress8(const SendParams &P, const float (&e_new)[8], int lanes_per_block,
                                                 unsigned (&ebits)[8], float &escale) {
@@ -181,11 +217,6 @@ __device__ __forceinline__ void state_compress8(const SendParams &P, const float
     }
 }
 
-__device__ __forceinline__ unsigned pack4_bytes(unsigned a, unsigned b, unsigned c, unsigned d) {
-    // low bytes of a, b, c, d -> one word, a lowest
-    return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
-}
-
 // Compensation value and Eq. 5's previous error for 8 elements, from the stored state.
 template <int STATE, int MODE>
 __device__ __forceinline__ void decode_state8(const SendParams &P, uint2 e8, const float (&ef)[8], float sscale,
@@ -194,8 +225,7 @@ __device__ __forceinline__ void decode_state8(const SendParams &P, uint2 e8, con
     for (int j = 0; j < 8; ++j) {
         if (STATE == ST_INT8) {
             const float ei = byte_to_float(j < 4 ? e8.x : e8.y, j & 3);
-            if (MODE == MODE_FIXED_RCP) c[j] = __fmul_rn(ei, P.inv_se);       // dec(e_k; s_e), Eq. 2
-            else if (MODE == MODE_FIXED_DIV) c[j] = __fdiv_rn(ei, P.s_e);
+            if (MODE == MODE_FIXED) c[j] = __fdiv_rn(ei, P.s_e);              // dec(e_k; s_e), Eq. 2
             else c[j] = __fmul_rn(ei, sscale);
             prev[j] = c[j];
         } else if (STATE == ST_FP32) {
@@ -205,7 +235,7 @@ __device__ __forceinline__ void decode_state8(const SendParams &P, uint2 e8, con
             prev[j] = ef[j];
             unsigned bits;
             const float r = round_clamp(__fmul_rn(ef[j], P.s_e), -128.0f, 127.0f, bits);
-            c[j] = (MODE == MODE_FIXED_RCP) ? __fmul_rn(r, P.inv_se) : __fdiv_rn(r, P.s_e);
+            c[j] = __fdiv_rn(r, P.s_e);
         } else {
             c[j] = 0.0f;
             prev[j] = 0.0f;
@@ -233,53 +263,42 @@ __device__ __forceinline__ void store_codes8(uint8_t *dst, const unsigned (&code
     }
 }
 
-// One warp row (256 elements starting at partition-local offset `o`, bucket element i0 = part*lp + o).
-// FULL: all 256 elements exist; otherwise elements >= n are treated as absent (code 0, no state).
-template <int GRAD, int STATE, int BITS, int MODE, bool FULL>
-__device__ __forceinline__ void send_row(const SendParams &P, unsigned long long part, unsigned long long o,
-                                         int lane, unsigned &nonfinite, unsigned &saturated) {
+// One warp row (256 elements starting at partition-local offset `o`, bucket element i0 = part*lp + o),
+// careful routine.  Elements >= n are treated as absent (code 0, no state).  Reads its inputs itself.
+// Out of line and with its own copy of the parameters, so that the fast routine's register allocation and
+// constant-bank accesses are not disturbed by this rarely taken path.  Returns the number of saturated
+// codes of this lane, plus 2^31 if the lane met a non-finite value.
+template <int GRAD, int STATE, int BITS, int MODE>
+__device__ __noinline__ unsigned send_row_careful(const SendParams P, unsigned long long part, unsigned long long o,
+                                                  int lane) {
+    unsigned nonfinite = 0u, saturated = 0u;
     const unsigned long long i0 = part * P.lp + o + static_cast<unsigned long long>(lane) * kLaneElems;
-    int valid = 8;
-    if (!FULL) {
-        valid = i0 >= P.n ? 0 : (P.n - i0 >= 8 ? 8 : static_cast<int>(P.n - i0));
-    }
+    const int valid = i0 >= P.n ? 0 : (P.n - i0 >= 8 ? 8 : static_cast<int>(P.n - i0));
     const int lanes_per_block = (MODE == MODE_BLOCK) ? (P.block_log2 >= 8 ? 32 : (1 << (P.block_log2 - 3))) : 1;
     const unsigned long long blk = (MODE == MODE_BLOCK) ? (i0 >> P.block_log2) : 0;
 
     float g[8], ef[8], c[8], prev[8];
-    uint2 e8 = make_uint2(0u, 0u);
     float sscale = 0.0f;
     int8_t *st8 = static_cast<int8_t *>(P.state);
     float *stf = static_cast<float *>(P.state);
     float *st_scales = reinterpret_cast<float *>(static_cast<uint8_t *>(P.state) + P.state_scale_off);
 
-    if (FULL) {
-        load_grad8<GRAD>(P.grad, i0, g);
-        if (STATE == ST_INT8) e8 = *reinterpret_cast<const uint2 *>(st8 + i0);
-        if (STATE == ST_FP32 || STATE == ST_Q8COMP) {
-            const float4 a = *reinterpret_cast<const float4 *>(stf + i0);
-            const float4 b = *(reinterpret_cast<const float4 *>(stf + i0) + 1);
-            ef[0] = a.x; ef[1] = a.y; ef[2] = a.z; ef[3] = a.w;
-            ef[4] = b.x; ef[5] = b.y; ef[6] = b.z; ef[7] = b.w;
-        }
-    } else {
-        unsigned lo_w = 0, hi_w = 0;
+    unsigned lo_w = 0, hi_w = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            g[j] = 0.0f;
-            ef[j] = 0.0f;
-            if (j < valid) {
-                g[j] = load_grad1<GRAD>(P.grad, i0 + j);
-                if (STATE == ST_INT8) {
-                    const unsigned b = static_cast<uint8_t>(st8[i0 + j]);
-                    if (j < 4) lo_w |= b << (8 * j); else hi_w |= b << (8 * (j - 4));
-                }
-                if (STATE == ST_FP32 || STATE == ST_Q8COMP) ef[j] = stf[i0 + j];
+    for (int j = 0; j < 8; ++j) {
+        g[j] = 0.0f;
+        ef[j] = 0.0f;
+        if (j < valid) {
+            g[j] = load_grad1<GRAD>(P.grad, i0 + j);
+            if (STATE == ST_INT8) {
+                const unsigned b = static_cast<uint8_t>(st8[i0 + j]);
+                if (j < 4) lo_w |= b << (8 * j); else hi_w |= b << (8 * (j - 4));
             }
+            if (STATE == ST_FP32 || STATE == ST_Q8COMP) ef[j] = stf[i0 + j];
         }
-        e8 = make_uint2(lo_w, hi_w);
     }
-    if (STATE == ST_INT8 && MODE == MODE_BLOCK) sscale = (FULL || valid > 0) ? st_scales[blk] : 0.0f;
+    const uint2 e8 = make_uint2(lo_w, hi_w);
+    if (STATE == ST_INT8 && MODE == MODE_BLOCK) sscale = valid > 0 ? st_scales[blk] : 0.0f;
 
     decode_state8<STATE, MODE>(P, e8, ef, sscale, c, prev);
 
@@ -297,7 +316,6 @@ __device__ __forceinline__ void send_row(const SendParams &P, unsigned long long
     }
 
     // Eq. 7: reset, or keep / compress the new error
-    if (STATE == ST_NONE) return;
     if (STATE == ST_INT8) {
         unsigned ebits[8];
         float escale = 0.0f;
@@ -307,83 +325,348 @@ __device__ __forceinline__ void send_row(const SendParams &P, unsigned long long
         } else {
             state_compress8<MODE>(P, e_new, lanes_per_block, ebits, escale);
         }
-        if (FULL) {
-            uint2 v;
-            v.x = pack4_bytes(ebits[0], ebits[1], ebits[2], ebits[3]);
-            v.y = pack4_bytes(ebits[4], ebits[5], ebits[6], ebits[7]);
-            *reinterpret_cast<uint2 *>(st8 + i0) = v;
-        } else {
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (j < valid) st8[i0 + j] = static_cast<int8_t>(ebits[j] & 0xffu);
-        }
+        for (int j = 0; j < 8; ++j)
+            if (j < valid) st8[i0 + j] = static_cast<int8_t>(ebits[j] & 0xffu);
         if (MODE == MODE_BLOCK) {
-            if ((lane & (lanes_per_block - 1)) == 0 && (i0 & ((1ull << P.block_log2) - 1)) == 0 && (FULL || valid > 0))
+            if ((lane & (lanes_per_block - 1)) == 0 && (i0 & ((1ull << P.block_log2) - 1)) == 0 && valid > 0)
                 st_scales[blk] = escale;
         }
+    } else if (STATE == ST_FP32 || STATE == ST_Q8COMP) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (j < valid) stf[i0 + j] = P.reset ? 0.0f : e_new[j];
+    }
+    return saturated | (nonfinite << 31);
+}
+
+// ------------------------------------------------------------------------------------------
+// send, fast routine: one full row whose inputs are already in registers.
+
+template <int GRAD, int STATE>
+struct RowIn {
+    static constexpr int GW = (GRAD == GRAD_BF16) ? 4 : 8;                       // gradient words per lane
+    static constexpr int SW = (STATE == ST_INT8) ? 2 : (STATE == ST_NONE ? 1 : 8);   // state words per lane
+    unsigned g[GW];
+    unsigned e[SW];
+    float sscale;                                                                // BLOCK + INT8
+};
+
+// Per-lane base pointers of one partition: everything a row needs is base + row * (bytes per row).
+struct LanePtrs {
+    const uint8_t *grad;      // this lane's 8 gradient elements of row 0
+    uint8_t *state;           // this lane's 8 state elements of row 0 (int8 or fp32)
+    uint8_t *codes;           // this lane's code bytes of row 0 in the partition's code area
+    float *wire_scales;       // BLOCK: the partition's scale area
+    float *state_scales;      // BLOCK + INT8: scale of the bucket's block 0
+    unsigned long long elem0; // bucket index of this lane's first element of row 0
+    unsigned lane_elem;       // partition-local index of this lane's first element of row 0
+};
+
+template <int GRAD, int STATE, int MODE>
+__device__ __forceinline__ void load_row(const LanePtrs &L, unsigned row, int block_log2, RowIn<GRAD, STATE> &in) {
+    constexpr unsigned gbytes = (GRAD == GRAD_BF16 ? 2u : 4u) * kRow;
+    const uint8_t *gp = L.grad + static_cast<size_t>(row) * gbytes;
+    if (GRAD == GRAD_BF16) {
+        const uint4 v = ld_stream16(gp);
+        in.g[0] = v.x; in.g[1] = v.y; in.g[2] = v.z; in.g[3] = v.w;
     } else {
-        if (P.reset) {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) e_new[j] = 0.0f;
-        }
-        if (FULL) {
-            *reinterpret_cast<float4 *>(stf + i0) = make_float4(e_new[0], e_new[1], e_new[2], e_new[3]);
-            *(reinterpret_cast<float4 *>(stf + i0) + 1) = make_float4(e_new[4], e_new[5], e_new[6], e_new[7]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (j < valid) stf[i0 + j] = e_new[j];
-        }
+        const uint4 a = ld_stream16(gp);
+        const uint4 b = ld_stream16(gp + 16);
+        in.g[0] = a.x; in.g[1] = a.y; in.g[2] = a.z; in.g[3] = a.w;
+        in.g[RowIn<GRAD, STATE>::GW - 4] = b.x; in.g[RowIn<GRAD, STATE>::GW - 3] = b.y;
+        in.g[RowIn<GRAD, STATE>::GW - 2] = b.z; in.g[RowIn<GRAD, STATE>::GW - 1] = b.w;
+    }
+    in.sscale = 0.0f;
+    if (STATE == ST_INT8) {
+        const uint2 v = ld_stream8(L.state + static_cast<size_t>(row) * kRow);
+        in.e[0] = v.x; in.e[1] = v.y;
+        if (MODE == MODE_BLOCK)
+            in.sscale = L.state_scales[(L.elem0 + static_cast<unsigned long long>(row) * kRow) >> block_log2];
+    } else if (STATE == ST_FP32 || STATE == ST_Q8COMP) {
+        const uint8_t *sp = L.state + static_cast<size_t>(row) * (4u * kRow);
+        const uint4 a = ld_stream16(sp);
+        const uint4 b = ld_stream16(sp + 16);
+        in.e[0] = a.x; in.e[1] = a.y; in.e[2] = a.z; in.e[3] = a.w;
+        in.e[RowIn<GRAD, STATE>::SW - 4] = b.x; in.e[RowIn<GRAD, STATE>::SW - 3] = b.y;
+        in.e[RowIn<GRAD, STATE>::SW - 2] = b.z; in.e[RowIn<GRAD, STATE>::SW - 1] = b.w;
+    } else {
+        in.e[0] = 0u;
     }
 }
 
+// Packs the 8 codes held in the low bits of the magic-biased floats mb[j] = bits(kMagic + 2^(p-1) + q_j):
+// sum_j mb[j] * R^j = kMagicBits * sum_j R^j + sum_j (q_j + 2^(p-1)) R^j  (mod 2^32), R = 2^p; removing the
+// constant and flipping each field's top bit turns the biased fields into two's complement.
+template <int BITS>
+__device__ __forceinline__ void store_codes_fast(uint8_t *dst, const unsigned (&mb)[8]) {
+    if (BITS == 4) {
+        unsigned acc = mb[7];
+#pragma unroll
+        for (int j = 6; j >= 0; --j) acc = acc * 16u + mb[j];
+        st_stream4(dst, (acc - kMagicBits * 0x11111111u) ^ 0x88888888u);
+    } else if (BITS == 8) {
+        unsigned a0 = mb[3], a1 = mb[7];
+#pragma unroll
+        for (int j = 2; j >= 0; --j) { a0 = a0 * 256u + mb[j]; a1 = a1 * 256u + mb[4 + j]; }
+        st_stream8(dst, make_uint2((a0 - kMagicBits * 0x01010101u) ^ 0x80808080u,
+                                   (a1 - kMagicBits * 0x01010101u) ^ 0x80808080u));
+    } else {
+        unsigned acc = mb[7];
+#pragma unroll
+        for (int j = 6; j >= 0; --j) acc = acc * 4u + mb[j];
+        *reinterpret_cast<uint16_t *>(dst) = static_cast<uint16_t>(((acc - kMagicBits * 0x5555u) ^ 0xAAAAu) & 0xffffu);
+    }
+}
+
+// The scalars of Algorithm 1 the fast routine needs, read from the parameters once per kernel.
+struct SendConsts {
+    float s, s_e, beta, omb, inv_s, inv_se, dq_a, dq_b, de_a, de_b;
+    int dq_mode, de_mode, block_log2, reset;
+};
+
+// Returns false (and stores nothing) if some lane of the warp met a non-finite compensated gradient:
+// the caller then redoes the row with the careful routine.
+// LEAN: both decompressors are the single fused multiply-add and no statistics are collected, so the
+// routine has no data-dependent branch at all.
+template <int GRAD, int STATE, int BITS, int MODE, bool LEAN>
+__device__ __forceinline__ bool send_row_fast(const SendConsts &K, const LanePtrs &L, const RowIn<GRAD, STATE> &in,
+                                              unsigned row, int lane, bool stats, unsigned &saturated) {
+    constexpr float lo = QRange<BITS>::lo, hi = QRange<BITS>::hi, qmagic = kMagic + QRange<BITS>::off;
+    constexpr float emagic = kMagic + 128.0f;
+    const int dq_mode = LEAN ? DEC_FMA : K.dq_mode, de_mode = LEAN ? DEC_FMA : K.de_mode;
+    const int lanes_per_block = (MODE == MODE_BLOCK) ? (K.block_log2 >= 8 ? 32 : (1 << (K.block_log2 - 3))) : 1;
+
+    float g[8], c[8], prev[8], h[8];
+    if (GRAD == GRAD_BF16) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            g[2 * j] = __uint_as_float(in.g[j] << 16);
+            g[2 * j + 1] = __uint_as_float(in.g[j] & 0xffff0000u);
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) g[j] = __uint_as_float(in.g[j]);
+    }
+
+    // step 1, Eq. 2: c = what is added to g, prev = e~_k of Eq. 5
+    if (STATE == ST_INT8) {
+        const unsigned x0 = in.e[0] ^ 0x80808080u, x1 = in.e[1] ^ 0x80808080u;    // bytes e + 128
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float m = __uint_as_float(__byte_perm(j < 4 ? x0 : x1, kMagicBits, 0x7650 + (j & 3)));   // kMagic + 128 + e
+            if (MODE == MODE_FIXED) c[j] = dec_fast(m, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se);
+            else c[j] = __fmul_rn(__fadd_rn(m, -emagic), in.sscale);
+            prev[j] = c[j];
+        }
+    } else if (STATE == ST_FP32) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = __uint_as_float(in.e[j]); prev[j] = c[j]; }
+    } else if (STATE == ST_Q8COMP) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            prev[j] = __uint_as_float(in.e[j]);
+            const float t = fminf(fmaxf(__fmul_rn(prev[j], K.s_e), -128.0f), 127.0f);
+            c[j] = dec_fast(__fadd_rn(t, emagic), emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se);
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = 0.0f; prev[j] = 0.0f; }
+    }
+    float nf = 0.0f;                     // stays 0 unless some h is NaN or +-Inf
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        h[j] = __fadd_rn(g[j], c[j]);
+        nf = __fmaf_rn(h[j], 0.0f, nf);
+    }
+    if (__any_sync(kFull, !(nf == 0.0f))) return false;
+
+    // Eq. 1 / Eq. 3: q = round_p-bit(h x s);  step 2: d, Eq. 5
+    float mult = K.s, scale = 0.0f;
+    if (MODE == MODE_BLOCK) {
+        float amax = fmaxf(fabsf(h[0]), fabsf(h[1]));
+#pragma unroll
+        for (int j = 2; j < 8; ++j) amax = fmaxf(amax, fabsf(h[j]));
+        amax = warp_group_max(amax, lanes_per_block);
+        scale = amax > 0.0f ? __fdiv_rn(amax, hi) : 0.0f;
+        mult = amax > 0.0f ? __fdiv_rn(hi, amax) : 0.0f;
+    }
+    unsigned mb[8];
+    float e_new[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const float y = __fmul_rn(h[j], mult);
+        const float m = __fadd_rn(fminf(fmaxf(y, lo), hi), qmagic);      // kMagic + 2^(p-1) + q
+        mb[j] = __float_as_uint(m);
+        float d;
+        if (MODE == MODE_FIXED) d = dec_fast(m, qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s);
+        else d = __fmul_rn(__fadd_rn(m, -qmagic), scale);
+        const float delta = __fsub_rn(h[j], d);
+        e_new[j] = __fadd_rn(__fmul_rn(K.omb, prev[j]), __fmul_rn(K.beta, delta));
+        if (!LEAN && MODE == MODE_FIXED && stats) {
+            if (y >= hi + 0.5f || y < lo - 0.5f) saturated += 1u;
+        }
+    }
+    store_codes_fast<BITS>(L.codes + static_cast<size_t>(row) * (kRow * BITS / 8), mb);
+    if (MODE == MODE_BLOCK) {
+        const unsigned ol = L.lane_elem + row * kRow;       // partition-local element index (rows are < 2^24)
+        if ((lane & (lanes_per_block - 1)) == 0 && ((ol & ((1u << K.block_log2) - 1)) == 0))
+            L.wire_scales[(static_cast<unsigned long long>(row) * kRow + L.lane_elem) >> K.block_log2] = scale;
+    }
+
+    // Eq. 7
+    if (STATE == ST_INT8) {
+        uint2 v = make_uint2(0u, 0u);
+        float escale = 0.0f;
+        if (!K.reset) {
+            float emult = K.s_e;
+            if (MODE == MODE_BLOCK) {
+                float amax = fmaxf(fabsf(e_new[0]), fabsf(e_new[1]));
+#pragma unroll
+                for (int j = 2; j < 8; ++j) amax = fmaxf(amax, fabsf(e_new[j]));
+                amax = warp_group_max(amax, lanes_per_block);
+                escale = amax > 0.0f ? __fdiv_rn(amax, 127.0f) : 0.0f;
+                emult = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+            }
+            int q[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) q[j] = __float2int_rn(__fmul_rn(e_new[j], emult));   // saturates, NaN -> 0
+            v.x = pack_sat_s8(q[0], q[1], pack_sat_s8(q[2], q[3], 0u));
+            v.y = pack_sat_s8(q[4], q[5], pack_sat_s8(q[6], q[7], 0u));
+        }
+        st_stream8(L.state + static_cast<size_t>(row) * kRow, v);
+        if (MODE == MODE_BLOCK) {
+            const unsigned long long i0 = L.elem0 + static_cast<unsigned long long>(row) * kRow;
+            if ((lane & (lanes_per_block - 1)) == 0 && (i0 & ((1ull << K.block_log2) - 1)) == 0)
+                L.state_scales[i0 >> K.block_log2] = escale;
+        }
+    } else if (STATE == ST_FP32 || STATE == ST_Q8COMP) {
+        if (K.reset) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) e_new[j] = 0.0f;
+        }
+        uint8_t *dst = L.state + static_cast<size_t>(row) * (4u * kRow);
+        st_stream16(dst, make_uint4(__float_as_uint(e_new[0]), __float_as_uint(e_new[1]), __float_as_uint(e_new[2]), __float_as_uint(e_new[3])));
+        st_stream16(dst + 16, make_uint4(__float_as_uint(e_new[4]), __float_as_uint(e_new[5]), __float_as_uint(e_new[6]), __float_as_uint(e_new[7])));
+    }
+    return true;
+}
+
 // grid = (ctas per partition, partitions).  Each warp walks the partition's rows with the
-// stride of all warps working on that partition.
-template <int GRAD, int STATE, int BITS, int MODE>
-__global__ void __launch_bounds__(kThreads) loco_send_kernel(const SendParams P) {
+// stride of all warps working on that partition, kUnroll rows per trip.
+// LEAN kernels are launched when the host proved both single-FMA decompressors and no statistics are
+// wanted (and for every block-scaled configuration); the others choose per element at run time.
+template <int GRAD, int STATE, int BITS, int MODE, bool LEAN>
+__global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams P) {
+    // bytes a lane loads per row decide how many rows a trip can afford in registers
+    constexpr int kLoadWords = RowIn<GRAD, STATE>::GW + (STATE == ST_NONE ? 0 : RowIn<GRAD, STATE>::SW);
+    constexpr int kUnroll = kLoadWords <= 6 ? 4 : 2;
     const int lane = threadIdx.x & 31;
     const unsigned long long part = blockIdx.y;
-    const unsigned long long warp = static_cast<unsigned long long>(blockIdx.x) * kWarps + (threadIdx.x >> 5);
-    const unsigned long long nwarps = static_cast<unsigned long long>(gridDim.x) * kWarps;
-    const unsigned long long rows = P.lp / kRow;
+    const unsigned warp = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    const unsigned nwarps = gridDim.x * kWarps;
+    const unsigned rows = static_cast<unsigned>(P.lp / kRow);
     const unsigned long long base = part * P.lp;
     // rows [0, full_rows) of this partition lie entirely below n
-    unsigned long long full_rows = 0;
+    unsigned full_rows = 0;
     if (P.n > base) {
         const unsigned long long avail = P.n - base;
-        full_rows = avail >= P.lp ? rows : avail / kRow;
+        full_rows = avail >= P.lp ? rows : static_cast<unsigned>(avail / kRow);
     }
-    unsigned nonfinite = 0u, saturated = 0u;
-    for (unsigned long long r = warp; r < rows; r += nwarps) {
-        if (r < full_rows) send_row<GRAD, STATE, BITS, MODE, true>(P, part, r * kRow, lane, nonfinite, saturated);
-        else send_row<GRAD, STATE, BITS, MODE, false>(P, part, r * kRow, lane, nonfinite, saturated);
+    unsigned saturated = 0u;
+    unsigned long long careful_acc = 0ull;
+    unsigned r = warp;
+    if (P.fast) {
+        LanePtrs L;
+        L.lane_elem = static_cast<unsigned>(lane) * kLaneElems;
+        L.elem0 = base + L.lane_elem;
+        L.grad = static_cast<const uint8_t *>(P.grad) + L.elem0 * (GRAD == GRAD_BF16 ? 2u : 4u);
+        L.state = static_cast<uint8_t *>(P.state) + L.elem0 * (STATE == ST_INT8 ? 1u : 4u);
+        uint8_t *pbase = P.comm + part * P.stride;
+        L.codes = pbase + static_cast<size_t>(L.lane_elem) * BITS / 8;
+        L.wire_scales = reinterpret_cast<float *>(pbase + P.code_bytes);
+        L.state_scales = reinterpret_cast<float *>(static_cast<uint8_t *>(P.state) + P.state_scale_off);
+        SendConsts K;
+        K.s = P.s; K.s_e = P.s_e; K.beta = P.beta; K.omb = P.omb; K.inv_s = P.inv_s; K.inv_se = P.inv_se;
+        K.dq_a = P.dq_a; K.dq_b = P.dq_b; K.de_a = P.de_a; K.de_b = P.de_b;
+        K.dq_mode = P.dq_mode; K.de_mode = P.de_mode; K.block_log2 = P.block_log2; K.reset = P.reset;
+        const bool stats = P.collect_stats != 0;
+        // full_rows <= rows < 2^32 - kUnroll * nwarps for every bucket this library accepts
+        for (; r + (kUnroll - 1) * nwarps < full_rows; r += kUnroll * nwarps) {
+            RowIn<GRAD, STATE> in[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) load_row<GRAD, STATE, MODE>(L, r + u * nwarps, K.block_log2, in[u]);
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                if (!send_row_fast<GRAD, STATE, BITS, MODE, LEAN>(K, L, in[u], r + u * nwarps, lane, stats, saturated))
+                    careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(r + u * nwarps) * kRow, lane);
+            }
+        }
+        for (; r < full_rows; r += nwarps) {
+            RowIn<GRAD, STATE> in;
+            load_row<GRAD, STATE, MODE>(L, r, K.block_log2, in);
+            if (!send_row_fast<GRAD, STATE, BITS, MODE, LEAN>(K, L, in, r, lane, stats, saturated))
+                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(r) * kRow, lane);
+        }
     }
-    if (__any_sync(0xffffffffu, nonfinite != 0u)) {
+    for (; r < rows; r += nwarps)
+        careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(r) * kRow, lane);
+    // each careful call adds at most 8 saturated codes and 2^31 per row with a non-finite value; the 64-bit
+    // sum keeps the flag apart from the count
+    const unsigned nonfinite = (careful_acc >> 31) != 0ull ? 1u : 0u;
+    saturated += static_cast<unsigned>(careful_acc & 0x7fffffffull);
+
+    if (__any_sync(kFull, nonfinite != 0u)) {
         if (lane == 0) atomicOr(P.status, static_cast<unsigned long long>(kFlagNonFinite));
     }
     if (P.collect_stats) {
-        for (int o = 16; o > 0; o >>= 1) saturated += __shfl_xor_sync(0xffffffffu, saturated, o);
+        for (int o = 16; o > 0; o >>= 1) saturated += __shfl_xor_sync(kFull, saturated, o);
         if (lane == 0 && saturated) atomicAdd(P.status + 1, static_cast<unsigned long long>(saturated));
     }
 }
 
 // ------------------------------------------------------------------------------------------
-// receive: Eq. 8 on one warp row of 256 outputs, 8 per lane.
+// receive: Eq. 8 on warp rows of 256 outputs, 8 per lane.
+
+template <int BITS> struct CodeWord { unsigned x, y; };   // the 8 codes of one lane and row, as loaded (y: 8-bit only)
 
 template <int BITS>
-__device__ __forceinline__ void load_codes8(const uint8_t *src, float (&q)[8]) {
+__device__ __forceinline__ void load_codeword(const uint8_t *src, CodeWord<BITS> &w) {
+    w.y = 0u;
+    if (BITS == 8) { const uint2 t = ld_stream8(src); w.x = t.x; w.y = t.y; }
+    else if (BITS == 4) w.x = ld_stream4(src);
+    else w.x = static_cast<unsigned>(__ldcs(reinterpret_cast<const unsigned short *>(src)));
+}
+
+// The 8 codes as exact floats.  Each field, with its top bit flipped (code + 2^(p-1)), is masked in place
+// into the mantissa of a power of two chosen so that the field's lowest bit weighs 1; subtracting that
+// power of two and the bias leaves the code.
+template <int BITS>
+__device__ __forceinline__ void codes_to_float(const CodeWord<BITS> &w, float (&q)[8]) {
     if (BITS == 8) {
-        const uint2 v = __ldg(reinterpret_cast<const uint2 *>(src));
+        const unsigned x0 = w.x ^ 0x80808080u, x1 = w.y ^ 0x80808080u;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) q[j] = byte_to_float(j < 4 ? v.x : v.y, j & 3);
+        for (int j = 0; j < 8; ++j)
+            q[j] = __fadd_rn(__uint_as_float(__byte_perm(j < 4 ? x0 : x1, 0x4B000000u, 0x7650 + (j & 3))), -(8388608.0f + 128.0f));
     } else if (BITS == 4) {
-        const unsigned w = __ldg(reinterpret_cast<const unsigned *>(src));
+        const unsigned x = w.x ^ 0x88888888u;
+        const unsigned xh = x >> 12;                         // fields 5..7 moved to positions 2..4
 #pragma unroll
-        for (int j = 0; j < 8; ++j) q[j] = __int2float_rn(static_cast<int>(w << (28 - 4 * j)) >> 28);
+        for (int j = 0; j < 8; ++j) {
+            const int pos = j < 5 ? j : j - 3;               // field position inside the word used
+            const unsigned src = j < 5 ? x : xh;
+            const unsigned expo = static_cast<unsigned>(127 + 23 - 4 * pos) << 23;        // 2^(23 - 4 pos)
+            const float m = __uint_as_float((src & (0xFu << (4 * pos))) | expo);
+            q[j] = __fadd_rn(m, -(__uint_as_float(expo) + 8.0f));
+        }
     } else {
-        const unsigned w = __ldg(reinterpret_cast<const uint16_t *>(src));
+        const unsigned x = w.x ^ 0xAAAAu;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) q[j] = __int2float_rn(static_cast<int>(w << (30 - 2 * j)) >> 30);
+        for (int j = 0; j < 8; ++j) {
+            const unsigned expo = static_cast<unsigned>(127 + 23 - 2 * j) << 23;
+            const float m = __uint_as_float((x & (0x3u << (2 * j))) | expo);
+            q[j] = __fadd_rn(m, -(__uint_as_float(expo) + 2.0f));
+        }
     }
 }
 
@@ -394,8 +677,74 @@ __device__ __forceinline__ unsigned pack_bf16x2_rn(float a, float b) {
     return r;
 }
 
+template <int OUT>
+__device__ __forceinline__ void store_out8(void *out, unsigned long long oi, const float (&res)[8], unsigned long long left) {
+    if (left >= 8) {
+        if (OUT == GRAD_BF16) {
+            st_stream16(static_cast<uint16_t *>(out) + oi,
+                        make_uint4(pack_bf16x2_rn(res[0], res[1]), pack_bf16x2_rn(res[2], res[3]),
+                                   pack_bf16x2_rn(res[4], res[5]), pack_bf16x2_rn(res[6], res[7])));
+        } else {
+            float *dst = static_cast<float *>(out) + oi;
+            st_stream16(dst, make_uint4(__float_as_uint(res[0]), __float_as_uint(res[1]), __float_as_uint(res[2]), __float_as_uint(res[3])));
+            st_stream16(dst + 4, make_uint4(__float_as_uint(res[4]), __float_as_uint(res[5]), __float_as_uint(res[6]), __float_as_uint(res[7])));
+        }
+    } else {
+        const int cnt = static_cast<int>(left);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (j < cnt) {
+                if (OUT == GRAD_BF16)
+                    static_cast<uint16_t *>(out)[oi + j] = static_cast<uint16_t>(pack_bf16x2_rn(res[j], 0.0f) & 0xffffu);
+                else
+                    static_cast<float *>(out)[oi + j] = res[j];
+            }
+        }
+    }
+}
+
+// acc / N as Eq. 8 writes it
+__device__ __forceinline__ float div_workers(const ReduceParams &P, float acc) {
+    if (P.div_mode == 0) return __fmul_rn(acc, P.inv_n);
+    if (P.div_mode == 1) {
+        const float q0 = __fmul_rn(acc, P.inv_n);
+        const float rem = __fmaf_rn(-q0, P.n_workers_f, acc);
+        return __fmaf_rn(rem, P.inv_n, q0);
+    }
+    return __fdiv_rn(acc, P.n_workers_f);
+}
+
+// Integer path (global power-of-two s, at most 16 workers): every dec(q; s) and every partial sum of Eq. 8
+// is an integer multiple of 1/s that fp32 holds exactly, so the sum over workers does not depend on the
+// order or the format it is taken in.  The codes, biased to be non-negative, are added side by side inside
+// 32-bit words (8-bit lanes for 2- and 4-bit codes, 16-bit lanes for 8-bit codes); the lane sums S reach
+// fp32 through the mantissa of kMagic and one fused multiply-add gives (S - bias N) / s (/ N).
+template <int BITS>
+struct LaneSums {
+    unsigned a, b, c, d;    // BITS 4: a = elements 0,2,4,6; b = 1,3,5,7.   BITS 8: a = 0,2  b = 1,3  c = 4,6  d = 5,7
+    __device__ __forceinline__ void clear() { a = b = c = d = 0u; }
+    __device__ __forceinline__ void add(const CodeWord<BITS> &w) {
+        if (BITS == 4) {
+            a += (w.x ^ 0x88888888u) & 0x0F0F0F0Fu;
+            b += ((w.x >> 4) ^ 0x08080808u) & 0x0F0F0F0Fu;
+        } else {
+            a += (w.x ^ 0x80808080u) & 0x00FF00FFu;
+            b += ((w.x >> 8) ^ 0x00800080u) & 0x00FF00FFu;
+            c += (w.y ^ 0x80808080u) & 0x00FF00FFu;
+            d += ((w.y >> 8) ^ 0x00800080u) & 0x00FF00FFu;
+        }
+    }
+    // kMagic + S_j as a float
+    __device__ __forceinline__ float get(int j) const {
+        if (BITS == 4) return __uint_as_float(__byte_perm((j & 1) ? b : a, kMagicBits, 0x7650 + (j >> 1)));
+        const unsigned src = j < 4 ? ((j & 1) ? b : a) : ((j & 1) ? d : c);
+        return __uint_as_float(__byte_perm(src, kMagicBits, ((j >> 1) & 1) ? 0x7632 : 0x7610));
+    }
+};
+
 template <int OUT, int BITS, int MODE>
 __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParams P) {
+    constexpr int kUnroll = 4;
     const int lane = threadIdx.x & 31;
     const unsigned long long part = blockIdx.y;                       // relative to P.first
     const unsigned long long warp = static_cast<unsigned long long>(blockIdx.x) * kWarps + (threadIdx.x >> 5);
@@ -407,60 +756,72 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
     const unsigned long long rows = (valid + kRow - 1) / kRow;
     const unsigned long long poff = part * P.stride;
     const unsigned long long out0 = part * P.lp;                      // output index of the part's first element
+    const unsigned long long lane_off = static_cast<unsigned long long>(lane) * kLaneElems;
+    const int N = P.num_workers;
+
+    if (MODE == MODE_FIXED && BITS != 2 && P.int_path) {
+        for (unsigned long long r = warp; r < rows; r += kUnroll * nwarps) {
+            LaneSums<BITS> sums[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) sums[u].clear();
+#pragma unroll 4
+            for (int w = 0; w < N; ++w) {
+                const uint8_t *src = P.parts[w] + poff;
+                CodeWord<BITS> cw[kUnroll];
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) {
+                    const unsigned long long o = (r + u * nwarps) * kRow + lane_off;
+                    // rows past the end are clamped to the last row: loaded, never stored
+                    const unsigned long long oc = (r + u * nwarps) < rows ? o : (rows - 1) * kRow + lane_off;
+                    load_codeword<BITS>(src + oc * BITS / 8, cw[u]);
+                }
+#pragma unroll
+                for (int u = 0; u < kUnroll; ++u) sums[u].add(cw[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const unsigned long long o = (r + u * nwarps) * kRow + lane_off;
+                if ((r + u * nwarps) >= rows || o >= valid) continue;
+                float res[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float acc = __fmaf_rn(sums[u].get(j), P.ra, P.rb);
+                    res[j] = P.div_mode == 0 ? acc : div_workers(P, acc);
+                }
+                store_out8<OUT>(P.out, out0 + o, res, valid - o);
+            }
+        }
+        return;
+    }
 
     for (unsigned long long r = warp; r < rows; r += nwarps) {
-        const unsigned long long o = r * kRow + static_cast<unsigned long long>(lane) * kLaneElems;
+        const unsigned long long o = r * kRow + lane_off;
         if (o >= valid) continue;
         float acc[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
 #pragma unroll 4
-        for (int w = 0; w < P.num_workers; ++w) {
+        for (int w = 0; w < N; ++w) {
             const uint8_t *src = P.parts[w] + poff;
-            float q[8];
-            load_codes8<BITS>(src + o * BITS / 8, q);
-            float sc = 0.0f;
+            CodeWord<BITS> cw;
+            load_codeword<BITS>(src + o * BITS / 8, cw);
+            float sc = P.gen_mul;
             if (MODE == MODE_BLOCK)
                 sc = __ldg(reinterpret_cast<const float *>(src + P.code_bytes) + (o >> P.block_log2));
+            float q[8];
+            codes_to_float<BITS>(cw, q);
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 float d;                                               // dec(q; s), Eq. 1
-                if (MODE == MODE_FIXED_RCP) d = __fmul_rn(q[j], P.inv_s);
-                else if (MODE == MODE_FIXED_DIV) d = __fdiv_rn(q[j], P.s);
+                if (MODE == MODE_FIXED && sc == 0.0f) d = __fdiv_rn(q[j], P.s);
                 else d = __fmul_rn(q[j], sc);
                 acc[j] = __fadd_rn(acc[j], d);
             }
         }
         float res[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j)                                    // the 1/N of Eq. 8
-            res[j] = P.inv_n_exact ? __fmul_rn(acc[j], P.inv_n) : __fdiv_rn(acc[j], P.n_workers_f);
-        const unsigned long long oi = out0 + o;
-        if (valid - o >= 8) {
-            if (OUT == GRAD_BF16) {
-                uint4 v;
-                v.x = pack_bf16x2_rn(res[0], res[1]);
-                v.y = pack_bf16x2_rn(res[2], res[3]);
-                v.z = pack_bf16x2_rn(res[4], res[5]);
-                v.w = pack_bf16x2_rn(res[6], res[7]);
-                *reinterpret_cast<uint4 *>(static_cast<uint16_t *>(P.out) + oi) = v;
-            } else {
-                float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(P.out) + oi);
-                dst[0] = make_float4(res[0], res[1], res[2], res[3]);
-                dst[1] = make_float4(res[4], res[5], res[6], res[7]);
-            }
-        } else {
-            const int cnt = static_cast<int>(valid - o);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if (j < cnt) {
-                    if (OUT == GRAD_BF16)
-                        static_cast<uint16_t *>(P.out)[oi + j] = static_cast<uint16_t>(pack_bf16x2_rn(res[j], 0.0f) & 0xffffu);
-                    else
-                        static_cast<float *>(P.out)[oi + j] = res[j];
-                }
-            }
-        }
+        for (int j = 0; j < 8; ++j) res[j] = div_workers(P, acc[j]);   // the 1/N of Eq. 8
+        store_out8<OUT>(P.out, out0 + o, res, valid - o);
     }
 }
 

@@ -55,6 +55,12 @@ class Worker:
         self.state_whole, state_view = guarded(max(self.state_bytes, 16))
         self.gstate = loco.State(gcfg, n, buffer=state_view)
         self.comm_whole, self.gcomm = guarded(max(self.packed_bytes, 16))
+        # a twin with the statistics switched the other way: the kernels take a different branch for it
+        import dataclasses
+        self.tcfg = dataclasses.replace(gcfg, collect_stats=0 if gcfg.collect_stats else 1)
+        self.tstate_whole, tstate_view = guarded(max(self.state_bytes, 16))
+        self.tstate = loco.State(self.tcfg, n, buffer=tstate_view)
+        self.tcomm_whole, self.tcomm = guarded(max(self.packed_bytes, 16))
         self.ostate = orc.new_state(ocfg, n)
         self.ocomm = orc.new_comm(ocfg, n, fill=CANARY)
         self.osat = 0
@@ -64,15 +70,20 @@ class Worker:
         bf16 = self.gcfg.grad_dtype == loco.BF16
         g = to_device(grad_np, bf16)
         loco.loco_compensate_quantize_pack(self.gstate, g, self.gcomm, k)
+        loco.loco_compensate_quantize_pack(self.tstate, g, self.tcomm, k)
         torch.cuda.synchronize()
         flags, sat = orc.send_step(self.ocfg, grad_np, self.ostate, self.ocomm, k)
         self.oflags |= flags
         self.osat += sat
 
     def compare(self, where=""):
+        self._compare(self.gcfg, self.gstate, self.gcomm, self.state_whole, self.comm_whole, where)
+        self._compare(self.tcfg, self.tstate, self.tcomm, self.tstate_whole, self.tcomm_whole, where + " (twin)")
+
+    def _compare(self, gcfg, gstate_obj, gcomm_t, state_whole, comm_whole, where):
         n, ocfg = self.n, self.ocfg
-        gcomm = self.gcomm.cpu().numpy()
-        gstate = self.gstate.buffer.cpu().numpy()
+        gcomm = gcomm_t.cpu().numpy()
+        gstate = gstate_obj.buffer.cpu().numpy()
         for j, ((gc, gs), (oc, os_)) in enumerate(zip(orc.comm_views(ocfg, n, gcomm), orc.comm_views(ocfg, n, self.ocomm))):
             bad = int((gc != oc).sum())
             assert bad == 0, "%s partition %d: %d code bytes differ (first at %d)" % (where, j, bad, int(np.argmax(gc != oc)))
@@ -95,12 +106,14 @@ class Worker:
             assert np.allclose(gv, ov, rtol=RTOL, atol=ATOL, equal_nan=True), "%s: fp32 state out of tolerance" % where
             nbad = int((gv.view(np.uint32) != ov.view(np.uint32)).sum())
             assert nbad == 0, "%s: %d fp32 state words are not bit-identical" % (where, nbad)
-        check_guards(self.state_whole, max(self.state_bytes, 16))
-        check_guards(self.comm_whole, max(self.packed_bytes, 16))
-        flags, sat = loco.loco_last_status(self.gstate)
+        check_guards(state_whole, max(self.state_bytes, 16))
+        check_guards(comm_whole, max(self.packed_bytes, 16))
+        flags, sat = loco.loco_last_status(gstate_obj)
         assert flags == self.oflags, "%s: flags %d vs %d" % (where, flags, self.oflags)
-        if self.gcfg.collect_stats:
+        if gcfg.collect_stats:
             assert sat == self.osat, "%s: saturated %d vs %d" % (where, sat, self.osat)
+        elif not gcfg.collect_stats:
+            assert sat == 0
 
 
 def reduce_both(gcfg, ocfg, n, workers, first=0, count=None):
