@@ -6,10 +6,11 @@ iteration on a Llama-2-7B-shaped gradient -- 6,738,415,616 bf16 elements cut int
 buckets of 25,000,000 (last one partial):
     phase A  for every bucket: send pass (Algorithm 1 steps 1-2: compensate, 4-bit codes,
              moving-average error into the 8-bit state, pack into the 8-part buffer);
-    phase B  for every bucket: receive pass (Eq. 8) over this rank's part, from its own
-             buffer and the buffers of the 7 other workers (resident in the same HBM).
+    phase B  for every bucket: receive pass (Eq. 8) over all 8 parts of the bucket, averaging this
+             worker's packed buffer with the buffers of the 7 other simulated workers (resident in
+             the same HBM), into the bf16 gradient handed to the optimizer.
 All inputs are synthetic and resident in HBM before the timed region; every bucket is read
-once per step and the step touches ~35 GB, far more than the 126 MB L2.
+once per step and the step touches ~70 GB, far more than the 126 MB L2.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
@@ -35,7 +36,7 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
-METRIC = "compensate+quantize and dequant-reduce GB/s of gradient per bucket pass (send + own-part reduce)"
+METRIC = "compensate+quantize and dequant-reduce GB/s of gradient per bucket pass (send, then 8-worker reduce)"
 BUCKET = 25_000_000
 WORKERS = 8
 L2_BYTES = 126 * 1024 * 1024
@@ -133,18 +134,19 @@ class RankWorkload:
         cfg = self.cfg
         sb = [loco.loco_state_bytes(cfg, hi - lo) for lo, hi in self.buckets]
         pb = [loco.loco_packed_bytes(cfg, hi - lo) for lo, hi in self.buckets]
-        self.stride = [loco.loco_partition_bytes(cfg, hi - lo) for lo, hi in self.buckets]
-        self.out_elems = [loco.loco_partition_elems(cfg, hi - lo, self.part) for lo, hi in self.buckets]
         self.state_buf = torch.empty(sum(sb), dtype=torch.uint8, device=device)
         self.comm_buf = torch.empty(sum(pb), dtype=torch.uint8, device=device)
-        # parts of the 7 other workers as they would sit after the all-to-all: any byte is two valid codes
+        # packed buffers of the 7 other workers as they would sit after the exchange: any byte is two valid codes
         gen = torch.Generator(device=device)
         gen.manual_seed(1234 + rank)
-        self.recv_buf = torch.randint(0, 256, (sum(self.stride) * (WORKERS - 1),), dtype=torch.uint8, device=device,
-                                      generator=gen)
-        self.out_buf = torch.empty(sum((e + 127) // 128 * 128 for e in self.out_elems), dtype=torch.bfloat16, device=device)
+        self.recv_buf = torch.empty(sum(pb) * (WORKERS - 1), dtype=torch.uint8, device=device)
+        chunk = 1 << 30
+        for off in range(0, self.recv_buf.numel(), chunk):
+            m = min(chunk, self.recv_buf.numel() - off)
+            self.recv_buf[off:off + m] = torch.randint(0, 256, (m,), dtype=torch.uint8, device=device, generator=gen)
+        self.out_buf = torch.empty(self.total, dtype=torch.bfloat16, device=device)
         self.states, self.grads, self.comms, self.packed, self.outs = [], [], [], [], []
-        so = co = ro = oo = 0
+        so = co = ro = 0
         for i, (lo, hi) in enumerate(self.buckets):
             n = hi - lo
             self.states.append(loco.State(cfg, n, buffer=self.state_buf[so:so + sb[i]]))
@@ -154,17 +156,16 @@ class RankWorkload:
             ptrs = []
             for w in range(WORKERS):
                 if w == self.part:
-                    ptrs.append(comm.data_ptr() + self.part * self.stride[i])
+                    ptrs.append(comm.data_ptr())
                 else:
                     ptrs.append(self.recv_buf.data_ptr() + ro)
-                    ro += self.stride[i]
+                    ro += pb[i]
             self.packed.append(ptrs)
-            self.outs.append(self.out_buf[oo:oo + self.out_elems[i]])
+            self.outs.append(self.out_buf[lo:hi])
             so += sb[i]
             co += pb[i]
-            oo += (self.out_elems[i] + 127) // 128 * 128
         self.send_bytes = SEND_BYTES_PER_ELEM * self.total
-        self.recv_bytes = sum(e * (WORKERS * 0.5 + 2) for e in self.out_elems)
+        self.recv_bytes = self.total * (WORKERS * 0.5 + 2)
         self.grad_bytes = 2 * self.total
 
     def send_phase(self, k: int):
@@ -175,30 +176,30 @@ class RankWorkload:
     def reduce_phase(self):
         f = self.loco.loco_unpack_dequant_reduce
         for i, (lo, hi) in enumerate(self.buckets):
-            f(self.cfg, self.packed[i], hi - lo, self.outs[i], first_partition=self.part, partition_count=1)
+            f(self.cfg, self.packed[i], hi - lo, self.outs[i])
 
 
 def run_e2e(wl: RankWorkload, steps: int, warmup: int):
-    """Same step through the host-buffer entry points: every bucket's gradient and the 8 packed parts are
-    copied from pinned host memory, the packed codes and the averaged part are copied back."""
+    """Same step through the host-buffer entry points: every bucket's gradient and the 8 workers' packed
+    buffers are copied from pinned host memory, the packed codes and the averaged gradient are copied back."""
     loco, cfg = wl.loco, wl.cfg
-    ring = 4
+    ring = 3
     nmax = BUCKET
+    pbytes = loco.loco_packed_bytes(cfg, nmax)
     h_grad = [torch.empty(nmax, dtype=torch.bfloat16).pin_memory() for _ in range(ring)]
-    h_comm = [torch.empty(loco.loco_packed_bytes(cfg, nmax), dtype=torch.uint8).pin_memory() for _ in range(ring)]
-    stride = loco.loco_partition_bytes(cfg, nmax)
-    h_parts = [[torch.randint(0, 256, (stride,), dtype=torch.uint8).pin_memory() for _ in range(WORKERS)] for _ in range(ring)]
-    h_out = [torch.empty(loco.loco_partition_capacity(cfg, nmax), dtype=torch.bfloat16).pin_memory() for _ in range(ring)]
+    h_comm = [torch.empty(pbytes, dtype=torch.uint8).pin_memory() for _ in range(ring)]
+    h_parts = [[torch.randint(0, 256, (pbytes,), dtype=torch.uint8).pin_memory() for _ in range(WORKERS)] for _ in range(ring)]
+    h_out = [torch.empty(nmax, dtype=torch.bfloat16).pin_memory() for _ in range(ring)]
     for r in range(ring):
         h_grad[r].copy_(wl.grads[r].cpu())
     dev = wl.grad.device
     w_send = torch.empty(loco.loco_send_host_workspace_bytes(cfg, nmax), dtype=torch.uint8, device=dev)
-    w_red = torch.empty(loco.loco_reduce_host_workspace_bytes(cfg, nmax, WORKERS, 1), dtype=torch.uint8, device=dev)
+    w_red = torch.empty(loco.loco_reduce_host_workspace_bytes(cfg, nmax, WORKERS, cfg.num_partitions), dtype=torch.uint8, device=dev)
     h2d = d2h = 0
     for i, (lo, hi) in enumerate(wl.buckets):
         n = hi - lo
-        h2d += 2 * n + WORKERS * loco.loco_partition_bytes(cfg, n)
-        d2h += loco.loco_packed_bytes(cfg, n) + 2 * wl.out_elems[i]
+        h2d += 2 * n + WORKERS * loco.loco_packed_bytes(cfg, n)
+        d2h += loco.loco_packed_bytes(cfg, n) + 2 * n
 
     def step(k):
         for i, (lo, hi) in enumerate(wl.buckets):
@@ -208,8 +209,7 @@ def run_e2e(wl: RankWorkload, steps: int, warmup: int):
         for i, (lo, hi) in enumerate(wl.buckets):
             n = hi - lo
             r = i % ring
-            loco.loco_unpack_dequant_reduce_host(cfg, h_parts[r], n, h_out[r], w_red, first_partition=wl.part,
-                                                 partition_count=1)
+            loco.loco_unpack_dequant_reduce_host(cfg, h_parts[r], n, h_out[r], w_red)
 
     for k in range(warmup):
         step(1000 + k)
@@ -226,7 +226,7 @@ def run_e2e(wl: RankWorkload, steps: int, warmup: int):
 
 def oracle_sample(threads: int, buckets_per_thread: int):
     """The oracle as it stands on `threads` host threads, each doing whole 25M-element buckets of the
-    workload (send pass, then this rank's part of the receive pass with 8 workers)."""
+    workload (send pass, then the receive pass over the whole bucket with 8 workers)."""
     import numpy as np
     from oracle import loco_oracle as orc
     ocfg = orc.OracleConfig(**CFG)
@@ -241,7 +241,7 @@ def oracle_sample(threads: int, buckets_per_thread: int):
     def work(t):
         for b in range(buckets_per_thread):
             orc.send_step(ocfg, g, states[t], comms[t], 1 + b)
-            orc.reduce(ocfg, n, [comms[t]] + [others[w % 2] for w in range(WORKERS - 1)], first=0, count=1)
+            orc.reduce(ocfg, n, [comms[t]] + [others[w % 2] for w in range(WORKERS - 1)])
 
     t0 = time.perf_counter()
     with ThreadPoolExecutor(max_workers=threads) as ex:
@@ -268,10 +268,10 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     cores = os.cpu_count() or 1
-    config = {"workload": "llama2-7b: 270 bf16 buckets of 25M elements (6,738,415,616), per-rank view of an 8-worker job",
+    config = {"workload": "llama2-7b: 270 bf16 buckets of 25M elements (6,738,415,616): one worker's send pass per bucket, then the 8-worker reduce of the bucket",
               "bits": 4, "scale": "fixed s=2^14, s_e=4s (Eq. 1)", "beta": 0.5, "T_c": 512, "state": "int8",
               "workers_on_reduce_side": WORKERS, "out": "bf16",
-              "l2": "inputs larger than L2: each step streams ~35 GB once, no reuse between launches"}
+              "l2": "inputs larger than L2: each step streams ~70 GB once, no reuse between launches"}
 
     if args.impl == "reference":
         if rank != 0:
@@ -286,7 +286,7 @@ def main():
             elems += e
         dt = time.perf_counter() - t0
         val = 2.0 * elems / dt / 1e9
-        sample = "%d buckets of 25M elements per step (one per host thread), send + own-part reduce" % cores
+        sample = "%d buckets of 25M elements per step (one per host thread), send + 8-worker reduce" % cores
         print(json.dumps({"impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus,
                           "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": dt / steps * 1e3,
                           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
@@ -393,13 +393,13 @@ def main():
     kernels = {"send": {"hbm_gbs": send_gbs, "frac_of_peak": send_gbs / peak, "gradient_gbs": wl.grad_bytes / (send_ms * 1e-3) / 1e9,
                         "ms_per_step": send_ms, "avg_launch_us": send_ms * 1e3 / nb, "bytes_per_elem": SEND_BYTES_PER_ELEM},
                "reduce": {"hbm_gbs": recv_gbs, "frac_of_peak": recv_gbs / peak,
-                          "gradient_gbs": 2 * sum(wl.out_elems) / (recv_ms * 1e-3) / 1e9, "ms_per_step": recv_ms,
+                          "gradient_gbs": wl.grad_bytes / (recv_ms * 1e-3) / 1e9, "ms_per_step": recv_ms,
                           "avg_launch_us": recv_ms * 1e3 / nb, "bytes_per_out_elem": WORKERS * 0.5 + 2}}
     cpu = None
     if not args.no_cpu_baseline:
         v, dt, elems = oracle_sample(cores, 2)
         cpu = {"value": v, "unit": "GB/s", "cores": cores, "kind": "oracle",
-               "sample": "%d buckets of 25M elements (2 per host thread), send + own-part reduce, %.1f s wall" % (2 * cores, dt)}
+               "sample": "%d buckets of 25M elements (2 per host thread), send + 8-worker reduce, %.1f s wall" % (2 * cores, dt)}
     line = {"metric": METRIC, "value": world * wl.grad_bytes / (step_ms * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": world,
             "steps": K, "warmup": max(3, args.warmup), "ms_per_step": step_ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,

@@ -591,23 +591,23 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams
         K.dq_a = P.dq_a; K.dq_b = P.dq_b; K.de_a = P.de_a; K.de_b = P.de_b;
         K.dq_mode = P.dq_mode; K.de_mode = P.de_mode; K.block_log2 = P.block_log2; K.reset = P.reset;
         const bool stats = P.collect_stats != 0;
-        // full_rows <= rows < 2^32 - kUnroll * nwarps for every bucket this library accepts
-        for (; r + (kUnroll - 1) * nwarps < full_rows; r += kUnroll * nwarps) {
+        // full_rows <= rows < 2^32 - kUnroll * nwarps for every bucket this library accepts.
+        // The last trip of a warp may hold fewer than kUnroll rows: its loads are still issued together.
+        for (; r < full_rows; r += kUnroll * nwarps) {
             RowIn<GRAD, STATE> in[kUnroll];
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) load_row<GRAD, STATE, MODE>(L, r + u * nwarps, K.block_log2, in[u]);
+            for (int u = 0; u < kUnroll; ++u)
+                if (u == 0 || r + u * nwarps < full_rows) load_row<GRAD, STATE, MODE>(L, r + u * nwarps, K.block_log2, in[u]);
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
-                if (!send_row_fast<GRAD, STATE, BITS, MODE, LEAN>(K, L, in[u], r + u * nwarps, lane, stats, saturated))
-                    careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(r + u * nwarps) * kRow, lane);
+                if (u == 0 || r + u * nwarps < full_rows) {
+                    if (!send_row_fast<GRAD, STATE, BITS, MODE, LEAN>(K, L, in[u], r + u * nwarps, lane, stats, saturated))
+                        careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(r + u * nwarps) * kRow, lane);
+                }
             }
         }
-        for (; r < full_rows; r += nwarps) {
-            RowIn<GRAD, STATE> in;
-            load_row<GRAD, STATE, MODE>(L, r, K.block_log2, in);
-            if (!send_row_fast<GRAD, STATE, BITS, MODE, LEAN>(K, L, in, r, lane, stats, saturated))
-                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(r) * kRow, lane);
-        }
+        // rows of this warp at or beyond full_rows (partial or padding rows) are left to the careful routine
+        r = warp + ((full_rows > warp ? (full_rows - warp + nwarps - 1) / nwarps : 0u)) * nwarps;
     }
     for (; r < rows; r += nwarps)
         careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(r) * kRow, lane);
@@ -744,44 +744,45 @@ struct LaneSums {
 
 template <int OUT, int BITS, int MODE>
 __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParams P) {
-    constexpr int kUnroll = 4;
+    constexpr unsigned kRowBytes = kRow * BITS / 8;                   // code bytes of one row
     const int lane = threadIdx.x & 31;
     const unsigned long long part = blockIdx.y;                       // relative to P.first
-    const unsigned long long warp = static_cast<unsigned long long>(blockIdx.x) * kWarps + (threadIdx.x >> 5);
-    const unsigned long long nwarps = static_cast<unsigned long long>(gridDim.x) * kWarps;
+    const unsigned warp = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    const unsigned nwarps = gridDim.x * kWarps;
     const unsigned long long base = (P.first + part) * P.lp;          // first bucket element of the part
     if (base >= P.n) return;
     const unsigned long long avail = P.n - base;
     const unsigned long long valid = avail >= P.lp ? P.lp : avail;
-    const unsigned long long rows = (valid + kRow - 1) / kRow;
+    const unsigned rows = static_cast<unsigned>((valid + kRow - 1) / kRow);
     const unsigned long long poff = part * P.stride;
     const unsigned long long out0 = part * P.lp;                      // output index of the part's first element
-    const unsigned long long lane_off = static_cast<unsigned long long>(lane) * kLaneElems;
+    const unsigned lane_elem = static_cast<unsigned>(lane) * kLaneElems;
+    const unsigned lane_byte = lane_elem * BITS / 8;
     const int N = P.num_workers;
 
     if (MODE == MODE_FIXED && BITS != 2 && P.int_path) {
-        for (unsigned long long r = warp; r < rows; r += kUnroll * nwarps) {
+        constexpr int kUnroll = 4;
+        for (unsigned r = warp; r < rows; r += kUnroll * nwarps) {
             LaneSums<BITS> sums[kUnroll];
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) sums[u].clear();
 #pragma unroll 4
             for (int w = 0; w < N; ++w) {
-                const uint8_t *src = P.parts[w] + poff;
+                const uint8_t *src = P.parts[w] + poff + lane_byte;
                 CodeWord<BITS> cw[kUnroll];
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
-                    const unsigned long long o = (r + u * nwarps) * kRow + lane_off;
-                    // rows past the end are clamped to the last row: loaded, never stored
-                    const unsigned long long oc = (r + u * nwarps) < rows ? o : (rows - 1) * kRow + lane_off;
-                    load_codeword<BITS>(src + oc * BITS / 8, cw[u]);
+                    cw[u].x = 0u; cw[u].y = 0u;
+                    if (u == 0 || r + u * nwarps < rows)
+                        load_codeword<BITS>(src + static_cast<size_t>(r + u * nwarps) * kRowBytes, cw[u]);
                 }
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) sums[u].add(cw[u]);
             }
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
-                const unsigned long long o = (r + u * nwarps) * kRow + lane_off;
-                if ((r + u * nwarps) >= rows || o >= valid) continue;
+                const unsigned long long o = static_cast<unsigned long long>(r + u * nwarps) * kRow + lane_elem;
+                if ((u != 0 && r + u * nwarps >= rows) || o >= valid) continue;
                 float res[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -794,34 +795,51 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
         return;
     }
 
-    for (unsigned long long r = warp; r < rows; r += nwarps) {
-        const unsigned long long o = r * kRow + lane_off;
-        if (o >= valid) continue;
-        float acc[8];
+    constexpr int kUnrollG = 2;
+    for (unsigned r = warp; r < rows; r += kUnrollG * nwarps) {
+        float acc[kUnrollG][8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
-#pragma unroll 4
+        for (int u = 0; u < kUnrollG; ++u)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[u][j] = 0.0f;
+#pragma unroll 2
         for (int w = 0; w < N; ++w) {
-            const uint8_t *src = P.parts[w] + poff;
-            CodeWord<BITS> cw;
-            load_codeword<BITS>(src + o * BITS / 8, cw);
-            float sc = P.gen_mul;
-            if (MODE == MODE_BLOCK)
-                sc = __ldg(reinterpret_cast<const float *>(src + P.code_bytes) + (o >> P.block_log2));
-            float q[8];
-            codes_to_float<BITS>(cw, q);
+            const uint8_t *wbase = P.parts[w] + poff;
+            CodeWord<BITS> cw[kUnrollG];
+            float sc[kUnrollG];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                float d;                                               // dec(q; s), Eq. 1
-                if (MODE == MODE_FIXED && sc == 0.0f) d = __fdiv_rn(q[j], P.s);
-                else d = __fmul_rn(q[j], sc);
-                acc[j] = __fadd_rn(acc[j], d);
+            for (int u = 0; u < kUnrollG; ++u) {
+                cw[u].x = 0u; cw[u].y = 0u;
+                sc[u] = P.gen_mul;
+                if (u == 0 || r + u * nwarps < rows) {
+                    load_codeword<BITS>(wbase + lane_byte + static_cast<size_t>(r + u * nwarps) * kRowBytes, cw[u]);
+                    if (MODE == MODE_BLOCK)
+                        sc[u] = __ldg(reinterpret_cast<const float *>(wbase + P.code_bytes) +
+                                      ((static_cast<unsigned long long>(r + u * nwarps) * kRow + lane_elem) >> P.block_log2));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kUnrollG; ++u) {
+                float q[8];
+                codes_to_float<BITS>(cw[u], q);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    float d;                                               // dec(q; s), Eq. 1
+                    if (MODE == MODE_FIXED && P.gen_mul == 0.0f) d = __fdiv_rn(q[j], P.s);
+                    else d = __fmul_rn(q[j], sc[u]);
+                    acc[u][j] = __fadd_rn(acc[u][j], d);
+                }
             }
         }
-        float res[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) res[j] = div_workers(P, acc[j]);   // the 1/N of Eq. 8
-        store_out8<OUT>(P.out, out0 + o, res, valid - o);
+        for (int u = 0; u < kUnrollG; ++u) {
+            const unsigned long long o = static_cast<unsigned long long>(r + u * nwarps) * kRow + lane_elem;
+            if ((u != 0 && r + u * nwarps >= rows) || o >= valid) continue;
+            float res[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) res[j] = div_workers(P, acc[u][j]);   // the 1/N of Eq. 8
+            store_out8<OUT>(P.out, out0 + o, res, valid - o);
+        }
     }
 }
 
