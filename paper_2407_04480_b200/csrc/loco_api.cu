@@ -154,16 +154,21 @@ int num_sms() {
 // ---- send dispatch -----------------------------------------------------------------------
 
 using SendFn = void (*)(const SendParams);
+struct SendKernel { SendFn fn; int smem_bytes; };
 
 template <int GRAD, int STATE, int BITS>
-SendFn pick_send_mode(int mode, bool lean) {
-    if (mode == MODE_FIXED)
-        return lean ? loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, true> : loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, false>;
-    if (STATE == ST_Q8COMP) return nullptr;                     // Q8COMP exists for the global scales only
-    return loco_send_kernel<GRAD, (STATE == ST_Q8COMP ? ST_FP32 : STATE), BITS, MODE_BLOCK, true>;
+SendKernel pick_send_mode(int mode, bool lean) {
+    if (mode == MODE_FIXED) {
+        const int smem = Ring<GRAD, STATE, MODE_FIXED>::kBytes;
+        if (lean) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, true>, smem};
+        return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, false>, smem};
+    }
+    if (STATE == ST_Q8COMP) return {nullptr, 0};                // Q8COMP exists for the global scales only
+    constexpr int ST = (STATE == ST_Q8COMP ? ST_FP32 : STATE);
+    return {loco_send_kernel<GRAD, ST, BITS, MODE_BLOCK, true>, Ring<GRAD, ST, MODE_BLOCK>::kBytes};
 }
 template <int GRAD, int STATE>
-SendFn pick_send_bits(int bits, int mode, bool lean) {
+SendKernel pick_send_bits(int bits, int mode, bool lean) {
     switch (bits) {
     case 2: return pick_send_mode<GRAD, STATE, 2>(mode, lean);
     case 4: return pick_send_mode<GRAD, STATE, 4>(mode, lean);
@@ -171,7 +176,7 @@ SendFn pick_send_bits(int bits, int mode, bool lean) {
     }
 }
 template <int GRAD>
-SendFn pick_send_state(int state, int bits, int mode, bool lean) {
+SendKernel pick_send_state(int state, int bits, int mode, bool lean) {
     switch (state) {
     case LOCO_STATE_INT8: return pick_send_bits<GRAD, ST_INT8>(bits, mode, lean);
     case LOCO_STATE_FP32: return pick_send_bits<GRAD, ST_FP32>(bits, mode, lean);
@@ -179,7 +184,7 @@ SendFn pick_send_state(int state, int bits, int mode, bool lean) {
     default: return pick_send_bits<GRAD, ST_Q8COMP>(bits, mode, lean);
     }
 }
-SendFn pick_send(const loco_config_t *c, int mode, bool lean) {
+SendKernel pick_send(const loco_config_t *c, int mode, bool lean) {
     return c->grad_dtype == LOCO_BF16 ? pick_send_state<GRAD_BF16>(c->state_fmt, c->bits, mode, lean)
                                       : pick_send_state<GRAD_F32>(c->state_fmt, c->bits, mode, lean);
 }
@@ -228,6 +233,7 @@ struct loco_state {
     int device;
     int mode;
     SendFn send_fn;
+    int send_smem_bytes;            // dynamic shared memory of the send kernel (its cp.async ring)
     int send_ctas_per_sm;
     Layout layout;
     DecChoice dq, de;               // how the kernels evaluate dec(q; s) and dec(e; s_e)
@@ -302,17 +308,31 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
         if (cfg->state_fmt == LOCO_STATE_INT8 || cfg->state_fmt == LOCO_STATE_FP32_Q8COMP)
             st->de = choose_dec(cfg->s_e, -128, 127, 128);
         st->fast = (st->dq.mode != DEC_DIVIDE && st->de.mode != DEC_DIVIDE) ? 1 : 0;
+        // the fast routine tests only g for NaN / Inf when the state is 8-bit: dec(e) must be too small to push a
+        // finite g to infinity (|e / s_e| <= 128 / s_e < 2^100)
+        if (cfg->state_fmt == LOCO_STATE_INT8 && !(cfg->s_e > 1e-28f)) st->fast = 0;
     }
     {
         const bool lean = st->mode == MODE_BLOCK ||
                           (st->dq.mode == DEC_FMA && st->de.mode == DEC_FMA && !cfg->collect_stats);
-        st->send_fn = pick_send(cfg, st->mode, lean);
+        const SendKernel k = pick_send(cfg, st->mode, lean);
+        st->send_fn = k.fn;
+        st->send_smem_bytes = k.smem_bytes;
     }
     st->send_ctas_per_sm = 1;
     if (!st->send_fn) { delete st; return LOCO_ERR_UNSUPPORTED; }
     if (cudaGetDevice(&st->device) != cudaSuccess) { delete st; return LOCO_ERR_CUDA; }
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, st->send_fn, kThreads, 0) != cudaSuccess || occ < 1) {
+    // the ring wants most of the SM's shared memory (3 CTAs x up to 72 KB)
+    if (cudaFuncSetAttribute(reinterpret_cast<const void *>(st->send_fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             st->send_smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(reinterpret_cast<const void *>(st->send_fn), cudaFuncAttributePreferredSharedMemoryCarveout,
+                             cudaSharedmemCarveoutMaxShared) != cudaSuccess) {
+        cudaGetLastError();
+        delete st;
+        return LOCO_ERR_CUDA;
+    }
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, st->send_fn, kThreads, static_cast<size_t>(st->send_smem_bytes)) != cudaSuccess || occ < 1) {
         cudaGetLastError();
         delete st;
         return LOCO_ERR_CUDA;
@@ -388,7 +408,7 @@ int loco_compensate_quantize_pack(loco_state_t *st, const void *d_grad, void *d_
     P.status = st->d_status;
     const uint64_t rows = P.lp / kRow;
     dim3 grid(grid_x_for(rows, c.num_partitions, st->send_ctas_per_sm), static_cast<unsigned>(c.num_partitions), 1);
-    st->send_fn<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(P);
+    st->send_fn<<<grid, kThreads, static_cast<size_t>(st->send_smem_bytes), static_cast<cudaStream_t>(stream)>>>(P);
     if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;
     g_launches.fetch_add(1);
     return LOCO_OK;
@@ -441,7 +461,7 @@ int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_pa
         }
         // Integer path: with s a power of two every partial sum of Eq. 8 is exact in fp32, so the codes can be
         // added as integers.  The lane sums are bounded by (2^p - 1) * N, which 8- and 16-bit lanes hold for N <= 16.
-        if (cfg->bits != 2 && num_workers <= 16 && is_pow2_float(cfg->s)) {
+        if (cfg->bits != 2 && num_workers <= 16 && is_pow2_float(cfg->s) && L.code_bytes < (1ull << 32)) {
             P.int_path = 1;
             const float inv_s = 1.0f / cfg->s;                                    // exact
             float ra = inv_s;

@@ -13,9 +13,12 @@
 //   * codes are packed by a Horner chain of integer multiply-adds (they run on the fp32 pipe);
 //   * non-finite inputs are detected with one fused multiply-add per element (h * 0 accumulates NaN)
 //     and the rare rows that contain one are redone by a plain, careful routine.
-// Work unit: a "row" of 256 consecutive elements handled by one warp, 8 consecutive elements per
-// lane, so that every warp-wide access covers one contiguous span.  A warp loads several rows before
-// it starts computing, which keeps enough bytes in flight to cover the HBM latency.
+//   * the fp32 steps of the send pass run two elements at a time on the packed fp32x2 instructions, which
+//     halves their issue slots; the inputs of a warp's next rows travel through a cp.async ring in shared
+//     memory, so the bytes in flight do not depend on registers or on the phase the warp is in.
+// Work unit of the send pass: a "wide row" of 512 consecutive elements handled by one warp, 16 consecutive
+// elements per lane; of the receive pass and of the careful routine: a row of 256 elements, 8 per lane.
+// Every warp-wide access covers one contiguous span.
 //
 // Rounding discipline: every floating-point step of Algorithm 1 is one IEEE fp32 operation rounded to
 // nearest even, written with intrinsics, so that nothing is contracted into an FMA by the compiler; an
@@ -341,82 +344,179 @@ __device__ __noinline__ unsigned send_row_careful(const SendParams P, unsigned l
 }
 
 // ------------------------------------------------------------------------------------------
-// send, fast routine: one full row whose inputs are already in registers.
+// send, fast routine: "wide rows" of 512 elements, 16 consecutive elements per lane, computed two at a
+// time with the packed fp32x2 instructions of sm_100 (one issue slot for two IEEE operations).
 
-template <int GRAD, int STATE>
-struct RowIn {
-    static constexpr int GW = (GRAD == GRAD_BF16) ? 4 : 8;                       // gradient words per lane
-    static constexpr int SW = (STATE == ST_INT8) ? 2 : (STATE == ST_NONE ? 1 : 8);   // state words per lane
-    unsigned g[GW];
-    unsigned e[SW];
-    float sscale;                                                                // BLOCK + INT8
-};
+constexpr int kWide = 512;         // elements per wide row
+constexpr int kWideLane = 16;      // elements per lane per wide row
 
-// Per-lane base pointers of one partition: everything a row needs is base + row * (bytes per row).
+typedef unsigned long long f32x2;  // two fp32 in one 64-bit register pair: low word = the even element
+
+__device__ __forceinline__ f32x2 pk2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ f32x2 dup2(float v) { return pk2(v, v); }
+__device__ __forceinline__ void unpk2(f32x2 v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fadd2(f32x2 a, f32x2 b) { f32x2 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 fsub2(f32x2 a, f32x2 b) { f32x2 d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 fmul2(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
+__device__ __forceinline__ f32x2 ffma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+// The assembler contracts a packed multiply that feeds a packed add or subtract into one packed FMA even
+// though both carry an explicit rounding mode (seen as single-rounded results on sm_100a, CUDA 12.9).  Where
+// Algorithm 1 rounds the product and the sum separately, the sum is therefore taken with scalar
+// instructions, which are never contracted.
+__device__ __forceinline__ f32x2 fadd2_after_mul(f32x2 a, f32x2 b) {
+    float a0, a1, b0, b1;
+    unpk2(a, a0, a1);
+    unpk2(b, b0, b1);
+    return pk2(__fadd_rn(a0, b0), __fadd_rn(a1, b1));
+}
+__device__ __forceinline__ f32x2 fsub2_after_mul(f32x2 a, f32x2 b) {
+    float a0, a1, b0, b1;
+    unpk2(a, a0, a1);
+    unpk2(b, b0, b1);
+    return pk2(__fsub_rn(a0, b0), __fsub_rn(a1, b1));
+}
+__device__ __forceinline__ unsigned hfma2_bf16(unsigned a, unsigned b, unsigned c) {
+    unsigned d;
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+// Per-lane base pointers of one partition: everything a wide row needs is base + row * (bytes per row).
 struct LanePtrs {
-    const uint8_t *grad;      // this lane's 8 gradient elements of row 0
-    uint8_t *state;           // this lane's 8 state elements of row 0 (int8 or fp32)
-    uint8_t *codes;           // this lane's code bytes of row 0 in the partition's code area
+    uint8_t *state;           // this lane's 16 state elements of wide row 0 (int8 or fp32)
+    uint8_t *codes;           // this lane's code bytes of wide row 0 in the partition's code area
     float *wire_scales;       // BLOCK: the partition's scale area
     float *state_scales;      // BLOCK + INT8: scale of the bucket's block 0
-    unsigned long long elem0; // bucket index of this lane's first element of row 0
-    unsigned lane_elem;       // partition-local index of this lane's first element of row 0
+    unsigned long long elem0; // bucket index of this lane's first element of wide row 0
+    unsigned lane_elem;       // partition-local index of this lane's first element of wide row 0
+};
+
+// ---- per-warp ring of asynchronous copies (cp.async) -------------------------------------------
+// Every warp stages the inputs of its next wide rows in shared memory with cp.async, in 16-byte chunks
+// laid out so that a copy instruction of the warp reads 512 contiguous bytes of global memory; the bytes in
+// flight occupy no registers, and the depth of the ring, not the phase a warp happens to be in, decides how
+// much of the HBM latency is covered.  A lane's own elements span several chunks that other lanes copied,
+// so a chunk c is stored at position c ^ ((c >> 3) & (chunks per lane - 1)): both the copies and the
+// 16-byte reads of 8 consecutive lanes then fall into 8 different bank groups.  cp.async.wait_group
+// followed by __syncwarp() orders the warp's reads after all of its lanes' copies.
+// Shared memory is addressed by its 32-bit window offset throughout.
+__device__ __forceinline__ void cp_async16(unsigned saddr, const void *gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(saddr), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async4(unsigned saddr, const void *gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(saddr), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
+__device__ __forceinline__ uint4 lds16(unsigned saddr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned lds4(unsigned saddr) {
+    unsigned v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(saddr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_stream32(void *p, const unsigned *v) {      // one 256-bit store
+    asm volatile("st.global.cs.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 :: "l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+}
+
+template <int GRAD, int STATE, int MODE>
+struct Ring {
+    static constexpr int kGradChunks = (GRAD == GRAD_BF16) ? 2 : 4;                          // 16-byte chunks per lane
+    static constexpr int kStateChunks = (STATE == ST_INT8) ? 1 : (STATE == ST_NONE ? 0 : 4);
+    static constexpr int kScaleBytes = (STATE == ST_INT8 && MODE == MODE_BLOCK) ? 4 : 0;
+    static constexpr int kWarpSlotBytes = (kGradChunks + kStateChunks) * 512 + kScaleBytes * 32;
+    static constexpr int kSlotStride = kWarpSlotBytes * kWarps;
+    static constexpr int kFit = 73728 / kSlotStride;
+    static constexpr int kDepth = kFit > 6 ? 6 : kFit;
+    static constexpr int kBytes = kDepth * kSlotStride;
+    static constexpr int kStateOff = kGradChunks * 512;
+    static constexpr int kScaleOff = (kGradChunks + kStateChunks) * 512;
+    static_assert(kDepth >= 2, "the ring needs at least two slots");
+};
+
+// The lane's own shared-memory addresses inside slot 0 of its warp's ring.
+template <int GRAD, int STATE>
+struct RingAddr {
+    static constexpr int GC = (GRAD == GRAD_BF16) ? 2 : 4;
+    static constexpr int SC = (STATE == ST_INT8 || STATE == ST_NONE) ? 1 : 4;
+    unsigned g_stage;       // where this lane's copy of chunk (32 k + lane) goes for k = 0; add 512 k
+    unsigned e_stage;
+    unsigned g_fetch[GC];   // where this lane's own chunks are
+    unsigned e_fetch[SC];
+    unsigned sc;            // state scale
 };
 
 template <int GRAD, int STATE, int MODE>
-__device__ __forceinline__ void load_row(const LanePtrs &L, unsigned row, int block_log2, RowIn<GRAD, STATE> &in) {
-    constexpr unsigned gbytes = (GRAD == GRAD_BF16 ? 2u : 4u) * kRow;
-    const uint8_t *gp = L.grad + static_cast<size_t>(row) * gbytes;
-    if (GRAD == GRAD_BF16) {
-        const uint4 v = ld_stream16(gp);
-        in.g[0] = v.x; in.g[1] = v.y; in.g[2] = v.z; in.g[3] = v.w;
+__device__ __forceinline__ void ring_addresses(unsigned ring0, int lane, int warp_in_cta, RingAddr<GRAD, STATE> &A) {
+    using R = Ring<GRAD, STATE, MODE>;
+    constexpr int GC = R::kGradChunks;
+    constexpr int SC = RingAddr<GRAD, STATE>::SC;
+    const unsigned wbase = ring0 + warp_in_cta * R::kWarpSlotBytes;
+    const unsigned L = static_cast<unsigned>(lane);
+    A.g_stage = wbase + ((L ^ ((L >> 3) & (GC - 1))) << 4);
+    const unsigned xg = (GC == 2) ? ((L >> 2) & 1u) : ((L >> 1) & 3u);
+#pragma unroll
+    for (int k = 0; k < GC; ++k) A.g_fetch[k] = wbase + ((GC * L + (static_cast<unsigned>(k) ^ xg)) << 4);
+    if (SC == 4) {
+        A.e_stage = wbase + R::kStateOff + ((L ^ ((L >> 3) & 3u)) << 4);
+        const unsigned xe = (L >> 1) & 3u;
+#pragma unroll
+        for (int k = 0; k < SC; ++k) A.e_fetch[k] = wbase + R::kStateOff + ((4 * L + (static_cast<unsigned>(k) ^ xe)) << 4);
     } else {
-        const uint4 a = ld_stream16(gp);
-        const uint4 b = ld_stream16(gp + 16);
-        in.g[0] = a.x; in.g[1] = a.y; in.g[2] = a.z; in.g[3] = a.w;
-        in.g[RowIn<GRAD, STATE>::GW - 4] = b.x; in.g[RowIn<GRAD, STATE>::GW - 3] = b.y;
-        in.g[RowIn<GRAD, STATE>::GW - 2] = b.z; in.g[RowIn<GRAD, STATE>::GW - 1] = b.w;
+        A.e_stage = wbase + R::kStateOff + (L << 4);
+        A.e_fetch[0] = A.e_stage;
     }
-    in.sscale = 0.0f;
-    if (STATE == ST_INT8) {
-        const uint2 v = ld_stream8(L.state + static_cast<size_t>(row) * kRow);
-        in.e[0] = v.x; in.e[1] = v.y;
-        if (MODE == MODE_BLOCK)
-            in.sscale = L.state_scales[(L.elem0 + static_cast<unsigned long long>(row) * kRow) >> block_log2];
-    } else if (STATE == ST_FP32 || STATE == ST_Q8COMP) {
-        const uint8_t *sp = L.state + static_cast<size_t>(row) * (4u * kRow);
-        const uint4 a = ld_stream16(sp);
-        const uint4 b = ld_stream16(sp + 16);
-        in.e[0] = a.x; in.e[1] = a.y; in.e[2] = a.z; in.e[3] = a.w;
-        in.e[RowIn<GRAD, STATE>::SW - 4] = b.x; in.e[RowIn<GRAD, STATE>::SW - 3] = b.y;
-        in.e[RowIn<GRAD, STATE>::SW - 2] = b.z; in.e[RowIn<GRAD, STATE>::SW - 1] = b.w;
-    } else {
-        in.e[0] = 0u;
-    }
+    A.sc = wbase + R::kScaleOff + (L << 2);
 }
 
-// Packs the 8 codes held in the low bits of the magic-biased floats mb[j] = bits(kMagic + 2^(p-1) + q_j):
-// sum_j mb[j] * R^j = kMagicBits * sum_j R^j + sum_j (q_j + 2^(p-1)) R^j  (mod 2^32), R = 2^p; removing the
-// constant and flipping each field's top bit turns the biased fields into two's complement.
-template <int BITS>
-__device__ __forceinline__ void store_codes_fast(uint8_t *dst, const unsigned (&mb)[8]) {
-    if (BITS == 4) {
-        unsigned acc = mb[7];
+// Issue the copies of one wide row.  g_row / e_row: global address of the row's first byte plus lane * 16.
+template <int GRAD, int STATE, int MODE>
+__device__ __forceinline__ void stage_row(const RingAddr<GRAD, STATE> &A, unsigned slot_off, const uint8_t *g_row,
+                                          const uint8_t *e_row, const float *scale_ptr) {
+    using R = Ring<GRAD, STATE, MODE>;
 #pragma unroll
-        for (int j = 6; j >= 0; --j) acc = acc * 16u + mb[j];
-        st_stream4(dst, (acc - kMagicBits * 0x11111111u) ^ 0x88888888u);
-    } else if (BITS == 8) {
-        unsigned a0 = mb[3], a1 = mb[7];
+    for (int k = 0; k < R::kGradChunks; ++k) cp_async16(A.g_stage + slot_off + 512 * k, g_row + 512 * k);
 #pragma unroll
-        for (int j = 2; j >= 0; --j) { a0 = a0 * 256u + mb[j]; a1 = a1 * 256u + mb[4 + j]; }
-        st_stream8(dst, make_uint2((a0 - kMagicBits * 0x01010101u) ^ 0x80808080u,
-                                   (a1 - kMagicBits * 0x01010101u) ^ 0x80808080u));
-    } else {
-        unsigned acc = mb[7];
+    for (int k = 0; k < R::kStateChunks; ++k) cp_async16(A.e_stage + slot_off + 512 * k, e_row + 512 * k);
+    if (R::kScaleBytes) cp_async4(A.sc + slot_off, scale_ptr);
+}
+
+template <int GRAD, int STATE>
+struct WideIn {
+    static constexpr int GW = (GRAD == GRAD_BF16) ? 8 : 16;                          // gradient words per lane
+    static constexpr int EW = (STATE == ST_INT8) ? 4 : (STATE == ST_NONE ? 1 : 16);  // state words per lane
+    unsigned g[GW];
+    unsigned e[EW];
+    float sscale;                                                                    // BLOCK + INT8
+};
+
+template <int GRAD, int STATE, int MODE>
+__device__ __forceinline__ void fetch_row(const RingAddr<GRAD, STATE> &A, unsigned slot_off, WideIn<GRAD, STATE> &in) {
+    using R = Ring<GRAD, STATE, MODE>;
+    constexpr int EW = WideIn<GRAD, STATE>::EW;
 #pragma unroll
-        for (int j = 6; j >= 0; --j) acc = acc * 4u + mb[j];
-        *reinterpret_cast<uint16_t *>(dst) = static_cast<uint16_t>(((acc - kMagicBits * 0x5555u) ^ 0xAAAAu) & 0xffffu);
+    for (int k = 0; k < R::kGradChunks; ++k) {
+        const uint4 v = lds16(A.g_fetch[k] + slot_off);
+        in.g[4 * k] = v.x; in.g[4 * k + 1] = v.y; in.g[4 * k + 2] = v.z; in.g[4 * k + 3] = v.w;
     }
+    in.e[0] = 0u;
+#pragma unroll
+    for (int k = 0; k < R::kStateChunks; ++k) {
+        const uint4 v = lds16(A.e_fetch[k % RingAddr<GRAD, STATE>::SC] + slot_off);
+        in.e[(4 * k) % EW] = v.x; in.e[(4 * k + 1) % EW] = v.y;
+        in.e[(4 * k + 2) % EW] = v.z; in.e[(4 * k + 3) % EW] = v.w;
+    }
+    in.sscale = R::kScaleBytes ? __uint_as_float(lds4(A.sc + slot_off)) : 0.0f;
 }
 
 // The scalars of Algorithm 1 the fast routine needs, read from the parameters once per kernel.
@@ -425,147 +525,245 @@ struct SendConsts {
     int dq_mode, de_mode, block_log2, reset;
 };
 
-// Returns false (and stores nothing) if some lane of the warp met a non-finite compensated gradient:
-// the caller then redoes the row with the careful routine.
-// LEAN: both decompressors are the single fused multiply-add and no statistics are collected, so the
-// routine has no data-dependent branch at all.
+// Field j of the packed codes sits in the low bits of mb[j] = bits(kMagic + 2^(p-1) + q_j):
+// sum_j mb[j] * R^j = kMagicBits * sum_j R^j + sum_j (q_j + 2^(p-1)) R^j  (mod 2^32), R = 2^p; removing the
+// constant and flipping each field's top bit turns the biased fields into two's complement.
+template <int BITS, int COUNT>
+__device__ __forceinline__ unsigned horner_codes(const unsigned *mb) {
+    unsigned acc = mb[COUNT - 1];
+#pragma unroll
+    for (int j = COUNT - 2; j >= 0; --j) acc = acc * (1u << BITS) + mb[j];
+    unsigned ones = 0u, flip = 0u;
+#pragma unroll
+    for (int j = 0; j < COUNT; ++j) { ones |= 1u << (BITS * j); flip |= (1u << (BITS - 1)) << (BITS * j); }
+    return (acc - kMagicBits * ones) ^ flip;
+}
+
+// One wide row.  Returns false (and stores nothing) if some lane of the warp met a value that the fast
+// arithmetic does not cover (NaN, +-Inf, or a magnitude that could overflow): the caller then redoes the row
+// with the careful routine.
+// LEAN: both decompressors are the single fused multiply-add and no statistics are collected.
 template <int GRAD, int STATE, int BITS, int MODE, bool LEAN>
-__device__ __forceinline__ bool send_row_fast(const SendConsts &K, const LanePtrs &L, const RowIn<GRAD, STATE> &in,
-                                              unsigned row, int lane, bool stats, unsigned &saturated) {
+__device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtrs &L, const WideIn<GRAD, STATE> &in,
+                                              unsigned wrow, int lane, bool stats, unsigned &saturated) {
     constexpr float lo = QRange<BITS>::lo, hi = QRange<BITS>::hi, qmagic = kMagic + QRange<BITS>::off;
     constexpr float emagic = kMagic + 128.0f;
+    constexpr bool kStateF32 = (STATE == ST_FP32 || STATE == ST_Q8COMP);
+    constexpr int GW = WideIn<GRAD, STATE>::GW, EW = WideIn<GRAD, STATE>::EW;
     const int dq_mode = LEAN ? DEC_FMA : K.dq_mode, de_mode = LEAN ? DEC_FMA : K.de_mode;
-    const int lanes_per_block = (MODE == MODE_BLOCK) ? (K.block_log2 >= 8 ? 32 : (1 << (K.block_log2 - 3))) : 1;
+    const int lanes_per_block = (MODE == MODE_BLOCK) ? (K.block_log2 >= 9 ? 32 : (1 << (K.block_log2 - 4))) : 1;
+    const f32x2 zero2 = 0ull;
 
-    float g[8], c[8], prev[8], h[8];
+    // ---- values outside the fast arithmetic -------------------------------------------------------------
+    // x * 0 is 0 for finite x and NaN otherwise; with fp32 state, g and e~ are first scaled by 4 so that
+    // anything whose sum could overflow is caught as well.  With the 8-bit state the host has checked that
+    // dec(e) is too small to push a finite g to infinity.
+    unsigned bad_bits;
+    f32x2 g2[8];
     if (GRAD == GRAD_BF16) {
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            g[2 * j] = __uint_as_float(in.g[j] << 16);
-            g[2 * j + 1] = __uint_as_float(in.g[j] & 0xffff0000u);
-        }
+        for (int k = 0; k < 8; ++k)
+            g2[k] = pk2(__uint_as_float(in.g[k % GW] << 16), __uint_as_float(in.g[k % GW] & 0xffff0000u));
     } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) g[j] = __uint_as_float(in.g[j]);
+        for (int k = 0; k < 8; ++k)
+            g2[k] = pk2(__uint_as_float(in.g[(2 * k) % GW]), __uint_as_float(in.g[(2 * k + 1) % GW]));
     }
-
-    // step 1, Eq. 2: c = what is added to g, prev = e~_k of Eq. 5
-    if (STATE == ST_INT8) {
-        const unsigned x0 = in.e[0] ^ 0x80808080u, x1 = in.e[1] ^ 0x80808080u;    // bytes e + 128
+    if (GRAD == GRAD_BF16 && !kStateF32) {
+        unsigned acc = 0u;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const float m = __uint_as_float(__byte_perm(j < 4 ? x0 : x1, kMagicBits, 0x7650 + (j & 3)));   // kMagic + 128 + e
-            if (MODE == MODE_FIXED) c[j] = dec_fast(m, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se);
-            else c[j] = __fmul_rn(__fadd_rn(m, -emagic), in.sscale);
-            prev[j] = c[j];
-        }
-    } else if (STATE == ST_FP32) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) { c[j] = __uint_as_float(in.e[j]); prev[j] = c[j]; }
-    } else if (STATE == ST_Q8COMP) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            prev[j] = __uint_as_float(in.e[j]);
-            const float t = fminf(fmaxf(__fmul_rn(prev[j], K.s_e), -128.0f), 127.0f);
-            c[j] = dec_fast(__fadd_rn(t, emagic), emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se);
-        }
+        for (int k = 0; k < 8; ++k) acc = hfma2_bf16(in.g[k % GW], 0u, acc);
+        bad_bits = acc & 0x7fff7fffu;
     } else {
+        f32x2 acc = zero2;
+        const f32x2 four2 = dup2(4.0f);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { c[j] = 0.0f; prev[j] = 0.0f; }
-    }
-    float nf = 0.0f;                     // stays 0 unless some h is NaN or +-Inf
+        for (int k = 0; k < 8; ++k) acc = ffma2(kStateF32 ? fmul2(g2[k], four2) : g2[k], zero2, acc);
+        if (kStateF32) {
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        h[j] = __fadd_rn(g[j], c[j]);
-        nf = __fmaf_rn(h[j], 0.0f, nf);
+            for (int k = 0; k < 8; ++k) {
+                const f32x2 e2 = pk2(__uint_as_float(in.e[(2 * k) % EW]), __uint_as_float(in.e[(2 * k + 1) % EW]));
+                acc = ffma2(fmul2(e2, four2), zero2, acc);
+            }
+        }
+        bad_bits = (static_cast<unsigned>(acc) | static_cast<unsigned>(acc >> 32)) & 0x7fffffffu;
     }
-    if (__any_sync(kFull, !(nf == 0.0f))) return false;
+    if (MODE != MODE_BLOCK) {
+        if (__any_sync(kFull, bad_bits != 0u)) return false;
+    }
 
-    // Eq. 1 / Eq. 3: q = round_p-bit(h x s);  step 2: d, Eq. 5
+    // ---- step 1, Eq. 2: c = what is added to g, prev = e~_k of Eq. 5, h = g + c -----------------------------
+    f32x2 prev2[8], h2[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        f32x2 c2;
+        if (STATE == ST_INT8) {
+            const unsigned x = in.e[(k >> 1) % EW] ^ 0x80808080u;                                   // bytes e + 128
+            const float m0 = __uint_as_float(__byte_perm(x, kMagicBits, 0x7650 + 2 * (k & 1)));     // kMagic + 128 + e
+            const float m1 = __uint_as_float(__byte_perm(x, kMagicBits, 0x7651 + 2 * (k & 1)));
+            if (MODE == MODE_BLOCK) {
+                c2 = fmul2(fadd2(pk2(m0, m1), dup2(-emagic)), dup2(in.sscale));
+            } else if (LEAN) {
+                c2 = ffma2(pk2(m0, m1), dup2(K.de_a), dup2(K.de_b));
+            } else {
+                c2 = pk2(dec_fast(m0, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se),
+                         dec_fast(m1, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se));
+            }
+            prev2[k] = c2;
+        } else if (kStateF32) {
+            prev2[k] = pk2(__uint_as_float(in.e[(2 * k) % EW]), __uint_as_float(in.e[(2 * k + 1) % EW]));
+            if (STATE == ST_FP32) {
+                c2 = prev2[k];
+            } else {
+                float y0, y1;
+                unpk2(fmul2(prev2[k], dup2(K.s_e)), y0, y1);
+                const f32x2 m2 = fadd2(pk2(fminf(fmaxf(y0, -128.0f), 127.0f), fminf(fmaxf(y1, -128.0f), 127.0f)), dup2(emagic));
+                if (LEAN) {
+                    c2 = ffma2(m2, dup2(K.de_a), dup2(K.de_b));
+                } else {
+                    float m0, m1;
+                    unpk2(m2, m0, m1);
+                    c2 = pk2(dec_fast(m0, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se),
+                             dec_fast(m1, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se));
+                }
+            }
+        } else {
+            c2 = zero2;
+            prev2[k] = zero2;
+        }
+        // g + 0 changes at most the sign of a zero, never a code; in block mode c is a product
+        h2[k] = (STATE == ST_NONE) ? g2[k] : ((MODE == MODE_BLOCK && STATE == ST_INT8) ? fadd2_after_mul(g2[k], c2) : fadd2(g2[k], c2));
+    }
+
+    // ---- block scale (extension): absmax of the block's h over the lanes that share it ---------------------------
     float mult = K.s, scale = 0.0f;
     if (MODE == MODE_BLOCK) {
-        float amax = fmaxf(fabsf(h[0]), fabsf(h[1]));
+        float amax = 0.0f;
+        f32x2 acc = zero2;
 #pragma unroll
-        for (int j = 2; j < 8; ++j) amax = fmaxf(amax, fabsf(h[j]));
+        for (int k = 0; k < 8; ++k) {
+            float a, b;
+            unpk2(h2[k], a, b);
+            amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+            acc = ffma2(h2[k], zero2, acc);
+        }
+        bad_bits |= (static_cast<unsigned>(acc) | static_cast<unsigned>(acc >> 32)) & 0x7fffffffu;
+        if (__any_sync(kFull, bad_bits != 0u)) return false;
         amax = warp_group_max(amax, lanes_per_block);
         scale = amax > 0.0f ? __fdiv_rn(amax, hi) : 0.0f;
         mult = amax > 0.0f ? __fdiv_rn(hi, amax) : 0.0f;
     }
-    unsigned mb[8];
-    float e_new[8];
+
+    // ---- Eq. 1 / Eq. 3: q = round_p-bit(h x s);  step 2: d, Eq. 5 ---------------------------------------------
+    unsigned mb[16];
+    f32x2 en2[8];
+    const f32x2 mult2 = dup2(mult), qmagic2 = dup2(qmagic), omb2 = dup2(K.omb), beta2 = dup2(K.beta);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const float y = __fmul_rn(h[j], mult);
-        const float m = __fadd_rn(fminf(fmaxf(y, lo), hi), qmagic);      // kMagic + 2^(p-1) + q
-        mb[j] = __float_as_uint(m);
-        float d;
-        if (MODE == MODE_FIXED) d = dec_fast(m, qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s);
-        else d = __fmul_rn(__fadd_rn(m, -qmagic), scale);
-        const float delta = __fsub_rn(h[j], d);
-        e_new[j] = __fadd_rn(__fmul_rn(K.omb, prev[j]), __fmul_rn(K.beta, delta));
-        if (!LEAN && MODE == MODE_FIXED && stats) {
-            if (y >= hi + 0.5f || y < lo - 0.5f) saturated += 1u;
+    for (int k = 0; k < 8; ++k) {
+        float y0, y1;
+        unpk2(fmul2(h2[k], mult2), y0, y1);
+        const f32x2 m2 = fadd2(pk2(fminf(fmaxf(y0, lo), hi), fminf(fmaxf(y1, lo), hi)), qmagic2);   // kMagic + 2^(p-1) + q
+        mb[2 * k] = static_cast<unsigned>(m2);
+        mb[2 * k + 1] = static_cast<unsigned>(m2 >> 32);
+        f32x2 d2;
+        if (MODE == MODE_BLOCK) {
+            d2 = fmul2(fadd2(m2, dup2(-qmagic)), dup2(scale));
+        } else if (LEAN) {
+            d2 = ffma2(m2, dup2(K.dq_a), dup2(K.dq_b));
+        } else {
+            d2 = pk2(dec_fast(__uint_as_float(mb[2 * k]), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s),
+                     dec_fast(__uint_as_float(mb[2 * k + 1]), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s));
+            if (stats) {
+                if (y0 >= hi + 0.5f || y0 < lo - 0.5f) saturated += 1u;
+                if (y1 >= hi + 0.5f || y1 < lo - 0.5f) saturated += 1u;
+            }
         }
+        const f32x2 delta2 = (MODE == MODE_BLOCK) ? fsub2_after_mul(h2[k], d2) : fsub2(h2[k], d2);
+        en2[k] = (STATE == ST_NONE) ? zero2 : fadd2_after_mul(fmul2(omb2, prev2[k]), fmul2(beta2, delta2));
     }
-    store_codes_fast<BITS>(L.codes + static_cast<size_t>(row) * (kRow * BITS / 8), mb);
+    uint8_t *cdst = L.codes + static_cast<size_t>(wrow) * (kWide * BITS / 8);
+    if (BITS == 4) {
+        st_stream8(cdst, make_uint2(horner_codes<4, 8>(mb), horner_codes<4, 8>(mb + 8)));
+    } else if (BITS == 8) {
+        st_stream16(cdst, make_uint4(horner_codes<8, 4>(mb), horner_codes<8, 4>(mb + 4), horner_codes<8, 4>(mb + 8), horner_codes<8, 4>(mb + 12)));
+    } else {
+        st_stream4(cdst, horner_codes<2, 16>(mb));
+    }
     if (MODE == MODE_BLOCK) {
-        const unsigned ol = L.lane_elem + row * kRow;       // partition-local element index (rows are < 2^24)
+        const unsigned ol = L.lane_elem + wrow * kWide;     // partition-local element index
         if ((lane & (lanes_per_block - 1)) == 0 && ((ol & ((1u << K.block_log2) - 1)) == 0))
-            L.wire_scales[(static_cast<unsigned long long>(row) * kRow + L.lane_elem) >> K.block_log2] = scale;
+            L.wire_scales[ol >> K.block_log2] = scale;
     }
 
-    // Eq. 7
+    // ---- Eq. 7 ---------------------------------------------------------------------------------------------------
     if (STATE == ST_INT8) {
-        uint2 v = make_uint2(0u, 0u);
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
         float escale = 0.0f;
         if (!K.reset) {
             float emult = K.s_e;
             if (MODE == MODE_BLOCK) {
-                float amax = fmaxf(fabsf(e_new[0]), fabsf(e_new[1]));
+                float amax = 0.0f;
 #pragma unroll
-                for (int j = 2; j < 8; ++j) amax = fmaxf(amax, fabsf(e_new[j]));
+                for (int k = 0; k < 8; ++k) {
+                    float a, b;
+                    unpk2(en2[k], a, b);
+                    amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+                }
                 amax = warp_group_max(amax, lanes_per_block);
                 escale = amax > 0.0f ? __fdiv_rn(amax, 127.0f) : 0.0f;
                 emult = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
             }
-            int q[8];
+            const f32x2 emult2 = dup2(emult);
+            int q[16];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) q[j] = __float2int_rn(__fmul_rn(e_new[j], emult));   // saturates, NaN -> 0
+            for (int k = 0; k < 8; ++k) {
+                float a, b;
+                unpk2(fmul2(en2[k], emult2), a, b);
+                q[2 * k] = __float2int_rn(a);                   // saturates, NaN -> 0
+                q[2 * k + 1] = __float2int_rn(b);
+            }
             v.x = pack_sat_s8(q[0], q[1], pack_sat_s8(q[2], q[3], 0u));
             v.y = pack_sat_s8(q[4], q[5], pack_sat_s8(q[6], q[7], 0u));
+            v.z = pack_sat_s8(q[8], q[9], pack_sat_s8(q[10], q[11], 0u));
+            v.w = pack_sat_s8(q[12], q[13], pack_sat_s8(q[14], q[15], 0u));
         }
-        st_stream8(L.state + static_cast<size_t>(row) * kRow, v);
+        st_stream16(L.state + static_cast<size_t>(wrow) * kWide, v);
         if (MODE == MODE_BLOCK) {
-            const unsigned long long i0 = L.elem0 + static_cast<unsigned long long>(row) * kRow;
+            const unsigned long long i0 = L.elem0 + static_cast<unsigned long long>(wrow) * kWide;
             if ((lane & (lanes_per_block - 1)) == 0 && (i0 & ((1ull << K.block_log2) - 1)) == 0)
                 L.state_scales[i0 >> K.block_log2] = escale;
         }
-    } else if (STATE == ST_FP32 || STATE == ST_Q8COMP) {
-        if (K.reset) {
+    } else if (kStateF32) {
+        unsigned w[16];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) e_new[j] = 0.0f;
+        for (int k = 0; k < 8; ++k) {
+            w[2 * k] = K.reset ? 0u : static_cast<unsigned>(en2[k]);
+            w[2 * k + 1] = K.reset ? 0u : static_cast<unsigned>(en2[k] >> 32);
         }
-        uint8_t *dst = L.state + static_cast<size_t>(row) * (4u * kRow);
-        st_stream16(dst, make_uint4(__float_as_uint(e_new[0]), __float_as_uint(e_new[1]), __float_as_uint(e_new[2]), __float_as_uint(e_new[3])));
-        st_stream16(dst + 16, make_uint4(__float_as_uint(e_new[4]), __float_as_uint(e_new[5]), __float_as_uint(e_new[6]), __float_as_uint(e_new[7])));
+        uint8_t *dst = L.state + static_cast<size_t>(wrow) * (4u * kWide);
+        st_stream32(dst, w);
+        st_stream32(dst + 32, w + 8);
     }
     return true;
 }
 
-// grid = (ctas per partition, partitions).  Each warp walks the partition's rows with the
-// stride of all warps working on that partition, kUnroll rows per trip.
+// grid = (ctas per partition, partitions).  Each warp walks the partition's wide rows with the stride of all
+// warps working on that partition; the inputs of its next rows are on their way through the cp.async ring.
+// What is left of the partition (a last half-wide row, partial and padding rows) goes to the careful routine.
 // LEAN kernels are launched when the host proved both single-FMA decompressors and no statistics are
 // wanted (and for every block-scaled configuration); the others choose per element at run time.
 template <int GRAD, int STATE, int BITS, int MODE, bool LEAN>
 __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams P) {
-    // bytes a lane loads per row decide how many rows a trip can afford in registers
-    constexpr int kLoadWords = RowIn<GRAD, STATE>::GW + (STATE == ST_NONE ? 0 : RowIn<GRAD, STATE>::SW);
-    constexpr int kUnroll = kLoadWords <= 6 ? 4 : 2;
+    using R = Ring<GRAD, STATE, MODE>;
+    constexpr int D = R::kDepth;
+    constexpr unsigned gbytes = (GRAD == GRAD_BF16 ? 2u : 4u) * kWide;       // gradient bytes of a wide row
+    constexpr unsigned ebytes = (STATE == ST_INT8 ? 1u : 4u) * kWide;        // state bytes of a wide row
+    extern __shared__ __align__(16) uint8_t ring[];
     const int lane = threadIdx.x & 31;
     const unsigned long long part = blockIdx.y;
     const unsigned warp = blockIdx.x * kWarps + (threadIdx.x >> 5);
     const unsigned nwarps = gridDim.x * kWarps;
-    const unsigned rows = static_cast<unsigned>(P.lp / kRow);
+    const unsigned rows = static_cast<unsigned>(P.lp / kRow);                // 256-element rows of the partition
     const unsigned long long base = part * P.lp;
     // rows [0, full_rows) of this partition lie entirely below n
     unsigned full_rows = 0;
@@ -575,41 +773,61 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams
     }
     unsigned saturated = 0u;
     unsigned long long careful_acc = 0ull;
-    unsigned r = warp;
+    unsigned first_careful = 0u;             // first 256-element row left to the careful routine
     if (P.fast) {
+        const unsigned full_wide = full_rows / 2;
+        first_careful = 2 * full_wide;
         LanePtrs L;
-        L.lane_elem = static_cast<unsigned>(lane) * kLaneElems;
+        L.lane_elem = static_cast<unsigned>(lane) * kWideLane;
         L.elem0 = base + L.lane_elem;
-        L.grad = static_cast<const uint8_t *>(P.grad) + L.elem0 * (GRAD == GRAD_BF16 ? 2u : 4u);
         L.state = static_cast<uint8_t *>(P.state) + L.elem0 * (STATE == ST_INT8 ? 1u : 4u);
         uint8_t *pbase = P.comm + part * P.stride;
         L.codes = pbase + static_cast<size_t>(L.lane_elem) * BITS / 8;
         L.wire_scales = reinterpret_cast<float *>(pbase + P.code_bytes);
         L.state_scales = reinterpret_cast<float *>(static_cast<uint8_t *>(P.state) + P.state_scale_off);
+        // staging reads: chunk `lane` of each 512-byte piece of the row
+        const uint8_t *g_stage = static_cast<const uint8_t *>(P.grad) + base * (GRAD == GRAD_BF16 ? 2u : 4u) + lane * 16;
+        const uint8_t *e_stage = static_cast<const uint8_t *>(P.state) + base * (STATE == ST_INT8 ? 1u : 4u) + lane * 16;
         SendConsts K;
         K.s = P.s; K.s_e = P.s_e; K.beta = P.beta; K.omb = P.omb; K.inv_s = P.inv_s; K.inv_se = P.inv_se;
         K.dq_a = P.dq_a; K.dq_b = P.dq_b; K.de_a = P.de_a; K.de_b = P.de_b;
         K.dq_mode = P.dq_mode; K.de_mode = P.de_mode; K.block_log2 = P.block_log2; K.reset = P.reset;
         const bool stats = P.collect_stats != 0;
-        // full_rows <= rows < 2^32 - kUnroll * nwarps for every bucket this library accepts.
-        // The last trip of a warp may hold fewer than kUnroll rows: its loads are still issued together.
-        for (; r < full_rows; r += kUnroll * nwarps) {
-            RowIn<GRAD, STATE> in[kUnroll];
+        RingAddr<GRAD, STATE> A;
+        ring_addresses<GRAD, STATE, MODE>(static_cast<unsigned>(__cvta_generic_to_shared(ring)), lane, threadIdx.x >> 5, A);
+        // this warp's wide rows are warp + i * nwarps, i < cnt
+        const unsigned cnt = full_wide > warp ? (full_wide - warp + nwarps - 1) / nwarps : 0u;
+        auto stage = [&](unsigned slot_off, unsigned wrow) {
+            const float *sp = L.state_scales + ((L.elem0 + static_cast<unsigned long long>(wrow) * kWide) >> K.block_log2);
+            stage_row<GRAD, STATE, MODE>(A, slot_off, g_stage + static_cast<size_t>(wrow) * gbytes,
+                                         e_stage + static_cast<size_t>(wrow) * ebytes, sp);
+        };
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u)
-                if (u == 0 || r + u * nwarps < full_rows) load_row<GRAD, STATE, MODE>(L, r + u * nwarps, K.block_log2, in[u]);
-#pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                if (u == 0 || r + u * nwarps < full_rows) {
-                    if (!send_row_fast<GRAD, STATE, BITS, MODE, LEAN>(K, L, in[u], r + u * nwarps, lane, stats, saturated))
-                        careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(r + u * nwarps) * kRow, lane);
-                }
-            }
+        for (int i = 0; i < D - 1; ++i) {
+            if (static_cast<unsigned>(i) < cnt) stage(i * R::kSlotStride, warp + i * nwarps);
+            cp_async_commit();
         }
-        // rows of this warp at or beyond full_rows (partial or padding rows) are left to the careful routine
-        r = warp + ((full_rows > warp ? (full_rows - warp + nwarps - 1) / nwarps : 0u)) * nwarps;
+        unsigned slot_off = 0u, stage_off = (D - 1) * R::kSlotStride;
+        unsigned wrow = warp, stage_wrow = warp + (D - 1) * nwarps;
+#pragma unroll 1
+        for (unsigned i = 0; i < cnt; ++i) {
+            cp_async_wait<D - 2>();            // every group but the newest D-2 has landed: this row is there
+            __syncwarp();                      // ... for all lanes; and every lane is done reading the slot refilled next
+            WideIn<GRAD, STATE> in;
+            fetch_row<GRAD, STATE, MODE>(A, slot_off, in);
+            if (stage_wrow < full_wide) stage(stage_off, stage_wrow);
+            cp_async_commit();                 // one group per iteration, empty near the end
+            if (!send_wide_row<GRAD, STATE, BITS, MODE, LEAN>(K, L, in, wrow, lane, stats, saturated)) {
+                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(wrow) * kWide, lane);
+                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(wrow) * kWide + kRow, lane);
+            }
+            slot_off = slot_off + R::kSlotStride == R::kBytes ? 0u : slot_off + R::kSlotStride;
+            stage_off = stage_off + R::kSlotStride == R::kBytes ? 0u : stage_off + R::kSlotStride;
+            wrow += nwarps;
+            stage_wrow += nwarps;
+        }
     }
-    for (; r < rows; r += nwarps)
+    for (unsigned r = first_careful + warp; r < rows; r += nwarps)
         careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(r) * kRow, lane);
     // each careful call adds at most 8 saturated codes and 2^31 per row with a non-finite value; the 64-bit
     // sum keeps the flag apart from the count
@@ -719,19 +937,26 @@ __device__ __forceinline__ float div_workers(const ReduceParams &P, float acc) {
 // order or the format it is taken in.  The codes, biased to be non-negative, are added side by side inside
 // 32-bit words (8-bit lanes for 2- and 4-bit codes, 16-bit lanes for 8-bit codes); the lane sums S reach
 // fp32 through the mantissa of kMagic and one fused multiply-add gives (S - bias N) / s (/ N).
+// (a ^ b) & c in one instruction
+__device__ __forceinline__ unsigned xor_and(unsigned a, unsigned b, unsigned c) {
+    unsigned d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x28;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 template <int BITS>
 struct LaneSums {
     unsigned a, b, c, d;    // BITS 4: a = elements 0,2,4,6; b = 1,3,5,7.   BITS 8: a = 0,2  b = 1,3  c = 4,6  d = 5,7
     __device__ __forceinline__ void clear() { a = b = c = d = 0u; }
     __device__ __forceinline__ void add(const CodeWord<BITS> &w) {
         if (BITS == 4) {
-            a += (w.x ^ 0x88888888u) & 0x0F0F0F0Fu;
-            b += ((w.x >> 4) ^ 0x08080808u) & 0x0F0F0F0Fu;
+            a += xor_and(w.x, 0x08080808u, 0x0F0F0F0Fu);
+            b += xor_and(w.x >> 4, 0x08080808u, 0x0F0F0F0Fu);
         } else {
-            a += (w.x ^ 0x80808080u) & 0x00FF00FFu;
-            b += ((w.x >> 8) ^ 0x00800080u) & 0x00FF00FFu;
-            c += (w.y ^ 0x80808080u) & 0x00FF00FFu;
-            d += ((w.y >> 8) ^ 0x00800080u) & 0x00FF00FFu;
+            a += xor_and(w.x, 0x00800080u, 0x00FF00FFu);
+            b += xor_and(w.x >> 8, 0x00800080u, 0x00FF00FFu);
+            c += xor_and(w.y, 0x00800080u, 0x00FF00FFu);
+            d += xor_and(w.y >> 8, 0x00800080u, 0x00FF00FFu);
         }
     }
     // kMagic + S_j as a float
@@ -761,20 +986,26 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
     const int N = P.num_workers;
 
     if (MODE == MODE_FIXED && BITS != 2 && P.int_path) {
+        // code areas below 4 GiB (checked by the host): row offsets fit 32 bits
         constexpr int kUnroll = 4;
         for (unsigned r = warp; r < rows; r += kUnroll * nwarps) {
             LaneSums<BITS> sums[kUnroll];
+            unsigned off[kUnroll];
+            bool ok[kUnroll];
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) sums[u].clear();
+            for (int u = 0; u < kUnroll; ++u) {
+                sums[u].clear();
+                ok[u] = (u == 0) || (r + u * nwarps < rows);
+                off[u] = (r + u * nwarps) * kRowBytes + lane_byte;
+            }
 #pragma unroll 4
             for (int w = 0; w < N; ++w) {
-                const uint8_t *src = P.parts[w] + poff + lane_byte;
+                const uint8_t *src = P.parts[w] + poff;
                 CodeWord<BITS> cw[kUnroll];
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
                     cw[u].x = 0u; cw[u].y = 0u;
-                    if (u == 0 || r + u * nwarps < rows)
-                        load_codeword<BITS>(src + static_cast<size_t>(r + u * nwarps) * kRowBytes, cw[u]);
+                    if (ok[u]) load_codeword<BITS>(src + off[u], cw[u]);
                 }
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) sums[u].add(cw[u]);
@@ -782,7 +1013,7 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 const unsigned long long o = static_cast<unsigned long long>(r + u * nwarps) * kRow + lane_elem;
-                if ((u != 0 && r + u * nwarps >= rows) || o >= valid) continue;
+                if (!ok[u] || o >= valid) continue;
                 float res[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
