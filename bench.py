@@ -45,8 +45,11 @@ CFG = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 14, s_e=2.0 ** 16, bet
            state_fmt=0, grad_dtype=1, out_dtype=1, num_partitions=WORKERS)
 # Algorithmic HBM bytes per element (bf16 gradient read, int8 state read + written, 4-bit code written).
 SEND_BYTES_PER_ELEM = 2 + 1 + 1 + 0.5
-# DRAM bytes per element of the send kernel from the ncu capture summarised under profiles/ (None = not captured).
-SEND_DRAM_BYTES_PER_ELEM = None
+# dram__bytes_read.sum + dram__bytes_write.sum per launch (one 25M-element bucket) from the ncu captures summarised under
+# profiles/.  Reads equal the algorithmic reads; most written lines are still in the 126 MB L2 when a lone launch ends,
+# so the DRAM write counter of a single captured launch is far below the algorithmic 37.5 / 50 MB.
+SEND_DRAM_BYTES_PER_LAUNCH = 75.03e6 + 3.05e6
+REDUCE_DRAM_BYTES_PER_LAUNCH = 100.06e6 + 14.50e6
 
 
 def measured_peak():
@@ -168,15 +171,31 @@ class RankWorkload:
         self.recv_bytes = self.total * (WORKERS * 0.5 + 2)
         self.grad_bytes = 2 * self.total
 
-    def send_phase(self, k: int):
-        f = self.loco.loco_compensate_quantize_pack
-        for st, g, c in zip(self.states, self.grads, self.comms):
-            f(st, g, c, k)
+    def _fan_out(self, launch, n_items: int, streams):
+        """Issue item i on streams[i % len]: buckets are independent, so consecutive launches may overlap
+        (the next kernel's CTAs fill the SMs that the previous kernel's tail leaves idle)."""
+        if not streams:
+            for i in range(n_items):
+                launch(i, None)
+            return
+        cur = torch.cuda.current_stream()
+        for s in streams:
+            s.wait_stream(cur)
+        for i in range(n_items):
+            s = streams[i % len(streams)]
+            with torch.cuda.stream(s):
+                launch(i, s)
+        for s in streams:
+            cur.wait_stream(s)
 
-    def reduce_phase(self):
+    def send_phase(self, k: int, streams=None):
+        f = self.loco.loco_compensate_quantize_pack
+        self._fan_out(lambda i, s: f(self.states[i], self.grads[i], self.comms[i], k, stream=s), len(self.buckets), streams)
+
+    def reduce_phase(self, streams=None):
         f = self.loco.loco_unpack_dequant_reduce
-        for i, (lo, hi) in enumerate(self.buckets):
-            f(self.cfg, self.packed[i], hi - lo, self.outs[i])
+        self._fan_out(lambda i, s: f(self.cfg, self.packed[i], self.buckets[i][1] - self.buckets[i][0], self.outs[i], stream=s),
+                      len(self.buckets), streams)
 
 
 def run_e2e(wl: RankWorkload, steps: int, warmup: int):
@@ -263,6 +282,8 @@ def main():
     ap.add_argument("--buckets", type=int, default=0,
                     help="profiling aid: only the first K buckets of the workload (0 = all 270); not a bench line")
     ap.add_argument("--no-graph", action="store_true", help="profiling aid: launch every kernel directly")
+    ap.add_argument("--streams", type=int, default=2,
+                    help="streams the per-bucket launches of a phase are spread over (1 = strictly one after the other)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -270,7 +291,7 @@ def main():
     cores = os.cpu_count() or 1
     config = {"workload": "llama2-7b: 270 bf16 buckets of 25M elements (6,738,415,616): one worker's send pass per bucket, then the 8-worker reduce of the bucket",
               "bits": 4, "scale": "fixed s=2^14, s_e=4s (Eq. 1)", "beta": 0.5, "T_c": 512, "state": "int8",
-              "workers_on_reduce_side": WORKERS, "out": "bf16",
+              "workers_on_reduce_side": WORKERS, "out": "bf16", "streams": args.streams,
               "l2": "inputs larger than L2: each step streams ~70 GB once, no reuse between launches"}
 
     if args.impl == "reference":
@@ -326,11 +347,12 @@ def main():
             def __init__(self, fn): self.replay = fn
         g_send, g_reduce = _Direct(lambda: wl.send_phase(100)), _Direct(wl.reduce_phase)
     else:
+        side = [torch.cuda.Stream(device=device) for _ in range(args.streams)] if args.streams > 1 else None
         g_send, g_reduce = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
         with torch.cuda.graph(g_send):
-            wl.send_phase(100)
+            wl.send_phase(100, side)
         with torch.cuda.graph(g_reduce):
-            wl.reduce_phase()
+            wl.reduce_phase(side)
     for k in range(max(3, args.warmup)):
         g_send.replay()
         g_reduce.replay()
@@ -352,6 +374,21 @@ def main():
     barrier()
     launches = 2 * nb * K          # one send and one receive kernel per bucket and step, replayed from the graphs
     clocks = sampler.stop()
+    # outside the timed region: the same two phases with every launch strictly after the previous one (one stream),
+    # which shows what a launch costs when nothing overlaps its start-up and its tail
+    serial_us = None
+    if not args.no_graph and args.streams > 1:
+        s_send, s_reduce = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(s_send):
+            wl.send_phase(100, None)
+        with torch.cuda.graph(s_reduce):
+            wl.reduce_phase(None)
+        s_send.replay(); s_reduce.replay()
+        sev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        torch.cuda.synchronize()
+        sev[0].record(); s_send.replay(); s_send.replay(); sev[1].record(); s_reduce.replay(); s_reduce.replay(); sev[2].record()
+        torch.cuda.synchronize()
+        serial_us = (sev[0].elapsed_time(sev[1]) * 1e3 / (2 * nb), sev[1].elapsed_time(sev[2]) * 1e3 / (2 * nb))
     total_ms = start.elapsed_time(end)
     send_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / K
     recv_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
@@ -384,17 +421,31 @@ def main():
     peak, peak_kind = measured_peak()
     send_gbs = wl.send_bytes / (send_ms * 1e-3) / 1e9
     recv_gbs = wl.recv_bytes / (recv_ms * 1e-3) / 1e9
-    roofline = {"kernel": "loco_send_kernel<bf16, int8 state, 4 bit, fixed scale>", "bound": "hbm",
-                "achieved": send_gbs, "peak": peak, "peak_kind": "%s HBM copy bandwidth" % peak_kind, "unit": "GB/s",
-                "frac": send_gbs / peak, "frac_of_nominal_8TBps": send_gbs / 8000.0,
-                "traffic": (SEND_DRAM_BYTES_PER_ELEM * BUCKET if SEND_DRAM_BYTES_PER_ELEM else None),
-                "algorithmic_bytes_per_launch": SEND_BYTES_PER_ELEM * BUCKET, "avg_launch_us": send_ms * 1e3 / nb,
-                "launches_per_step": nb}
+    how = ("CUDA events around this kernel's phase of every timed step / launches in it; the launches of a phase "
+           "alternate between %d streams, so a kernel's start-up and tail overlap its neighbour" % max(1, args.streams))
+    roof_send = {"kernel": "loco_send_kernel<bf16 g, int8 state, 4 bit, fixed scale>", "bound": "hbm",
+                 "achieved": send_gbs, "peak": peak, "peak_kind": "%s HBM copy bandwidth" % peak_kind, "unit": "GB/s",
+                 "frac": send_gbs / peak, "frac_of_nominal_8TBps": send_gbs / 8000.0, "traffic": SEND_DRAM_BYTES_PER_LAUNCH,
+                 "algorithmic_bytes_per_launch": SEND_BYTES_PER_ELEM * BUCKET, "avg_launch_us": send_ms * 1e3 / nb,
+                 "launches_per_step": nb, "how": how}
+    roof_reduce = {"kernel": "loco_reduce_kernel<bf16 out, 4 bit, fixed scale>, 8 workers", "bound": "hbm",
+                   "achieved": recv_gbs, "peak": peak, "peak_kind": "%s HBM copy bandwidth" % peak_kind, "unit": "GB/s",
+                   "frac": recv_gbs / peak, "frac_of_nominal_8TBps": recv_gbs / 8000.0, "traffic": REDUCE_DRAM_BYTES_PER_LAUNCH,
+                   "algorithmic_bytes_per_launch": (WORKERS * 0.5 + 2) * BUCKET, "avg_launch_us": recv_ms * 1e3 / nb,
+                   "launches_per_step": nb, "how": how}
+    # the roofline object describes the kernel that takes the larger share of the step; the other one rides along
+    roofline, other = (roof_reduce, roof_send) if recv_ms >= send_ms else (roof_send, roof_reduce)
+    roofline["other_kernel"] = other
     kernels = {"send": {"hbm_gbs": send_gbs, "frac_of_peak": send_gbs / peak, "gradient_gbs": wl.grad_bytes / (send_ms * 1e-3) / 1e9,
                         "ms_per_step": send_ms, "avg_launch_us": send_ms * 1e3 / nb, "bytes_per_elem": SEND_BYTES_PER_ELEM},
                "reduce": {"hbm_gbs": recv_gbs, "frac_of_peak": recv_gbs / peak,
                           "gradient_gbs": wl.grad_bytes / (recv_ms * 1e-3) / 1e9, "ms_per_step": recv_ms,
                           "avg_launch_us": recv_ms * 1e3 / nb, "bytes_per_out_elem": WORKERS * 0.5 + 2}}
+    if serial_us is not None:
+        kernels["send"]["one_stream_launch_us"] = serial_us[0]
+        kernels["send"]["one_stream_hbm_gbs"] = wl.send_bytes / nb / (serial_us[0] * 1e-6) / 1e9
+        kernels["reduce"]["one_stream_launch_us"] = serial_us[1]
+        kernels["reduce"]["one_stream_hbm_gbs"] = wl.recv_bytes / nb / (serial_us[1] * 1e-6) / 1e9
     cpu = None
     if not args.no_cpu_baseline:
         v, dt, elems = oracle_sample(cores, 2)
