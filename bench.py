@@ -270,6 +270,143 @@ def oracle_sample(threads: int, buckets_per_thread: int):
     return 2.0 * elems / dt / 1e9, dt, elems
 
 
+# ------------------------------------------------------------------------------------------------ sweep (config 5)
+
+def _time_launches(launch, n_sets: int, launches: int, streams):
+    """Average device time of `launch(set_index, stream)` over `launches` launches that walk round-robin over n_sets
+    independent working sets and alternate between the streams (CUDA events on the current stream around all)."""
+    def run(count):
+        cur = torch.cuda.current_stream()
+        for st in streams:
+            st.wait_stream(cur)
+        for i in range(count):
+            st = streams[i % len(streams)]
+            with torch.cuda.stream(st):
+                launch(i % n_sets, st)
+        for st in streams:
+            cur.wait_stream(st)
+
+    run(min(launches, 2 * n_sets))
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()                       # replayed, so that the host's launch cost is not what is timed
+    with torch.cuda.graph(graph):
+        run(launches)
+    graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / launches          # microseconds
+
+
+def sweep(args, device):
+    """Throughput table over bucket size, gradient type, state format, code width, scale rule and worker count
+    (Gaussian gradients, seed 4).  Every launch touches a working set that the previous launches did not leave in L2
+    unless the row says so."""
+    from paper_2407_04480_b200 import inputs, loco
+    peak, peak_kind = measured_peak()
+    streams = [torch.cuda.Stream(device=device) for _ in range(max(1, args.streams))]
+    rows = []
+    budget = 6 << 30                    # device bytes per case
+
+    def sets_for(bytes_per_set):
+        want = max(3, -(-(1 << 30) // bytes_per_set))
+        return int(max(1, min(want, 256, budget // max(1, bytes_per_set))))
+
+    def send_case(label, n, **kw):
+        base = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=512, state_fmt=0,
+                    grad_dtype=1, out_dtype=1, num_partitions=8)
+        base.update(kw)
+        cfg = loco.Config(**base)
+        gsz = 2 if cfg.grad_dtype == loco.BF16 else 4
+        sb, pb = loco.loco_state_bytes(cfg, n), loco.loco_packed_bytes(cfg, n)
+        nsets = sets_for(n * gsz + sb + pb)
+        dt = torch.bfloat16 if gsz == 2 else torch.float32
+        grads = [inputs.gaussian(n, 1e-3, seed=4, worker=i, dtype=dt, device=device) for i in range(nsets)]
+        states = [loco.State(cfg, n) for _ in range(nsets)]
+        comms = [torch.empty(max(pb, 16), dtype=torch.uint8, device=device) for _ in range(nsets)]
+        for i in range(nsets):                      # a first iteration, so that the timed ones meet a non-zero state
+            loco.loco_compensate_quantize_pack(states[i], grads[i], comms[i], 1)
+        torch.cuda.synchronize()
+        us = _time_launches(lambda i, st: loco.loco_compensate_quantize_pack(states[i], grads[i], comms[i], 2, stream=st),
+                            nsets, max(12, min(200, 4 * nsets)), streams)
+        state_rw = {0: 2, 1: 8, 2: 0, 3: 8}[cfg.state_fmt]
+        scale_b = (4.0 / cfg.block_size) * (3 if cfg.state_fmt == 0 else 1) if cfg.scale_mode == 1 else 0.0
+        bpe = gsz + state_rw + cfg.bits / 8 + scale_b
+        gbs = bpe * n / us / 1e3
+        rows.append(dict(kernel="send", case=label, n=n, bytes_per_elem=round(bpe, 3), us=round(us, 2), hbm_gbs=round(gbs, 1),
+                         frac=round(gbs / peak, 3), grad_gbs=round(gsz * n / us / 1e3, 1),
+                         l2_resident=bool(nsets * (n * gsz + sb + pb) < L2_BYTES)))
+        print(json.dumps(rows[-1]), flush=True)
+
+    def reduce_case(label, n, workers, **kw):
+        base = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=512, state_fmt=2,
+                    grad_dtype=1, out_dtype=1, num_partitions=8)
+        base.update(kw)
+        cfg = loco.Config(**base)
+        osz = 2 if cfg.out_dtype == loco.BF16 else 4
+        pb = loco.loco_packed_bytes(cfg, n)
+        nsets = sets_for(workers * pb + n * osz)
+        gen = torch.Generator(device=device)
+        gen.manual_seed(4)
+        packed = []
+        for i in range(nsets):
+            if cfg.scale_mode == 1:                 # block scales must be real numbers: compress real gradients
+                bufs = []
+                for w in range(workers):
+                    st = loco.State(cfg, n)
+                    c = torch.empty(max(pb, 16), dtype=torch.uint8, device=device)
+                    loco.loco_compensate_quantize_pack(st, inputs.gaussian(n, 1e-3, seed=4, worker=w, step=i, dtype=torch.bfloat16, device=device), c, 1)
+                    bufs.append(c)
+                packed.append(bufs)
+            else:
+                packed.append([torch.randint(0, 256, (max(pb, 16),), dtype=torch.uint8, device=device, generator=gen) for _ in range(workers)])
+        outs = [torch.empty(n, dtype=torch.bfloat16 if osz == 2 else torch.float32, device=device) for _ in range(nsets)]
+        torch.cuda.synchronize()
+        us = _time_launches(lambda i, st: loco.loco_unpack_dequant_reduce(cfg, packed[i], n, outs[i], stream=st),
+                            nsets, max(12, min(200, 4 * nsets)), streams)
+        bpe = workers * cfg.bits / 8 + osz + (workers * 4.0 / cfg.block_size if cfg.scale_mode == 1 else 0.0)
+        gbs = bpe * n / us / 1e3
+        rows.append(dict(kernel="reduce", case=label, n=n, workers=workers, bytes_per_elem=round(bpe, 3), us=round(us, 2),
+                         hbm_gbs=round(gbs, 1), frac=round(gbs / peak, 3), grad_gbs=round(osz * n / us / 1e3, 1),
+                         l2_resident=bool(nsets * (workers * pb + n * osz) < L2_BYTES)))
+        print(json.dumps(rows[-1]), flush=True)
+
+    M = 25_000_000
+    for log2n in (16, 18, 20, 22, 24, 27, 30):
+        send_case("bf16 g, int8 state, 4 bit, fixed", 1 << log2n)
+    for log2n in (16, 20, 24, 27, 30):
+        send_case("fp32 g, int8 state, 4 bit, fixed", 1 << log2n, grad_dtype=0)
+    for bits in (2, 4, 8):
+        send_case("bf16 g, int8 state, %d bit, fixed" % bits, M, bits=bits)
+        send_case("fp32 g, int8 state, %d bit, fixed" % bits, M, bits=bits, grad_dtype=0)
+    send_case("bf16 g, int8 state, 4 bit, fixed, s_e = 6 s (Newton-Raphson decompressor)", M, s_e=6 * 2.0 ** 11)
+    send_case("bf16 g, int8 state, 4 bit, fixed, statistics on", M, collect_stats=1)
+    send_case("bf16 g, fp32 state, 4 bit, fixed", M, state_fmt=1)
+    send_case("bf16 g, fp32 state + 8-bit compensation, 4 bit, fixed", M, state_fmt=3)
+    send_case("bf16 g, no state, 4 bit, fixed", M, state_fmt=2)
+    for B in (256, 64, 32):
+        send_case("bf16 g, int8 state, 4 bit, block-%d absmax" % B, M, scale_mode=1, block_size=B)
+    send_case("fp32 g, int8 state, 4 bit, block-256 absmax", M, scale_mode=1, grad_dtype=0)
+    for log2n in (16, 20, 24, 27, 30):
+        reduce_case("4 bit, bf16 out, fixed", 1 << log2n, 8)
+    for bits in (2, 4, 8):
+        for od in (1, 0):
+            for N in (1, 2, 4, 8, 16):
+                reduce_case("%d bit, %s out, fixed" % (bits, "bf16" if od else "fp32"), M, N, bits=bits, out_dtype=od)
+    reduce_case("4 bit, bf16 out, fixed, s = 3000 (generic path)", M, 8, s=3000.0)
+    reduce_case("4 bit, bf16 out, fixed, 3 workers (division by 3)", M, 3)
+    reduce_case("4 bit, bf16 out, block-256 absmax", M, 8, scale_mode=1)
+    reduce_case("4 bit, bf16 out, block-32 absmax", M, 8, scale_mode=1, block_size=32)
+    print("| kernel | case | n | workers | B/elem | us/launch | HBM GB/s | of %s peak %.0f | gradient GB/s | L2-resident |" % (peak_kind, peak))
+    print("|---|---|---|---|---|---|---|---|---|---|")
+    for r in rows:
+        print("| %s | %s | %d | %s | %s | %s | %s | %.3f | %s | %s |" % (r["kernel"], r["case"], r["n"], r.get("workers", "-"), r["bytes_per_elem"],
+                                                                      r["us"], r["hbm_gbs"], r["frac"], r["grad_gbs"], "yes" if r["l2_resident"] else ""))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -282,6 +419,8 @@ def main():
     ap.add_argument("--buckets", type=int, default=0,
                     help="profiling aid: only the first K buckets of the workload (0 = all 270); not a bench line")
     ap.add_argument("--no-graph", action="store_true", help="profiling aid: launch every kernel directly")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the bench line: the size / type / width / worker-count table (one JSON line per case, then markdown)")
     ap.add_argument("--streams", type=int, default=2,
                     help="streams the per-bucket launches of a phase are spread over (1 = strictly one after the other)")
     args = ap.parse_args()
@@ -333,6 +472,10 @@ def main():
 
     from paper_2407_04480_b200 import loco
     loco.lib()
+    if args.sweep:
+        if rank == 0:
+            sweep(args, device)
+        return
     wl = RankWorkload(rank, device, args.buckets)
     nb = len(wl.buckets)
     if args.buckets > 0:
