@@ -316,6 +316,8 @@ def sweep(args, device):
         return int(max(1, min(want, 256, budget // max(1, bytes_per_set))))
 
     def send_case(label, n, **kw):
+        if args.sweep_filter and args.sweep_filter not in "send: " + label:
+            return
         base = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=512, state_fmt=0,
                     grad_dtype=1, out_dtype=1, num_partitions=8)
         base.update(kw)
@@ -342,6 +344,8 @@ def sweep(args, device):
         print(json.dumps(rows[-1]), flush=True)
 
     def reduce_case(label, n, workers, **kw):
+        if args.sweep_filter and args.sweep_filter not in "reduce: " + label:
+            return
         base = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=512, state_fmt=2,
                     grad_dtype=1, out_dtype=1, num_partitions=8)
         base.update(kw)
@@ -421,6 +425,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="profiling aid: launch every kernel directly")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the bench line: the size / type / width / worker-count table (one JSON line per case, then markdown)")
+    ap.add_argument("--sweep-filter", default="", help="with --sweep: only the cases whose 'kernel: label' contains this text")
     ap.add_argument("--streams", type=int, default=2,
                     help="streams the per-bucket launches of a phase are spread over (1 = strictly one after the other)")
     args = ap.parse_args()

@@ -194,21 +194,22 @@ SendKernel pick_send(const loco_config_t *c, int mode, bool lean) {
 using ReduceFn = void (*)(const ReduceParams);
 
 template <int OUT, int BITS>
-ReduceFn pick_reduce_mode(int mode) {
-    if (mode == MODE_FIXED) return loco_reduce_kernel<OUT, BITS, MODE_FIXED>;
-    return loco_reduce_kernel<OUT, BITS, MODE_BLOCK>;
+ReduceFn pick_reduce_mode(int mode, bool int_path) {
+    if (mode == MODE_FIXED)
+        return int_path ? loco_reduce_kernel<OUT, BITS, MODE_FIXED, true> : loco_reduce_kernel<OUT, BITS, MODE_FIXED, false>;
+    return loco_reduce_kernel<OUT, BITS, MODE_BLOCK, false>;
 }
 template <int OUT>
-ReduceFn pick_reduce_bits(int bits, int mode) {
+ReduceFn pick_reduce_bits(int bits, int mode, bool int_path) {
     switch (bits) {
-    case 2: return pick_reduce_mode<OUT, 2>(mode);
-    case 4: return pick_reduce_mode<OUT, 4>(mode);
-    default: return pick_reduce_mode<OUT, 8>(mode);
+    case 2: return pick_reduce_mode<OUT, 2>(mode, int_path);
+    case 4: return pick_reduce_mode<OUT, 4>(mode, int_path);
+    default: return pick_reduce_mode<OUT, 8>(mode, int_path);
     }
 }
-ReduceFn pick_reduce(const loco_config_t *c, int mode) {
-    return c->out_dtype == LOCO_BF16 ? pick_reduce_bits<GRAD_BF16>(c->bits, mode)
-                                     : pick_reduce_bits<GRAD_F32>(c->bits, mode);
+ReduceFn pick_reduce(const loco_config_t *c, int mode, bool int_path) {
+    return c->out_dtype == LOCO_BF16 ? pick_reduce_bits<GRAD_BF16>(c->bits, mode, int_path)
+                                     : pick_reduce_bits<GRAD_F32>(c->bits, mode, int_path);
 }
 
 unsigned grid_x_for(uint64_t rows_per_partition, int partitions, int ctas_per_sm) {
@@ -452,16 +453,34 @@ int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_pa
     const bool n_pow2 = is_pow2(static_cast<uint64_t>(num_workers));
     P.div_mode = n_pow2 ? 0 : 2;          // a multiply by 1/N is the division only for powers of two
     P.gen_mul = 0.0f;
+    P.gen_mode = 2;
+    P.inv_s = 0.0f;
     P.int_path = 0;
+    P.out_align32 = (reinterpret_cast<uintptr_t>(d_out) & 31u) == 0 ? 1 : 0;
     if (mode == MODE_FIXED) {
         const int half = 1 << (cfg->bits - 1);
-        if (reciprocal_exact(cfg->s, -half, half - 1)) {
-            const volatile float inv = 1.0f / cfg->s;
-            P.gen_mul = inv;
+        {
+            const volatile float vinv = 1.0f / cfg->s;
+            const float inv = vinv;
+            P.inv_s = inv;
+            if (reciprocal_exact(cfg->s, -half, half - 1)) {
+                P.gen_mul = inv;
+                P.gen_mode = 0;
+            } else if (std::isfinite(inv) && inv != 0.0f) {
+                bool nr_ok = true;
+                for (int q = -half; q < half && nr_ok; ++q) {
+                    const float fq = static_cast<float>(q);
+                    const volatile float want = fq / cfg->s;
+                    const volatile float q0 = fq * inv;
+                    const float rem = std::fmaf(q0, -cfg->s, fq);
+                    nr_ok = same_bits(std::fmaf(rem, inv, q0), want);
+                }
+                if (nr_ok) P.gen_mode = 1;
+            }
         }
         // Integer path: with s a power of two every partial sum of Eq. 8 is exact in fp32, so the codes can be
         // added as integers.  The lane sums are bounded by (2^p - 1) * N, which 8- and 16-bit lanes hold for N <= 16.
-        if (cfg->bits != 2 && num_workers <= 16 && is_pow2_float(cfg->s) && L.code_bytes < (1ull << 32)) {
+        if (num_workers <= 16 && is_pow2_float(cfg->s) && L.code_bytes < (1ull << 32)) {
             P.int_path = 1;
             const float inv_s = 1.0f / cfg->s;                                    // exact
             float ra = inv_s;
@@ -482,9 +501,9 @@ int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_pa
             }
         }
     }
-    ReduceFn fn = pick_reduce(cfg, mode);
-    static int occ_cache[2][3][2] = {};
-    int &occ = occ_cache[cfg->out_dtype == LOCO_BF16][cfg->bits == 2 ? 0 : (cfg->bits == 4 ? 1 : 2)][mode];
+    ReduceFn fn = pick_reduce(cfg, mode, P.int_path != 0);
+    static int occ_cache[2][3][2][2] = {};
+    int &occ = occ_cache[cfg->out_dtype == LOCO_BF16][cfg->bits == 2 ? 0 : (cfg->bits == 4 ? 1 : 2)][mode][P.int_path != 0];
     if (occ == 0) {
         int v = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, fn, kThreads, 0) != cudaSuccess || v < 1) {
@@ -493,7 +512,7 @@ int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_pa
         }
         occ = v;
     }
-    const uint64_t rows = L.lp / kRow;
+    const uint64_t rows = (L.lp + kWide - 1) / kWide;
     dim3 grid(grid_x_for(rows, partition_count, occ), static_cast<unsigned>(partition_count), 1);
     fn<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(P);
     if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;

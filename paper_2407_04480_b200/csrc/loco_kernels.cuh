@@ -80,7 +80,10 @@ struct ReduceParams {
     int int_path;                    // codes may be summed as integers (power-of-two s, N <= 16)
     float ra, rb;                    // int path: sum/s (and /N when exact) = fma(kMagic + S, ra, rb)
     int div_mode;                    // division by N: 0 folded into ra/rb or a multiply, 1 Newton-Raphson, 2 IEEE
-    float gen_mul;                   // generic FIXED path: multiplier that reproduces q/s, 0 if division is needed
+    float gen_mul;                   // generic FIXED path, gen_mode 0: fl(1/s), which reproduces q/s for every code
+    float inv_s;                     // fl(1/s) for gen_mode 1
+    int gen_mode;                    // generic FIXED path: 0 multiply, 1 Newton-Raphson division, 2 IEEE division
+    int out_align32;                 // the output pointer is 32-byte aligned: 256-bit stores may be used
 };
 
 // ------------------------------------------------------------------------------------------
@@ -740,9 +743,9 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             w[2 * k] = K.reset ? 0u : static_cast<unsigned>(en2[k]);
             w[2 * k + 1] = K.reset ? 0u : static_cast<unsigned>(en2[k] >> 32);
         }
-        uint8_t *dst = L.state + static_cast<size_t>(wrow) * (4u * kWide);
-        st_stream32(dst, w);
-        st_stream32(dst + 32, w + 8);
+        uint8_t *dst = L.state + static_cast<size_t>(wrow) * (4u * kWide);   // 16-byte aligned by contract, not more
+#pragma unroll
+        for (int j = 0; j < 4; ++j) st_stream16(dst + 16 * j, make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]));
     }
     return true;
 }
@@ -844,47 +847,48 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams
 }
 
 // ------------------------------------------------------------------------------------------
-// receive: Eq. 8 on warp rows of 256 outputs, 8 per lane.
+// receive: Eq. 8 on wide rows of 512 outputs, 16 per lane.
 
-template <int BITS> struct CodeWord { unsigned x, y; };   // the 8 codes of one lane and row, as loaded (y: 8-bit only)
+template <int BITS> struct WideCodes {                       // the 16 codes of one lane and wide row, as loaded
+    static constexpr int W = BITS / 2;                       // 32-bit words: 1, 2 or 4
+    unsigned w[W];
+};
 
 template <int BITS>
-__device__ __forceinline__ void load_codeword(const uint8_t *src, CodeWord<BITS> &w) {
-    w.y = 0u;
-    if (BITS == 8) { const uint2 t = ld_stream8(src); w.x = t.x; w.y = t.y; }
-    else if (BITS == 4) w.x = ld_stream4(src);
-    else w.x = static_cast<unsigned>(__ldcs(reinterpret_cast<const unsigned short *>(src)));
+__device__ __forceinline__ void load_codes(const uint8_t *src, WideCodes<BITS> &c) {
+    if (BITS == 8) { const uint4 t = ld_stream16(src); c.w[0] = t.x; c.w[1 % WideCodes<BITS>::W] = t.y; c.w[2 % WideCodes<BITS>::W] = t.z; c.w[3 % WideCodes<BITS>::W] = t.w; }
+    else if (BITS == 4) { const uint2 t = ld_stream8(src); c.w[0] = t.x; c.w[1 % WideCodes<BITS>::W] = t.y; }
+    else c.w[0] = ld_stream4(src);
 }
 
-// The 8 codes as exact floats.  Each field, with its top bit flipped (code + 2^(p-1)), is masked in place
-// into the mantissa of a power of two chosen so that the field's lowest bit weighs 1; subtracting that
-// power of two and the bias leaves the code.
+// (a & b) | c in one instruction (the mask and the exponent live in registers)
+__device__ __forceinline__ unsigned and_or(unsigned a, unsigned b, unsigned c) {
+    unsigned d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+// The magic float 2^e + (code + 2^(p-1)) of field j: the field, with its top bit already flipped in x, is masked in
+// place into the mantissa of a power of two chosen so that the field's lowest bit weighs 1.  `k` receives that
+// power of two plus the bias, i.e. what has to be subtracted to leave the code.
 template <int BITS>
-__device__ __forceinline__ void codes_to_float(const CodeWord<BITS> &w, float (&q)[8]) {
+__device__ __forceinline__ float field_magic(const unsigned (&x)[WideCodes<BITS>::W], const unsigned (&xh)[WideCodes<BITS>::W], int j, float &k) {
     if (BITS == 8) {
-        const unsigned x0 = w.x ^ 0x80808080u, x1 = w.y ^ 0x80808080u;
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-            q[j] = __fadd_rn(__uint_as_float(__byte_perm(j < 4 ? x0 : x1, 0x4B000000u, 0x7650 + (j & 3))), -(8388608.0f + 128.0f));
+        k = 8388608.0f + 128.0f;
+        return __uint_as_float(__byte_perm(x[(j >> 2) % WideCodes<BITS>::W], 0x4B000000u, 0x7650 + (j & 3)));
     } else if (BITS == 4) {
-        const unsigned x = w.x ^ 0x88888888u;
-        const unsigned xh = x >> 12;                         // fields 5..7 moved to positions 2..4
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int pos = j < 5 ? j : j - 3;               // field position inside the word used
-            const unsigned src = j < 5 ? x : xh;
-            const unsigned expo = static_cast<unsigned>(127 + 23 - 4 * pos) << 23;        // 2^(23 - 4 pos)
-            const float m = __uint_as_float((src & (0xFu << (4 * pos))) | expo);
-            q[j] = __fadd_rn(m, -(__uint_as_float(expo) + 8.0f));
-        }
+        const int jj = j & 7;
+        const int pos = jj < 5 ? jj : jj - 3;                // fields 5..7 are taken from the word shifted right by 12
+        const unsigned src = jj < 5 ? x[(j >> 3) % WideCodes<BITS>::W] : xh[(j >> 3) % WideCodes<BITS>::W];
+        const unsigned expo = static_cast<unsigned>(127 + 23 - 4 * pos) << 23;        // 2^(23 - 4 pos)
+        k = __uint_as_float(expo) + 8.0f;
+        return __uint_as_float(and_or(src, 0xFu << (4 * pos), expo));
     } else {
-        const unsigned x = w.x ^ 0xAAAAu;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const unsigned expo = static_cast<unsigned>(127 + 23 - 2 * j) << 23;
-            const float m = __uint_as_float((x & (0x3u << (2 * j))) | expo);
-            q[j] = __fadd_rn(m, -(__uint_as_float(expo) + 2.0f));
-        }
+        const int pos = j < 11 ? j : j - 8;                  // fields 11..15 are taken from the word shifted right by 16
+        const unsigned src = j < 11 ? x[0] : xh[0];
+        const unsigned expo = static_cast<unsigned>(127 + 23 - 2 * pos) << 23;
+        k = __uint_as_float(expo) + 2.0f;
+        return __uint_as_float(and_or(src, 0x3u << (2 * pos), expo));
     }
 }
 
@@ -895,22 +899,38 @@ __device__ __forceinline__ unsigned pack_bf16x2_rn(float a, float b) {
     return r;
 }
 
+// 16 results of one lane to out[oi ..]; `left` = elements that exist from oi on; wide32: out + oi is 32-byte aligned.
 template <int OUT>
-__device__ __forceinline__ void store_out8(void *out, unsigned long long oi, const float (&res)[8], unsigned long long left) {
-    if (left >= 8) {
+__device__ __forceinline__ void store_out16(void *out, unsigned long long oi, const float (&res)[16], unsigned long long left, bool wide32) {
+    if (left >= 16) {
         if (OUT == GRAD_BF16) {
-            st_stream16(static_cast<uint16_t *>(out) + oi,
-                        make_uint4(pack_bf16x2_rn(res[0], res[1]), pack_bf16x2_rn(res[2], res[3]),
-                                   pack_bf16x2_rn(res[4], res[5]), pack_bf16x2_rn(res[6], res[7])));
+            unsigned w[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[j] = pack_bf16x2_rn(res[2 * j], res[2 * j + 1]);
+            uint16_t *dst = static_cast<uint16_t *>(out) + oi;
+            if (wide32) {
+                st_stream32(dst, w);
+            } else {
+                st_stream16(dst, make_uint4(w[0], w[1], w[2], w[3]));
+                st_stream16(dst + 8, make_uint4(w[4], w[5], w[6], w[7]));
+            }
         } else {
+            unsigned w[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) w[j] = __float_as_uint(res[j]);
             float *dst = static_cast<float *>(out) + oi;
-            st_stream16(dst, make_uint4(__float_as_uint(res[0]), __float_as_uint(res[1]), __float_as_uint(res[2]), __float_as_uint(res[3])));
-            st_stream16(dst + 4, make_uint4(__float_as_uint(res[4]), __float_as_uint(res[5]), __float_as_uint(res[6]), __float_as_uint(res[7])));
+            if (wide32) {
+                st_stream32(dst, w);
+                st_stream32(dst + 8, w + 8);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) st_stream16(dst + 4 * j, make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]));
+            }
         }
     } else {
         const int cnt = static_cast<int>(left);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
+        for (int j = 0; j < 16; ++j) {
             if (j < cnt) {
                 if (OUT == GRAD_BF16)
                     static_cast<uint16_t *>(out)[oi + j] = static_cast<uint16_t>(pack_bf16x2_rn(res[j], 0.0f) & 0xffffu);
@@ -932,11 +952,6 @@ __device__ __forceinline__ float div_workers(const ReduceParams &P, float acc) {
     return __fdiv_rn(acc, P.n_workers_f);
 }
 
-// Integer path (global power-of-two s, at most 16 workers): every dec(q; s) and every partial sum of Eq. 8
-// is an integer multiple of 1/s that fp32 holds exactly, so the sum over workers does not depend on the
-// order or the format it is taken in.  The codes, biased to be non-negative, are added side by side inside
-// 32-bit words (8-bit lanes for 2- and 4-bit codes, 16-bit lanes for 8-bit codes); the lane sums S reach
-// fp32 through the mantissa of kMagic and one fused multiply-add gives (S - bias N) / s (/ N).
 // (a ^ b) & c in one instruction
 __device__ __forceinline__ unsigned xor_and(unsigned a, unsigned b, unsigned c) {
     unsigned d;
@@ -944,32 +959,50 @@ __device__ __forceinline__ unsigned xor_and(unsigned a, unsigned b, unsigned c) 
     return d;
 }
 
+// Integer path (global power-of-two s, at most 16 workers): every dec(q; s) and every partial sum of Eq. 8
+// is an integer multiple of 1/s that fp32 holds exactly, so the sum over workers does not depend on the
+// order or the format it is taken in.  The codes, biased to be non-negative, are added side by side inside
+// 32-bit words (8-bit lanes for 2- and 4-bit codes, 16-bit lanes for 8-bit codes); the lane sums S reach
+// fp32 through the mantissa of kMagic and one fused multiply-add gives (S - bias N) / s (/ N).
 template <int BITS>
-struct LaneSums {
-    unsigned a, b, c, d;    // BITS 4: a = elements 0,2,4,6; b = 1,3,5,7.   BITS 8: a = 0,2  b = 1,3  c = 4,6  d = 5,7
-    __device__ __forceinline__ void clear() { a = b = c = d = 0u; }
-    __device__ __forceinline__ void add(const CodeWord<BITS> &w) {
-        if (BITS == 4) {
-            a += xor_and(w.x, 0x08080808u, 0x0F0F0F0Fu);
-            b += xor_and(w.x >> 4, 0x08080808u, 0x0F0F0F0Fu);
-        } else {
-            a += xor_and(w.x, 0x00800080u, 0x00FF00FFu);
-            b += xor_and(w.x >> 8, 0x00800080u, 0x00FF00FFu);
-            c += xor_and(w.y, 0x00800080u, 0x00FF00FFu);
-            d += xor_and(w.y >> 8, 0x00800080u, 0x00FF00FFu);
+struct WideSums {
+    static constexpr int S = (BITS == 8) ? 8 : 4;
+    unsigned s[S];
+    __device__ __forceinline__ void clear() {
+#pragma unroll
+        for (int i = 0; i < S; ++i) s[i] = 0u;
+    }
+    __device__ __forceinline__ void add(const WideCodes<BITS> &c) {
+        if (BITS == 4) {            // s[2h] holds elements 8h + {0,2,4,6}, s[2h+1] elements 8h + {1,3,5,7}
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                s[(2 * h) % S] += xor_and(c.w[h % WideCodes<BITS>::W], 0x08080808u, 0x0F0F0F0Fu);
+                s[(2 * h + 1) % S] += xor_and(c.w[h % WideCodes<BITS>::W] >> 4, 0x08080808u, 0x0F0F0F0Fu);
+            }
+        } else if (BITS == 8) {     // s[2h] holds elements 4h + {0,2}, s[2h+1] elements 4h + {1,3}, in 16-bit lanes
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                s[(2 * h) % S] += xor_and(c.w[h % WideCodes<BITS>::W], 0x00800080u, 0x00FF00FFu);
+                s[(2 * h + 1) % S] += xor_and(c.w[h % WideCodes<BITS>::W] >> 8, 0x00800080u, 0x00FF00FFu);
+            }
+        } else {                    // byte b of s[k] holds element 4b + k
+#pragma unroll
+            for (int k = 0; k < 4; ++k) s[k % S] += xor_and(c.w[0] >> (2 * k), 0x02020202u, 0x03030303u);
         }
     }
     // kMagic + S_j as a float
     __device__ __forceinline__ float get(int j) const {
-        if (BITS == 4) return __uint_as_float(__byte_perm((j & 1) ? b : a, kMagicBits, 0x7650 + (j >> 1)));
-        const unsigned src = j < 4 ? ((j & 1) ? b : a) : ((j & 1) ? d : c);
-        return __uint_as_float(__byte_perm(src, kMagicBits, ((j >> 1) & 1) ? 0x7632 : 0x7610));
+        if (BITS == 4) return __uint_as_float(__byte_perm(s[(2 * (j >> 3) + (j & 1)) % S], kMagicBits, 0x7650 + ((j & 7) >> 1)));
+        if (BITS == 8) return __uint_as_float(__byte_perm(s[(2 * (j >> 2) + (j & 1)) % S], kMagicBits, ((j & 3) >> 1) ? 0x7632 : 0x7610));
+        return __uint_as_float(__byte_perm(s[(j & 3) % S], kMagicBits, 0x7650 + (j >> 2)));
     }
 };
 
-template <int OUT, int BITS, int MODE>
+// INT: the integer-sum path (only with the global scale); otherwise the generic path.  Two kernels, so that each path
+// gets the registers and the occupancy it wants.
+template <int OUT, int BITS, int MODE, bool INT>
 __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParams P) {
-    constexpr unsigned kRowBytes = kRow * BITS / 8;                   // code bytes of one row
+    constexpr unsigned kRowBytes = kWide * BITS / 8;                  // code bytes of one wide row
     const int lane = threadIdx.x & 31;
     const unsigned long long part = blockIdx.y;                       // relative to P.first
     const unsigned warp = blockIdx.x * kWarps + (threadIdx.x >> 5);
@@ -978,99 +1011,140 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
     if (base >= P.n) return;
     const unsigned long long avail = P.n - base;
     const unsigned long long valid = avail >= P.lp ? P.lp : avail;
-    const unsigned rows = static_cast<unsigned>((valid + kRow - 1) / kRow);
+    const unsigned rows = static_cast<unsigned>((valid + kWide - 1) / kWide);
     const unsigned long long poff = part * P.stride;
     const unsigned long long out0 = part * P.lp;                      // output index of the part's first element
-    const unsigned lane_elem = static_cast<unsigned>(lane) * kLaneElems;
+    const unsigned lane_elem = static_cast<unsigned>(lane) * kWideLane;
     const unsigned lane_byte = lane_elem * BITS / 8;
     const int N = P.num_workers;
+    const bool wide32 = P.out_align32 != 0;
 
-    if (MODE == MODE_FIXED && BITS != 2 && P.int_path) {
+    if (INT) {
         // code areas below 4 GiB (checked by the host): row offsets fit 32 bits
-        constexpr int kUnroll = 4;
+        constexpr int kUnroll = 2;
         for (unsigned r = warp; r < rows; r += kUnroll * nwarps) {
-            LaneSums<BITS> sums[kUnroll];
+            WideSums<BITS> sums[kUnroll];
             unsigned off[kUnroll];
             bool ok[kUnroll];
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 sums[u].clear();
-                ok[u] = (u == 0) || (r + u * nwarps < rows);
+                // a lane loads only if its 16 elements start below the part's valid length (they then lie inside the code area)
+                ok[u] = (r + u * nwarps < rows) && (static_cast<unsigned long long>(r + u * nwarps) * kWide + lane_elem < valid);
                 off[u] = (r + u * nwarps) * kRowBytes + lane_byte;
             }
 #pragma unroll 4
             for (int w = 0; w < N; ++w) {
                 const uint8_t *src = P.parts[w] + poff;
-                CodeWord<BITS> cw[kUnroll];
+                WideCodes<BITS> cw[kUnroll];
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
-                    cw[u].x = 0u; cw[u].y = 0u;
-                    if (ok[u]) load_codeword<BITS>(src + off[u], cw[u]);
+#pragma unroll
+                    for (int i = 0; i < WideCodes<BITS>::W; ++i) cw[u].w[i] = 0u;
+                    if (ok[u]) load_codes<BITS>(src + off[u], cw[u]);
                 }
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) sums[u].add(cw[u]);
             }
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
-                const unsigned long long o = static_cast<unsigned long long>(r + u * nwarps) * kRow + lane_elem;
-                if (!ok[u] || o >= valid) continue;
-                float res[8];
+                if (!ok[u]) continue;
+                const unsigned long long o = static_cast<unsigned long long>(r + u * nwarps) * kWide + lane_elem;
+                float res[16];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
+                for (int j = 0; j < 16; ++j) {
                     const float acc = __fmaf_rn(sums[u].get(j), P.ra, P.rb);
                     res[j] = P.div_mode == 0 ? acc : div_workers(P, acc);
                 }
-                store_out8<OUT>(P.out, out0 + o, res, valid - o);
+                store_out16<OUT>(P.out, out0 + o, res, valid - o, wide32);
             }
         }
         return;
     }
 
-    constexpr int kUnrollG = 2;
-    for (unsigned r = warp; r < rows; r += kUnrollG * nwarps) {
-        float acc[kUnrollG][8];
+    // Generic path: dec(q) and the sum in worker order, each operation rounded as Eq. 8 and Eq. 1 state them.
+    // gen_mode 0: q * (1/s) equals q / s for every code (or block scales: q * scale); 1: Newton-Raphson division,
+    // checked on the host for every code; 2: IEEE division.
+    // The workers of a row are taken four at a time; while one group is being summed, the loads of the next group
+    // (of this row or of the warp's next row) are already in flight.
+    constexpr int kGroup = 4;
+    struct Group {
+        WideCodes<BITS> c[kGroup];
+        float sc[kGroup];
+    };
+    const int groups = (N + kGroup - 1) / kGroup;
+    auto load_group = [&](unsigned row, int g, Group &G) {
+        const unsigned long long o = static_cast<unsigned long long>(row) * kWide + lane_elem;
+        const bool in = row < rows && o < valid;
+        const unsigned off = row * kRowBytes + lane_byte;
+        const unsigned long long sidx = o >> P.block_log2;
 #pragma unroll
-        for (int u = 0; u < kUnrollG; ++u)
+        for (int i = 0; i < kGroup; ++i) {
+            const int w = g * kGroup + i;
 #pragma unroll
-            for (int j = 0; j < 8; ++j) acc[u][j] = 0.0f;
-#pragma unroll 2
-        for (int w = 0; w < N; ++w) {
-            const uint8_t *wbase = P.parts[w] + poff;
-            CodeWord<BITS> cw[kUnrollG];
-            float sc[kUnrollG];
-#pragma unroll
-            for (int u = 0; u < kUnrollG; ++u) {
-                cw[u].x = 0u; cw[u].y = 0u;
-                sc[u] = P.gen_mul;
-                if (u == 0 || r + u * nwarps < rows) {
-                    load_codeword<BITS>(wbase + lane_byte + static_cast<size_t>(r + u * nwarps) * kRowBytes, cw[u]);
-                    if (MODE == MODE_BLOCK)
-                        sc[u] = __ldg(reinterpret_cast<const float *>(wbase + P.code_bytes) +
-                                      ((static_cast<unsigned long long>(r + u * nwarps) * kRow + lane_elem) >> P.block_log2));
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < kUnrollG; ++u) {
-                float q[8];
-                codes_to_float<BITS>(cw[u], q);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    float d;                                               // dec(q; s), Eq. 1
-                    if (MODE == MODE_FIXED && P.gen_mul == 0.0f) d = __fdiv_rn(q[j], P.s);
-                    else d = __fmul_rn(q[j], sc[u]);
-                    acc[u][j] = __fadd_rn(acc[u][j], d);
-                }
+            for (int t = 0; t < WideCodes<BITS>::W; ++t) G.c[i].w[t] = 0u;
+            G.sc[i] = P.gen_mul;
+            if (in && w < N) {
+                const uint8_t *wbase = P.parts[w] + poff;
+                load_codes<BITS>(wbase + off, G.c[i]);
+                if (MODE == MODE_BLOCK) G.sc[i] = __ldg(reinterpret_cast<const float *>(wbase + P.code_bytes) + sidx);
             }
         }
+    };
+    Group cur;
+    if (warp < rows) load_group(warp, 0, cur);
+    for (unsigned r = warp; r < rows; r += nwarps) {
+        const unsigned long long o = static_cast<unsigned long long>(r) * kWide + lane_elem;
+        f32x2 acc2[8];
 #pragma unroll
-        for (int u = 0; u < kUnrollG; ++u) {
-            const unsigned long long o = static_cast<unsigned long long>(r + u * nwarps) * kRow + lane_elem;
-            if ((u != 0 && r + u * nwarps >= rows) || o >= valid) continue;
-            float res[8];
+        for (int i = 0; i < 8; ++i) acc2[i] = 0ull;
+        for (int g = 0; g < groups; ++g) {
+            Group nxt;
+            if (g + 1 < groups) load_group(r, g + 1, nxt);
+            else load_group(r + nwarps, 0, nxt);
 #pragma unroll
-            for (int j = 0; j < 8; ++j) res[j] = div_workers(P, acc[u][j]);   // the 1/N of Eq. 8
-            store_out8<OUT>(P.out, out0 + o, res, valid - o);
+            for (int i = 0; i < kGroup; ++i) {
+                if (g * kGroup + i >= N) break;
+                unsigned x[WideCodes<BITS>::W], xh[WideCodes<BITS>::W];
+#pragma unroll
+                for (int t = 0; t < WideCodes<BITS>::W; ++t) {
+                    x[t] = cur.c[i].w[t] ^ (BITS == 8 ? 0x80808080u : (BITS == 4 ? 0x88888888u : 0xAAAAAAAAu));
+                    xh[t] = x[t] >> (BITS == 4 ? 12 : 16);
+                }
+                const f32x2 sc2 = dup2(cur.sc[i]);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    float k0, k1;
+                    const float m0 = field_magic<BITS>(x, xh, 2 * k, k0);
+                    const float m1 = field_magic<BITS>(x, xh, 2 * k + 1, k1);
+                    const f32x2 q2 = fadd2(pk2(m0, m1), pk2(-k0, -k1));                 // the two codes, exact
+                    if (MODE == MODE_BLOCK || P.gen_mode == 0) {
+                        acc2[k] = fadd2_after_mul(acc2[k], fmul2(q2, sc2));             // product and sum rounded separately
+                    } else if (P.gen_mode == 1) {
+                        const f32x2 inv2 = dup2(P.inv_s);
+                        const f32x2 q0 = fmul2(q2, inv2);
+                        const f32x2 rem = ffma2(q0, dup2(-P.s), q2);
+                        acc2[k] = fadd2(acc2[k], ffma2(rem, inv2, q0));
+                    } else {
+                        float a, b, c, d;
+                        unpk2(q2, a, b);
+                        unpk2(acc2[k], c, d);
+                        acc2[k] = pk2(__fadd_rn(c, __fdiv_rn(a, P.s)), __fadd_rn(d, __fdiv_rn(b, P.s)));
+                    }
+                }
+            }
+            cur = nxt;
         }
+        if (o >= valid) continue;
+        float res[16];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float a, b;
+            unpk2(acc2[i], a, b);
+            res[2 * i] = div_workers(P, a);                                          // the 1/N of Eq. 8
+            res[2 * i + 1] = div_workers(P, b);
+        }
+        store_out16<OUT>(P.out, out0 + o, res, valid - o, wide32);
     }
 }
 
