@@ -223,6 +223,16 @@ int loco_unpack_dequant_reduce_host_noalloc(const loco_config_t *cfg, const void
  */
 int loco_last_status(loco_state_t *st, uint32_t *flags, uint64_t *n_saturated, void *stream);
 
+/*
+ * Diagnostic for the block-scaled extension (no counterpart in the paper).  The send kernel forms a block's scale
+ * amax/qmax and its inverse qmax/amax with short multiply-add sequences instead of the general division routine;
+ * this call runs both sequences against the IEEE division for every positive finite fp32 amax and qmax in
+ * {1, 7, 127} on the current device (about a second, synchronous, allocates and frees 16 bytes) and writes the number
+ * of differing results: mismatches[0] for amax/qmax, mismatches[1] for qmax/amax.  Both must be 0.
+ * Errors: ARG (null), CUDA.
+ */
+int loco_selfcheck_block_division(uint64_t *mismatches /* host, 2 elements */);
+
 /* Human-readable name of a loco_status_t. */
 const char *loco_status_string(int status);
 

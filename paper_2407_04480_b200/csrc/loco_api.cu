@@ -650,6 +650,25 @@ int loco_unpack_dequant_reduce_host_noalloc(const loco_config_t *cfg, const void
                                            d_scratch, LOCO_NOALLOC_SCRATCH_BYTES, stream);
 }
 
+int loco_selfcheck_block_division(uint64_t *mismatches) {
+    if (!mismatches) return LOCO_ERR_ARG;
+    unsigned long long *d = nullptr;
+    if (cudaMalloc(reinterpret_cast<void **>(&d), 16) != cudaSuccess) { cudaGetLastError(); return LOCO_ERR_CUDA; }
+    unsigned long long h[2] = {0, 0};
+    cudaError_t e = cudaMemset(d, 0, 16);
+    if (e == cudaSuccess) {
+        loco_division_selfcheck_kernel<<<num_sms() * 8, 256>>>(d);
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaMemcpy(h, d, 16, cudaMemcpyDeviceToHost);
+    cudaFree(d);
+    if (e != cudaSuccess) { cudaGetLastError(); return LOCO_ERR_CUDA; }
+    g_launches.fetch_add(1);
+    mismatches[0] = h[0];
+    mismatches[1] = h[1];
+    return LOCO_OK;
+}
+
 int loco_last_status(loco_state_t *st, uint32_t *flags, uint64_t *n_saturated, void *stream) {
     if (!st) return LOCO_ERR_ARG;
     unsigned long long host[2] = {0, 0};

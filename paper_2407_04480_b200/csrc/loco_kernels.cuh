@@ -542,6 +542,46 @@ __device__ __forceinline__ unsigned horner_codes(const unsigned *mb) {
     return (acc - kMagicBits * ones) ^ flip;
 }
 
+// ---- the two divisions of a block scale, without the general division routine --------------------------------
+// scale = amax / qmax and 1/scale = qmax / amax must carry the bits of the IEEE division (the oracle divides).
+// amax / c for the three constants that occur (1, 7, 127): multiply by fl(1/c) and correct once with two fused
+// multiply-adds.  qmax / amax: the hardware's approximate reciprocal, corrected the same way, for amax in
+// [2^-100, 2^100]; outside that range the general division is used.  Both short forms are compared against
+// __fdiv_rn for EVERY positive finite float by loco_selfcheck_block_division() (and by the GPU tests).
+__device__ __forceinline__ float div_by_qmax(float a, float c, float rc) {
+    const float q0 = __fmul_rn(a, rc);
+    const float rem = __fmaf_rn(-q0, c, a);
+    return __fmaf_rn(rem, rc, q0);
+}
+__device__ __forceinline__ float qmax_over(float c, float a) {
+    if (__float_as_uint(a) - 0x0d800000u <= 0x71800000u - 0x0d800000u) {      // 2^-100 <= a <= 2^100
+        float x;
+        asm("rcp.approx.f32 %0, %1;" : "=f"(x) : "f"(a));
+        const float q0 = __fmul_rn(c, x);
+        const float rem = __fmaf_rn(-q0, a, c);
+        return __fmaf_rn(rem, x, q0);
+    }
+    return __fdiv_rn(c, a);
+}
+
+// mismatch[0]: amax / c, mismatch[1]: c / amax, over all positive finite floats, for c = 1, 7, 127
+__global__ void loco_division_selfcheck_kernel(unsigned long long *mismatch) {
+    const float cs[3] = {1.0f, 7.0f, 127.0f};
+    unsigned long long bad0 = 0, bad1 = 0;
+    for (unsigned long long b = blockIdx.x * static_cast<unsigned long long>(blockDim.x) + threadIdx.x + 1; b <= 0x7f7fffffull;
+         b += static_cast<unsigned long long>(gridDim.x) * blockDim.x) {
+        const float a = __uint_as_float(static_cast<unsigned>(b));
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            const float c = cs[i];
+            if (__float_as_uint(div_by_qmax(a, c, __frcp_rn(c))) != __float_as_uint(__fdiv_rn(a, c))) ++bad0;
+            if (__float_as_uint(qmax_over(c, a)) != __float_as_uint(__fdiv_rn(c, a))) ++bad1;
+        }
+    }
+    if (bad0) atomicAdd(mismatch, bad0);
+    if (bad1) atomicAdd(mismatch + 1, bad1);
+}
+
 // One wide row.  Returns false (and stores nothing) if some lane of the warp met a value that the fast
 // arithmetic does not cover (NaN, +-Inf, or a magnitude that could overflow): the caller then redoes the row
 // with the careful routine.
@@ -653,8 +693,8 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         bad_bits |= (static_cast<unsigned>(acc) | static_cast<unsigned>(acc >> 32)) & 0x7fffffffu;
         if (__any_sync(kFull, bad_bits != 0u)) return false;
         amax = warp_group_max(amax, lanes_per_block);
-        scale = amax > 0.0f ? __fdiv_rn(amax, hi) : 0.0f;
-        mult = amax > 0.0f ? __fdiv_rn(hi, amax) : 0.0f;
+        scale = amax > 0.0f ? div_by_qmax(amax, hi, 1.0f / hi) : 0.0f;
+        mult = amax > 0.0f ? qmax_over(hi, amax) : 0.0f;
     }
 
     // ---- Eq. 1 / Eq. 3: q = round_p-bit(h x s);  step 2: d, Eq. 5 ---------------------------------------------
@@ -713,8 +753,8 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
                     amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
                 }
                 amax = warp_group_max(amax, lanes_per_block);
-                escale = amax > 0.0f ? __fdiv_rn(amax, 127.0f) : 0.0f;
-                emult = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
+                escale = amax > 0.0f ? div_by_qmax(amax, 127.0f, 1.0f / 127.0f) : 0.0f;
+                emult = amax > 0.0f ? qmax_over(127.0f, amax) : 0.0f;
             }
             const f32x2 emult2 = dup2(emult);
             int q[16];

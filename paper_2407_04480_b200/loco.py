@@ -29,7 +29,7 @@ EXPORTS = ("loco_state_bytes", "loco_packed_bytes", "loco_partition_bytes", "loc
            "loco_last_status", "loco_status_string", "loco_launch_count",
            "loco_send_host_workspace_bytes", "loco_reduce_host_workspace_bytes",
            "loco_compensate_quantize_pack_host", "loco_unpack_dequant_reduce_host",
-           "loco_unpack_dequant_reduce_host_noalloc")
+           "loco_unpack_dequant_reduce_host_noalloc", "loco_selfcheck_block_division")
 NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
@@ -108,6 +108,8 @@ def lib() -> C.CDLL:
         L.loco_unpack_dequant_reduce_host.argtypes = [cp, C.POINTER(vp), i32, u64, i32, i32, vp, vp, u64, vp]
         L.loco_unpack_dequant_reduce_host_noalloc.restype = C.c_int
         L.loco_unpack_dequant_reduce_host_noalloc.argtypes = [cp, C.POINTER(vp), i32, u64, i32, i32, vp, vp]
+        L.loco_selfcheck_block_division.restype = C.c_int
+        L.loco_selfcheck_block_division.argtypes = [C.POINTER(u64)]
         L.loco_last_status.restype = C.c_int
         L.loco_last_status.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(u64), vp]
         L.loco_status_string.restype = C.c_char_p
@@ -295,3 +297,11 @@ def loco_unpack_dequant_reduce_host_noalloc(cfg: Config, h_packed: Sequence[torc
     _check(lib().loco_unpack_dequant_reduce_host_noalloc(C.byref(cfg.c()), ptrs, len(h_packed), n, first_partition,
                                                          partition_count, _host_ptr(h_out), _stream_ptr(stream)),
            "loco_unpack_dequant_reduce_host_noalloc")
+
+
+def loco_selfcheck_block_division():
+    """(mismatches of amax/qmax, mismatches of qmax/amax) of the kernels' short division sequences against the IEEE
+    division over every positive finite fp32 amax; both must be 0.  Synchronous, about a second."""
+    out = (C.c_uint64 * 2)(0, 0)
+    _check(lib().loco_selfcheck_block_division(out), "loco_selfcheck_block_division")
+    return int(out[0]), int(out[1])

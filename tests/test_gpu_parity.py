@@ -301,3 +301,9 @@ def test_host_buffer_variants(mode):
         loco.loco_unpack_dequant_reduce_host(gcfg, [c[first * stride:] for c in h_comms], n, h_out, w_red[:-1],
                                              first_partition=first, partition_count=count)
     assert ei.value.code == loco.ERR_SIZE
+
+
+def test_block_scale_divisions_are_ieee_for_every_amax():
+    """The block-scaled send path divides with short multiply-add sequences; the library checks them against the IEEE
+    division for every positive finite fp32 amax and qmax in {1, 7, 127}."""
+    assert loco.loco_selfcheck_block_division() == (0, 0)
