@@ -157,36 +157,38 @@ using SendFn = void (*)(const SendParams);
 struct SendKernel { SendFn fn; int smem_bytes; };
 
 template <int GRAD, int STATE, int BITS>
-SendKernel pick_send_mode(int mode, bool lean) {
+SendKernel pick_send_mode(int mode, int var) {
     if (mode == MODE_FIXED) {
         const int smem = Ring<GRAD, STATE, MODE_FIXED>::kBytes;
-        if (lean) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, true>, smem};
-        return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, false>, smem};
+        if (var == VAR_LEAN) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_LEAN>, smem};
+        if (var == VAR_LEAN_NR && (STATE == ST_INT8 || STATE == ST_Q8COMP))
+            return {loco_send_kernel<GRAD, (STATE == ST_INT8 || STATE == ST_Q8COMP) ? STATE : ST_INT8, BITS, MODE_FIXED, VAR_LEAN_NR>, smem};
+        return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_GENERAL>, smem};
     }
     if (STATE == ST_Q8COMP) return {nullptr, 0};                // Q8COMP exists for the global scales only
     constexpr int ST = (STATE == ST_Q8COMP ? ST_FP32 : STATE);
-    return {loco_send_kernel<GRAD, ST, BITS, MODE_BLOCK, true>, Ring<GRAD, ST, MODE_BLOCK>::kBytes};
+    return {loco_send_kernel<GRAD, ST, BITS, MODE_BLOCK, VAR_LEAN>, Ring<GRAD, ST, MODE_BLOCK>::kBytes};
 }
 template <int GRAD, int STATE>
-SendKernel pick_send_bits(int bits, int mode, bool lean) {
+SendKernel pick_send_bits(int bits, int mode, int var) {
     switch (bits) {
-    case 2: return pick_send_mode<GRAD, STATE, 2>(mode, lean);
-    case 4: return pick_send_mode<GRAD, STATE, 4>(mode, lean);
-    default: return pick_send_mode<GRAD, STATE, 8>(mode, lean);
+    case 2: return pick_send_mode<GRAD, STATE, 2>(mode, var);
+    case 4: return pick_send_mode<GRAD, STATE, 4>(mode, var);
+    default: return pick_send_mode<GRAD, STATE, 8>(mode, var);
     }
 }
 template <int GRAD>
-SendKernel pick_send_state(int state, int bits, int mode, bool lean) {
+SendKernel pick_send_state(int state, int bits, int mode, int var) {
     switch (state) {
-    case LOCO_STATE_INT8: return pick_send_bits<GRAD, ST_INT8>(bits, mode, lean);
-    case LOCO_STATE_FP32: return pick_send_bits<GRAD, ST_FP32>(bits, mode, lean);
-    case LOCO_STATE_NONE: return pick_send_bits<GRAD, ST_NONE>(bits, mode, lean);
-    default: return pick_send_bits<GRAD, ST_Q8COMP>(bits, mode, lean);
+    case LOCO_STATE_INT8: return pick_send_bits<GRAD, ST_INT8>(bits, mode, var);
+    case LOCO_STATE_FP32: return pick_send_bits<GRAD, ST_FP32>(bits, mode, var);
+    case LOCO_STATE_NONE: return pick_send_bits<GRAD, ST_NONE>(bits, mode, var);
+    default: return pick_send_bits<GRAD, ST_Q8COMP>(bits, mode, var);
     }
 }
-SendKernel pick_send(const loco_config_t *c, int mode, bool lean) {
-    return c->grad_dtype == LOCO_BF16 ? pick_send_state<GRAD_BF16>(c->state_fmt, c->bits, mode, lean)
-                                      : pick_send_state<GRAD_F32>(c->state_fmt, c->bits, mode, lean);
+SendKernel pick_send(const loco_config_t *c, int mode, int var) {
+    return c->grad_dtype == LOCO_BF16 ? pick_send_state<GRAD_BF16>(c->state_fmt, c->bits, mode, var)
+                                      : pick_send_state<GRAD_F32>(c->state_fmt, c->bits, mode, var);
 }
 
 // ---- reduce dispatch ---------------------------------------------------------------------
@@ -194,22 +196,26 @@ SendKernel pick_send(const loco_config_t *c, int mode, bool lean) {
 using ReduceFn = void (*)(const ReduceParams);
 
 template <int OUT, int BITS>
-ReduceFn pick_reduce_mode(int mode, bool int_path) {
-    if (mode == MODE_FIXED)
-        return int_path ? loco_reduce_kernel<OUT, BITS, MODE_FIXED, true> : loco_reduce_kernel<OUT, BITS, MODE_FIXED, false>;
-    return loco_reduce_kernel<OUT, BITS, MODE_BLOCK, false>;
-}
-template <int OUT>
-ReduceFn pick_reduce_bits(int bits, int mode, bool int_path) {
-    switch (bits) {
-    case 2: return pick_reduce_mode<OUT, 2>(mode, int_path);
-    case 4: return pick_reduce_mode<OUT, 4>(mode, int_path);
-    default: return pick_reduce_mode<OUT, 8>(mode, int_path);
+ReduceFn pick_reduce_mode(int mode, int path) {
+    if (mode != MODE_FIXED) return loco_reduce_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>;
+    switch (path) {
+    case PATH_INT: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_INT>;
+    case PATH_MUL: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>;
+    case PATH_NEWTON: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON>;
+    default: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE>;
     }
 }
-ReduceFn pick_reduce(const loco_config_t *c, int mode, bool int_path) {
-    return c->out_dtype == LOCO_BF16 ? pick_reduce_bits<GRAD_BF16>(c->bits, mode, int_path)
-                                     : pick_reduce_bits<GRAD_F32>(c->bits, mode, int_path);
+template <int OUT>
+ReduceFn pick_reduce_bits(int bits, int mode, int path) {
+    switch (bits) {
+    case 2: return pick_reduce_mode<OUT, 2>(mode, path);
+    case 4: return pick_reduce_mode<OUT, 4>(mode, path);
+    default: return pick_reduce_mode<OUT, 8>(mode, path);
+    }
+}
+ReduceFn pick_reduce(const loco_config_t *c, int mode, int path) {
+    return c->out_dtype == LOCO_BF16 ? pick_reduce_bits<GRAD_BF16>(c->bits, mode, path)
+                                     : pick_reduce_bits<GRAD_F32>(c->bits, mode, path);
 }
 
 unsigned grid_x_for(uint64_t rows_per_partition, int partitions, int ctas_per_sm) {
@@ -314,9 +320,11 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
         if (cfg->state_fmt == LOCO_STATE_INT8 && !(cfg->s_e > 1e-28f)) st->fast = 0;
     }
     {
-        const bool lean = st->mode == MODE_BLOCK ||
-                          (st->dq.mode == DEC_FMA && st->de.mode == DEC_FMA && !cfg->collect_stats);
-        const SendKernel k = pick_send(cfg, st->mode, lean);
+        int var = VAR_GENERAL;
+        if (st->mode == MODE_BLOCK) var = VAR_LEAN;
+        else if (!cfg->collect_stats && st->dq.mode == DEC_FMA && st->de.mode == DEC_FMA) var = VAR_LEAN;
+        else if (!cfg->collect_stats && st->dq.mode == DEC_FMA && st->de.mode == DEC_NEWTON) var = VAR_LEAN_NR;
+        const SendKernel k = pick_send(cfg, st->mode, var);
         st->send_fn = k.fn;
         st->send_smem_bytes = k.smem_bytes;
     }
@@ -501,9 +509,11 @@ int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_pa
             }
         }
     }
-    ReduceFn fn = pick_reduce(cfg, mode, P.int_path != 0);
-    static int occ_cache[2][3][2][2] = {};
-    int &occ = occ_cache[cfg->out_dtype == LOCO_BF16][cfg->bits == 2 ? 0 : (cfg->bits == 4 ? 1 : 2)][mode][P.int_path != 0];
+    const int path = mode == MODE_BLOCK ? PATH_MUL
+                     : (P.int_path ? PATH_INT : (P.gen_mode == 0 ? PATH_MUL : (P.gen_mode == 1 ? PATH_NEWTON : PATH_DIVIDE)));
+    ReduceFn fn = pick_reduce(cfg, mode, path);
+    static int occ_cache[2][3][2][4] = {};
+    int &occ = occ_cache[cfg->out_dtype == LOCO_BF16][cfg->bits == 2 ? 0 : (cfg->bits == 4 ? 1 : 2)][mode][path];
     if (occ == 0) {
         int v = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, fn, kThreads, 0) != cudaSuccess || v < 1) {

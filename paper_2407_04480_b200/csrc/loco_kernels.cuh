@@ -585,15 +585,37 @@ __global__ void loco_division_selfcheck_kernel(unsigned long long *mismatch) {
 // One wide row.  Returns false (and stores nothing) if some lane of the warp met a value that the fast
 // arithmetic does not cover (NaN, +-Inf, or a magnitude that could overflow): the caller then redoes the row
 // with the careful routine.
-// LEAN: both decompressors are the single fused multiply-add and no statistics are collected.
-template <int GRAD, int STATE, int BITS, int MODE, bool LEAN>
+// VAR_LEAN: both decompressors are the single fused multiply-add and no statistics are collected;
+// VAR_LEAN_NR: the same, but dec(e; s_e) is the Newton-Raphson form (s_e = 6 s of the paper), still packed;
+// VAR_GENERAL: the forms are chosen per call at run time (scalar code) and statistics may be collected.
+enum : int { VAR_LEAN = 0, VAR_LEAN_NR = 1, VAR_GENERAL = 2 };
+
+// dec(e; s_e) of a pair from the magic floats m2 = kMagic + 128 + e
+template <int VAR>
+__device__ __forceinline__ f32x2 dec_state2(const SendConsts &K, f32x2 m2, float emagic, int de_mode) {
+    if (VAR == VAR_LEAN) return ffma2(m2, dup2(K.de_a), dup2(K.de_b));
+    if (VAR == VAR_LEAN_NR) {
+        const f32x2 e2 = fadd2(m2, dup2(-emagic));                   // the codes, exact
+        const f32x2 inv2 = dup2(K.inv_se);
+        const f32x2 q0 = fmul2(e2, inv2);
+        const f32x2 rem = ffma2(q0, dup2(-K.s_e), e2);
+        return ffma2(rem, inv2, q0);
+    }
+    float m0, m1;
+    unpk2(m2, m0, m1);
+    return pk2(dec_fast(m0, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se),
+               dec_fast(m1, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se));
+}
+
+template <int GRAD, int STATE, int BITS, int MODE, int VAR>
 __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtrs &L, const WideIn<GRAD, STATE> &in,
                                               unsigned wrow, int lane, bool stats, unsigned &saturated) {
     constexpr float lo = QRange<BITS>::lo, hi = QRange<BITS>::hi, qmagic = kMagic + QRange<BITS>::off;
     constexpr float emagic = kMagic + 128.0f;
     constexpr bool kStateF32 = (STATE == ST_FP32 || STATE == ST_Q8COMP);
     constexpr int GW = WideIn<GRAD, STATE>::GW, EW = WideIn<GRAD, STATE>::EW;
-    const int dq_mode = LEAN ? DEC_FMA : K.dq_mode, de_mode = LEAN ? DEC_FMA : K.de_mode;
+    constexpr bool LEAN = (VAR != VAR_GENERAL);
+    const int dq_mode = LEAN ? DEC_FMA : K.dq_mode, de_mode = K.de_mode;
     const int lanes_per_block = (MODE == MODE_BLOCK) ? (K.block_log2 >= 9 ? 32 : (1 << (K.block_log2 - 4))) : 1;
     const f32x2 zero2 = 0ull;
 
@@ -646,11 +668,8 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             const float m1 = __uint_as_float(__byte_perm(x, kMagicBits, 0x7651 + 2 * (k & 1)));
             if (MODE == MODE_BLOCK) {
                 c2 = fmul2(fadd2(pk2(m0, m1), dup2(-emagic)), dup2(in.sscale));
-            } else if (LEAN) {
-                c2 = ffma2(pk2(m0, m1), dup2(K.de_a), dup2(K.de_b));
             } else {
-                c2 = pk2(dec_fast(m0, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se),
-                         dec_fast(m1, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se));
+                c2 = dec_state2<VAR>(K, pk2(m0, m1), emagic, de_mode);
             }
             prev2[k] = c2;
         } else if (kStateF32) {
@@ -661,14 +680,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
                 float y0, y1;
                 unpk2(fmul2(prev2[k], dup2(K.s_e)), y0, y1);
                 const f32x2 m2 = fadd2(pk2(fminf(fmaxf(y0, -128.0f), 127.0f), fminf(fmaxf(y1, -128.0f), 127.0f)), dup2(emagic));
-                if (LEAN) {
-                    c2 = ffma2(m2, dup2(K.de_a), dup2(K.de_b));
-                } else {
-                    float m0, m1;
-                    unpk2(m2, m0, m1);
-                    c2 = pk2(dec_fast(m0, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se),
-                             dec_fast(m1, emagic, de_mode, K.de_a, K.de_b, K.s_e, K.inv_se));
-                }
+                c2 = dec_state2<VAR>(K, m2, emagic, de_mode);
             }
         } else {
             c2 = zero2;
@@ -793,9 +805,9 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
 // grid = (ctas per partition, partitions).  Each warp walks the partition's wide rows with the stride of all
 // warps working on that partition; the inputs of its next rows are on their way through the cp.async ring.
 // What is left of the partition (a last half-wide row, partial and padding rows) goes to the careful routine.
-// LEAN kernels are launched when the host proved both single-FMA decompressors and no statistics are
-// wanted (and for every block-scaled configuration); the others choose per element at run time.
-template <int GRAD, int STATE, int BITS, int MODE, bool LEAN>
+// VAR_LEAN / VAR_LEAN_NR kernels are launched when the host proved the corresponding decompressor forms and no
+// statistics are wanted (VAR_LEAN also for every block-scaled configuration); VAR_GENERAL chooses at run time.
+template <int GRAD, int STATE, int BITS, int MODE, int VAR>
 __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams P) {
     using R = Ring<GRAD, STATE, MODE>;
     constexpr int D = R::kDepth;
@@ -860,7 +872,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams
             fetch_row<GRAD, STATE, MODE>(A, slot_off, in);
             if (stage_wrow < full_wide) stage(stage_off, stage_wrow);
             cp_async_commit();                 // one group per iteration, empty near the end
-            if (!send_wide_row<GRAD, STATE, BITS, MODE, LEAN>(K, L, in, wrow, lane, stats, saturated)) {
+            if (!send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, wrow, lane, stats, saturated)) {
                 careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(wrow) * kWide, lane);
                 careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(wrow) * kWide + kRow, lane);
             }
@@ -1038,9 +1050,11 @@ struct WideSums {
     }
 };
 
-// INT: the integer-sum path (only with the global scale); otherwise the generic path.  Two kernels, so that each path
-// gets the registers and the occupancy it wants.
-template <int OUT, int BITS, int MODE, bool INT>
+// PATH_INT: the integer-sum path (only with the global scale); otherwise the generic path with dec(q; s) as a multiply
+// (also the block-scaled form), as the Newton-Raphson division, or as the IEEE division.  Separate kernels, so that each
+// path gets the registers and the occupancy it wants and no per-element choice is left.
+enum : int { PATH_INT = 0, PATH_MUL = 1, PATH_NEWTON = 2, PATH_DIVIDE = 3 };
+template <int OUT, int BITS, int MODE, int PATH>
 __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParams P) {
     constexpr unsigned kRowBytes = kWide * BITS / 8;                  // code bytes of one wide row
     const int lane = threadIdx.x & 31;
@@ -1059,7 +1073,7 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
     const int N = P.num_workers;
     const bool wide32 = P.out_align32 != 0;
 
-    if (INT) {
+    if (PATH == PATH_INT) {
         // code areas below 4 GiB (checked by the host): row offsets fit 32 bits
         constexpr int kUnroll = 2;
         for (unsigned r = warp; r < rows; r += kUnroll * nwarps) {
@@ -1103,8 +1117,8 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
     }
 
     // Generic path: dec(q) and the sum in worker order, each operation rounded as Eq. 8 and Eq. 1 state them.
-    // gen_mode 0: q * (1/s) equals q / s for every code (or block scales: q * scale); 1: Newton-Raphson division,
-    // checked on the host for every code; 2: IEEE division.
+    // PATH_MUL: q * (1/s) equals q / s for every code (or block scales: q * scale); PATH_NEWTON: Newton-Raphson
+    // division, checked on the host for every code; PATH_DIVIDE: IEEE division.
     // The workers of a row are taken four at a time; while one group is being summed, the loads of the next group
     // (of this row or of the warp's next row) are already in flight.
     constexpr int kGroup = 4;
@@ -1131,6 +1145,7 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
             }
         }
     };
+    const f32x2 inv2 = dup2(P.inv_s), negs2 = dup2(-P.s);
     Group cur;
     if (warp < rows) load_group(warp, 0, cur);
     for (unsigned r = warp; r < rows; r += nwarps) {
@@ -1158,12 +1173,11 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
                     const float m0 = field_magic<BITS>(x, xh, 2 * k, k0);
                     const float m1 = field_magic<BITS>(x, xh, 2 * k + 1, k1);
                     const f32x2 q2 = fadd2(pk2(m0, m1), pk2(-k0, -k1));                 // the two codes, exact
-                    if (MODE == MODE_BLOCK || P.gen_mode == 0) {
+                    if (PATH == PATH_MUL) {
                         acc2[k] = fadd2_after_mul(acc2[k], fmul2(q2, sc2));             // product and sum rounded separately
-                    } else if (P.gen_mode == 1) {
-                        const f32x2 inv2 = dup2(P.inv_s);
+                    } else if (PATH == PATH_NEWTON) {
                         const f32x2 q0 = fmul2(q2, inv2);
-                        const f32x2 rem = ffma2(q0, dup2(-P.s), q2);
+                        const f32x2 rem = ffma2(q0, negs2, q2);
                         acc2[k] = fadd2(acc2[k], ffma2(rem, inv2, q0));
                     } else {
                         float a, b, c, d;
