@@ -57,3 +57,13 @@ def loco_step(g, e_tilde, e_code, k, *, s, s_e, beta, T_c, p=4, p_e=8, state="in
 def average(ds):
     """Eq. 8: the mean of the workers' dequantised vectors."""
     return np.mean(np.asarray(ds, dtype=np.float64), axis=0)
+
+
+def adam_family_step(g, m, v, theta, *, lr, beta1, beta2, delta):
+    """The paper's Adam-family equations with Adam's pre-conditioner: m = (1-b1) m + b1 g, v = (1-b2) v + b2 g^2,
+    theta = theta - lr / sqrt(v + delta) * m  (no bias correction, delta inside the root).  Returns (m, v, theta)."""
+    g, m, v, theta = (np.asarray(a, dtype=np.float64) for a in (g, m, v, theta))
+    m = (1.0 - beta1) * m + beta1 * g
+    v = (1.0 - beta2) * v + beta2 * g * g
+    theta = theta - lr / np.sqrt(v + delta) * m
+    return m, v, theta

@@ -22,6 +22,7 @@
  *   moving-average error ................. Algorithm 1 step 2, Eq. 5
  *   reset / 8-bit error compression ...... Algorithm 1 step 2, Eq. 7
  *   average of the N dequantised parts ... Algorithm 1 step 3, Eq. 8
+ *   Adam-family update with g~ ............ Algorithm 1 step 3, Adam-family equations (Sec. on LoCo-integrated Adam)
  *   partition of the vector into N parts . Sec. 3.3 (FSDP / all2all paragraph)
  *
  * Readings where the paper is silent (all restated in the design notes):
@@ -39,7 +40,9 @@
  *     amax/qmax, and is defined here only so that both sides agree;
  *   - non-finite h: NaN gives code 0, +-Inf the saturated code, and in both
  *     cases the compression error of that element is taken as 0;
- *   - Eq. 8 is summed in worker order in fp32, then divided by (float)N.
+ *   - Eq. 8 is summed in worker order in fp32, then divided by (float)N;
+ *   - the Adam-family step is taken exactly as printed (no bias correction, delta inside the root), with
+ *     eta_k = eta / sqrt(v_k + delta) evaluated as one square root and one division.
  *
  * Pins (tests/test_oracle_pins.py): code range, half-step bound and saturation
  * error of Lemma "round", brute-force nearest code, idempotence, identity
@@ -47,7 +50,9 @@
  * unrolling of Eq. 5, the identity of Lemma 1 in its three storage forms, the
  * telescoping sum of Lemma 2's proof, reset, averaging versus the real-number
  * mean, storage sizes of Table 1's text, brute force over all byte values of
- * the packing, and a hand-worked example (tests/golden/).
+ * the packing, and a hand-worked example (tests/golden/); for the fused Adam-family step: the sign-update special
+ * case (beta1 = beta2 = 1, delta = 0), the closed form of the moments under a constant gradient, a zero gradient,
+ * agreement with the textbook formulas in float64, and a hand-worked dyadic example.
  * Unpinned by anything in the paper: the value of beta, the block size and the
  * block-scaled variant as a whole ("parity unpinned" for SCALE_BLOCK_ABSMAX:
  * it is pinned only by the invariants that do not depend on the scale rule).
@@ -423,6 +428,72 @@ int orc_reduce(const orc_config *cfg, uint64_t n, const uint8_t *const *parts, i
             const float g = acc / (float)num_workers;                      /* the 1/N of Eq. 8 */
             if (cfg->out_dtype == ORC_BF16) ((uint16_t *)out)[w_out] = f32_to_bf16_rne(g);
             else ((float *)out)[w_out] = g;
+            ++w_out;
+        }
+    }
+    return 0;
+}
+
+/*
+ * Receive side followed by the Adam-family update of the same elements (Algorithm 1 step 3: "use g~_k to update
+ * theta_k"; the Adam-family equations of the section on LoCo-integrated Adam-family optimizers):
+ *     g      = (1/N) sum_n dec(q^n)                       Eq. 8, in fp32, NOT rounded to the output type first
+ *     m_k    = (1 - beta1) m_{k-1} + beta1 g              (beta1 weights the new gradient, as the paper writes it)
+ *     v_k    = (1 - beta2) v_{k-1} + beta2 g^2
+ *     eta_k  = eta / sqrt(v_k + delta)                    Adam's pre-conditioner v(.) = 1/sqrt(v_k + delta)
+ *     theta  = theta - eta_k * m_k
+ * There is no bias correction and delta sits inside the square root: that is what the paper prints.
+ * Every operation is one IEEE fp32 operation; (1 - beta) is rounded once.  m, v, theta hold the valid elements of
+ * the `count` partitions contiguously and are updated in place; grad_out (may be NULL) receives g in out_dtype.
+ */
+typedef struct { float lr, beta1, beta2, delta; } orc_adam;
+
+int orc_reduce_adam(const orc_config *cfg, uint64_t n, const uint8_t *const *parts, int32_t num_workers,
+                    int32_t first, int32_t count, const orc_adam *ad, float *m, float *v, float *theta,
+                    void *grad_out) {
+    if (!config_ok(cfg) || !ad || num_workers < 1 || first < 0 || count < 0 ||
+        first + count > cfg->num_partitions) return -1;
+    if (n == 0 || count == 0) return 0;
+    const int p = cfg->bits;
+    const int fixed = cfg->scale_mode == ORC_SCALE_FIXED;
+    const uint64_t lp = orc_partition_capacity(cfg, n);
+    const uint64_t stride = orc_partition_bytes(cfg, n);
+    const uint64_t cbytes = code_bytes_of(cfg, lp);
+    const uint64_t B = fixed ? 1 : (uint64_t)cfg->block_size;
+    const float omb1 = 1.0f - ad->beta1, omb2 = 1.0f - ad->beta2;
+    uint64_t w_out = 0;
+    for (int32_t j = first; j < first + count; ++j) {
+        const uint64_t valid = orc_partition_elems(cfg, n, j);
+        const uint64_t off = (uint64_t)(j - first) * stride;
+        for (uint64_t o = 0; o < valid; ++o) {
+            float acc = 0.0f;
+            for (int32_t w = 0; w < num_workers; ++w) {
+                const uint8_t *base = parts[w] + off;
+                const int32_t q = get_code(base, o, p);
+                float d;
+                if (fixed) {
+                    d = (float)q / cfg->s;
+                } else {
+                    float sc;
+                    memcpy(&sc, base + cbytes + (o / B) * 4, 4);
+                    d = (float)q * sc;
+                }
+                acc = acc + d;
+            }
+            const float g = acc / (float)num_workers;                       /* Eq. 8 */
+            const float mk = (omb1 * m[w_out]) + (ad->beta1 * g);
+            const float gg = g * g;
+            const float vk = (omb2 * v[w_out]) + (ad->beta2 * gg);
+            const float den = sqrtf(vk + ad->delta);
+            const float eta_k = ad->lr / den;
+            const float upd = eta_k * mk;
+            m[w_out] = mk;
+            v[w_out] = vk;
+            theta[w_out] = theta[w_out] - upd;
+            if (grad_out) {
+                if (cfg->out_dtype == ORC_BF16) ((uint16_t *)grad_out)[w_out] = f32_to_bf16_rne(g);
+                else ((float *)grad_out)[w_out] = g;
+            }
             ++w_out;
         }
     }

@@ -42,6 +42,10 @@ class _Cfg(C.Structure):
                 ("grad_dtype", C.c_int32), ("out_dtype", C.c_int32), ("num_partitions", C.c_int32)]
 
 
+class _Adam(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("delta", C.c_float)]
+
+
 class _Trace(C.Structure):
     _fields_ = [("c", C.c_void_p), ("h", C.c_void_p), ("q", C.c_void_p),
                 ("d", C.c_void_p), ("delta", C.c_void_p), ("e_new", C.c_void_p)]
@@ -94,6 +98,8 @@ def lib():
         L.orc_send_step.argtypes = [cp, u64, vp, vp, vp, i64, C.POINTER(_Trace), vp]
         L.orc_reduce.restype = C.c_int
         L.orc_reduce.argtypes = [cp, u64, C.POINTER(vp), i32, i32, i32, vp]
+        L.orc_reduce_adam.restype = C.c_int
+        L.orc_reduce_adam.argtypes = [cp, u64, C.POINTER(vp), i32, i32, i32, C.POINTER(_Adam), vp, vp, vp, vp]
         L.orc_f32_to_bf16.restype = C.c_uint16
         L.orc_f32_to_bf16.argtypes = [C.c_float]
         L.orc_bf16_to_f32.restype = C.c_float
@@ -202,6 +208,28 @@ def reduce(cfg: OracleConfig, n: int, comms, first: int = 0, count: int | None =
     out = np.zeros(n_out, dtype=np.uint16 if cfg.out_dtype == BF16 else np.float32)
     ptrs = (C.c_void_p * len(comms))(*[_ptr(c) + first * stride for c in comms])
     rc = lib().orc_reduce(C.byref(cfg.c()), n, ptrs, len(comms), first, count, _ptr(out) if n_out else None)
+    if rc != 0:
+        raise ValueError("oracle: bad configuration")
+    return out
+
+
+def reduce_adam(cfg: OracleConfig, n: int, comms, m: np.ndarray, v: np.ndarray, theta: np.ndarray, *, lr: float,
+                beta1: float, beta2: float, delta: float, first: int = 0, count: int | None = None,
+                want_grad: bool = False):
+    """Eq. 8 followed by the paper's Adam-family step on the same elements; m, v, theta (float32) are updated in
+    place.  Returns the averaged gradient (out_dtype) when want_grad is set."""
+    if count is None:
+        count = cfg.num_partitions - first
+    stride = partition_bytes(cfg, n)
+    n_out = sum(partition_elems(cfg, n, j) for j in range(first, first + count))
+    for a in (m, v, theta):
+        assert a.dtype == np.float32 and a.size >= n_out and a.flags["C_CONTIGUOUS"]
+    out = np.zeros(n_out, dtype=np.uint16 if cfg.out_dtype == BF16 else np.float32) if want_grad else None
+    ptrs = (C.c_void_p * len(comms))(*[_ptr(c) + first * stride for c in comms])
+    ad = _Adam(lr, beta1, beta2, delta)
+    rc = lib().orc_reduce_adam(C.byref(cfg.c()), n, ptrs, len(comms), first, count, C.byref(ad),
+                               _ptr(m) if n_out else None, _ptr(v) if n_out else None, _ptr(theta) if n_out else None,
+                               _ptr(out) if (want_grad and n_out) else None)
     if rc != 0:
         raise ValueError("oracle: bad configuration")
     return out

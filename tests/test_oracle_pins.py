@@ -2,6 +2,7 @@
 
 None of these tests touches the CUDA library.  Each names the statement it checks.
 """
+import dataclasses
 import itertools
 import os
 
@@ -501,3 +502,110 @@ def test_non_finite_inputs():
     assert list(tr["q"]) == [0, 7, -8, 1, 7] and sat == 1
     e = state.view(np.float32)[:5]
     assert e[0] == 0 and e[1] == 0 and e[2] == 0 and np.isfinite(e).all()
+
+
+# ---------------------------------------------------------------- Adam-family step fused behind Eq. 8
+
+def _codes_to_comm(cfg, qs):
+    """A one-partition communication buffer holding the given codes (via the oracle's own packing routine)."""
+    n = len(qs)
+    comm = orc.new_comm(cfg, n)
+    packed = orc.pack_codes(np.asarray(qs, dtype=np.int32), cfg.bits)
+    comm[:packed.size] = packed
+    return comm
+
+
+def test_adam_family_hand_worked_example():
+    ex = {}
+    for line in open(os.path.join(GOLDEN, "adam_family_worked_example.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        k, *vals = line.split()
+        ex[k] = [float(x) for x in vals]
+    cfg = orc.OracleConfig(bits=int(ex["p"][0]), s=ex["s"][0], state_fmt=orc.STATE_NONE, grad_dtype=orc.F32, out_dtype=orc.F32)
+    comms = [_codes_to_comm(cfg, [int(q) for q in ex["qa"]]), _codes_to_comm(cfg, [int(q) for q in ex["qb"]])]
+    m, v, th = (np.array(ex[k], dtype=np.float32) for k in ("m0", "v0", "theta0"))
+    g = orc.reduce_adam(cfg, 4, comms, m, v, th, lr=ex["eta"][0], beta1=ex["beta1"][0], beta2=ex["beta2"][0],
+                        delta=ex["delta"][0], want_grad=True)
+    assert g.tolist() == ex["g"] and m.tolist() == ex["m1"] and v.tolist() == ex["v1"] and th.tolist() == ex["theta1"]
+
+
+def test_adam_family_sign_update_special_case():
+    """beta1 = beta2 = 1, delta = 0: m = g, v = g^2, so theta moves by eta * sign(g) wherever g != 0 (up to the
+    rounding of the square, the root, the quotient and the product: a few ulp of eta)."""
+    rng = np.random.default_rng(3)
+    n = 4096
+    cfg = orc.OracleConfig(bits=4, s=2.0 ** 6, state_fmt=orc.STATE_NONE, grad_dtype=orc.F32, out_dtype=orc.F32)
+    comms = [_codes_to_comm(cfg, rng.integers(-8, 8, n)) for _ in range(3)]
+    g = orc.reduce(cfg, n, comms)
+    m, v = rng.normal(size=n).astype(np.float32), rng.random(n).astype(np.float32)
+    th0 = rng.normal(size=n).astype(np.float32)
+    th = th0.copy()
+    orc.reduce_adam(cfg, n, comms, m, v, th, lr=0.125, beta1=1.0, beta2=1.0, delta=0.0)
+    nz = g != 0
+    assert nz.sum() > n // 2
+    assert np.array_equal(m, g) and np.array_equal(v, g * g)
+    step = (th0.astype(np.float64) - th.astype(np.float64))
+    assert np.allclose(step[nz], 0.125 * np.sign(g[nz]), rtol=0, atol=1e-6)
+    assert np.array_equal(th[~nz], th0[~nz]) or np.isnan(th[~nz]).all()      # g = 0: 0/0, the update is undefined there
+
+
+def test_adam_family_constant_gradient_closed_form():
+    """From m = v = 0 under a constant gradient: m_k = (1 - (1-b1)^k) g, v_k = (1 - (1-b2)^k) g^2."""
+    n, K, b1, b2 = 64, 6, 0.1, 0.01
+    cfg = orc.OracleConfig(bits=8, s=2.0 ** 4, state_fmt=orc.STATE_NONE, grad_dtype=orc.F32, out_dtype=orc.F32)
+    comms = [_codes_to_comm(cfg, np.arange(-32, 32))]
+    g = orc.reduce(cfg, n, comms).astype(np.float64)
+    m, v, th = np.zeros(n, np.float32), np.zeros(n, np.float32), np.ones(n, np.float32)
+    th64 = np.ones(n)
+    for k in range(1, K + 1):
+        orc.reduce_adam(cfg, n, comms, m, v, th, lr=1e-3, beta1=b1, beta2=b2, delta=1e-8)
+        mk, vk = (1 - (1 - b1) ** k) * g, (1 - (1 - b2) ** k) * g * g
+        th64 = th64 - 1e-3 / np.sqrt(vk + 1e-8) * mk
+        assert np.allclose(m, mk, rtol=1e-5, atol=1e-9) and np.allclose(v, vk, rtol=1e-5, atol=1e-12)
+    assert np.allclose(th, th64, rtol=1e-5, atol=1e-7)
+
+
+def test_adam_family_matches_float64_definition_and_unfused_path():
+    """Random moments and codes: the fused step equals Eq. 8 followed by the float64 formulas; a swapped beta, a
+    missing square or delta outside the root would all break the tolerance."""
+    rng = np.random.default_rng(11)
+    n = 5000
+    for mode in (orc.SCALE_FIXED, orc.SCALE_BLOCK_ABSMAX):
+        cfg = orc.OracleConfig(bits=4, scale_mode=mode, block_size=64, s=2.0 ** 10, s_e=2.0 ** 12, state_fmt=orc.STATE_NONE,
+                               grad_dtype=orc.F32, out_dtype=orc.BF16, num_partitions=3)
+        comms = []
+        for w in range(4):
+            comm = orc.new_comm(cfg, n)
+            orc.send_step(cfg, rng.normal(0, 2e-3, n).astype(np.float32), orc.new_state(cfg, n), comm, 1)
+            comms.append(comm)
+        cfg32 = dataclasses.replace(cfg, out_dtype=orc.F32)
+        g = orc.reduce(cfg32, n, comms).astype(np.float64)
+        m0, v0, th0 = rng.normal(0, 1e-3, n).astype(np.float32), (rng.random(n) * 1e-6).astype(np.float32), rng.normal(size=n).astype(np.float32)
+        m, v, th = m0.copy(), v0.copy(), th0.copy()
+        gb = orc.reduce_adam(cfg, n, comms, m, v, th, lr=1e-2, beta1=0.1, beta2=0.05, delta=1e-10, want_grad=True)
+        assert np.array_equal(gb, orc.reduce(cfg, n, comms)), "the optional gradient output is Eq. 8 in the output type"
+        wm, wv, wth = defn.adam_family_step(g, m0, v0, th0, lr=1e-2, beta1=0.1, beta2=0.05, delta=1e-10)
+        assert np.allclose(m, wm, rtol=1e-5, atol=1e-9) and np.allclose(v, wv, rtol=1e-5, atol=1e-13)
+        assert np.allclose(th, wth, rtol=1e-5, atol=1e-6)
+        # the planted mistakes are far outside those tolerances
+        bm, bv, bth = defn.adam_family_step(g, m0, v0, th0, lr=1e-2, beta1=0.9, beta2=0.05, delta=1e-10)
+        assert not np.allclose(m, bm, rtol=1e-3, atol=1e-7)
+        # part by part gives the same as all parts at once
+        m2, v2, th2 = m0.copy(), v0.copy(), th0.copy()
+        pos = 0
+        for j in range(3):
+            cnt = orc.partition_elems(cfg, n, j)
+            orc.reduce_adam(cfg, n, comms, m2[pos:pos + cnt], v2[pos:pos + cnt], th2[pos:pos + cnt], lr=1e-2, beta1=0.1,
+                            beta2=0.05, delta=1e-10, first=j, count=1)
+            pos += cnt
+        assert np.array_equal(m2, m) and np.array_equal(v2, v) and np.array_equal(th2, th)
+
+
+def test_adam_family_zero_gradient_decays_the_moments():
+    n = 256
+    cfg = orc.OracleConfig(bits=4, s=2.0 ** 8, state_fmt=orc.STATE_NONE, grad_dtype=orc.F32, out_dtype=orc.F32)
+    comms = [orc.new_comm(cfg, n), orc.new_comm(cfg, n)]          # all codes 0
+    m, v, th = np.full(n, 0.5, np.float32), np.full(n, 4.0, np.float32), np.zeros(n, np.float32)
+    orc.reduce_adam(cfg, n, comms, m, v, th, lr=1.0, beta1=0.5, beta2=0.75, delta=0.0)
+    assert (m == 0.25).all() and (v == 1.0).all() and (th == -0.25).all()
