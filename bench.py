@@ -378,6 +378,33 @@ def sweep(args, device):
                          l2_resident=bool(nsets * (workers * pb + n * osz) < L2_BYTES)))
         print(json.dumps(rows[-1]), flush=True)
 
+    def adam_case(label, n, workers, **kw):
+        if args.sweep_filter and args.sweep_filter not in "reduce+adam: " + label:
+            return
+        base = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=512, state_fmt=2,
+                    grad_dtype=1, out_dtype=1, num_partitions=8)
+        base.update(kw)
+        cfg = loco.Config(**base)
+        pb = loco.loco_packed_bytes(cfg, n)
+        nsets = sets_for(workers * pb + n * 12)
+        gen = torch.Generator(device=device)
+        gen.manual_seed(4)
+        packed = [[torch.randint(0, 256, (max(pb, 16),), dtype=torch.uint8, device=device, generator=gen) for _ in range(workers)]
+                  for _ in range(nsets)]
+        ms = [torch.zeros(n, dtype=torch.float32, device=device) for _ in range(nsets)]
+        vs = [torch.zeros(n, dtype=torch.float32, device=device) for _ in range(nsets)]
+        ths = [torch.ones(n, dtype=torch.float32, device=device) for _ in range(nsets)]
+        torch.cuda.synchronize()
+        us = _time_launches(lambda i, st: loco.loco_unpack_dequant_reduce_adam(cfg, packed[i], n, ms[i], vs[i], ths[i], lr=1e-3, beta1=0.1,
+                                                                                 beta2=0.001, delta=1e-16, stream=st),
+                            nsets, max(12, min(200, 4 * nsets)), streams)
+        bpe = workers * cfg.bits / 8 + 24
+        gbs = bpe * n / us / 1e3
+        rows.append(dict(kernel="reduce+adam", case=label, n=n, workers=workers, bytes_per_elem=round(bpe, 3), us=round(us, 2),
+                         hbm_gbs=round(gbs, 1), frac=round(gbs / peak, 3), grad_gbs=round(4 * n / us / 1e3, 1),
+                         l2_resident=bool(nsets * (workers * pb + n * 12) < L2_BYTES)))
+        print(json.dumps(rows[-1]), flush=True)
+
     M = 25_000_000
     for log2n in (16, 18, 20, 22, 24, 27, 30):
         send_case("bf16 g, int8 state, 4 bit, fixed", 1 << log2n)
@@ -404,6 +431,10 @@ def sweep(args, device):
     reduce_case("4 bit, bf16 out, fixed, 3 workers (division by 3)", M, 3)
     reduce_case("4 bit, bf16 out, block-256 absmax", M, 8, scale_mode=1)
     reduce_case("4 bit, bf16 out, block-32 absmax", M, 8, scale_mode=1, block_size=32)
+    for N in (1, 8, 16):
+        adam_case("4 bit, fixed, Adam-family step fused, no gradient output", M, N)
+    adam_case("8 bit, fixed, Adam-family step fused, no gradient output", M, 8, bits=8)
+    adam_case("4 bit, fixed, Adam-family step fused, no gradient output", 1 << 27, 8)
     print("| kernel | case | n | workers | B/elem | us/launch | HBM GB/s | of %s peak %.0f | gradient GB/s | L2-resident |" % (peak_kind, peak))
     print("|---|---|---|---|---|---|---|---|---|---|")
     for r in rows:

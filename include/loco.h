@@ -152,6 +152,30 @@ int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_pa
                                int32_t num_workers, uint64_t n, int32_t first_partition,
                                int32_t partition_count, void *d_out, void *stream);
 
+/*
+ * Receive pass fused with the optimizer's update -- Algorithm 1 step 3 ("use g~_k to update theta_k") with the paper's
+ * Adam-family equations and Adam's pre-conditioner:
+ *     g      = Eq. 8 (as loco_unpack_dequant_reduce, kept in fp32)
+ *     m      = (1 - beta1) m + beta1 g          beta1, beta2 weight the NEW term, as the paper writes them
+ *     v      = (1 - beta2) v + beta2 g^2
+ *     theta  = theta - lr / sqrt(v + delta) * m      no bias correction, delta inside the root (the printed form)
+ * d_m, d_v, d_theta: fp32 DEVICE arrays holding the same elements d_out would (the valid elements of the parts,
+ * contiguously), 16-byte aligned, updated in place.  d_grad_out may be NULL; otherwise it also receives g in out_dtype.
+ * The averaged gradient then never travels through HBM: 24 B/element of optimizer state plus the packed codes.
+ * One launch, no allocation, no synchronisation.  Errors: as loco_unpack_dequant_reduce, plus ARG for a null adam /
+ * moment pointer or beta outside [0, 1], non-finite lr, negative delta.
+ */
+typedef struct {
+    float lr;       /* eta */
+    float beta1;    /* weight of the new gradient in the first moment  */
+    float beta2;    /* weight of the new squared gradient in the second moment */
+    float delta;    /* >= 0, added to v inside the square root */
+} loco_adam_t;
+int loco_unpack_dequant_reduce_adam(const loco_config_t *cfg, const void *const *d_packed, int32_t num_workers,
+                                    uint64_t n, int32_t first_partition, int32_t partition_count,
+                                    const loco_adam_t *adam, float *d_m, float *d_v, float *d_theta,
+                                    void *d_grad_out, void *stream);
+
 /* ---- host-buffer variants ------------------------------------------------------------------
  * The same two passes for callers whose gradient and communication buffers live in HOST memory
  * (pinned memory makes the copies asynchronous).  Each call enqueues, on `stream`: the

@@ -195,27 +195,31 @@ SendKernel pick_send(const loco_config_t *c, int mode, int var) {
 
 using ReduceFn = void (*)(const ReduceParams);
 
-template <int OUT, int BITS>
-ReduceFn pick_reduce_mode(int mode, int path) {
-    if (mode != MODE_FIXED) return loco_reduce_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>;
+template <int OUT, int BITS, bool ADAM>
+ReduceFn pick_reduce_path(int mode, int path) {
+    if (mode != MODE_FIXED) return loco_reduce_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL, ADAM>;
     switch (path) {
-    case PATH_INT: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_INT>;
-    case PATH_MUL: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>;
-    case PATH_NEWTON: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON>;
-    default: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE>;
+    case PATH_INT: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_INT, ADAM>;
+    case PATH_MUL: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_MUL, ADAM>;
+    case PATH_NEWTON: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON, ADAM>;
+    default: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE, ADAM>;
     }
+}
+template <int OUT, int BITS>
+ReduceFn pick_reduce_mode(int mode, int path, bool adam) {
+    return adam ? pick_reduce_path<OUT, BITS, true>(mode, path) : pick_reduce_path<OUT, BITS, false>(mode, path);
 }
 template <int OUT>
-ReduceFn pick_reduce_bits(int bits, int mode, int path) {
+ReduceFn pick_reduce_bits(int bits, int mode, int path, bool adam) {
     switch (bits) {
-    case 2: return pick_reduce_mode<OUT, 2>(mode, path);
-    case 4: return pick_reduce_mode<OUT, 4>(mode, path);
-    default: return pick_reduce_mode<OUT, 8>(mode, path);
+    case 2: return pick_reduce_mode<OUT, 2>(mode, path, adam);
+    case 4: return pick_reduce_mode<OUT, 4>(mode, path, adam);
+    default: return pick_reduce_mode<OUT, 8>(mode, path, adam);
     }
 }
-ReduceFn pick_reduce(const loco_config_t *c, int mode, int path) {
-    return c->out_dtype == LOCO_BF16 ? pick_reduce_bits<GRAD_BF16>(c->bits, mode, path)
-                                     : pick_reduce_bits<GRAD_F32>(c->bits, mode, path);
+ReduceFn pick_reduce(const loco_config_t *c, int mode, int path, bool adam) {
+    return c->out_dtype == LOCO_BF16 ? pick_reduce_bits<GRAD_BF16>(c->bits, mode, path, adam)
+                                     : pick_reduce_bits<GRAD_F32>(c->bits, mode, path, adam);
 }
 
 unsigned grid_x_for(uint64_t rows_per_partition, int partitions, int ctas_per_sm) {
@@ -423,19 +427,29 @@ int loco_compensate_quantize_pack(loco_state_t *st, const void *d_grad, void *d_
     return LOCO_OK;
 }
 
-int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_packed, int32_t num_workers,
-                               uint64_t n, int32_t first_partition, int32_t partition_count, void *d_out,
-                               void *stream) {
+}  // extern "C"
+
+namespace {
+
+// The receive pass; with `ad` the Adam-family step is applied to the averaged gradient in the same kernel and d_out
+// (the gradient itself) becomes optional.
+int reduce_launch(const loco_config_t *cfg, const void *const *d_packed, int32_t num_workers, uint64_t n,
+                  int32_t first_partition, int32_t partition_count, void *d_out, const loco_adam_t *ad, float *d_m,
+                  float *d_v, float *d_theta, void *stream) {
     const int rc = check_config(cfg);
     if (rc != LOCO_OK) return rc;
     if (num_workers < 1 || first_partition < 0 || partition_count < 0 ||
         first_partition + partition_count > cfg->num_partitions) return LOCO_ERR_ARG;
     if (num_workers > 64) return LOCO_ERR_UNSUPPORTED;
+    if (ad && !(std::isfinite(ad->lr) && ad->beta1 >= 0.0f && ad->beta1 <= 1.0f && ad->beta2 >= 0.0f && ad->beta2 <= 1.0f &&
+                ad->delta >= 0.0f && std::isfinite(ad->delta))) return LOCO_ERR_ARG;
     if (n == 0 || partition_count == 0) return LOCO_OK;
     const Layout L = make_layout(cfg, n);
     if (static_cast<uint64_t>(first_partition) * L.lp >= n) return LOCO_OK;      // nothing valid there
-    if (!d_packed || !d_out) return LOCO_ERR_ARG;
+    if (!d_packed || (!ad && !d_out)) return LOCO_ERR_ARG;
+    if (ad && (!d_m || !d_v || !d_theta)) return LOCO_ERR_ARG;
     if (!aligned16(d_out)) return LOCO_ERR_ALIGN;
+    if (ad && (!aligned16(d_m) || !aligned16(d_v) || !aligned16(d_theta))) return LOCO_ERR_ALIGN;
     ReduceParams P;
     std::memset(&P, 0, sizeof(P));
     for (int w = 0; w < num_workers; ++w) {
@@ -511,9 +525,15 @@ int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_pa
     }
     const int path = mode == MODE_BLOCK ? PATH_MUL
                      : (P.int_path ? PATH_INT : (P.gen_mode == 0 ? PATH_MUL : (P.gen_mode == 1 ? PATH_NEWTON : PATH_DIVIDE)));
-    ReduceFn fn = pick_reduce(cfg, mode, path);
-    static int occ_cache[2][3][2][4] = {};
-    int &occ = occ_cache[cfg->out_dtype == LOCO_BF16][cfg->bits == 2 ? 0 : (cfg->bits == 4 ? 1 : 2)][mode][path];
+    if (ad) {
+        P.adam_m = d_m; P.adam_v = d_v; P.adam_theta = d_theta;
+        P.lr = ad->lr; P.beta1 = ad->beta1; P.beta2 = ad->beta2; P.delta = ad->delta;
+        const volatile float o1 = 1.0f - ad->beta1, o2 = 1.0f - ad->beta2;       // rounded once to fp32
+        P.omb1 = o1; P.omb2 = o2;
+    }
+    ReduceFn fn = pick_reduce(cfg, mode, path, ad != nullptr);
+    static int occ_cache[2][3][2][4][2] = {};
+    int &occ = occ_cache[cfg->out_dtype == LOCO_BF16][cfg->bits == 2 ? 0 : (cfg->bits == 4 ? 1 : 2)][mode][path][ad != nullptr];
     if (occ == 0) {
         int v = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, fn, kThreads, 0) != cudaSuccess || v < 1) {
@@ -528,6 +548,25 @@ int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_pa
     if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;
     g_launches.fetch_add(1);
     return LOCO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int loco_unpack_dequant_reduce(const loco_config_t *cfg, const void *const *d_packed, int32_t num_workers,
+                               uint64_t n, int32_t first_partition, int32_t partition_count, void *d_out,
+                               void *stream) {
+    return reduce_launch(cfg, d_packed, num_workers, n, first_partition, partition_count, d_out, nullptr, nullptr, nullptr,
+                         nullptr, stream);
+}
+
+int loco_unpack_dequant_reduce_adam(const loco_config_t *cfg, const void *const *d_packed, int32_t num_workers,
+                                    uint64_t n, int32_t first_partition, int32_t partition_count, const loco_adam_t *adam,
+                                    float *d_m, float *d_v, float *d_theta, void *d_grad_out, void *stream) {
+    if (!adam) return LOCO_ERR_ARG;
+    return reduce_launch(cfg, d_packed, num_workers, n, first_partition, partition_count, d_grad_out, adam, d_m, d_v,
+                         d_theta, stream);
 }
 
 uint64_t loco_send_host_workspace_bytes(const loco_config_t *cfg, uint64_t n) {

@@ -84,6 +84,9 @@ struct ReduceParams {
     float inv_s;                     // fl(1/s) for gen_mode 1
     int gen_mode;                    // generic FIXED path: 0 multiply, 1 Newton-Raphson division, 2 IEEE division
     int out_align32;                 // the output pointer is 32-byte aligned: 256-bit stores may be used
+    // fused Adam-family step (kernels instantiated with ADAM): moments and weights of the same elements as `out`
+    float *adam_m, *adam_v, *adam_theta;
+    float lr, beta1, beta2, omb1, omb2, delta;
 };
 
 // ------------------------------------------------------------------------------------------
@@ -1004,6 +1007,60 @@ __device__ __forceinline__ float div_workers(const ReduceParams &P, float acc) {
     return __fdiv_rn(acc, P.n_workers_f);
 }
 
+// The paper's Adam-family step on the 16 averaged gradients of one lane (Algorithm 1 step 3: the update that
+// consumes g~): m = (1-b1) m + b1 g; v = (1-b2) v + b2 g^2; theta -= eta / sqrt(v + delta) * m.  One IEEE fp32
+// operation per written operation (scalar intrinsics: nothing is contracted), IEEE square root and division.
+// The averaged gradient never goes through HBM unless the caller asks for it.
+struct AdamRegs { float m[16], v[16], t[16]; };
+
+// Start the loads of a lane's 16 moments and weights (issued before the workers' codes are summed, so that they
+// are in flight meanwhile).  Only for lanes whose 16 elements all exist.
+__device__ __forceinline__ void adam_load16(const ReduceParams &P, unsigned long long oi, AdamRegs &R) {
+    const float *pm = P.adam_m + oi, *pv = P.adam_v + oi, *pt = P.adam_theta + oi;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const uint4 a = ld_stream16(pm + 4 * j), b = ld_stream16(pv + 4 * j), c = ld_stream16(pt + 4 * j);
+        R.m[4 * j] = __uint_as_float(a.x); R.m[4 * j + 1] = __uint_as_float(a.y); R.m[4 * j + 2] = __uint_as_float(a.z); R.m[4 * j + 3] = __uint_as_float(a.w);
+        R.v[4 * j] = __uint_as_float(b.x); R.v[4 * j + 1] = __uint_as_float(b.y); R.v[4 * j + 2] = __uint_as_float(b.z); R.v[4 * j + 3] = __uint_as_float(b.w);
+        R.t[4 * j] = __uint_as_float(c.x); R.t[4 * j + 1] = __uint_as_float(c.y); R.t[4 * j + 2] = __uint_as_float(c.z); R.t[4 * j + 3] = __uint_as_float(c.w);
+    }
+}
+
+template <int OUT>
+__device__ __forceinline__ void adam_finish16(const ReduceParams &P, unsigned long long oi, const float (&g)[16],
+                                              unsigned long long left, bool wide32, AdamRegs &R) {
+    float *pm = P.adam_m + oi, *pv = P.adam_v + oi, *pt = P.adam_theta + oi;
+    if (left >= 16) {                                    // R was loaded by adam_load16
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            R.m[j] = __fadd_rn(__fmul_rn(P.omb1, R.m[j]), __fmul_rn(P.beta1, g[j]));
+            R.v[j] = __fadd_rn(__fmul_rn(P.omb2, R.v[j]), __fmul_rn(P.beta2, __fmul_rn(g[j], g[j])));
+            const float eta_k = __fdiv_rn(P.lr, __fsqrt_rn(__fadd_rn(R.v[j], P.delta)));
+            R.t[j] = __fsub_rn(R.t[j], __fmul_rn(eta_k, R.m[j]));
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            st_stream16(pm + 4 * j, make_uint4(__float_as_uint(R.m[4 * j]), __float_as_uint(R.m[4 * j + 1]), __float_as_uint(R.m[4 * j + 2]), __float_as_uint(R.m[4 * j + 3])));
+            st_stream16(pv + 4 * j, make_uint4(__float_as_uint(R.v[4 * j]), __float_as_uint(R.v[4 * j + 1]), __float_as_uint(R.v[4 * j + 2]), __float_as_uint(R.v[4 * j + 3])));
+            st_stream16(pt + 4 * j, make_uint4(__float_as_uint(R.t[4 * j]), __float_as_uint(R.t[4 * j + 1]), __float_as_uint(R.t[4 * j + 2]), __float_as_uint(R.t[4 * j + 3])));
+        }
+    } else {
+        const int cnt = static_cast<int>(left);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            if (j < cnt) {
+                const float mk = __fadd_rn(__fmul_rn(P.omb1, pm[j]), __fmul_rn(P.beta1, g[j]));
+                const float vk = __fadd_rn(__fmul_rn(P.omb2, pv[j]), __fmul_rn(P.beta2, __fmul_rn(g[j], g[j])));
+                const float eta_k = __fdiv_rn(P.lr, __fsqrt_rn(__fadd_rn(vk, P.delta)));
+                pm[j] = mk;
+                pv[j] = vk;
+                pt[j] = __fsub_rn(pt[j], __fmul_rn(eta_k, mk));
+            }
+        }
+    }
+    if (P.out) store_out16<OUT>(P.out, oi, g, left, wide32);
+}
+
 // (a ^ b) & c in one instruction
 __device__ __forceinline__ unsigned xor_and(unsigned a, unsigned b, unsigned c) {
     unsigned d;
@@ -1053,9 +1110,10 @@ struct WideSums {
 // PATH_INT: the integer-sum path (only with the global scale); otherwise the generic path with dec(q; s) as a multiply
 // (also the block-scaled form), as the Newton-Raphson division, or as the IEEE division.  Separate kernels, so that each
 // path gets the registers and the occupancy it wants and no per-element choice is left.
+// ADAM: the Adam-family update of the optimizer is applied to the averaged gradient in the same pass.
 enum : int { PATH_INT = 0, PATH_MUL = 1, PATH_NEWTON = 2, PATH_DIVIDE = 3 };
-template <int OUT, int BITS, int MODE, int PATH>
-__global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParams P) {
+template <int OUT, int BITS, int MODE, int PATH, bool ADAM>
+__global__ void __launch_bounds__(kThreads, ADAM ? 3 : 1) loco_reduce_kernel(const ReduceParams P) {
     constexpr unsigned kRowBytes = kWide * BITS / 8;                  // code bytes of one wide row
     const int lane = threadIdx.x & 31;
     const unsigned long long part = blockIdx.y;                       // relative to P.first
@@ -1075,11 +1133,16 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
 
     if (PATH == PATH_INT) {
         // code areas below 4 GiB (checked by the host): row offsets fit 32 bits
-        constexpr int kUnroll = 2;
+        constexpr int kUnroll = ADAM ? 1 : 2;
         for (unsigned r = warp; r < rows; r += kUnroll * nwarps) {
             WideSums<BITS> sums[kUnroll];
             unsigned off[kUnroll];
             bool ok[kUnroll];
+            AdamRegs AR;
+            if (ADAM) {
+                const unsigned long long o = static_cast<unsigned long long>(r) * kWide + lane_elem;
+                if (o + 16 <= valid) adam_load16(P, out0 + o, AR);
+            }
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 sums[u].clear();
@@ -1110,7 +1173,8 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
                     const float acc = __fmaf_rn(sums[u].get(j), P.ra, P.rb);
                     res[j] = P.div_mode == 0 ? acc : div_workers(P, acc);
                 }
-                store_out16<OUT>(P.out, out0 + o, res, valid - o, wide32);
+                if (ADAM) adam_finish16<OUT>(P, out0 + o, res, valid - o, wide32, AR);
+                else store_out16<OUT>(P.out, out0 + o, res, valid - o, wide32);
             }
         }
         return;
@@ -1153,6 +1217,8 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
         f32x2 acc2[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc2[i] = 0ull;
+        AdamRegs AR;
+        if (ADAM && o + 16 <= valid) adam_load16(P, out0 + o, AR);
         for (int g = 0; g < groups; ++g) {
             Group nxt;
             if (g + 1 < groups) load_group(r, g + 1, nxt);
@@ -1198,7 +1264,8 @@ __global__ void __launch_bounds__(kThreads) loco_reduce_kernel(const ReduceParam
             res[2 * i] = div_workers(P, a);                                          // the 1/N of Eq. 8
             res[2 * i + 1] = div_workers(P, b);
         }
-        store_out16<OUT>(P.out, out0 + o, res, valid - o, wide32);
+        if (ADAM) adam_finish16<OUT>(P, out0 + o, res, valid - o, wide32, AR);
+        else store_out16<OUT>(P.out, out0 + o, res, valid - o, wide32);
     }
 }
 

@@ -29,7 +29,8 @@ EXPORTS = ("loco_state_bytes", "loco_packed_bytes", "loco_partition_bytes", "loc
            "loco_last_status", "loco_status_string", "loco_launch_count",
            "loco_send_host_workspace_bytes", "loco_reduce_host_workspace_bytes",
            "loco_compensate_quantize_pack_host", "loco_unpack_dequant_reduce_host",
-           "loco_unpack_dequant_reduce_host_noalloc", "loco_selfcheck_block_division")
+           "loco_unpack_dequant_reduce_host_noalloc", "loco_selfcheck_block_division",
+           "loco_unpack_dequant_reduce_adam")
 NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
@@ -44,6 +45,10 @@ class loco_config_t(C.Structure):
                 ("s", C.c_float), ("s_e", C.c_float), ("beta", C.c_float),
                 ("reset_period", C.c_int32), ("state_fmt", C.c_int32), ("grad_dtype", C.c_int32),
                 ("out_dtype", C.c_int32), ("num_partitions", C.c_int32), ("collect_stats", C.c_int32)]
+
+
+class loco_adam_t(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("delta", C.c_float)]
 
 
 @dataclass
@@ -108,6 +113,8 @@ def lib() -> C.CDLL:
         L.loco_unpack_dequant_reduce_host.argtypes = [cp, C.POINTER(vp), i32, u64, i32, i32, vp, vp, u64, vp]
         L.loco_unpack_dequant_reduce_host_noalloc.restype = C.c_int
         L.loco_unpack_dequant_reduce_host_noalloc.argtypes = [cp, C.POINTER(vp), i32, u64, i32, i32, vp, vp]
+        L.loco_unpack_dequant_reduce_adam.restype = C.c_int
+        L.loco_unpack_dequant_reduce_adam.argtypes = [cp, C.POINTER(vp), i32, u64, i32, i32, C.POINTER(loco_adam_t), vp, vp, vp, vp, vp]
         L.loco_selfcheck_block_division.restype = C.c_int
         L.loco_selfcheck_block_division.argtypes = [C.POINTER(u64)]
         L.loco_last_status.restype = C.c_int
@@ -305,3 +312,25 @@ def loco_selfcheck_block_division():
     out = (C.c_uint64 * 2)(0, 0)
     _check(lib().loco_selfcheck_block_division(out), "loco_selfcheck_block_division")
     return int(out[0]), int(out[1])
+
+
+def loco_unpack_dequant_reduce_adam(cfg: Config, packed: Sequence, n: int, m: torch.Tensor, v: torch.Tensor, theta: torch.Tensor,
+                                    *, lr: float, beta1: float, beta2: float, delta: float, grad_out: Optional[torch.Tensor] = None,
+                                    first_partition: int = 0, partition_count: Optional[int] = None, stream=None) -> None:
+    """Receive pass (Eq. 8) fused with the paper's Adam-family step: m, v, theta (fp32 CUDA tensors covering the valid
+    elements of the parts) are updated in place; grad_out, if given, also receives the averaged gradient."""
+    if partition_count is None:
+        partition_count = cfg.num_partitions - first_partition
+    ptrs = (C.c_void_p * len(packed))(*[p if isinstance(p, int) else _dev_ptr(p) for p in packed])
+    need = sum(loco_partition_elems(cfg, n, j) for j in range(first_partition, first_partition + partition_count))
+    for t in (m, v, theta):
+        if t.dtype != torch.float32 or t.numel() < need:
+            raise ValueError("m, v, theta must be float32 with at least %d elements" % need)
+    if grad_out is not None:
+        want = torch.bfloat16 if cfg.out_dtype == BF16 else torch.float32
+        if grad_out.dtype != want or grad_out.numel() < need:
+            raise ValueError("grad_out must be %s with at least %d elements" % (want, need))
+    ad = loco_adam_t(lr, beta1, beta2, delta)
+    _check(lib().loco_unpack_dequant_reduce_adam(C.byref(cfg.c()), ptrs, len(packed), n, first_partition, partition_count,
+                                                 C.byref(ad), _dev_ptr(m), _dev_ptr(v), _dev_ptr(theta), _dev_ptr(grad_out),
+                                                 _stream_ptr(stream)), "loco_unpack_dequant_reduce_adam")
