@@ -567,6 +567,26 @@ __device__ __forceinline__ float qmax_over(float c, float a) {
     return __fdiv_rn(c, a);
 }
 
+// The same without the fallback, for callers that have already sent every a outside [2^-100, 2^100] elsewhere.
+__device__ __forceinline__ float qmax_over_midrange(float c, float a) {
+    float x;
+    asm("rcp.approx.f32 %0, %1;" : "=f"(x) : "f"(a));
+    const float q0 = __fmul_rn(c, x);
+    const float rem = __fmaf_rn(-q0, a, c);
+    return __fmaf_rn(rem, x, q0);
+}
+__device__ __forceinline__ bool in_midrange(float a) { return __float_as_uint(a) - 0x0d800000u <= 0x71800000u - 0x0d800000u; }
+
+// max over aligned groups of `lanes` lanes (2, 4, 8 or 16) in a fixed number of steps, without a loop
+__device__ __forceinline__ float group_max16(float v, int lanes) {
+#pragma unroll
+    for (int o = 1; o < 16; o <<= 1) {
+        const float w = __shfl_xor_sync(kFull, v, o);
+        v = o < lanes ? fmaxf(v, w) : v;
+    }
+    return v;
+}
+
 // mismatch[0]: amax / c, mismatch[1]: c / amax, over all positive finite floats, for c = 1, 7, 127
 __global__ void loco_division_selfcheck_kernel(unsigned long long *mismatch) {
     const float cs[3] = {1.0f, 7.0f, 127.0f};
@@ -579,6 +599,7 @@ __global__ void loco_division_selfcheck_kernel(unsigned long long *mismatch) {
             const float c = cs[i];
             if (__float_as_uint(div_by_qmax(a, c, __frcp_rn(c))) != __float_as_uint(__fdiv_rn(a, c))) ++bad0;
             if (__float_as_uint(qmax_over(c, a)) != __float_as_uint(__fdiv_rn(c, a))) ++bad1;
+            if (in_midrange(a) && __float_as_uint(qmax_over_midrange(c, a)) != __float_as_uint(__fdiv_rn(c, a))) ++bad1;
         }
     }
     if (bad0) atomicAdd(mismatch, bad0);
@@ -697,19 +718,18 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     float mult = K.s, scale = 0.0f;
     if (MODE == MODE_BLOCK) {
         float amax = 0.0f;
-        f32x2 acc = zero2;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             float a, b;
             unpk2(h2[k], a, b);
             amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
-            acc = ffma2(h2[k], zero2, acc);
         }
-        bad_bits |= (static_cast<unsigned>(acc) | static_cast<unsigned>(acc >> 32)) & 0x7fffffffu;
-        if (__any_sync(kFull, bad_bits != 0u)) return false;
-        amax = warp_group_max(amax, lanes_per_block);
+        amax = group_max16(amax, lanes_per_block);
+        // g is finite here, so h can only be +-Inf (an overflowing sum), never NaN, and the maximum shows it.  A block
+        // maximum outside [2^-100, 2^100] (other than 0) also leaves the row to the careful routine, which divides.
+        if (__any_sync(kFull, bad_bits != 0u || !(amax == 0.0f || in_midrange(amax)))) return false;
         scale = amax > 0.0f ? div_by_qmax(amax, hi, 1.0f / hi) : 0.0f;
-        mult = amax > 0.0f ? qmax_over(hi, amax) : 0.0f;
+        mult = amax > 0.0f ? qmax_over_midrange(hi, amax) : 0.0f;
     }
 
     // ---- Eq. 1 / Eq. 3: q = round_p-bit(h x s);  step 2: d, Eq. 5 ---------------------------------------------
@@ -767,9 +787,11 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
                     unpk2(en2[k], a, b);
                     amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
                 }
-                amax = warp_group_max(amax, lanes_per_block);
+                amax = group_max16(amax, lanes_per_block);
+                // nothing of the state has been written yet, and the codes stored above are what the careful routine stores
+                if (__any_sync(kFull, !(amax == 0.0f || in_midrange(amax)))) return false;
                 escale = amax > 0.0f ? div_by_qmax(amax, 127.0f, 1.0f / 127.0f) : 0.0f;
-                emult = amax > 0.0f ? qmax_over(127.0f, amax) : 0.0f;
+                emult = amax > 0.0f ? qmax_over_midrange(127.0f, amax) : 0.0f;
             }
             const f32x2 emult2 = dup2(emult);
             int q[16];
