@@ -40,6 +40,8 @@
  *     amax/qmax, and is defined here only so that both sides agree;
  *   - non-finite h: NaN gives code 0, +-Inf the saturated code, and in both
  *     cases the compression error of that element is taken as 0;
+ *   - the element-wise clipping of g named in the experiments section has no stated threshold: `clip` is a
+ *     parameter (0 = off), applied to g before step 1;
  *   - Eq. 8 is summed in worker order in fp32, then divided by (float)N;
  *   - the Adam-family step is taken exactly as printed (no bias correction, delta inside the root), with
  *     eta_k = eta / sqrt(v_k + delta) evaluated as one square root and one division.
@@ -80,6 +82,8 @@ typedef struct {
     int32_t grad_dtype;     /* ORC_F32 / ORC_BF16 */
     int32_t out_dtype;      /* ORC_F32 / ORC_BF16 */
     int32_t num_partitions; /* N parts of Sec. 3.3 */
+    float   clip;           /* > 0: element-wise clipping of the local gradient to [-clip, clip] before Algorithm 1
+                               (the Sky-MoE pre-training runs of the experiments section); 0 = off */
 } orc_config;
 
 /* Optional per-element record of one send step, for the invariant tests. */
@@ -154,6 +158,7 @@ static int config_ok(const orc_config *c) {
     if (c->grad_dtype != ORC_F32 && c->grad_dtype != ORC_BF16) return 0;
     if (c->out_dtype != ORC_F32 && c->out_dtype != ORC_BF16) return 0;
     if (c->num_partitions < 1) return 0;
+    if (!(c->clip >= 0.0f) || !isfinite(c->clip)) return 0;
     return 1;
 }
 
@@ -233,8 +238,13 @@ void orc_unpack_codes(const uint8_t *bytes, uint64_t n, int32_t p, int32_t *q) {
 }
 
 static float load_grad(const orc_config *c, const void *grad, uint64_t i) {
-    if (c->grad_dtype == ORC_BF16) return bf16_to_f32(((const uint16_t *)grad)[i]);
-    return ((const float *)grad)[i];
+    float g = c->grad_dtype == ORC_BF16 ? bf16_to_f32(((const uint16_t *)grad)[i]) : ((const float *)grad)[i];
+    /* element-wise clipping of g (experiments section); a NaN stays a NaN, +-Inf becomes +-clip */
+    if (c->clip > 0.0f && !isnan(g)) {
+        if (g > c->clip) g = c->clip;
+        if (g < -c->clip) g = -c->clip;
+    }
+    return g;
 }
 
 /* Quantise one compensated value against a multiplier (s, or the block's inverse scale).

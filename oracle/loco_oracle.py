@@ -39,7 +39,8 @@ class _Cfg(C.Structure):
     _fields_ = [("bits", C.c_int32), ("scale_mode", C.c_int32), ("block_size", C.c_int32),
                 ("s", C.c_float), ("s_e", C.c_float), ("beta", C.c_float),
                 ("reset_period", C.c_int32), ("state_fmt", C.c_int32),
-                ("grad_dtype", C.c_int32), ("out_dtype", C.c_int32), ("num_partitions", C.c_int32)]
+                ("grad_dtype", C.c_int32), ("out_dtype", C.c_int32), ("num_partitions", C.c_int32),
+                ("clip", C.c_float)]
 
 
 class _Adam(C.Structure):
@@ -65,11 +66,12 @@ class OracleConfig:
     grad_dtype: int = F32
     out_dtype: int = F32
     num_partitions: int = 1
+    clip: float = 0.0
 
     def c(self) -> _Cfg:
         return _Cfg(self.bits, self.scale_mode, self.block_size, self.s, self.s_e, self.beta,
                     self.reset_period, self.state_fmt, self.grad_dtype, self.out_dtype,
-                    self.num_partitions)
+                    self.num_partitions, self.clip)
 
 
 _lib = None

@@ -609,3 +609,43 @@ def test_adam_family_zero_gradient_decays_the_moments():
     m, v, th = np.full(n, 0.5, np.float32), np.full(n, 4.0, np.float32), np.zeros(n, np.float32)
     orc.reduce_adam(cfg, n, comms, m, v, th, lr=1.0, beta1=0.5, beta2=0.75, delta=0.0)
     assert (m == 0.25).all() and (v == 1.0).all() and (th == -0.25).all()
+
+
+# ---------------------------------------------------------------- element-wise clipping of the local gradient
+
+@pytest.mark.parametrize("mode", [orc.SCALE_FIXED, orc.SCALE_BLOCK_ABSMAX])
+def test_clipping_equals_clipping_the_input_first(mode):
+    """send(clip = c, g) must be send(clip = 0, clamp(g, -c, c)) byte for byte over several iterations; a very large
+    threshold changes nothing; +-Inf becomes +-c and raises no flag; NaN is still flagged."""
+    rng = np.random.default_rng(8)
+    n, c = 3000, 2e-3
+    kw = dict(bits=4, scale_mode=mode, block_size=64, s=2.0 ** 10, s_e=2.0 ** 12, beta=0.5, reset_period=0,
+              state_fmt=orc.STATE_INT8, grad_dtype=orc.F32, out_dtype=orc.F32, num_partitions=2)
+    a, b, big = orc.OracleConfig(clip=c, **kw), orc.OracleConfig(**kw), orc.OracleConfig(clip=1e30, **kw)
+    sa, sb, sg = (orc.new_state(a, n) for _ in range(3))
+    ca, cb, cg = (orc.new_comm(a, n) for _ in range(3))
+    changed = 0
+    for k in range(1, 4):
+        g = rng.normal(0, 2e-3, n).astype(np.float32)
+        g[5], g[6] = np.inf, -np.inf
+        gc = np.clip(g, -c, c).astype(np.float32)
+        changed += int((gc != g).sum())
+        fa = orc.send_step(a, g, sa, ca, k)
+        fb = orc.send_step(b, gc, sb, cb, k)
+        assert fa == fb and fa[0] == 0
+        assert np.array_equal(ca, cb) and np.array_equal(sa, sb)
+        g2 = g.copy()
+        g2[5], g2[6] = 1.0, -1.0
+        orc.send_step(big, g2, sg, cg, k)
+    assert changed > 100
+    sref, cref = orc.new_state(b, n), orc.new_comm(b, n)
+    rng = np.random.default_rng(8)
+    for k in range(1, 4):
+        g = rng.normal(0, 2e-3, n).astype(np.float32)
+        g[5], g[6] = 1.0, -1.0
+        orc.send_step(b, g, sref, cref, k)
+    assert np.array_equal(cg, cref) and np.array_equal(sg, sref), "a threshold nothing reaches must change nothing"
+    g = rng.normal(0, 2e-3, n).astype(np.float32)
+    g[7] = np.nan
+    flags, _ = orc.send_step(a, g, sa, ca, 9)
+    assert flags & orc.FLAG_NONFINITE
