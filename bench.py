@@ -415,6 +415,8 @@ def sweep(args, device):
         send_case("fp32 g, int8 state, %d bit, fixed" % bits, M, bits=bits, grad_dtype=0)
     send_case("bf16 g, int8 state, 4 bit, fixed, s_e = 6 s (Newton-Raphson decompressor)", M, s_e=6 * 2.0 ** 11)
     send_case("bf16 g, int8 state, 4 bit, fixed, statistics on", M, collect_stats=1)
+    send_case("bf16 g, int8 state, 4 bit, fixed, element-wise clipping at 2 sigma", M, clip=2e-3)
+    send_case("bf16 weights, no state, 8 bit, block-256 absmax (Zero++-style weight payload)", M, bits=8, scale_mode=1, state_fmt=2)
     send_case("bf16 g, fp32 state, 4 bit, fixed", M, state_fmt=1)
     send_case("bf16 g, fp32 state + 8-bit compensation, 4 bit, fixed", M, state_fmt=3)
     send_case("bf16 g, no state, 4 bit, fixed", M, state_fmt=2)
@@ -431,6 +433,7 @@ def sweep(args, device):
     reduce_case("4 bit, bf16 out, fixed, 3 workers (division by 3)", M, 3)
     reduce_case("4 bit, bf16 out, block-256 absmax", M, 8, scale_mode=1)
     reduce_case("4 bit, bf16 out, block-32 absmax", M, 8, scale_mode=1, block_size=32)
+    reduce_case("8 bit, bf16 out, block-256 absmax, 1 worker (Zero++-style weight payload)", M, 1, bits=8, scale_mode=1)
     for N in (1, 8, 16):
         adam_case("4 bit, fixed, Adam-family step fused, no gradient output", M, N)
     adam_case("8 bit, fixed, Adam-family step fused, no gradient output", M, 8, bits=8)

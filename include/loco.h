@@ -91,6 +91,10 @@ typedef struct {
     int32_t num_partitions;  /* P >= 1: parts of the all-to-all layout (Sec. 3.3)                 */
     int32_t collect_stats;   /* non-zero: count saturated gradient codes (second case of the
                                 rounding lemma) during send; costs a few instructions/element   */
+    float   clip;            /* > 0: clip every element of the local gradient to [-clip, clip] before
+                                step 1 (the element-wise clipping of the Sky-MoE runs in the paper's
+                                experiments; the paper states no threshold); 0 = off.  +-Inf becomes
+                                +-clip, NaN stays NaN                                             */
 } loco_config_t;
 
 /* Per-bucket, per-worker handle: a host object holding the configuration, the bucket

@@ -41,6 +41,7 @@ int check_config(const loco_config_t *c) {
     if (c->grad_dtype != LOCO_F32 && c->grad_dtype != LOCO_BF16) return LOCO_ERR_ARG;
     if (c->out_dtype != LOCO_F32 && c->out_dtype != LOCO_BF16) return LOCO_ERR_ARG;
     if (c->num_partitions < 1 || c->num_partitions > 65535) return LOCO_ERR_ARG;
+    if (!(c->clip >= 0.0f) || !std::isfinite(c->clip)) return LOCO_ERR_ARG;
     if (c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX && c->block_size > 256) return LOCO_ERR_UNSUPPORTED;
     return LOCO_OK;
 }
@@ -410,6 +411,7 @@ int loco_compensate_quantize_pack(loco_state_t *st, const void *d_grad, void *d_
     P.dq_a = st->dq.a; P.dq_b = st->dq.b; P.dq_mode = st->dq.mode;
     P.de_a = st->de.a; P.de_b = st->de.b; P.de_mode = st->de.mode;
     P.fast = st->fast;
+    P.clip = c.clip;
     P.beta = c.beta;
     {
         const volatile float omb = 1.0f - c.beta;    // (1 - beta), rounded once to fp32

@@ -65,6 +65,7 @@ struct SendParams {
     int block_log2;                  // log2(B), BLOCK mode
     int reset;                       // k % T_c == 0
     int collect_stats;
+    float clip;                      // > 0: element-wise clipping of g to [-clip, clip] before step 1
     unsigned long long *status;      // [0] flags, [1] saturated codes
 };
 
@@ -299,6 +300,7 @@ __device__ __noinline__ unsigned send_row_careful(const SendParams P, unsigned l
         ef[j] = 0.0f;
         if (j < valid) {
             g[j] = load_grad1<GRAD>(P.grad, i0 + j);
+            if (P.clip > 0.0f && g[j] == g[j]) g[j] = fminf(fmaxf(g[j], -P.clip), P.clip);    // NaN stays NaN
             if (STATE == ST_INT8) {
                 const unsigned b = static_cast<uint8_t>(st8[i0 + j]);
                 if (j < 4) lo_w |= b << (8 * j); else hi_w |= b << (8 * (j - 4));
@@ -527,7 +529,7 @@ __device__ __forceinline__ void fetch_row(const RingAddr<GRAD, STATE> &A, unsign
 
 // The scalars of Algorithm 1 the fast routine needs, read from the parameters once per kernel.
 struct SendConsts {
-    float s, s_e, beta, omb, inv_s, inv_se, dq_a, dq_b, de_a, de_b;
+    float s, s_e, beta, omb, inv_s, inv_se, dq_a, dq_b, de_a, de_b, clip;
     int dq_mode, de_mode, block_log2, reset;
 };
 
@@ -679,6 +681,16 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     }
     if (MODE != MODE_BLOCK) {
         if (__any_sync(kFull, bad_bits != 0u)) return false;
+    }
+
+    // ---- optional element-wise clipping of g (finite here, or the row is redone by the careful routine) ------------
+    if (K.clip > 0.0f) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            float a, b;
+            unpk2(g2[k], a, b);
+            g2[k] = pk2(fminf(fmaxf(a, -K.clip), K.clip), fminf(fmaxf(b, -K.clip), K.clip));
+        }
     }
 
     // ---- step 1, Eq. 2: c = what is added to g, prev = e~_k of Eq. 5, h = g + c -----------------------------
@@ -871,7 +883,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams
         SendConsts K;
         K.s = P.s; K.s_e = P.s_e; K.beta = P.beta; K.omb = P.omb; K.inv_s = P.inv_s; K.inv_se = P.inv_se;
         K.dq_a = P.dq_a; K.dq_b = P.dq_b; K.de_a = P.de_a; K.de_b = P.de_b;
-        K.dq_mode = P.dq_mode; K.de_mode = P.de_mode; K.block_log2 = P.block_log2; K.reset = P.reset;
+        K.dq_mode = P.dq_mode; K.de_mode = P.de_mode; K.block_log2 = P.block_log2; K.reset = P.reset; K.clip = P.clip;
         const bool stats = P.collect_stats != 0;
         RingAddr<GRAD, STATE> A;
         ring_addresses<GRAD, STATE, MODE>(static_cast<unsigned>(__cvta_generic_to_shared(ring)), lane, threadIdx.x >> 5, A);

@@ -44,7 +44,8 @@ class loco_config_t(C.Structure):
     _fields_ = [("bits", C.c_int32), ("scale_mode", C.c_int32), ("block_size", C.c_int32),
                 ("s", C.c_float), ("s_e", C.c_float), ("beta", C.c_float),
                 ("reset_period", C.c_int32), ("state_fmt", C.c_int32), ("grad_dtype", C.c_int32),
-                ("out_dtype", C.c_int32), ("num_partitions", C.c_int32), ("collect_stats", C.c_int32)]
+                ("out_dtype", C.c_int32), ("num_partitions", C.c_int32), ("collect_stats", C.c_int32),
+                ("clip", C.c_float)]
 
 
 class loco_adam_t(C.Structure):
@@ -66,11 +67,12 @@ class Config:
     out_dtype: int = BF16
     num_partitions: int = 1
     collect_stats: int = 0
+    clip: float = 0.0
 
     def c(self) -> loco_config_t:
         return loco_config_t(self.bits, self.scale_mode, self.block_size, self.s, self.s_e, self.beta,
                              self.reset_period, self.state_fmt, self.grad_dtype, self.out_dtype,
-                             self.num_partitions, self.collect_stats)
+                             self.num_partitions, self.collect_stats, self.clip)
 
 
 _lib = None

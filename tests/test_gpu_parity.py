@@ -307,3 +307,51 @@ def test_block_scale_divisions_are_ieee_for_every_amax():
     """The block-scaled send path divides with short multiply-add sequences; the library checks them against the IEEE
     division for every positive finite fp32 amax and qmax in {1, 7, 127}."""
     assert loco.loco_selfcheck_block_division() == (0, 0)
+
+
+# ---------------------------------------------------------------- element-wise clipping of the local gradient
+
+@pytest.mark.parametrize("mode", [loco.SCALE_FIXED, loco.SCALE_BLOCK_ABSMAX])
+@pytest.mark.parametrize("fmt", [loco.STATE_INT8, loco.STATE_FP32, loco.STATE_NONE])
+def test_gradient_clipping(mode, fmt):
+    """clip > 0: every gradient element is clamped to [-clip, clip] before Algorithm 1 (heavy-tailed values, so that many
+    are clamped; a few +-Inf, which become +-clip, and NaN, which stay NaN)."""
+    n = 200_003
+    for gd in (loco.BF16, loco.F32):
+        gcfg, ocfg = both_configs(bits=4, scale_mode=mode, block_size=128, s=2.0 ** 12, s_e=2.0 ** 14, beta=0.5, reset_period=0,
+                                  state_fmt=fmt, grad_dtype=gd, out_dtype=loco.F32, num_partitions=3, clip=3e-4)
+        w = Worker(gcfg, ocfg, n)
+        dt = torch.bfloat16 if gd == loco.BF16 else torch.float32
+        for k in range(3):
+            g = inputs.student_t(n, 3.0, 1e-4, seed=15, step=k, dtype=torch.float32, device="cuda")
+            g[1000 + k] = float("inf")
+            g[70_000 + k] = float("-inf")
+            if k == 1:
+                g[150_000] = float("nan")
+            assert int((g.abs() > 3e-4).sum()) > n // 20
+            w.step(grad_bits(g.to(dt)), k + 1)
+            w.compare("step %d" % k)
+        assert w.oflags & orc.FLAG_NONFINITE
+        got, want = reduce_both(gcfg, ocfg, n, [w])
+        assert_reduced_equal(got, want, False)
+
+
+def test_zero_plus_plus_style_weight_payload():
+    """The 8-bit block-quantised weight payload of the LoCo-Zero++ variant is the send pass without error state (8-bit codes,
+    one scale per block) and the receive pass with a single worker: round trip within half a quantisation step of the block."""
+    n, B = 1_000_003, 256
+    gcfg, ocfg = both_configs(bits=8, scale_mode=loco.SCALE_BLOCK_ABSMAX, block_size=B, state_fmt=loco.STATE_NONE,
+                              grad_dtype=loco.BF16, out_dtype=loco.BF16, num_partitions=8)
+    wgt = inputs.gaussian(n, 0.02, seed=16, dtype=torch.bfloat16, device="cuda")
+    w = Worker(gcfg, ocfg, n)
+    w.step(grad_bits(wgt), 0)
+    w.compare("weights")
+    got, want = reduce_both(gcfg, ocfg, n, [w])
+    assert_reduced_equal(got, want, True)
+    back = torch.from_numpy(got.view(np.int16)).view(torch.bfloat16).float()
+    x = wgt.float().cpu()
+    pad = (-n) % B
+    amax = torch.nn.functional.pad(x.abs(), (0, pad)).view(-1, B).max(dim=1).values
+    step = (amax / 127.0).repeat_interleave(B)[:n]
+    # half a step from the rounding to a code plus half a bf16 ulp of the result
+    assert bool(((back - x).abs() <= 0.5 * step * 1.001 + x.abs() * 2.0 ** -8).all())
