@@ -42,6 +42,8 @@
  *     cases the compression error of that element is taken as 0;
  *   - the element-wise clipping of g named in the experiments section has no stated threshold: `clip` is a
  *     parameter (0 = off), applied to g before step 1;
+ *   - stochastic rounding (not in the paper, which rounds to nearest): floor(h x s + u) with u from a
+ *     Philox4x32-10 stream keyed by a seed and indexed by (element, iteration), so that it can be reproduced anywhere;
  *   - Eq. 8 is summed in worker order in fp32, then divided by (float)N;
  *   - the Adam-family step is taken exactly as printed (no bias correction, delta inside the root), with
  *     eta_k = eta / sqrt(v_k + delta) evaluated as one square root and one division.
@@ -84,7 +86,38 @@ typedef struct {
     int32_t num_partitions; /* N parts of Sec. 3.3 */
     float   clip;           /* > 0: element-wise clipping of the local gradient to [-clip, clip] before Algorithm 1
                                (the Sky-MoE pre-training runs of the experiments section); 0 = off */
+    int32_t rounding;       /* 0: nearest integer, Eq. 1 (the paper);  1: stochastic rounding (extension) */
+    uint32_t seed_lo, seed_hi;  /* key of the Philox stream used by stochastic rounding */
 } orc_config;
+
+/* ---------- Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", SC'11) ----------
+ * Counter-based generator: out = philox(counter[4], key[2]); ten rounds of two 32x32->64 multiplications by fixed
+ * constants, xors with the key, and a Weyl bump of the key between rounds.  Written from the published definition;
+ * the tests check the published known-answer vectors. */
+void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int r = 0; r < 10; ++r) {
+        if (r > 0) { k0 += W0; k1 += W1; }
+        const uint64_t p0 = (uint64_t)M0 * c0, p1 = (uint64_t)M1 * c2;
+        const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0, hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+        const uint32_t n0 = hi1 ^ c1 ^ k0, n1 = lo1, n2 = hi0 ^ c3 ^ k1, n3 = lo0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* The uniform number in [0, 1) that stochastic rounding adds to element i of the bucket at iteration k:
+ * word (i mod 4) of philox(counter = (i/4 low, i/4 high, k low, k high), key = seed), top 24 bits times 2^-24. */
+static float sr_uniform(const orc_config *c, uint64_t i, int64_t k) {
+    const uint64_t blk = i >> 2;
+    const uint32_t ctr[4] = {(uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)(uint64_t)k, (uint32_t)((uint64_t)k >> 32)};
+    const uint32_t key[2] = {c->seed_lo, c->seed_hi};
+    uint32_t out[4];
+    orc_philox4x32_10(ctr, key, out);
+    return (float)(out[i & 3] >> 8) * 5.9604644775390625e-8f;      /* 2^-24, exact */
+}
+float orc_sr_uniform(const orc_config *c, uint64_t i, int64_t k) { return sr_uniform(c, i, k); }
 
 /* Optional per-element record of one send step, for the invariant tests. */
 typedef struct {
@@ -159,6 +192,7 @@ static int config_ok(const orc_config *c) {
     if (c->out_dtype != ORC_F32 && c->out_dtype != ORC_BF16) return 0;
     if (c->num_partitions < 1) return 0;
     if (!(c->clip >= 0.0f) || !isfinite(c->clip)) return 0;
+    if (c->rounding != 0 && c->rounding != 1) return 0;
     return 1;
 }
 
@@ -249,11 +283,21 @@ static float load_grad(const orc_config *c, const void *grad, uint64_t i) {
 
 /* Quantise one compensated value against a multiplier (s, or the block's inverse scale).
  * Returns the code; *err0 is set when the element's compression error is defined as 0. */
-static int32_t quantise(float h, float mult, int p, int *err0, uint64_t *status) {
+static int32_t quantise(const orc_config *c, uint64_t i, int64_t k, float h, float mult, int p, int *err0, uint64_t *status) {
     *err0 = 0;
     if (isnan(h)) { *err0 = 1; status[0] |= ORC_FLAG_NONFINITE; return 0; }
     if (isinf(h)) { *err0 = 1; status[0] |= ORC_FLAG_NONFINITE; return h > 0 ? qmax_of(p) : qmin_of(p); }
     float y = h * mult;                       /* h x s of Eq. 1 */
+    if (c->rounding == 1) {
+        /* stochastic rounding (extension): floor(y + u), u uniform in [0, 1): up with probability frac(y) */
+        const float t = y + sr_uniform(c, i, k);
+        float r = floorf(t);
+        const float lo = (float)qmin_of(p), hi = (float)qmax_of(p);
+        if (r < lo || r > hi) status[1] += 1;
+        if (r < lo) r = lo;
+        if (r > hi) r = hi;
+        return (int32_t)r;
+    }
     float r = rintf(y);
     /* saturated: the nearest integer falls outside the p-bit range (second case of Lemma "round") */
     if (r < (float)qmin_of(p) || r > (float)qmax_of(p)) status[1] += 1;
@@ -351,7 +395,7 @@ int orc_send_step(const orc_config *cfg, uint64_t n, const void *grad, void *sta
         for (uint64_t t = 0; t < len; ++t) {
             const uint64_t i = b0 + t;
             int err0;
-            const int32_t q = quantise(hb[t], mult, p, &err0, status);
+            const int32_t q = quantise(cfg, i, k, hb[t], mult, p, &err0, status);
             const float d = fixed ? (float)q / cfg->s : (float)q * scale;
             const float delta = err0 ? 0.0f : hb[t] - d;
             const float e_new = (omb * pb[t]) + (beta * delta);      /* Eq. 5 */

@@ -40,7 +40,7 @@ class _Cfg(C.Structure):
                 ("s", C.c_float), ("s_e", C.c_float), ("beta", C.c_float),
                 ("reset_period", C.c_int32), ("state_fmt", C.c_int32),
                 ("grad_dtype", C.c_int32), ("out_dtype", C.c_int32), ("num_partitions", C.c_int32),
-                ("clip", C.c_float)]
+                ("clip", C.c_float), ("rounding", C.c_int32), ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32)]
 
 
 class _Adam(C.Structure):
@@ -67,11 +67,13 @@ class OracleConfig:
     out_dtype: int = F32
     num_partitions: int = 1
     clip: float = 0.0
+    rounding: int = 0
+    seed: int = 0
 
     def c(self) -> _Cfg:
         return _Cfg(self.bits, self.scale_mode, self.block_size, self.s, self.s_e, self.beta,
                     self.reset_period, self.state_fmt, self.grad_dtype, self.out_dtype,
-                    self.num_partitions, self.clip)
+                    self.num_partitions, self.clip, self.rounding, self.seed & 0xFFFFFFFF, (self.seed >> 32) & 0xFFFFFFFF)
 
 
 _lib = None
@@ -102,6 +104,10 @@ def lib():
         L.orc_reduce.argtypes = [cp, u64, C.POINTER(vp), i32, i32, i32, vp]
         L.orc_reduce_adam.restype = C.c_int
         L.orc_reduce_adam.argtypes = [cp, u64, C.POINTER(vp), i32, i32, i32, C.POINTER(_Adam), vp, vp, vp, vp]
+        L.orc_philox4x32_10.restype = None
+        L.orc_philox4x32_10.argtypes = [vp, vp, vp]
+        L.orc_sr_uniform.restype = C.c_float
+        L.orc_sr_uniform.argtypes = [cp, u64, i64]
         L.orc_f32_to_bf16.restype = C.c_uint16
         L.orc_f32_to_bf16.argtypes = [C.c_float]
         L.orc_bf16_to_f32.restype = C.c_float
@@ -235,6 +241,19 @@ def reduce_adam(cfg: OracleConfig, n: int, comms, m: np.ndarray, v: np.ndarray, 
     if rc != 0:
         raise ValueError("oracle: bad configuration")
     return out
+
+
+def philox4x32_10(ctr, key) -> np.ndarray:
+    """The four output words of Philox4x32-10 for a 4-word counter and a 2-word key."""
+    c = np.asarray(ctr, dtype=np.uint32).copy()
+    k = np.asarray(key, dtype=np.uint32).copy()
+    out = np.zeros(4, dtype=np.uint32)
+    lib().orc_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def sr_uniform(cfg: OracleConfig, i: int, k: int) -> float:
+    return float(lib().orc_sr_uniform(C.byref(cfg.c()), i, k))
 
 
 def state_views(cfg: OracleConfig, n: int, state: np.ndarray):

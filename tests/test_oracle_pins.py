@@ -649,3 +649,55 @@ def test_clipping_equals_clipping_the_input_first(mode):
     g[7] = np.nan
     flags, _ = orc.send_step(a, g, sa, ca, 9)
     assert flags & orc.FLAG_NONFINITE
+
+
+# ---------------------------------------------------------------- stochastic rounding on a Philox stream (extension)
+
+def test_philox_known_answer_vectors():
+    """The three known-answer vectors published with the generator (Random123 kat_vectors, philox4x32 10 rounds)."""
+    kat = [((0, 0, 0, 0), (0, 0), (0x6627e8d5, 0xe169c58d, 0xbc57ac4c, 0x9b00dbd8)),
+           ((0xffffffff,) * 4, (0xffffffff,) * 2, (0x408f276d, 0x41c83b0e, 0xa20bc7c6, 0x6d5451fd)),
+           ((0x243f6a88, 0x85a308d3, 0x13198a2e, 0x03707344), (0xa4093822, 0x299f31d0), (0xd16cfe09, 0x94fdcceb, 0x5001e420, 0x24126ea1))]
+    for ctr, key, want in kat:
+        assert tuple(int(x) for x in orc.philox4x32_10(ctr, key)) == want
+
+
+def test_stochastic_rounding_properties():
+    """q is floor or ceil of h x s (inside the range), integers are never moved, the mean over many draws is h x s, the
+    stream depends on (element, iteration, seed) only, and the uniform numbers are 24-bit fractions in [0, 1)."""
+    n, s = 1 << 14, 4.0
+    kw = dict(bits=8, s=s, s_e=16.0, beta=0.5, reset_period=0, state_fmt=orc.STATE_NONE, grad_dtype=orc.F32, out_dtype=orc.F32)
+    cfg = orc.OracleConfig(rounding=1, seed=12345, **kw)
+    rng = np.random.default_rng(5)
+    h = rng.uniform(-20, 20, n).astype(np.float32) / np.float32(s)
+    h[:64] = np.arange(-32, 32, dtype=np.float32) / np.float32(s)            # exact integers after scaling
+    y = (h * np.float32(s)).astype(np.float64)
+    draws = []
+    for k in range(1, 201):
+        comm = orc.new_comm(cfg, n)
+        orc.send_step(cfg, h, orc.new_state(cfg, n), comm, k)
+        q = orc.unpack_codes(comm, n, 8)
+        assert ((q == np.floor(y)) | (q == np.ceil(y))).all()
+        assert (q[:64] == np.arange(-32, 32)).all()
+        draws.append(q)
+    mean = np.mean(draws, axis=0)
+    frac = y - np.floor(y)
+    # binomial standard error of 200 draws is at most 0.036; 5 sigma
+    assert np.abs(mean - y).max() < 0.18 and abs(float(np.mean(mean - y))) < 2e-3
+    # same (seed, element, iteration) -> same code; another seed or iteration -> another stream
+    comm2 = orc.new_comm(cfg, n)
+    orc.send_step(cfg, h, orc.new_state(cfg, n), comm2, 200)
+    assert np.array_equal(orc.unpack_codes(comm2, n, 8), draws[-1])
+    other = orc.OracleConfig(rounding=1, seed=12346, **kw)
+    comm3 = orc.new_comm(other, n)
+    orc.send_step(other, h, orc.new_state(other, n), comm3, 200)
+    assert (orc.unpack_codes(comm3, n, 8) != draws[-1]).mean() > 0.2
+    us = np.array([orc.sr_uniform(cfg, i, 7) for i in range(4096)])
+    assert us.min() >= 0.0 and us.max() < 1.0 and abs(us.mean() - 0.5) < 0.02
+    assert np.array_equal(us * 2 ** 24, np.round(us * 2 ** 24))
+    # the position inside a bucket matters, not the bucket's partitioning
+    cfgp = orc.OracleConfig(rounding=1, seed=12345, num_partitions=4, **kw)
+    commp = orc.new_comm(cfgp, n)
+    orc.send_step(cfgp, h, orc.new_state(cfgp, n), commp, 200)
+    qp = np.concatenate([orc.unpack_codes(c, orc.partition_elems(cfgp, n, j), 8) for j, (c, _) in enumerate(orc.comm_views(cfgp, n, commp))])
+    assert np.array_equal(qp, draws[-1])
