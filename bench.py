@@ -417,6 +417,7 @@ def sweep(args, device):
     send_case("bf16 g, int8 state, 4 bit, fixed, statistics on", M, collect_stats=1)
     send_case("bf16 g, int8 state, 4 bit, fixed, element-wise clipping at 2 sigma", M, clip=2e-3)
     send_case("bf16 weights, no state, 8 bit, block-256 absmax (Zero++-style weight payload)", M, bits=8, scale_mode=1, state_fmt=2)
+    send_case("bf16 g, int8 state, 4 bit, fixed, stochastic rounding (Philox4x32-10)", M, rounding=1, seed=7)
     send_case("bf16 g, fp32 state, 4 bit, fixed", M, state_fmt=1)
     send_case("bf16 g, fp32 state + 8-bit compensation, 4 bit, fixed", M, state_fmt=3)
     send_case("bf16 g, no state, 4 bit, fixed", M, state_fmt=2)

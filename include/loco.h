@@ -64,6 +64,8 @@ typedef enum {
     LOCO_SCALE_BLOCK_ABSMAX = 1  /* extension, not in the paper: fp32 scale amax/qmax per B      */
 } loco_scale_mode_t;
 
+typedef enum { LOCO_ROUND_NEAREST = 0, LOCO_ROUND_STOCHASTIC = 1 } loco_rounding_t;
+
 typedef enum {
     LOCO_STATE_INT8 = 0,         /* the paper's 8-bit error e_k (Eq. 7); Eq. 5 uses dec(e_k)     */
     LOCO_STATE_FP32 = 1,         /* uncompressed error, the ablation without error compression   */
@@ -79,7 +81,8 @@ typedef enum {
 typedef struct {
     int32_t bits;            /* p of Eq. 1 for the gradient codes: 2, 4 or 8 (the paper uses 4)   */
     int32_t scale_mode;      /* loco_scale_mode_t                                                 */
-    int32_t block_size;      /* B, BLOCK_ABSMAX only: power of two in [32, 4096]                  */
+    int32_t block_size;      /* B, BLOCK_ABSMAX only: power of two in [32, 4096]; this build runs
+                                32..256 and returns LOCO_ERR_UNSUPPORTED above                    */
     float   s;               /* Eq. 1 / Eq. 3 scale, FIXED only (> 0, finite)                     */
     float   s_e;             /* Eq. 2 / Eq. 7 scale of the 8-bit error, FIXED only                */
     float   beta;            /* Eq. 5, in [0, 1]: weight of the NEW compression error             */
@@ -95,6 +98,11 @@ typedef struct {
                                 step 1 (the element-wise clipping of the Sky-MoE runs in the paper's
                                 experiments; the paper states no threshold); 0 = off.  +-Inf becomes
                                 +-clip, NaN stays NaN                                             */
+    int32_t rounding;        /* loco_rounding_t: 0 = nearest integer as Eq. 1 states (the paper), 1 =
+                                stochastic rounding, an extension: floor(h x s + u), u uniform in
+                                [0, 1) from Philox4x32-10 with counter (element/4, iteration) and key
+                                `seed`; word element%4, top 24 bits                               */
+    uint32_t seed_lo, seed_hi; /* key of that stream (ignored with rounding 0)                      */
 } loco_config_t;
 
 /* Per-bucket, per-worker handle: a host object holding the configuration, the bucket

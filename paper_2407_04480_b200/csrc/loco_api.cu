@@ -42,6 +42,7 @@ int check_config(const loco_config_t *c) {
     if (c->out_dtype != LOCO_F32 && c->out_dtype != LOCO_BF16) return LOCO_ERR_ARG;
     if (c->num_partitions < 1 || c->num_partitions > 65535) return LOCO_ERR_ARG;
     if (!(c->clip >= 0.0f) || !std::isfinite(c->clip)) return LOCO_ERR_ARG;
+    if (c->rounding != LOCO_ROUND_NEAREST && c->rounding != LOCO_ROUND_STOCHASTIC) return LOCO_ERR_ARG;
     if (c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX && c->block_size > 256) return LOCO_ERR_UNSUPPORTED;
     return LOCO_OK;
 }
@@ -164,10 +165,13 @@ SendKernel pick_send_mode(int mode, int var) {
         if (var == VAR_LEAN) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_LEAN>, smem};
         if (var == VAR_LEAN_NR && (STATE == ST_INT8 || STATE == ST_Q8COMP))
             return {loco_send_kernel<GRAD, (STATE == ST_INT8 || STATE == ST_Q8COMP) ? STATE : ST_INT8, BITS, MODE_FIXED, VAR_LEAN_NR>, smem};
+        if (var == VAR_STOCHASTIC) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_STOCHASTIC>, smem};
         return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_GENERAL>, smem};
     }
     if (STATE == ST_Q8COMP) return {nullptr, 0};                // Q8COMP exists for the global scales only
     constexpr int ST = (STATE == ST_Q8COMP ? ST_FP32 : STATE);
+    if (var == VAR_GENERAL) return {loco_send_kernel<GRAD, ST, BITS, MODE_BLOCK, VAR_GENERAL>, Ring<GRAD, ST, MODE_BLOCK>::kBytes};
+    if (var == VAR_STOCHASTIC) return {loco_send_kernel<GRAD, ST, BITS, MODE_BLOCK, VAR_STOCHASTIC>, Ring<GRAD, ST, MODE_BLOCK>::kBytes};
     return {loco_send_kernel<GRAD, ST, BITS, MODE_BLOCK, VAR_LEAN>, Ring<GRAD, ST, MODE_BLOCK>::kBytes};
 }
 template <int GRAD, int STATE>
@@ -326,7 +330,11 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
     }
     {
         int var = VAR_GENERAL;
-        if (st->mode == MODE_BLOCK) var = VAR_LEAN;
+        if (cfg->rounding == LOCO_ROUND_STOCHASTIC) {
+            var = VAR_STOCHASTIC;
+            if (st->mode == MODE_BLOCK) st->fast = 0;        // block scales with stochastic rounding: careful routine only
+        } else if (cfg->clip > 0.0f) var = VAR_GENERAL;           // only the general variants carry the clipping
+        else if (st->mode == MODE_BLOCK) var = VAR_LEAN;
         else if (!cfg->collect_stats && st->dq.mode == DEC_FMA && st->de.mode == DEC_FMA) var = VAR_LEAN;
         else if (!cfg->collect_stats && st->dq.mode == DEC_FMA && st->de.mode == DEC_NEWTON) var = VAR_LEAN_NR;
         const SendKernel k = pick_send(cfg, st->mode, var);
@@ -412,6 +420,9 @@ int loco_compensate_quantize_pack(loco_state_t *st, const void *d_grad, void *d_
     P.de_a = st->de.a; P.de_b = st->de.b; P.de_mode = st->de.mode;
     P.fast = st->fast;
     P.clip = c.clip;
+    P.stochastic = c.rounding == LOCO_ROUND_STOCHASTIC ? 1 : 0;
+    P.seed_lo = c.seed_lo; P.seed_hi = c.seed_hi;
+    P.k_lo = static_cast<unsigned>(static_cast<uint64_t>(step_k)); P.k_hi = static_cast<unsigned>(static_cast<uint64_t>(step_k) >> 32);
     P.beta = c.beta;
     {
         const volatile float omb = 1.0f - c.beta;    // (1 - beta), rounded once to fp32

@@ -66,6 +66,9 @@ struct SendParams {
     int reset;                       // k % T_c == 0
     int collect_stats;
     float clip;                      // > 0: element-wise clipping of g to [-clip, clip] before step 1
+    int stochastic;                  // stochastic rounding of the gradient codes (extension)
+    unsigned seed_lo, seed_hi;       // key of its Philox stream
+    unsigned k_lo, k_hi;             // the iteration counter, part of the Philox counter
     unsigned long long *status;      // [0] flags, [1] saturated codes
 };
 
@@ -107,6 +110,28 @@ __device__ __forceinline__ float round_clamp(float y, float lo, float hi, unsign
     float m = __fadd_rn(t, kMagic);
     bits = __float_as_uint(m);
     return __fadd_rn(m, -kMagic);
+}
+
+// Philox4x32-10 (Salmon et al., SC'11), from its published definition: ten rounds of two 32x32->64 multiplications by
+// fixed constants, xors with the key, a Weyl bump of the key between rounds.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, unsigned k0, unsigned k1) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        if (r > 0) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+        const unsigned hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+        const unsigned hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+    }
+    return c;
+}
+// The four uniform numbers in [0, 1) of bucket elements 4 blk .. 4 blk + 3 at iteration (k_hi, k_lo): top 24 bits of the words.
+__device__ __forceinline__ void sr_uniform4(unsigned long long blk, unsigned k_lo, unsigned k_hi, unsigned seed_lo, unsigned seed_hi,
+                                            float (&u)[4]) {
+    const uint4 r = philox4x32_10(make_uint4(static_cast<unsigned>(blk), static_cast<unsigned>(blk >> 32), k_lo, k_hi), seed_lo, seed_hi);
+    u[0] = __uint2float_rn(r.x >> 8) * 5.9604644775390625e-8f;
+    u[1] = __uint2float_rn(r.y >> 8) * 5.9604644775390625e-8f;
+    u[2] = __uint2float_rn(r.z >> 8) * 5.9604644775390625e-8f;
+    u[3] = __uint2float_rn(r.w >> 8) * 5.9604644775390625e-8f;
 }
 
 __device__ __forceinline__ float warp_group_max(float v, int lanes) {
@@ -164,9 +189,9 @@ __device__ __forceinline__ void st_stream4(void *p, unsigned v) { __stcs(static_
 //  prev   e~_k as Eq. 5 sees it;  c  what is added to g (dec(e_k), e~_k, or dec(comp(e~_k)))
 //  valid  number of leading elements that exist
 //  Outputs: code bits (low byte of each word = code), e_new = e~_{k+1}, scale of the block.
-template <int STATE, int BITS, int MODE>
+template <int STATE, int BITS, int MODE, bool STOCH>
 __device__ __forceinline__ void send_core(const SendParams &P, const float (&g)[8], const float (&c)[8],
-                                          const float (&prev)[8], int valid, int lanes_per_block,
+                                          const float (&prev)[8], int valid, int lanes_per_block, unsigned long long i0,
                                           unsigned (&code)[8], float (&e_new)[8], float &scale,
                                           unsigned &nonfinite, unsigned &saturated) {
     constexpr float lo = QRange<BITS>::lo, hi = QRange<BITS>::hi;
@@ -188,18 +213,34 @@ __device__ __forceinline__ void send_core(const SendParams &P, const float (&g)[
         scale = amax > 0.0f ? __fdiv_rn(amax, hi) : 0.0f;
         mult = amax > 0.0f ? __fdiv_rn(hi, amax) : 0.0f;
     }
+    float u8[8];
+    if (STOCH) {                                            // i0 is a multiple of 8: two counters
+        float ua[4], ub[4];
+        sr_uniform4(i0 >> 2, P.k_lo, P.k_hi, P.seed_lo, P.seed_hi, ua);
+        sr_uniform4((i0 >> 2) + 1, P.k_lo, P.k_hi, P.seed_lo, P.seed_hi, ub);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { u8[j] = ua[j]; u8[4 + j] = ub[j]; }
+    }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
         const float hq = (h[j] != h[j]) ? 0.0f : h[j];      // NaN is sent as code 0
         float y = __fmul_rn(hq, mult);                      // h x s of Eq. 1
         if (!fin[j]) y = hq;                                // +-Inf saturates whatever the scale
-        const float r = round_clamp(y, lo, hi, code[j]);    // round_p-bit
+        float r;
+        if (STOCH && fin[j]) {                              // floor(y + u): up with probability frac(y)
+            const float fl = floorf(__fadd_rn(y, u8[j]));
+            if (P.collect_stats && j < valid && (fl < lo || fl > hi)) saturated += 1u;
+            r = fminf(fmaxf(fl, lo), hi);
+            code[j] = static_cast<unsigned>(__float2int_rn(r));
+        } else {
+            r = round_clamp(y, lo, hi, code[j]);            // round_p-bit
+        }
         float d;                                            // step 2: dec(q; s)
         if (MODE == MODE_FIXED) d = __fdiv_rn(r, P.s);
         else d = __fmul_rn(r, scale);
         const float delta = fin[j] ? __fsub_rn(h[j], d) : 0.0f;
         e_new[j] = __fadd_rn(__fmul_rn(P.omb, prev[j]), __fmul_rn(P.beta, delta));   // Eq. 5
-        if (MODE != MODE_BLOCK && P.collect_stats) {
+        if (MODE != MODE_BLOCK && P.collect_stats && !STOCH) {
             // nearest integer outside the range: y >= hi + 1/2 (hi is odd, the tie goes up and out)
             // or y < lo - 1/2 (lo is even, the tie stays in)
             if (fin[j] && j < valid && (y >= hi + 0.5f || y < lo - 0.5f)) saturated += 1u;
@@ -275,11 +316,11 @@ __device__ __forceinline__ void store_codes8(uint8_t *dst, const unsigned (&code
 
 // One warp row (256 elements starting at partition-local offset `o`, bucket element i0 = part*lp + o),
 // careful routine.  Elements >= n are treated as absent (code 0, no state).  Reads its inputs itself.
-// Out of line and with its own copy of the parameters, so that the fast routine's register allocation and
-// constant-bank accesses are not disturbed by this rarely taken path.  Returns the number of saturated
+// Out of line, reading the kernel's parameters in place (they are __grid_constant__, so their address can be taken
+// without a local copy), so that the fast routine's register allocation is not disturbed by this rarely taken path.  Returns the number of saturated
 // codes of this lane, plus 2^31 if the lane met a non-finite value.
-template <int GRAD, int STATE, int BITS, int MODE>
-__device__ __noinline__ unsigned send_row_careful(const SendParams P, unsigned long long part, unsigned long long o,
+template <int GRAD, int STATE, int BITS, int MODE, bool STOCH>
+__device__ __noinline__ unsigned send_row_careful(const SendParams &P, unsigned long long part, unsigned long long o,
                                                   int lane) {
     unsigned nonfinite = 0u, saturated = 0u;
     const unsigned long long i0 = part * P.lp + o + static_cast<unsigned long long>(lane) * kLaneElems;
@@ -315,7 +356,7 @@ __device__ __noinline__ unsigned send_row_careful(const SendParams P, unsigned l
 
     unsigned code[8];
     float e_new[8], scale;
-    send_core<STATE, BITS, MODE>(P, g, c, prev, valid, lanes_per_block, code, e_new, scale, nonfinite, saturated);
+    send_core<STATE, BITS, MODE, STOCH>(P, g, c, prev, valid, lanes_per_block, i0, code, e_new, scale, nonfinite, saturated);
 
     // codes (and the block's scale) into the partition's areas of the communication buffer
     uint8_t *pbase = P.comm + part * P.stride;
@@ -531,6 +572,7 @@ __device__ __forceinline__ void fetch_row(const RingAddr<GRAD, STATE> &A, unsign
 struct SendConsts {
     float s, s_e, beta, omb, inv_s, inv_se, dq_a, dq_b, de_a, de_b, clip;
     int dq_mode, de_mode, block_log2, reset;
+    unsigned seed_lo, seed_hi, k_lo, k_hi;
 };
 
 // Field j of the packed codes sits in the low bits of mb[j] = bits(kMagic + 2^(p-1) + q_j):
@@ -614,7 +656,8 @@ __global__ void loco_division_selfcheck_kernel(unsigned long long *mismatch) {
 // VAR_LEAN: both decompressors are the single fused multiply-add and no statistics are collected;
 // VAR_LEAN_NR: the same, but dec(e; s_e) is the Newton-Raphson form (s_e = 6 s of the paper), still packed;
 // VAR_GENERAL: the forms are chosen per call at run time (scalar code) and statistics may be collected.
-enum : int { VAR_LEAN = 0, VAR_LEAN_NR = 1, VAR_GENERAL = 2 };
+// VAR_STOCHASTIC: VAR_GENERAL with stochastic rounding of the gradient codes (extension; global scale only).
+enum : int { VAR_LEAN = 0, VAR_LEAN_NR = 1, VAR_GENERAL = 2, VAR_STOCHASTIC = 3 };
 
 // dec(e; s_e) of a pair from the magic floats m2 = kMagic + 128 + e
 template <int VAR>
@@ -640,7 +683,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     constexpr float emagic = kMagic + 128.0f;
     constexpr bool kStateF32 = (STATE == ST_FP32 || STATE == ST_Q8COMP);
     constexpr int GW = WideIn<GRAD, STATE>::GW, EW = WideIn<GRAD, STATE>::EW;
-    constexpr bool LEAN = (VAR != VAR_GENERAL);
+    constexpr bool LEAN = (VAR == VAR_LEAN || VAR == VAR_LEAN_NR);
     const int dq_mode = LEAN ? DEC_FMA : K.dq_mode, de_mode = K.de_mode;
     const int lanes_per_block = (MODE == MODE_BLOCK) ? (K.block_log2 >= 9 ? 32 : (1 << (K.block_log2 - 4))) : 1;
     const f32x2 zero2 = 0ull;
@@ -683,8 +726,9 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         if (__any_sync(kFull, bad_bits != 0u)) return false;
     }
 
-    // ---- optional element-wise clipping of g (finite here, or the row is redone by the careful routine) ------------
-    if (K.clip > 0.0f) {
+    // ---- optional element-wise clipping of g (finite here, or the row is redone by the careful routine); only the
+    //      general variants carry it, the host never launches a lean kernel with clip > 0 ---------------------------
+    if ((VAR == VAR_GENERAL || VAR == VAR_STOCHASTIC) && K.clip > 0.0f) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             float a, b;
@@ -752,7 +796,17 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     for (int k = 0; k < 8; ++k) {
         float y0, y1;
         unpk2(fmul2(h2[k], mult2), y0, y1);
-        const f32x2 m2 = fadd2(pk2(fminf(fmaxf(y0, lo), hi), fminf(fmaxf(y1, lo), hi)), qmagic2);   // kMagic + 2^(p-1) + q
+        float t0 = y0, t1 = y1;
+        bool sat0 = false, sat1 = false;
+        if (VAR == VAR_STOCHASTIC) {                       // floor(y + u): up with probability frac(y)
+            float u[4];
+            sr_uniform4((L.elem0 + static_cast<unsigned long long>(wrow) * kWide + 2 * (k & ~1)) >> 2, K.k_lo, K.k_hi, K.seed_lo, K.seed_hi, u);
+            t0 = floorf(__fadd_rn(y0, u[2 * (k & 1)]));
+            t1 = floorf(__fadd_rn(y1, u[2 * (k & 1) + 1]));
+            sat0 = t0 < lo || t0 > hi;
+            sat1 = t1 < lo || t1 > hi;
+        }
+        const f32x2 m2 = fadd2(pk2(fminf(fmaxf(t0, lo), hi), fminf(fmaxf(t1, lo), hi)), qmagic2);   // kMagic + 2^(p-1) + q
         mb[2 * k] = static_cast<unsigned>(m2);
         mb[2 * k + 1] = static_cast<unsigned>(m2 >> 32);
         f32x2 d2;
@@ -764,8 +818,12 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             d2 = pk2(dec_fast(__uint_as_float(mb[2 * k]), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s),
                      dec_fast(__uint_as_float(mb[2 * k + 1]), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s));
             if (stats) {
-                if (y0 >= hi + 0.5f || y0 < lo - 0.5f) saturated += 1u;
-                if (y1 >= hi + 0.5f || y1 < lo - 0.5f) saturated += 1u;
+                if (VAR == VAR_STOCHASTIC) {
+                    saturated += (sat0 ? 1u : 0u) + (sat1 ? 1u : 0u);
+                } else {
+                    if (y0 >= hi + 0.5f || y0 < lo - 0.5f) saturated += 1u;
+                    if (y1 >= hi + 0.5f || y1 < lo - 0.5f) saturated += 1u;
+                }
             }
         }
         const f32x2 delta2 = (MODE == MODE_BLOCK) ? fsub2_after_mul(h2[k], d2) : fsub2(h2[k], d2);
@@ -845,7 +903,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
 // VAR_LEAN / VAR_LEAN_NR kernels are launched when the host proved the corresponding decompressor forms and no
 // statistics are wanted (VAR_LEAN also for every block-scaled configuration); VAR_GENERAL chooses at run time.
 template <int GRAD, int STATE, int BITS, int MODE, int VAR>
-__global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams P) {
+__global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_constant__ SendParams P) {
     using R = Ring<GRAD, STATE, MODE>;
     constexpr int D = R::kDepth;
     constexpr unsigned gbytes = (GRAD == GRAD_BF16 ? 2u : 4u) * kWide;       // gradient bytes of a wide row
@@ -884,6 +942,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams
         K.s = P.s; K.s_e = P.s_e; K.beta = P.beta; K.omb = P.omb; K.inv_s = P.inv_s; K.inv_se = P.inv_se;
         K.dq_a = P.dq_a; K.dq_b = P.dq_b; K.de_a = P.de_a; K.de_b = P.de_b;
         K.dq_mode = P.dq_mode; K.de_mode = P.de_mode; K.block_log2 = P.block_log2; K.reset = P.reset; K.clip = P.clip;
+        K.seed_lo = P.seed_lo; K.seed_hi = P.seed_hi; K.k_lo = P.k_lo; K.k_hi = P.k_hi;
         const bool stats = P.collect_stats != 0;
         RingAddr<GRAD, STATE> A;
         ring_addresses<GRAD, STATE, MODE>(static_cast<unsigned>(__cvta_generic_to_shared(ring)), lane, threadIdx.x >> 5, A);
@@ -910,8 +969,8 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams
             if (stage_wrow < full_wide) stage(stage_off, stage_wrow);
             cp_async_commit();                 // one group per iteration, empty near the end
             if (!send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, wrow, lane, stats, saturated)) {
-                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(wrow) * kWide, lane);
-                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(wrow) * kWide + kRow, lane);
+                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, VAR == VAR_STOCHASTIC>(P, part, static_cast<unsigned long long>(wrow) * kWide, lane);
+                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, VAR == VAR_STOCHASTIC>(P, part, static_cast<unsigned long long>(wrow) * kWide + kRow, lane);
             }
             slot_off = slot_off + R::kSlotStride == R::kBytes ? 0u : slot_off + R::kSlotStride;
             stage_off = stage_off + R::kSlotStride == R::kBytes ? 0u : stage_off + R::kSlotStride;
@@ -920,7 +979,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const SendParams
         }
     }
     for (unsigned r = first_careful + warp; r < rows; r += nwarps)
-        careful_acc += send_row_careful<GRAD, STATE, BITS, MODE>(P, part, static_cast<unsigned long long>(r) * kRow, lane);
+        careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, VAR == VAR_STOCHASTIC>(P, part, static_cast<unsigned long long>(r) * kRow, lane);
     // each careful call adds at most 8 saturated codes and 2^31 per row with a non-finite value; the 64-bit
     // sum keeps the flag apart from the count
     const unsigned nonfinite = (careful_acc >> 31) != 0ull ? 1u : 0u;

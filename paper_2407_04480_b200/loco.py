@@ -21,6 +21,7 @@ OK, ERR_ARG, ERR_ALIGN, ERR_SIZE, ERR_CUDA, ERR_UNSUPPORTED = 0, -1, -2, -3, -4,
 F32, BF16 = 0, 1
 SCALE_FIXED, SCALE_BLOCK_ABSMAX = 0, 1
 STATE_INT8, STATE_FP32, STATE_NONE, STATE_FP32_Q8COMP = 0, 1, 2, 3
+ROUND_NEAREST, ROUND_STOCHASTIC = 0, 1
 FLAG_NONFINITE = 1
 
 EXPORTS = ("loco_state_bytes", "loco_packed_bytes", "loco_partition_bytes", "loco_partition_capacity",
@@ -45,7 +46,7 @@ class loco_config_t(C.Structure):
                 ("s", C.c_float), ("s_e", C.c_float), ("beta", C.c_float),
                 ("reset_period", C.c_int32), ("state_fmt", C.c_int32), ("grad_dtype", C.c_int32),
                 ("out_dtype", C.c_int32), ("num_partitions", C.c_int32), ("collect_stats", C.c_int32),
-                ("clip", C.c_float)]
+                ("clip", C.c_float), ("rounding", C.c_int32), ("seed_lo", C.c_uint32), ("seed_hi", C.c_uint32)]
 
 
 class loco_adam_t(C.Structure):
@@ -68,11 +69,14 @@ class Config:
     num_partitions: int = 1
     collect_stats: int = 0
     clip: float = 0.0
+    rounding: int = 0
+    seed: int = 0
 
     def c(self) -> loco_config_t:
         return loco_config_t(self.bits, self.scale_mode, self.block_size, self.s, self.s_e, self.beta,
                              self.reset_period, self.state_fmt, self.grad_dtype, self.out_dtype,
-                             self.num_partitions, self.collect_stats, self.clip)
+                             self.num_partitions, self.collect_stats, self.clip, self.rounding,
+                             self.seed & 0xFFFFFFFF, (self.seed >> 32) & 0xFFFFFFFF)
 
 
 _lib = None

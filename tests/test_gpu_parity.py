@@ -355,3 +355,34 @@ def test_zero_plus_plus_style_weight_payload():
     step = (amax / 127.0).repeat_interleave(B)[:n]
     # half a step from the rounding to a code plus half a bf16 ulp of the result
     assert bool(((back - x).abs() <= 0.5 * step * 1.001 + x.abs() * 2.0 ** -8).all())
+
+
+# ---------------------------------------------------------------- stochastic rounding on the shared Philox stream
+
+@pytest.mark.parametrize("mode", [loco.SCALE_FIXED, loco.SCALE_BLOCK_ABSMAX])
+@pytest.mark.parametrize("fmt", [loco.STATE_INT8, loco.STATE_FP32, loco.STATE_NONE])
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_stochastic_rounding(mode, fmt, bits):
+    """rounding = stochastic: the library and the oracle draw the same Philox4x32-10 numbers for (element, iteration, seed)
+    and must produce the same codes, state and statistics bit for bit; ragged size, several parts, both gradient types."""
+    n = 150_001
+    for gd in (loco.BF16, loco.F32):
+        gcfg, ocfg = both_configs(bits=bits, scale_mode=mode, block_size=64, s=2.0 ** 9, s_e=2.0 ** 11, beta=0.5, reset_period=0,
+                                  state_fmt=fmt, grad_dtype=gd, out_dtype=loco.F32, num_partitions=3, rounding=1,
+                                  seed=0x1234567890ABCDEF)
+        w = run_steps(gcfg, ocfg, n, 3, 2e-3, seed=17, k0=5)
+        got, want = reduce_both(gcfg, ocfg, n, [w])
+        assert_reduced_equal(got, want, False)
+
+
+def test_stochastic_rounding_differs_from_nearest_and_between_seeds():
+    n = 1 << 16
+    g = inputs.gaussian(n, 2e-3, seed=18, dtype=torch.bfloat16, device="cuda")
+    codes = []
+    for kw in (dict(rounding=0), dict(rounding=1, seed=1), dict(rounding=1, seed=2)):
+        cfg = loco.Config(bits=4, s=2.0 ** 9, s_e=2.0 ** 11, state_fmt=loco.STATE_NONE, grad_dtype=loco.BF16, **kw)
+        comm = torch.zeros(loco.loco_packed_bytes(cfg, n), dtype=torch.uint8, device="cuda")
+        loco.loco_compensate_quantize_pack(loco.State(cfg, n), g, comm, 3)
+        torch.cuda.synchronize()
+        codes.append(comm.cpu().numpy())
+    assert (codes[0] != codes[1]).mean() > 0.2 and (codes[1] != codes[2]).mean() > 0.2
