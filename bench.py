@@ -320,6 +320,7 @@ def sweep(args, device):
             return
         base = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=512, state_fmt=0,
                     grad_dtype=1, out_dtype=1, num_partitions=8)
+        scatter = kw.pop("scatter", False)
         base.update(kw)
         cfg = loco.Config(**base)
         gsz = 2 if cfg.grad_dtype == loco.BF16 else 4
@@ -329,11 +330,17 @@ def sweep(args, device):
         grads = [inputs.gaussian(n, 1e-3, seed=4, worker=i, dtype=dt, device=device) for i in range(nsets)]
         states = [loco.State(cfg, n) for _ in range(nsets)]
         comms = [torch.empty(max(pb, 16), dtype=torch.uint8, device=device) for _ in range(nsets)]
+        if scatter:                                 # part j of every set goes to a buffer of its own ("worker j's receive slot")
+            part = loco.loco_partition_bytes(cfg, n)
+            dsts = [[torch.empty(max(part, 16), dtype=torch.uint8, device=device) for _ in range(cfg.num_partitions)]
+                    for _ in range(nsets)]
+            send = lambda i, k, st=None: loco.loco_compensate_quantize_pack_scatter(states[i], grads[i], dsts[i], k, stream=st)
+        else:
+            send = lambda i, k, st=None: loco.loco_compensate_quantize_pack(states[i], grads[i], comms[i], k, stream=st)
         for i in range(nsets):                      # a first iteration, so that the timed ones meet a non-zero state
-            loco.loco_compensate_quantize_pack(states[i], grads[i], comms[i], 1)
+            send(i, 1)
         torch.cuda.synchronize()
-        us = _time_launches(lambda i, st: loco.loco_compensate_quantize_pack(states[i], grads[i], comms[i], 2, stream=st),
-                            nsets, max(12, min(200, 4 * nsets)), streams)
+        us = _time_launches(lambda i, st: send(i, 2, st), nsets, max(12, min(200, 4 * nsets)), streams)
         state_rw = {0: 2, 1: 8, 2: 0, 3: 8}[cfg.state_fmt]
         scale_b = (4.0 / cfg.block_size) * (3 if cfg.state_fmt == 0 else 1) if cfg.scale_mode == 1 else 0.0
         bpe = gsz + state_rw + cfg.bits / 8 + scale_b
@@ -418,6 +425,7 @@ def sweep(args, device):
     send_case("bf16 g, int8 state, 4 bit, fixed, element-wise clipping at 2 sigma", M, clip=2e-3)
     send_case("bf16 weights, no state, 8 bit, block-256 absmax (Zero++-style weight payload)", M, bits=8, scale_mode=1, state_fmt=2)
     send_case("bf16 g, int8 state, 4 bit, fixed, stochastic rounding (Philox4x32-10)", M, rounding=1, seed=7)
+    send_case("bf16 g, int8 state, 4 bit, fixed, parts scattered to 8 receive slots (all-to-all in the stores)", M, scatter=True)
     send_case("bf16 g, fp32 state, 4 bit, fixed", M, state_fmt=1)
     send_case("bf16 g, fp32 state + 8-bit compensation, 4 bit, fixed", M, state_fmt=3)
     send_case("bf16 g, no state, 4 bit, fixed", M, state_fmt=2)

@@ -148,6 +148,28 @@ int loco_compensate_quantize_pack(loco_state_t *st, const void *d_grad, void *d_
                                   int64_t step_k, void *stream);
 
 /*
+ * The same send pass with the all-to-all of Sec. 3.3 folded into its stores: part j of the
+ * communication buffer (codes, then scales, loco_partition_bytes() in all) is written to
+ * d_part_dst[j] instead of d_comm + j * loco_partition_bytes().
+ *   d_part_dst  HOST array of num_partitions DEVICE pointers, 16-byte aligned each, every one
+ *               with loco_partition_bytes() writable bytes.  A pointer may lie in this GPU's
+ *               memory or in a peer GPU's memory that the caller has made accessible from this
+ *               device (peer access enabled, or a mapped inter-process / symmetric-memory
+ *               handle): worker r passes, as d_part_dst[j], slot r of worker j's receive area,
+ *               and after every worker's pass has completed, worker j holds part j of all
+ *               workers in its own memory and reduces it with loco_unpack_dequant_reduce
+ *               (first_partition = j, partition_count = 1) from local pointers only.
+ *               The table is copied into the launch; the array may be reused on return.
+ * The kernel only stores to these addresses (plain global stores, no loads, no waits, no flags):
+ * making "every worker's pass has completed" known to the readers is the caller's business (an
+ * event, a barrier of its communication library, or stream order on one GPU).
+ * num_partitions <= 64 here (UNSUPPORTED beyond).  One launch, no allocation, no synchronisation.
+ * Errors: ARG (null table or entry, step_k < 0), ALIGN, UNSUPPORTED, CUDA.
+ */
+int loco_compensate_quantize_pack_scatter(loco_state_t *st, const void *d_grad,
+                                          void *const *d_part_dst, int64_t step_k, void *stream);
+
+/*
  * Receive pass -- Eq. 8: for `partition_count` consecutive parts starting at
  * `first_partition`, average the dequantised codes of `num_workers` workers (summed in
  * worker order in fp32, divided by N) and write out_dtype values to d_out.

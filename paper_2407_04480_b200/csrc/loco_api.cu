@@ -395,15 +395,29 @@ int loco_state_destroy(loco_state_t *st) {
     return rc;
 }
 
-int loco_compensate_quantize_pack(loco_state_t *st, const void *d_grad, void *d_comm, int64_t step_k,
-                                  void *stream) {
+}  // extern "C"
+
+namespace {
+
+// The send pass.  Its partitions go to d_comm + j * stride, or, with d_part_dst, to d_part_dst[j].
+int send_launch(loco_state_t *st, const void *d_grad, void *d_comm, void *const *d_part_dst, int64_t step_k,
+                void *stream) {
     if (!st || step_k < 0) return LOCO_ERR_ARG;
-    if (st->n == 0) return LOCO_OK;
-    if (!d_grad || !d_comm) return LOCO_ERR_ARG;
-    if (!aligned16(d_grad) || !aligned16(d_comm)) return LOCO_ERR_ALIGN;
     const loco_config_t &c = st->cfg;
+    if (d_part_dst && c.num_partitions > kMaxScatter) return LOCO_ERR_UNSUPPORTED;
+    if (st->n == 0) return LOCO_OK;
+    if (!d_grad || (!d_comm && !d_part_dst)) return LOCO_ERR_ARG;
+    if (!aligned16(d_grad) || !aligned16(d_comm)) return LOCO_ERR_ALIGN;
     SendParams P;
     std::memset(&P, 0, sizeof(P));
+    if (d_part_dst) {
+        for (int j = 0; j < c.num_partitions; ++j) {
+            if (!d_part_dst[j]) return LOCO_ERR_ARG;
+            if (!aligned16(d_part_dst[j])) return LOCO_ERR_ALIGN;
+            P.part_dst[j] = static_cast<uint8_t *>(d_part_dst[j]);
+        }
+        P.scatter = 1;
+    }
     P.grad = d_grad;
     P.state = st->d_state;
     P.comm = static_cast<uint8_t *>(d_comm);
@@ -438,6 +452,22 @@ int loco_compensate_quantize_pack(loco_state_t *st, const void *d_grad, void *d_
     if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;
     g_launches.fetch_add(1);
     return LOCO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int loco_compensate_quantize_pack(loco_state_t *st, const void *d_grad, void *d_comm, int64_t step_k,
+                                  void *stream) {
+    if (st && st->n != 0 && !d_comm) return LOCO_ERR_ARG;
+    return send_launch(st, d_grad, d_comm, nullptr, step_k, stream);
+}
+
+int loco_compensate_quantize_pack_scatter(loco_state_t *st, const void *d_grad, void *const *d_part_dst,
+                                          int64_t step_k, void *stream) {
+    if (!d_part_dst) return LOCO_ERR_ARG;
+    return send_launch(st, d_grad, nullptr, d_part_dst, step_k, stream);
 }
 
 }  // extern "C"

@@ -46,6 +46,7 @@ constexpr unsigned kMagicBits = 0x4B400000u;
 constexpr float kFltMax = 3.402823466e+38f;
 constexpr unsigned kFlagNonFinite = 1u;
 constexpr unsigned kFull = 0xffffffffu;
+constexpr int kMaxScatter = 64;    // most partitions a scattering send pass can address
 
 struct SendParams {
     const void *grad;
@@ -70,6 +71,8 @@ struct SendParams {
     unsigned seed_lo, seed_hi;       // key of its Philox stream
     unsigned k_lo, k_hi;             // the iteration counter, part of the Philox counter
     unsigned long long *status;      // [0] flags, [1] saturated codes
+    int scatter;                     // 1: partition j is written to part_dst[j] instead of comm + j * stride
+    uint8_t *part_dst[kMaxScatter];  // destinations of the partitions (this GPU's memory or a peer's)
 };
 
 struct ReduceParams {
@@ -359,7 +362,7 @@ __device__ __noinline__ unsigned send_row_careful(const SendParams &P, unsigned 
     send_core<STATE, BITS, MODE, STOCH>(P, g, c, prev, valid, lanes_per_block, i0, code, e_new, scale, nonfinite, saturated);
 
     // codes (and the block's scale) into the partition's areas of the communication buffer
-    uint8_t *pbase = P.comm + part * P.stride;
+    uint8_t *pbase = P.scatter ? P.part_dst[part] : P.comm + part * P.stride;
     const unsigned long long ol = o + static_cast<unsigned long long>(lane) * kLaneElems;
     store_codes8<BITS>(pbase + ol * BITS / 8, code);
     if (MODE == MODE_BLOCK) {
@@ -931,7 +934,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_con
         L.lane_elem = static_cast<unsigned>(lane) * kWideLane;
         L.elem0 = base + L.lane_elem;
         L.state = static_cast<uint8_t *>(P.state) + L.elem0 * (STATE == ST_INT8 ? 1u : 4u);
-        uint8_t *pbase = P.comm + part * P.stride;
+        uint8_t *pbase = P.scatter ? P.part_dst[part] : P.comm + part * P.stride;
         L.codes = pbase + static_cast<size_t>(L.lane_elem) * BITS / 8;
         L.wire_scales = reinterpret_cast<float *>(pbase + P.code_bytes);
         L.state_scales = reinterpret_cast<float *>(static_cast<uint8_t *>(P.state) + P.state_scale_off);

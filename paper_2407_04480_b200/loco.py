@@ -31,7 +31,7 @@ EXPORTS = ("loco_state_bytes", "loco_packed_bytes", "loco_partition_bytes", "loc
            "loco_send_host_workspace_bytes", "loco_reduce_host_workspace_bytes",
            "loco_compensate_quantize_pack_host", "loco_unpack_dequant_reduce_host",
            "loco_unpack_dequant_reduce_host_noalloc", "loco_selfcheck_block_division",
-           "loco_unpack_dequant_reduce_adam")
+           "loco_unpack_dequant_reduce_adam", "loco_compensate_quantize_pack_scatter")
 NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
@@ -113,6 +113,8 @@ def lib() -> C.CDLL:
         L.loco_send_host_workspace_bytes.argtypes = [cp, u64]
         L.loco_reduce_host_workspace_bytes.restype = u64
         L.loco_reduce_host_workspace_bytes.argtypes = [cp, u64, i32, i32]
+        L.loco_compensate_quantize_pack_scatter.restype = C.c_int
+        L.loco_compensate_quantize_pack_scatter.argtypes = [vp, vp, vp, i64, vp]
         L.loco_compensate_quantize_pack_host.restype = C.c_int
         L.loco_compensate_quantize_pack_host.argtypes = [vp, vp, vp, vp, u64, i64, vp]
         L.loco_unpack_dequant_reduce_host.restype = C.c_int
@@ -232,6 +234,24 @@ def loco_compensate_quantize_pack(st: State, grad: torch.Tensor, comm: torch.Ten
         raise ValueError("communication buffer too small or not uint8")
     _check(lib().loco_compensate_quantize_pack(st.handle, _dev_ptr(grad), _dev_ptr(comm), step_k,
                                                _stream_ptr(stream)), "loco_compensate_quantize_pack")
+
+
+def loco_compensate_quantize_pack_scatter(st: State, grad: torch.Tensor, part_dst: Sequence, step_k: int,
+                                          stream=None) -> None:
+    """Send pass whose part j goes to part_dst[j] (a uint8 CUDA tensor of at least loco_partition_bytes(), or an
+    int device address -- this GPU's memory or a peer's mapped here) instead of one contiguous buffer."""
+    want = torch.bfloat16 if st.cfg.grad_dtype == BF16 else torch.float32
+    if grad.dtype != want or grad.numel() != st.n:
+        raise ValueError("gradient must be %s with %d elements" % (want, st.n))
+    if len(part_dst) != st.cfg.num_partitions:
+        raise ValueError("one destination per partition is needed (%d)" % st.cfg.num_partitions)
+    need = loco_partition_bytes(st.cfg, st.n)
+    for d in part_dst:
+        if not isinstance(d, int) and (d.dtype != torch.uint8 or d.numel() < need):
+            raise ValueError("a destination is too small or not uint8")
+    ptrs = (C.c_void_p * len(part_dst))(*[d if isinstance(d, int) else _dev_ptr(d) for d in part_dst])
+    _check(lib().loco_compensate_quantize_pack_scatter(st.handle, _dev_ptr(grad), ptrs, step_k, _stream_ptr(stream)),
+           "loco_compensate_quantize_pack_scatter")
 
 
 def loco_unpack_dequant_reduce(cfg: Config, packed: Sequence, n: int, out: torch.Tensor,
