@@ -270,6 +270,69 @@ def oracle_sample(threads: int, buckets_per_thread: int):
     return 2.0 * elems / dt / 1e9, dt, elems
 
 
+# ------------------------------------------------------------------------------------------------ real exchange
+
+def run_exchange(args, rank: int, world: int, device, config):
+    """The same buckets with the exchange of Sec. 3.3 between the ranks: every rank compresses its own gradient into
+    `world` parts, the parts travel (NCCL all-to-all, or the send kernel's own stores into the peers' receive slots),
+    every rank averages the `world` copies of its part.  One stream per rank, bucket after bucket; no CUDA graph, since
+    the collective sits between the two kernels.  value = gradient bytes entering the path on all ranks per second."""
+    import torch.distributed as dist
+    from paper_2407_04480_b200 import exchange, inputs, loco
+    if not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29531")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=device)
+    cfg = loco.Config(**{**CFG, "num_partitions": world})
+    layout = inputs.llama2_7b()
+    scales = inputs.group_scales(1, layout.n_groups)
+    buckets = inputs.bucket_ranges(layout.numel, BUCKET)
+    if args.buckets > 0:
+        buckets = buckets[:args.buckets]
+    total = buckets[-1][1]
+    grad = torch.empty(total, dtype=torch.bfloat16, device=device)
+    for lo, hi in buckets:
+        grad[lo:hi] = inputs.layout_slice(layout, lo, hi, scales, 1e-4, seed=1, worker=rank, step=0, device=device)
+    transport = exchange.Transport(cfg, BUCKET, kind=args.exchange, device=device)
+    exs = [exchange.BucketExchange(cfg, hi - lo, shared=transport) for lo, hi in buckets]
+    shard = torch.empty(max(e.shard_elems() for e in exs), dtype=torch.bfloat16, device=device)
+
+    def step(k):
+        for e, (lo, hi) in zip(exs, buckets):
+            e.step(grad[lo:hi], k, shard)
+
+    for k in range(max(3, args.warmup)):
+        step(k)
+    dist.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(device.index)
+    sampler.start()
+    before = loco.loco_launch_count()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for k in range(args.steps):
+        step(100 + k)
+    end.record()
+    dist.barrier()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    t = torch.tensor([start.elapsed_time(end) / args.steps], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    lt = torch.tensor([loco.loco_launch_count() - before], device=device, dtype=torch.int64)
+    dist.all_reduce(lt)
+    step_ms = float(t.item())
+    if rank == 0:
+        config = dict(config, exchange=args.exchange, streams=1, workers_on_reduce_side=world,
+                      workload=config["workload"].split(":")[0] + ": %d bf16 buckets per rank; per bucket: send pass, exchange "
+                      "of %d parts between the ranks, average of this rank's part" % (len(buckets), world))
+        print(json.dumps({"metric": METRIC + " -- with the real exchange", "value": world * 2 * total / (step_ms * 1e-3) / 1e9,
+                          "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+                          "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                          "dtype": "f32", "data": "synthetic", "config": config, "clocks": clocks, "e2e": None,
+                          "gpu_launches": int(lt.item()), "roofline": None, "cpu_baseline": None}))
+    dist.destroy_process_group()
+
+
 # ------------------------------------------------------------------------------------------------ sweep (config 5)
 
 def _time_launches(launch, n_sets: int, launches: int, streams):
@@ -469,6 +532,10 @@ def main():
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the bench line: the size / type / width / worker-count table (one JSON line per case, then markdown)")
     ap.add_argument("--sweep-filter", default="", help="with --sweep: only the cases whose 'kernel: label' contains this text")
+    ap.add_argument("--exchange", choices=("none", "collective", "peer_store"), default="none",
+                    help="none (default): every rank runs the two passes on its own buckets, no data-path collective; "
+                         "collective / peer_store: the real exchange of Sec. 3.3 between the ranks (NCCL all-to-all, or the "
+                         "send kernel storing into the peers' receive slots), each rank reducing its own shard")
     ap.add_argument("--streams", type=int, default=2,
                     help="streams the per-bucket launches of a phase are spread over (1 = strictly one after the other)")
     args = ap.parse_args()
@@ -523,6 +590,9 @@ def main():
     if args.sweep:
         if rank == 0:
             sweep(args, device)
+        return
+    if args.exchange != "none":
+        run_exchange(args, rank, world, device, config)
         return
     wl = RankWorkload(rank, device, args.buckets)
     nb = len(wl.buckets)

@@ -199,30 +199,37 @@ SendKernel pick_send(const loco_config_t *c, int mode, int var) {
 // ---- reduce dispatch ---------------------------------------------------------------------
 
 using ReduceFn = void (*)(const ReduceParams);
+struct ReduceKernel { ReduceFn fn; int smem_bytes; };     // smem_bytes: the kernel's cp.async ring (0: none)
 
-template <int OUT, int BITS, bool ADAM>
-ReduceFn pick_reduce_path(int mode, int path) {
-    if (mode != MODE_FIXED) return loco_reduce_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL, ADAM>;
-    switch (path) {
-    case PATH_INT: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_INT, ADAM>;
-    case PATH_MUL: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_MUL, ADAM>;
-    case PATH_NEWTON: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON, ADAM>;
-    default: return loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE, ADAM>;
-    }
-}
 template <int OUT, int BITS>
-ReduceFn pick_reduce_mode(int mode, int path, bool adam) {
-    return adam ? pick_reduce_path<OUT, BITS, true>(mode, path) : pick_reduce_path<OUT, BITS, false>(mode, path);
+ReduceKernel pick_reduce_path(int mode, int path, bool adam) {
+    if (adam) {
+        if (mode != MODE_FIXED) return {loco_reduce_adam_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>, 0};
+        switch (path) {
+        case PATH_INT: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_INT>, 0};
+        case PATH_MUL: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, 0};
+        case PATH_NEWTON: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON>, 0};
+        default: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE>, 0};
+        }
+    }
+    if (mode != MODE_FIXED) return {loco_reduce_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>, static_cast<int>(RecvRing<BITS, MODE_BLOCK>::kCtaBytes)};
+    const int smem = static_cast<int>(RecvRing<BITS, MODE_FIXED>::kCtaBytes);
+    switch (path) {
+    case PATH_INT: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_INT>, smem};
+    case PATH_MUL: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, smem};
+    case PATH_NEWTON: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON>, smem};
+    default: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE>, smem};
+    }
 }
 template <int OUT>
-ReduceFn pick_reduce_bits(int bits, int mode, int path, bool adam) {
+ReduceKernel pick_reduce_bits(int bits, int mode, int path, bool adam) {
     switch (bits) {
-    case 2: return pick_reduce_mode<OUT, 2>(mode, path, adam);
-    case 4: return pick_reduce_mode<OUT, 4>(mode, path, adam);
-    default: return pick_reduce_mode<OUT, 8>(mode, path, adam);
+    case 2: return pick_reduce_path<OUT, 2>(mode, path, adam);
+    case 4: return pick_reduce_path<OUT, 4>(mode, path, adam);
+    default: return pick_reduce_path<OUT, 8>(mode, path, adam);
     }
 }
-ReduceFn pick_reduce(const loco_config_t *c, int mode, int path, bool adam) {
+ReduceKernel pick_reduce(const loco_config_t *c, int mode, int path, bool adam) {
     return c->out_dtype == LOCO_BF16 ? pick_reduce_bits<GRAD_BF16>(c->bits, mode, path, adam)
                                      : pick_reduce_bits<GRAD_F32>(c->bits, mode, path, adam);
 }
@@ -574,12 +581,27 @@ int reduce_launch(const loco_config_t *cfg, const void *const *d_packed, int32_t
         const volatile float o1 = 1.0f - ad->beta1, o2 = 1.0f - ad->beta2;       // rounded once to fp32
         P.omb1 = o1; P.omb2 = o2;
     }
-    ReduceFn fn = pick_reduce(cfg, mode, path, ad != nullptr);
-    static int occ_cache[2][3][2][4][2] = {};
-    int &occ = occ_cache[cfg->out_dtype == LOCO_BF16][cfg->bits == 2 ? 0 : (cfg->bits == 4 ? 1 : 2)][mode][path][ad != nullptr];
+    const ReduceKernel rk = pick_reduce(cfg, mode, path, ad != nullptr);
+    const ReduceFn fn = rk.fn;
+    const int smem = rk.smem_bytes;
+    // per device and kernel, once: the shared-memory attributes of the kernel and the CTAs of it that fit an SM
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return LOCO_ERR_CUDA;
+    }
+    static int occ_cache[64][2][3][2][4][2] = {};
+    int &occ = occ_cache[dev][cfg->out_dtype == LOCO_BF16][cfg->bits == 2 ? 0 : (cfg->bits == 4 ? 1 : 2)][mode][path][ad != nullptr];
     if (occ == 0) {
         int v = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, fn, kThreads, 0) != cudaSuccess || v < 1) {
+        if (smem > 0) {
+            if (cudaFuncSetAttribute(reinterpret_cast<const void *>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+                cudaFuncSetAttribute(reinterpret_cast<const void *>(fn), cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess) {
+                cudaGetLastError();
+                return LOCO_ERR_CUDA;
+            }
+        }
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, fn, kThreads, smem) != cudaSuccess || v < 1) {
             cudaGetLastError();
             return LOCO_ERR_CUDA;
         }
@@ -587,7 +609,7 @@ int reduce_launch(const loco_config_t *cfg, const void *const *d_packed, int32_t
     }
     const uint64_t rows = (L.lp + kWide - 1) / kWide;
     dim3 grid(grid_x_for(rows, partition_count, occ), static_cast<unsigned>(partition_count), 1);
-    fn<<<grid, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(P);
+    fn<<<grid, kThreads, static_cast<size_t>(smem), static_cast<cudaStream_t>(stream)>>>(P);
     if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;
     g_launches.fetch_add(1);
     return LOCO_OK;

@@ -464,11 +464,19 @@ __device__ __forceinline__ void cp_async16(unsigned saddr, const void *gmem) {
 __device__ __forceinline__ void cp_async4(unsigned saddr, const void *gmem) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(saddr), "l"(gmem) : "memory");
 }
+__device__ __forceinline__ void cp_async8(unsigned saddr, const void *gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" :: "r"(saddr), "l"(gmem) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
 __device__ __forceinline__ uint4 lds16(unsigned saddr) {
     uint4 v;
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint2 lds8(unsigned saddr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(saddr) : "memory");
     return v;
 }
 __device__ __forceinline__ unsigned lds4(unsigned saddr) {
@@ -1206,10 +1214,14 @@ struct WideSums {
 // PATH_INT: the integer-sum path (only with the global scale); otherwise the generic path with dec(q; s) as a multiply
 // (also the block-scaled form), as the Newton-Raphson division, or as the IEEE division.  Separate kernels, so that each
 // path gets the registers and the occupancy it wants and no per-element choice is left.
-// ADAM: the Adam-family update of the optimizer is applied to the averaged gradient in the same pass.
 enum : int { PATH_INT = 0, PATH_MUL = 1, PATH_NEWTON = 2, PATH_DIVIDE = 3 };
-template <int OUT, int BITS, int MODE, int PATH, bool ADAM>
-__global__ void __launch_bounds__(kThreads, ADAM ? 3 : 1) loco_reduce_kernel(const ReduceParams P) {
+
+// The receive pass with the Adam-family update of the optimizer applied to the averaged gradient in the same pass.
+// Its traffic is dominated by the lane's 48 optimizer words, which are loaded into registers at the start of a row;
+// the codes are read with plain loads (one wide row at a time on the integer path, groups of four workers with the
+// next group's loads in flight on the others).
+template <int OUT, int BITS, int MODE, int PATH>
+__global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const ReduceParams P) {
     constexpr unsigned kRowBytes = kWide * BITS / 8;                  // code bytes of one wide row
     const int lane = threadIdx.x & 31;
     const unsigned long long part = blockIdx.y;                       // relative to P.first
@@ -1229,13 +1241,13 @@ __global__ void __launch_bounds__(kThreads, ADAM ? 3 : 1) loco_reduce_kernel(con
 
     if (PATH == PATH_INT) {
         // code areas below 4 GiB (checked by the host): row offsets fit 32 bits
-        constexpr int kUnroll = ADAM ? 1 : 2;
+        constexpr int kUnroll = 1;
         for (unsigned r = warp; r < rows; r += kUnroll * nwarps) {
             WideSums<BITS> sums[kUnroll];
             unsigned off[kUnroll];
             bool ok[kUnroll];
             AdamRegs AR;
-            if (ADAM) {
+            {
                 const unsigned long long o = static_cast<unsigned long long>(r) * kWide + lane_elem;
                 if (o + 16 <= valid) adam_load16(P, out0 + o, AR);
             }
@@ -1269,8 +1281,7 @@ __global__ void __launch_bounds__(kThreads, ADAM ? 3 : 1) loco_reduce_kernel(con
                     const float acc = __fmaf_rn(sums[u].get(j), P.ra, P.rb);
                     res[j] = P.div_mode == 0 ? acc : div_workers(P, acc);
                 }
-                if (ADAM) adam_finish16<OUT>(P, out0 + o, res, valid - o, wide32, AR);
-                else store_out16<OUT>(P.out, out0 + o, res, valid - o, wide32);
+                adam_finish16<OUT>(P, out0 + o, res, valid - o, wide32, AR);
             }
         }
         return;
@@ -1314,7 +1325,7 @@ __global__ void __launch_bounds__(kThreads, ADAM ? 3 : 1) loco_reduce_kernel(con
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc2[i] = 0ull;
         AdamRegs AR;
-        if (ADAM && o + 16 <= valid) adam_load16(P, out0 + o, AR);
+        if (o + 16 <= valid) adam_load16(P, out0 + o, AR);
         for (int g = 0; g < groups; ++g) {
             Group nxt;
             if (g + 1 < groups) load_group(r, g + 1, nxt);
@@ -1360,9 +1371,264 @@ __global__ void __launch_bounds__(kThreads, ADAM ? 3 : 1) loco_reduce_kernel(con
             res[2 * i] = div_workers(P, a);                                          // the 1/N of Eq. 8
             res[2 * i + 1] = div_workers(P, b);
         }
-        if (ADAM) adam_finish16<OUT>(P, out0 + o, res, valid - o, wide32, AR);
-        else store_out16<OUT>(P.out, out0 + o, res, valid - o, wide32);
+        adam_finish16<OUT>(P, out0 + o, res, valid - o, wide32, AR);
     }
+}
+
+// ------------------------------------------------------------------------------------------
+// The receive pass with the workers' codes travelling through a per-warp cp.async ring.
+//
+// The unit of the ring is a group of up to 4 entries (entry = one worker's wide row: 512 codes, and in block mode
+// the scales of its blocks): with N >= 4 workers a group is 4 workers of one row (a row takes ceil(N/4) groups),
+// with fewer workers it is all workers of 4/N rows, so that the bytes in flight per warp do not shrink with N.
+// All copies are 16 bytes wide (the narrower forms of cp.async move fewer bytes per instruction and are slower):
+// a 16-byte chunk holds the codes of 16 / (2 BITS) lanes, so one copy instruction of the warp fills 1, 2 or 4
+// entries, and cp.async.wait_group followed by __syncwarp() orders every lane's reads after all lanes' copies.
+// One cp.async group per ring group; the ring holds kGroups of them, kGroups - 1 are in flight while one is summed.
+template <int BITS, int MODE> struct RecvRing {
+    static constexpr unsigned kLaneBytes = 2u * BITS;                       // the 16 codes of one lane
+    static constexpr unsigned kCodeBytes = 32u * kLaneBytes;                // one worker's wide row
+    static constexpr unsigned kEntry = kCodeBytes + (MODE == MODE_BLOCK ? 64u : 0u);   // + up to 16 block scales
+    static constexpr unsigned kGroupBytes = 4u * kEntry;
+    static constexpr unsigned kWarpBytes = 8192u;
+    static constexpr int kGroups = (kWarpBytes / kGroupBytes) > 8u ? 8 : static_cast<int>(kWarpBytes / kGroupBytes);
+    static constexpr unsigned kCtaBytes = kWarps * kGroups * kGroupBytes;
+    static constexpr int kEntriesPerCopy = 16 / kLaneBytes;                 // entries one copy instruction fills: 4, 2, 1
+    static constexpr int kCopies = 4 / kEntriesPerCopy;                     // copy instructions per group: 1, 2, 4
+    static constexpr int kLanesPerEntry = 32 / kEntriesPerCopy;             // 8, 16, 32
+    static constexpr unsigned kChunkElems = 128u / BITS;                    // codes in a 16-byte chunk
+    static_assert(kGroups >= 3, "the ring must hold at least three groups");
+};
+
+template <int OUT, int BITS, int MODE, int PATH>
+__global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_constant__ ReduceParams P) {
+    using R = RecvRing<BITS, MODE>;
+    constexpr int G = R::kGroups;
+    constexpr unsigned kRowBytes = kWide * BITS / 8;                  // code bytes of one wide row
+    extern __shared__ __align__(16) uint8_t ring[];
+    const int lane = threadIdx.x & 31;
+    const unsigned long long part = blockIdx.y;                       // relative to P.first
+    const unsigned warp = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    const unsigned nwarps = gridDim.x * kWarps;
+    const unsigned long long base = (P.first + part) * P.lp;          // first bucket element of the part
+    if (base >= P.n) return;
+    const unsigned long long avail = P.n - base;
+    const unsigned long long valid = avail >= P.lp ? P.lp : avail;
+    const unsigned rows = static_cast<unsigned>((valid + kWide - 1) / kWide);
+    const unsigned long long poff = part * P.stride;
+    const unsigned long long out0 = part * P.lp;                      // output index of the part's first element
+    const unsigned lane_elem = static_cast<unsigned>(lane) * kWideLane;
+    const unsigned lane_byte = static_cast<unsigned>(lane) * R::kLaneBytes;
+    const int N = P.num_workers;
+    const bool wide32 = P.out_align32 != 0;
+    const int C = N < 4 ? N : 4;                                      // workers per group
+    const int group_entries = (4 / C) * C;                            // 4, 4, 3, 4: (rows per group) x C
+    const int chunks = (N + C - 1) / C;                               // groups per row
+    const unsigned row_step = static_cast<unsigned>(4 / C) * nwarps;  // a group's rows are r, r + nwarps, ...
+    const unsigned my_ring = static_cast<unsigned>(__cvta_generic_to_shared(ring)) +
+                             (threadIdx.x >> 5) * (G * R::kGroupBytes);
+
+    // What this lane copies for a group: in copy instruction i it serves entry j = i * kEntriesPerCopy + lane / kLanesPerEntry
+    // (entry j = worker j % C of the group's row j / C) with the 16-byte chunk lane % kLanesPerEntry of that entry's codes.
+    unsigned cp_dst[R::kCopies], cp_row[R::kCopies], cp_src[R::kCopies];   // ring offset, row offset (in rows), byte offset in the row
+    int cp_w[R::kCopies], cp_lim[R::kCopies];                                // worker within the group
+#pragma unroll
+    for (int i = 0; i < R::kCopies; ++i) {
+        const int j = i * R::kEntriesPerCopy + lane / R::kLanesPerEntry;
+        const unsigned chunk = static_cast<unsigned>(lane % R::kLanesPerEntry);
+        const int rr = C == 1 ? j : (C == 2 ? (j >> 1) : 0);
+        cp_w[i] = j - rr * C;
+        cp_lim[i] = j < group_entries ? N - cp_w[i] : 0;              // the entry's worker exists in chunk c iff c * C < cp_lim
+        cp_row[i] = static_cast<unsigned>(rr) * nwarps;
+        cp_src[i] = chunk * 16u;
+        cp_dst[i] = static_cast<unsigned>(j) * R::kEntry + chunk * 16u;
+    }
+    // block mode: copy instruction i (of 2) brings the scales of entries 2i and 2i+1, lane % 16 = block within the row
+    const unsigned blocks_per_row = MODE == MODE_BLOCK ? (static_cast<unsigned>(kWide) >> P.block_log2) : 0u;
+    int sc_w[2], sc_lim[2];
+    unsigned sc_row[2], sc_dst[2];
+    if (MODE == MODE_BLOCK) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int j = 2 * i + (lane >> 4);
+            const int rr = C == 1 ? j : (C == 2 ? (j >> 1) : 0);
+            sc_w[i] = j - rr * C;
+            sc_lim[i] = (j < group_entries && static_cast<unsigned>(lane & 15) < blocks_per_row) ? N - sc_w[i] : 0;
+            sc_row[i] = static_cast<unsigned>(rr) * nwarps;
+            sc_dst[i] = static_cast<unsigned>(j) * R::kEntry + R::kCodeBytes + 4u * static_cast<unsigned>(lane & 15);
+        }
+    }
+
+    // copy the entries of group (first row r0, chunk c) into ring slot `slot`
+    const unsigned full_rows = static_cast<unsigned>(valid / kWide);  // rows all of whose 512 elements exist
+    auto stage = [&](unsigned slot, unsigned r0, int c) {
+        const unsigned dst = my_ring + slot * R::kGroupBytes;
+        const int w0 = c * C;
+        // every row of the group is a full one: no per-chunk bounds to check (r0 + 3 nwarps covers all group shapes)
+        const bool interior = r0 + 3u * nwarps < full_rows;
+#pragma unroll
+        for (int i = 0; i < R::kCopies; ++i) {
+            const unsigned row = r0 + cp_row[i];
+            bool go = w0 < cp_lim[i];                                 // this lane has an entry and its worker exists
+            if (!interior)
+                go = go && row < rows && static_cast<unsigned long long>(row) * kWide + (cp_src[i] >> 4) * R::kChunkElems < valid;
+            if (go)
+                cp_async16(dst + cp_dst[i], P.parts[w0 + cp_w[i]] + poff + static_cast<unsigned long long>(row) * kRowBytes + cp_src[i]);
+        }
+        if (MODE == MODE_BLOCK) {
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const unsigned row = r0 + sc_row[i];
+                const unsigned long long blk = ((static_cast<unsigned long long>(row) * kWide) >> P.block_log2) + static_cast<unsigned>(lane & 15);
+                bool go = w0 < sc_lim[i];
+                if (!interior) go = go && row < rows && (blk << P.block_log2) < valid;
+                if (go)
+                    cp_async4(dst + sc_dst[i], reinterpret_cast<const float *>(P.parts[w0 + sc_w[i]] + poff + P.code_bytes) + blk);
+            }
+        }
+    };
+
+    WideSums<BITS> sums;                                              // PATH_INT
+    f32x2 acc2[8];                                                    // the other paths
+    const f32x2 inv2 = dup2(P.inv_s), negs2 = dup2(-P.s);
+    const unsigned scale_off = R::kCodeBytes + 4u * (lane_elem >> P.block_log2);      // this lane's scale within an entry
+
+    auto begin_row = [&]() {
+        if (PATH == PATH_INT) sums.clear();
+        else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc2[i] = 0ull;
+        }
+    };
+    auto fetch = [&](unsigned entry, WideCodes<BITS> &cw, float &scale) {             // this lane's codes (and scale) of an entry
+        if (BITS == 8) { const uint4 t = lds16(entry + lane_byte); cw.w[0] = t.x; cw.w[1 % WideCodes<BITS>::W] = t.y; cw.w[2 % WideCodes<BITS>::W] = t.z; cw.w[3 % WideCodes<BITS>::W] = t.w; }
+        else if (BITS == 4) { const uint2 t = lds8(entry + lane_byte); cw.w[0] = t.x; cw.w[1 % WideCodes<BITS>::W] = t.y; }
+        else cw.w[0] = lds4(entry + lane_byte);
+        scale = (PATH != PATH_INT && MODE == MODE_BLOCK) ? __uint_as_float(lds4(entry + scale_off)) : P.gen_mul;
+    };
+    auto accumulate = [&](const WideCodes<BITS> &cw, float scale) {                   // one worker's codes into the row's sums
+        if (PATH == PATH_INT) {
+            sums.add(cw);
+            return;
+        }
+        unsigned x[WideCodes<BITS>::W], xh[WideCodes<BITS>::W];
+#pragma unroll
+        for (int t = 0; t < WideCodes<BITS>::W; ++t) {
+            x[t] = cw.w[t] ^ (BITS == 8 ? 0x80808080u : (BITS == 4 ? 0x88888888u : 0xAAAAAAAAu));
+            xh[t] = x[t] >> (BITS == 4 ? 12 : 16);
+        }
+        const f32x2 sc2 = dup2(scale);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            float k0, k1;
+            const float m0 = field_magic<BITS>(x, xh, 2 * k, k0);
+            const float m1 = field_magic<BITS>(x, xh, 2 * k + 1, k1);
+            const f32x2 q2 = fadd2(pk2(m0, m1), pk2(-k0, -k1));                 // the two codes, exact
+            if (PATH == PATH_MUL) {
+                acc2[k] = fadd2_after_mul(acc2[k], fmul2(q2, sc2));             // product and sum rounded separately
+            } else if (PATH == PATH_NEWTON) {
+                const f32x2 q0 = fmul2(q2, inv2);
+                const f32x2 rem = ffma2(q0, negs2, q2);
+                acc2[k] = fadd2(acc2[k], ffma2(rem, inv2, q0));
+            } else {
+                float a, b, cc, d;
+                unpk2(q2, a, b);
+                unpk2(acc2[k], cc, d);
+                acc2[k] = pk2(__fadd_rn(cc, __fdiv_rn(a, P.s)), __fadd_rn(d, __fdiv_rn(b, P.s)));
+            }
+        }
+    };
+    auto finish_row = [&](unsigned long long o) {                                    // the 1/N of Eq. 8 and the store
+        if (o >= valid) return;
+        float res[16];
+        if (PATH == PATH_INT) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float acc = __fmaf_rn(sums.get(i), P.ra, P.rb);
+                res[i] = P.div_mode == 0 ? acc : div_workers(P, acc);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float a, b;
+                unpk2(acc2[i], a, b);
+                res[2 * i] = div_workers(P, a);
+                res[2 * i + 1] = div_workers(P, b);
+            }
+        }
+        store_out16<OUT>(P.out, out0 + o, res, valid - o, wide32);
+    };
+
+    // producer: this warp's groups in order -- rows warp, warp + row_step, ...; within a row its chunks
+    unsigned p_row = warp, p_slot = 0u, c_slot = 0u;
+    int p_chunk = 0;
+    auto produce = [&]() {                     // one cp.async group per call, empty past the end
+        if (p_row < rows) stage(p_slot, p_row, p_chunk);
+        cp_async_commit();
+        if (++p_chunk == chunks) { p_chunk = 0; p_row += row_step; }
+        p_slot = p_slot + 1 == static_cast<unsigned>(G) ? 0u : p_slot + 1;
+    };
+    auto next_group = [&]() -> unsigned {      // wait for the oldest group, refill the slot summed last, return the group's ring address
+        cp_async_wait<G - 2>();                // all groups but the newest G-2 have landed
+        __syncwarp();                          // ... for all lanes; and all lanes are done with the slot that is refilled now
+        produce();
+        const unsigned src = my_ring + c_slot * R::kGroupBytes;
+        c_slot = c_slot + 1 == static_cast<unsigned>(G) ? 0u : c_slot + 1;
+        return src;
+    };
+#pragma unroll 1
+    for (int i = 0; i < G - 1; ++i) produce();
+
+    if (N >= 4) {
+        // a group = 4 workers (fewer in a row's last group) of one row
+#pragma unroll 1
+        for (unsigned row = warp; row < rows; row += nwarps) {
+            const unsigned long long o = static_cast<unsigned long long>(row) * kWide + lane_elem;
+            begin_row();
+#pragma unroll 1
+            for (int left = N; left > 0; left -= 4) {
+                const unsigned src = next_group();
+                if (left >= 4) {
+                    WideCodes<BITS> cw[4];
+                    float sc[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) fetch(src + e * R::kEntry, cw[e], sc[e]);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) accumulate(cw[e], sc[e]);
+                } else {
+#pragma unroll 1
+                    for (int e = 0; e < left; ++e) {
+                        WideCodes<BITS> cw;
+                        float sc;
+                        fetch(src + e * R::kEntry, cw, sc);
+                        accumulate(cw, sc);
+                    }
+                }
+            }
+            finish_row(o);
+        }
+    } else {
+        // a group = all N workers of 4 / N rows
+#pragma unroll 1
+        for (unsigned r0 = warp; r0 < rows; r0 += row_step) {
+            unsigned src = next_group();
+#pragma unroll 1
+            for (unsigned row = r0; row < rows && row < r0 + row_step; row += nwarps) {
+                const unsigned long long o = static_cast<unsigned long long>(row) * kWide + lane_elem;
+                begin_row();
+#pragma unroll 1
+                for (int e = 0; e < N; ++e) {
+                    WideCodes<BITS> cw;
+                    float sc;
+                    fetch(src, cw, sc);
+                    accumulate(cw, sc);
+                    src += R::kEntry;
+                }
+                finish_row(o);
+            }
+        }
+    }
+    cp_async_wait<0>();
 }
 
 }  // namespace loco

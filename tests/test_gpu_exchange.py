@@ -130,3 +130,55 @@ def test_scatter_argument_errors():
         loco.loco_compensate_quantize_pack_scatter(st2, g2, [buf.data_ptr()] * 65, 0)
     assert e.value.code == loco.ERR_UNSUPPORTED
     torch.cuda.synchronize()
+
+
+# ---- the torch.distributed plumbing, on the one GPU there is: a group of one rank ----------------------------------
+
+def _free_port():
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+@pytest.fixture(scope="module")
+def one_rank_group():
+    import os
+    import torch.distributed as dist
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(_free_port())
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    yield dist.group.WORLD
+    torch.cuda.synchronize()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("transport", ["collective", "peer_store"])
+def test_bucket_exchange_group_of_one(one_rank_group, transport):
+    """With one rank the exchange is the send pass, a transfer to itself and a one-worker average: the result is
+    dec(q) of the oracle's codes, and the state is the oracle's, over several iterations (both areas get used)."""
+    from paper_2407_04480_b200 import exchange
+    n = 700_001
+    kw = dict(bits=4, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=0, state_fmt=0, grad_dtype=1, out_dtype=0)
+    gcfg, ocfg = parity.both_configs(num_partitions=1, collect_stats=0, **kw)
+    try:
+        ex = exchange.BucketExchange(gcfg, n, group=one_rank_group, transport=transport)
+    except (RuntimeError, ImportError, AttributeError) as err:
+        if transport == "peer_store":
+            pytest.skip("symmetric memory is not available here: %s" % str(err).splitlines()[0])
+        raise
+    assert ex.shard_elems() == n
+    ostate, ocomm = orc.new_state(ocfg, n), orc.new_comm(ocfg, n)
+    out = torch.empty(n, dtype=torch.float32, device="cuda")
+    for k in range(3):
+        g = inputs.gaussian(n, 1e-3, seed=9, worker=0, step=k, dtype=torch.bfloat16)
+        gnp = inputs.as_numpy_bits(g)
+        ex.step(parity.to_device(gnp, True), k, out)
+        torch.cuda.synchronize()
+        orc.send_step(ocfg, gnp, ostate, ocomm, k)
+        want = orc.reduce(ocfg, n, [ocomm])
+        got = out.cpu().numpy()
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), "step %d" % k
+        gv, _ = orc.state_views(ocfg, n, ex.state.buffer.cpu().numpy())
+        ov, _ = orc.state_views(ocfg, n, ostate)
+        assert np.array_equal(gv, ov)
