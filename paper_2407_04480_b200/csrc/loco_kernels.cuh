@@ -1423,69 +1423,82 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
     const bool wide32 = P.out_align32 != 0;
     const int C = N < 4 ? N : 4;                                      // workers per group
     const int group_entries = (4 / C) * C;                            // 4, 4, 3, 4: (rows per group) x C
-    const int chunks = (N + C - 1) / C;                               // groups per row
     const unsigned row_step = static_cast<unsigned>(4 / C) * nwarps;  // a group's rows are r, r + nwarps, ...
     const unsigned my_ring = static_cast<unsigned>(__cvta_generic_to_shared(ring)) +
                              (threadIdx.x >> 5) * (G * R::kGroupBytes);
 
     // What this lane copies for a group: in copy instruction i it serves entry j = i * kEntriesPerCopy + lane / kLanesPerEntry
     // (entry j = worker j % C of the group's row j / C) with the 16-byte chunk lane % kLanesPerEntry of that entry's codes.
-    unsigned cp_dst[R::kCopies], cp_row[R::kCopies], cp_src[R::kCopies];   // ring offset, row offset (in rows), byte offset in the row
-    int cp_w[R::kCopies], cp_lim[R::kCopies];                                // worker within the group
+    // Per copy the lane keeps: where it goes in the ring group, which worker of the group it reads, the two limits that
+    // decide whether there is anything to copy (w0 < cp_lim: the worker exists; p_row < cp_rowlim: the chunk lies below the
+    // part's valid length), and the running byte offset of the chunk inside a worker's part.
+    const unsigned full_rows = static_cast<unsigned>(valid / kWide);  // rows all of whose 512 elements exist
+    const unsigned tail = static_cast<unsigned>(valid - static_cast<unsigned long long>(full_rows) * kWide);   // elements of the partial row
+    unsigned cp_dst[R::kCopies], cp_rowlim[R::kCopies];
+    int cp_w[R::kCopies], cp_lim[R::kCopies];
+    unsigned long long cp_off[R::kCopies];
 #pragma unroll
     for (int i = 0; i < R::kCopies; ++i) {
         const int j = i * R::kEntriesPerCopy + lane / R::kLanesPerEntry;
         const unsigned chunk = static_cast<unsigned>(lane % R::kLanesPerEntry);
         const int rr = C == 1 ? j : (C == 2 ? (j >> 1) : 0);
+        const unsigned row_off = static_cast<unsigned>(rr) * nwarps;
+        const unsigned lim_row = full_rows + (chunk * R::kChunkElems < tail ? 1u : 0u);
         cp_w[i] = j - rr * C;
-        cp_lim[i] = j < group_entries ? N - cp_w[i] : 0;              // the entry's worker exists in chunk c iff c * C < cp_lim
-        cp_row[i] = static_cast<unsigned>(rr) * nwarps;
-        cp_src[i] = chunk * 16u;
+        cp_lim[i] = j < group_entries ? N - cp_w[i] : 0;
+        cp_rowlim[i] = lim_row > row_off ? lim_row - row_off : 0u;
         cp_dst[i] = static_cast<unsigned>(j) * R::kEntry + chunk * 16u;
+        cp_off[i] = poff + static_cast<unsigned long long>(warp + row_off) * kRowBytes + chunk * 16u;
     }
     // block mode: copy instruction i (of 2) brings the scales of entries 2i and 2i+1, lane % 16 = block within the row
-    const unsigned blocks_per_row = MODE == MODE_BLOCK ? (static_cast<unsigned>(kWide) >> P.block_log2) : 0u;
     int sc_w[2], sc_lim[2];
-    unsigned sc_row[2], sc_dst[2];
+    unsigned sc_rowlim[2], sc_dst[2];
+    unsigned long long sc_off[2];
     if (MODE == MODE_BLOCK) {
+        const unsigned blocks_per_row = static_cast<unsigned>(kWide) >> P.block_log2;
+        const unsigned idx = static_cast<unsigned>(lane & 15);
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int j = 2 * i + (lane >> 4);
             const int rr = C == 1 ? j : (C == 2 ? (j >> 1) : 0);
+            const unsigned row_off = static_cast<unsigned>(rr) * nwarps;
+            const unsigned lim_row = full_rows + ((idx << P.block_log2) < tail ? 1u : 0u);
             sc_w[i] = j - rr * C;
-            sc_lim[i] = (j < group_entries && static_cast<unsigned>(lane & 15) < blocks_per_row) ? N - sc_w[i] : 0;
-            sc_row[i] = static_cast<unsigned>(rr) * nwarps;
-            sc_dst[i] = static_cast<unsigned>(j) * R::kEntry + R::kCodeBytes + 4u * static_cast<unsigned>(lane & 15);
+            sc_lim[i] = (j < group_entries && idx < blocks_per_row) ? N - sc_w[i] : 0;
+            sc_rowlim[i] = lim_row > row_off ? lim_row - row_off : 0u;
+            sc_dst[i] = static_cast<unsigned>(j) * R::kEntry + R::kCodeBytes + 4u * idx;
+            sc_off[i] = poff + P.code_bytes + 4ull * (((static_cast<unsigned long long>(warp + row_off) * kWide) >> P.block_log2) + idx);
         }
     }
+    const unsigned long long code_step = static_cast<unsigned long long>(row_step) * kRowBytes;             // per advance of p_row
+    const unsigned long long scale_step = 4ull * ((static_cast<unsigned long long>(row_step) * kWide) >> P.block_log2);
 
-    // copy the entries of group (first row r0, chunk c) into ring slot `slot`
-    const unsigned full_rows = static_cast<unsigned>(valid / kWide);  // rows all of whose 512 elements exist
-    auto stage = [&](unsigned slot, unsigned r0, int c) {
-        const unsigned dst = my_ring + slot * R::kGroupBytes;
-        const int w0 = c * C;
-        // every row of the group is a full one: no per-chunk bounds to check (r0 + 3 nwarps covers all group shapes)
-        const bool interior = r0 + 3u * nwarps < full_rows;
+    // producer: this warp's groups in order -- rows warp, warp + row_step, ...; within a row its chunks of C workers
+    unsigned p_row = warp, p_slot = 0u, c_slot = 0u;
+    int p_w0 = 0;                                                      // first worker of the producer's chunk
+    auto produce = [&]() {                     // one cp.async group per call, empty past the end
+        const unsigned dst = my_ring + p_slot * R::kGroupBytes;
 #pragma unroll
-        for (int i = 0; i < R::kCopies; ++i) {
-            const unsigned row = r0 + cp_row[i];
-            bool go = w0 < cp_lim[i];                                 // this lane has an entry and its worker exists
-            if (!interior)
-                go = go && row < rows && static_cast<unsigned long long>(row) * kWide + (cp_src[i] >> 4) * R::kChunkElems < valid;
-            if (go)
-                cp_async16(dst + cp_dst[i], P.parts[w0 + cp_w[i]] + poff + static_cast<unsigned long long>(row) * kRowBytes + cp_src[i]);
-        }
+        for (int i = 0; i < R::kCopies; ++i)
+            if (p_w0 < cp_lim[i] && p_row < cp_rowlim[i]) cp_async16(dst + cp_dst[i], P.parts[p_w0 + cp_w[i]] + cp_off[i]);
         if (MODE == MODE_BLOCK) {
 #pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const unsigned row = r0 + sc_row[i];
-                const unsigned long long blk = ((static_cast<unsigned long long>(row) * kWide) >> P.block_log2) + static_cast<unsigned>(lane & 15);
-                bool go = w0 < sc_lim[i];
-                if (!interior) go = go && row < rows && (blk << P.block_log2) < valid;
-                if (go)
-                    cp_async4(dst + sc_dst[i], reinterpret_cast<const float *>(P.parts[w0 + sc_w[i]] + poff + P.code_bytes) + blk);
+            for (int i = 0; i < 2; ++i)
+                if (p_w0 < sc_lim[i] && p_row < sc_rowlim[i]) cp_async4(dst + sc_dst[i], P.parts[p_w0 + sc_w[i]] + sc_off[i]);
+        }
+        cp_async_commit();
+        p_w0 += C;
+        if (p_w0 >= N) {
+            p_w0 = 0;
+            p_row += row_step;
+#pragma unroll
+            for (int i = 0; i < R::kCopies; ++i) cp_off[i] += code_step;
+            if (MODE == MODE_BLOCK) {
+#pragma unroll
+                for (int i = 0; i < 2; ++i) sc_off[i] += scale_step;
             }
         }
+        p_slot = p_slot + 1 == static_cast<unsigned>(G) ? 0u : p_slot + 1;
     };
 
     WideSums<BITS> sums;                                              // PATH_INT
@@ -1509,32 +1522,32 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
     auto accumulate = [&](const WideCodes<BITS> &cw, float scale) {                   // one worker's codes into the row's sums
         if (PATH == PATH_INT) {
             sums.add(cw);
-            return;
-        }
-        unsigned x[WideCodes<BITS>::W], xh[WideCodes<BITS>::W];
+        } else {
+            unsigned x[WideCodes<BITS>::W], xh[WideCodes<BITS>::W];
 #pragma unroll
-        for (int t = 0; t < WideCodes<BITS>::W; ++t) {
-            x[t] = cw.w[t] ^ (BITS == 8 ? 0x80808080u : (BITS == 4 ? 0x88888888u : 0xAAAAAAAAu));
-            xh[t] = x[t] >> (BITS == 4 ? 12 : 16);
-        }
-        const f32x2 sc2 = dup2(scale);
+            for (int t = 0; t < WideCodes<BITS>::W; ++t) {
+                x[t] = cw.w[t] ^ (BITS == 8 ? 0x80808080u : (BITS == 4 ? 0x88888888u : 0xAAAAAAAAu));
+                xh[t] = x[t] >> (BITS == 4 ? 12 : 16);
+            }
+            const f32x2 sc2 = dup2(scale);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            float k0, k1;
-            const float m0 = field_magic<BITS>(x, xh, 2 * k, k0);
-            const float m1 = field_magic<BITS>(x, xh, 2 * k + 1, k1);
-            const f32x2 q2 = fadd2(pk2(m0, m1), pk2(-k0, -k1));                 // the two codes, exact
-            if (PATH == PATH_MUL) {
-                acc2[k] = fadd2_after_mul(acc2[k], fmul2(q2, sc2));             // product and sum rounded separately
-            } else if (PATH == PATH_NEWTON) {
-                const f32x2 q0 = fmul2(q2, inv2);
-                const f32x2 rem = ffma2(q0, negs2, q2);
-                acc2[k] = fadd2(acc2[k], ffma2(rem, inv2, q0));
-            } else {
-                float a, b, cc, d;
-                unpk2(q2, a, b);
-                unpk2(acc2[k], cc, d);
-                acc2[k] = pk2(__fadd_rn(cc, __fdiv_rn(a, P.s)), __fadd_rn(d, __fdiv_rn(b, P.s)));
+            for (int k = 0; k < 8; ++k) {
+                float k0, k1;
+                const float m0 = field_magic<BITS>(x, xh, 2 * k, k0);
+                const float m1 = field_magic<BITS>(x, xh, 2 * k + 1, k1);
+                const f32x2 q2 = fadd2(pk2(m0, m1), pk2(-k0, -k1));                 // the two codes, exact
+                if (PATH == PATH_MUL) {
+                    acc2[k] = fadd2_after_mul(acc2[k], fmul2(q2, sc2));             // product and sum rounded separately
+                } else if (PATH == PATH_NEWTON) {
+                    const f32x2 q0 = fmul2(q2, inv2);
+                    const f32x2 rem = ffma2(q0, negs2, q2);
+                    acc2[k] = fadd2(acc2[k], ffma2(rem, inv2, q0));
+                } else {
+                    float a, b, cc, d;
+                    unpk2(q2, a, b);
+                    unpk2(acc2[k], cc, d);
+                    acc2[k] = pk2(__fadd_rn(cc, __fdiv_rn(a, P.s)), __fadd_rn(d, __fdiv_rn(b, P.s)));
+                }
             }
         }
     };
@@ -1543,31 +1556,29 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
         float res[16];
         if (PATH == PATH_INT) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float acc = __fmaf_rn(sums.get(i), P.ra, P.rb);
-                res[i] = P.div_mode == 0 ? acc : div_workers(P, acc);
-            }
+            for (int i = 0; i < 16; ++i) res[i] = __fmaf_rn(sums.get(i), P.ra, P.rb);
         } else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float a, b;
-                unpk2(acc2[i], a, b);
-                res[2 * i] = div_workers(P, a);
-                res[2 * i + 1] = div_workers(P, b);
+            for (int i = 0; i < 8; ++i) unpk2(acc2[i], res[2 * i], res[2 * i + 1]);
+        }
+        // one branch per row, not per element: which form the division by N takes is the same for the whole launch
+        if (PATH != PATH_INT && P.div_mode == 0) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) res[i] = __fmul_rn(res[i], P.inv_n);
+        } else if (P.div_mode == 1) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float q0 = __fmul_rn(res[i], P.inv_n);
+                const float rem = __fmaf_rn(-q0, P.n_workers_f, res[i]);
+                res[i] = __fmaf_rn(rem, P.inv_n, q0);
             }
+        } else if (P.div_mode == 2) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) res[i] = __fdiv_rn(res[i], P.n_workers_f);
         }
         store_out16<OUT>(P.out, out0 + o, res, valid - o, wide32);
     };
 
-    // producer: this warp's groups in order -- rows warp, warp + row_step, ...; within a row its chunks
-    unsigned p_row = warp, p_slot = 0u, c_slot = 0u;
-    int p_chunk = 0;
-    auto produce = [&]() {                     // one cp.async group per call, empty past the end
-        if (p_row < rows) stage(p_slot, p_row, p_chunk);
-        cp_async_commit();
-        if (++p_chunk == chunks) { p_chunk = 0; p_row += row_step; }
-        p_slot = p_slot + 1 == static_cast<unsigned>(G) ? 0u : p_slot + 1;
-    };
     auto next_group = [&]() -> unsigned {      // wait for the oldest group, refill the slot summed last, return the group's ring address
         cp_async_wait<G - 2>();                // all groups but the newest G-2 have landed
         __syncwarp();                          // ... for all lanes; and all lanes are done with the slot that is refilled now

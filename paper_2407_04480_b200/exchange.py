@@ -89,6 +89,9 @@ class Transport:
             self.areas = [torch.empty(nbytes, dtype=torch.uint8, device=device)]
             self.peer_ptrs = None
         else:
+            import os
+            # this transport only stores through plain peer pointers: no NVLink multicast object is needed for it
+            os.environ.setdefault("TORCH_SYMM_MEM_DISABLE_MULTICAST", "1")
             import torch.distributed._symmetric_memory as symm_mem
             self.areas, self.peer_ptrs, self._handles = [], [], []
             for _ in range(2):

@@ -170,6 +170,22 @@ def test_reduce_workers(N, bits, mode, s):
         assert_reduced_equal(got, want, od == loco.BF16)
 
 
+@pytest.mark.parametrize("N", [4, 6, 7, 9, 17, 33, 64])
+@pytest.mark.parametrize("mode,s,B", [(loco.SCALE_FIXED, 2.0 ** 12, 256), (loco.SCALE_FIXED, 3000.0, 256),
+                                      (loco.SCALE_BLOCK_ABSMAX, 1.0, 32), (loco.SCALE_BLOCK_ABSMAX, 1.0, 128)])
+def test_reduce_group_shapes(N, mode, s, B):
+    """Worker counts around the receive kernel's groups of four (one full group, a short last group, many groups, the
+    maximum; 17+ workers leave the integer path) and bucket sizes from less than one wide row to a few rows per warp."""
+    for n, bits in ((300, 4), (513, 8), (40_000, 2), (150_001, 4)):
+        gcfg, ocfg = both_configs(bits=bits, scale_mode=mode, block_size=B, s=s, s_e=4 * s, beta=0.5,
+                                  reset_period=0, state_fmt=loco.STATE_NONE, grad_dtype=loco.BF16, out_dtype=loco.BF16,
+                                  num_partitions=2)
+        base = [run_steps(gcfg, ocfg, n, 1, 5e-4, seed=33, worker=w) for w in range(min(N, 5))]
+        ws = [base[w % len(base)] for w in range(N)]
+        got, want = reduce_both(gcfg, ocfg, n, ws)
+        assert_reduced_equal(got, want, True, "n=%d bits=%d N=%d" % (n, bits, N))
+
+
 # ---------------------------------------------------------------- Llama-2-7B-shaped buckets, 8 workers
 
 def test_llama_buckets_sampled():
