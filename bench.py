@@ -48,8 +48,8 @@ SEND_BYTES_PER_ELEM = 2 + 1 + 1 + 0.5
 # dram__bytes_read.sum + dram__bytes_write.sum per launch (one 25M-element bucket) from the ncu captures summarised under
 # profiles/.  Reads equal the algorithmic reads; most written lines are still in the 126 MB L2 when a lone launch ends,
 # so the DRAM write counter of a single captured launch is far below the algorithmic 37.5 / 50 MB.
-SEND_DRAM_BYTES_PER_LAUNCH = 75.02e6 + 3.12e6
-REDUCE_DRAM_BYTES_PER_LAUNCH = 100.03e6 + 7.79e6
+SEND_DRAM_BYTES_PER_LAUNCH = 75.03e6 + 3.12e6
+REDUCE_DRAM_BYTES_PER_LAUNCH = 100.03e6 + 14.08e6
 
 
 def measured_peak():
@@ -650,6 +650,31 @@ def main():
         sev[0].record(); s_send.replay(); s_send.replay(); sev[1].record(); s_reduce.replay(); s_reduce.replay(); sev[2].record()
         torch.cuda.synchronize()
         serial_us = (sev[0].elapsed_time(sev[1]) * 1e3 / (2 * nb), sev[1].elapsed_time(sev[2]) * 1e3 / (2 * nb))
+    # also outside the timed region, for scale: a plain device-to-device copy (the driver's cudaMemcpyAsync, issued by
+    # torch) that moves as many bytes per launch as the send kernel does, one launch per bucket over memory not in L2
+    copy_us = None
+    if not args.no_graph:
+        half = int(SEND_BYTES_PER_ELEM * BUCKET / 2) // 256 * 256          # bytes copied = half of read + written
+        src8, dst8 = wl.grad.view(torch.uint8), wl.out_buf.view(torch.uint8)
+        span = min(src8.numel(), dst8.numel())
+        count = max(1, min(nb, span // half))
+
+        def copies(streams):
+            wl._fan_out(lambda i, st: dst8[i * half:(i + 1) * half].copy_(src8[i * half:(i + 1) * half]), count, streams)
+
+        res = []
+        for strs in (None, side if args.streams > 1 else None):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                copies(strs)
+            g.replay()
+            ce = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+            torch.cuda.synchronize()
+            ce[0].record(); g.replay(); g.replay(); ce[1].record()
+            torch.cuda.synchronize()
+            res.append(ce[0].elapsed_time(ce[1]) * 1e3 / (2 * count))
+        copy_us = {"bytes_moved_per_launch": 2 * half, "one_stream_launch_us": res[0], "one_stream_gbs": 2 * half / res[0] / 1e3,
+                   "two_stream_launch_us": res[1], "two_stream_gbs": 2 * half / res[1] / 1e3}
     total_ms = start.elapsed_time(end)
     send_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / K
     recv_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
@@ -707,6 +732,8 @@ def main():
         kernels["send"]["one_stream_hbm_gbs"] = wl.send_bytes / nb / (serial_us[0] * 1e-6) / 1e9
         kernels["reduce"]["one_stream_launch_us"] = serial_us[1]
         kernels["reduce"]["one_stream_hbm_gbs"] = wl.recv_bytes / nb / (serial_us[1] * 1e-6) / 1e9
+    if copy_us is not None:
+        kernels["device_copy_same_bytes_as_send"] = copy_us
     cpu = None
     if not args.no_cpu_baseline:
         v, dt, elems = oracle_sample(cores, 2)
