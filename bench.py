@@ -220,15 +220,25 @@ def run_e2e(wl: RankWorkload, steps: int, warmup: int):
         h2d += 2 * n + WORKERS * loco.loco_packed_bytes(cfg, n)
         d2h += loco.loco_packed_bytes(cfg, n) + 2 * n
 
+    # Two streams: the send pass of bucket i+1 (gradient in, codes out) runs while the receive pass of bucket i (8 packed
+    # buffers in, averaged gradient out) is still copying, so that both directions of the host link are busy; the receive
+    # pass of a bucket starts only after its send pass has finished.
+    s_send, s_recv = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    done = [torch.cuda.Event() for _ in wl.buckets]
+
     def step(k):
+        cur = torch.cuda.current_stream()
+        s_send.wait_stream(cur)
+        s_recv.wait_stream(cur)
         for i, (lo, hi) in enumerate(wl.buckets):
             n = hi - lo
             r = i % ring
-            loco.loco_compensate_quantize_pack_host(wl.states[i], h_grad[r][:n], h_comm[r], w_send, k)
-        for i, (lo, hi) in enumerate(wl.buckets):
-            n = hi - lo
-            r = i % ring
-            loco.loco_unpack_dequant_reduce_host(cfg, h_parts[r], n, h_out[r], w_red)
+            loco.loco_compensate_quantize_pack_host(wl.states[i], h_grad[r][:n], h_comm[r], w_send, k, stream=s_send)
+            done[i].record(s_send)
+            s_recv.wait_event(done[i])
+            loco.loco_unpack_dequant_reduce_host(cfg, h_parts[r], n, h_out[r], w_red, stream=s_recv)
+        cur.wait_stream(s_send)
+        cur.wait_stream(s_recv)
 
     for k in range(warmup):
         step(1000 + k)
@@ -696,7 +706,8 @@ def main():
             e_ms = float(t.item())
         e2e = {"value": world * wl.grad_bytes / (e_ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d * world,
                "d2h_bytes_per_step": d2h * world, "ms_per_step": e_ms, "steps": args.e2e_steps,
-               "how": "loco_*_host entry points, pinned host buffers, copies inside the timed region"}
+               "how": "loco_*_host entry points, pinned host buffers, copies inside the timed region; send and receive passes "
+                      "on two streams so that host-to-device and device-to-host copies overlap"}
     if dist is not None:
         dist.barrier()
     if rank != 0:
