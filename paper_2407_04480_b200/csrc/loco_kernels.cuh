@@ -668,13 +668,16 @@ __global__ void loco_division_selfcheck_kernel(unsigned long long *mismatch) {
 // VAR_LEAN_NR: the same, but dec(e; s_e) is the Newton-Raphson form (s_e = 6 s of the paper), still packed;
 // VAR_GENERAL: the forms are chosen per call at run time (scalar code) and statistics may be collected.
 // VAR_STOCHASTIC: VAR_GENERAL with stochastic rounding of the gradient codes (extension; global scale only).
-enum : int { VAR_LEAN = 0, VAR_LEAN_NR = 1, VAR_GENERAL = 2, VAR_STOCHASTIC = 3 };
+// VAR_LEAN_X / VAR_LEAN_NR_X: the lean forms plus what a call may ask for on top (statistics, clipping of g).
+enum : int { VAR_LEAN = 0, VAR_LEAN_NR = 1, VAR_GENERAL = 2, VAR_STOCHASTIC = 3, VAR_LEAN_X = 4, VAR_LEAN_NR_X = 5 };
+__host__ __device__ constexpr bool var_is_lean(int var) { return var == VAR_LEAN || var == VAR_LEAN_NR || var == VAR_LEAN_X || var == VAR_LEAN_NR_X; }
+__host__ __device__ constexpr bool var_has_extras(int var) { return var != VAR_LEAN && var != VAR_LEAN_NR; }
 
 // dec(e; s_e) of a pair from the magic floats m2 = kMagic + 128 + e
 template <int VAR>
 __device__ __forceinline__ f32x2 dec_state2(const SendConsts &K, f32x2 m2, float emagic, int de_mode) {
-    if (VAR == VAR_LEAN) return ffma2(m2, dup2(K.de_a), dup2(K.de_b));
-    if (VAR == VAR_LEAN_NR) {
+    if (VAR == VAR_LEAN || VAR == VAR_LEAN_X) return ffma2(m2, dup2(K.de_a), dup2(K.de_b));
+    if (VAR == VAR_LEAN_NR || VAR == VAR_LEAN_NR_X) {
         const f32x2 e2 = fadd2(m2, dup2(-emagic));                   // the codes, exact
         const f32x2 inv2 = dup2(K.inv_se);
         const f32x2 q0 = fmul2(e2, inv2);
@@ -694,7 +697,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     constexpr float emagic = kMagic + 128.0f;
     constexpr bool kStateF32 = (STATE == ST_FP32 || STATE == ST_Q8COMP);
     constexpr int GW = WideIn<GRAD, STATE>::GW, EW = WideIn<GRAD, STATE>::EW;
-    constexpr bool LEAN = (VAR == VAR_LEAN || VAR == VAR_LEAN_NR);
+    constexpr bool LEAN = var_is_lean(VAR), EXTRAS = var_has_extras(VAR);
     const int dq_mode = LEAN ? DEC_FMA : K.dq_mode, de_mode = K.de_mode;
     const int lanes_per_block = (MODE == MODE_BLOCK) ? (K.block_log2 >= 9 ? 32 : (1 << (K.block_log2 - 4))) : 1;
     const f32x2 zero2 = 0ull;
@@ -737,9 +740,9 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         if (__any_sync(kFull, bad_bits != 0u)) return false;
     }
 
-    // ---- optional element-wise clipping of g (finite here, or the row is redone by the careful routine); only the
-    //      general variants carry it, the host never launches a lean kernel with clip > 0 ---------------------------
-    if ((VAR == VAR_GENERAL || VAR == VAR_STOCHASTIC) && K.clip > 0.0f) {
+    // ---- optional element-wise clipping of g (finite here, or the row is redone by the careful routine); the plain
+    //      lean variants do not carry it, the host never launches one of them with clip > 0 ----------------------------
+    if (EXTRAS && K.clip > 0.0f) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
             float a, b;
@@ -828,13 +831,13 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         } else {
             d2 = pk2(dec_fast(__uint_as_float(mb[2 * k]), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s),
                      dec_fast(__uint_as_float(mb[2 * k + 1]), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s));
-            if (stats) {
-                if (VAR == VAR_STOCHASTIC) {
-                    saturated += (sat0 ? 1u : 0u) + (sat1 ? 1u : 0u);
-                } else {
-                    if (y0 >= hi + 0.5f || y0 < lo - 0.5f) saturated += 1u;
-                    if (y1 >= hi + 0.5f || y1 < lo - 0.5f) saturated += 1u;
-                }
+        }
+        if (MODE != MODE_BLOCK && EXTRAS && stats) {
+            if (VAR == VAR_STOCHASTIC) {
+                saturated += (sat0 ? 1u : 0u) + (sat1 ? 1u : 0u);
+            } else {
+                if (y0 >= hi + 0.5f || y0 < lo - 0.5f) saturated += 1u;
+                if (y1 >= hi + 0.5f || y1 < lo - 0.5f) saturated += 1u;
             }
         }
         const f32x2 delta2 = (MODE == MODE_BLOCK) ? fsub2_after_mul(h2[k], d2) : fsub2(h2[k], d2);
@@ -911,8 +914,9 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
 // grid = (ctas per partition, partitions).  Each warp walks the partition's wide rows with the stride of all
 // warps working on that partition; the inputs of its next rows are on their way through the cp.async ring.
 // What is left of the partition (a last half-wide row, partial and padding rows) goes to the careful routine.
-// VAR_LEAN / VAR_LEAN_NR kernels are launched when the host proved the corresponding decompressor forms and no
-// statistics are wanted (VAR_LEAN also for every block-scaled configuration); VAR_GENERAL chooses at run time.
+// VAR_LEAN / VAR_LEAN_NR kernels are launched when the host proved the corresponding decompressor forms and neither
+// statistics nor clipping are wanted (VAR_LEAN also for every block-scaled configuration), VAR_LEAN_X / VAR_LEAN_NR_X
+// when they are; VAR_GENERAL chooses the decompressor forms at run time.
 template <int GRAD, int STATE, int BITS, int MODE, int VAR>
 __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_constant__ SendParams P) {
     using R = Ring<GRAD, STATE, MODE>;
