@@ -433,6 +433,13 @@ __device__ __forceinline__ f32x2 fsub2_after_mul(f32x2 a, f32x2 b) {
     unpk2(b, b0, b1);
     return pk2(__fsub_rn(a0, b0), __fsub_rn(a1, b1));
 }
+// For a running sum that starts at +0 the sign of a zero product never shows (acc is never -0), so there the product
+// may be taken as fma(a, b, +0): the rounded product up to the sign of zero, which no later add can be contracted with.
+__device__ __forceinline__ f32x2 fmul2_pz(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(0ull));
+    return d;
+}
 __device__ __forceinline__ unsigned hfma2_bf16(unsigned a, unsigned b, unsigned c) {
     unsigned d;
     asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
@@ -1351,7 +1358,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const Red
                     const float m1 = field_magic<BITS>(x, xh, 2 * k + 1, k1);
                     const f32x2 q2 = fadd2(pk2(m0, m1), pk2(-k0, -k1));                 // the two codes, exact
                     if (PATH == PATH_MUL) {
-                        acc2[k] = fadd2_after_mul(acc2[k], fmul2(q2, sc2));             // product and sum rounded separately
+                        acc2[k] = fadd2(acc2[k], fmul2_pz(q2, sc2));                 // product and sum rounded separately
                     } else if (PATH == PATH_NEWTON) {
                         const f32x2 q0 = fmul2(q2, inv2);
                         const f32x2 rem = ffma2(q0, negs2, q2);
@@ -1541,7 +1548,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
                 const float m1 = field_magic<BITS>(x, xh, 2 * k + 1, k1);
                 const f32x2 q2 = fadd2(pk2(m0, m1), pk2(-k0, -k1));                 // the two codes, exact
                 if (PATH == PATH_MUL) {
-                    acc2[k] = fadd2_after_mul(acc2[k], fmul2(q2, sc2));             // product and sum rounded separately
+                    acc2[k] = fadd2(acc2[k], fmul2_pz(q2, sc2));                 // product and sum rounded separately
                 } else if (PATH == PATH_NEWTON) {
                     const f32x2 q0 = fmul2(q2, inv2);
                     const f32x2 rem = ffma2(q0, negs2, q2);
