@@ -107,15 +107,18 @@ void orc_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t ou
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-/* The uniform number in [0, 1) that stochastic rounding adds to element i of the bucket at iteration k:
- * word (i mod 4) of philox(counter = (i/4 low, i/4 high, k low, k high), key = seed), top 24 bits times 2^-24. */
+/* The number in (0, 1) that stochastic rounding adds to element i of the bucket at iteration k: one byte of the 16 that
+ * philox(counter = (i/16 low, i/16 high, k low, k high), key = seed) returns -- byte (i mod 4) of word ((i mod 16) / 4),
+ * least significant byte first -- taken as (byte + 1/2) / 256: 256 equally likely values, each in the middle of its
+ * cell, so that the probability of rounding up equals frac(y) to within 1/512. */
 static float sr_uniform(const orc_config *c, uint64_t i, int64_t k) {
-    const uint64_t blk = i >> 2;
+    const uint64_t blk = i >> 4;
     const uint32_t ctr[4] = {(uint32_t)blk, (uint32_t)(blk >> 32), (uint32_t)(uint64_t)k, (uint32_t)((uint64_t)k >> 32)};
     const uint32_t key[2] = {c->seed_lo, c->seed_hi};
     uint32_t out[4];
     orc_philox4x32_10(ctr, key, out);
-    return (float)(out[i & 3] >> 8) * 5.9604644775390625e-8f;      /* 2^-24, exact */
+    const uint32_t byte = (out[(i >> 2) & 3] >> (8 * (unsigned)(i & 3))) & 0xFFu;
+    return ((float)byte + 0.5f) * 0.00390625f;                     /* (byte + 1/2) / 256, exact */
 }
 float orc_sr_uniform(const orc_config *c, uint64_t i, int64_t k) { return sr_uniform(c, i, k); }
 
@@ -289,7 +292,7 @@ static int32_t quantise(const orc_config *c, uint64_t i, int64_t k, float h, flo
     if (isinf(h)) { *err0 = 1; status[0] |= ORC_FLAG_NONFINITE; return h > 0 ? qmax_of(p) : qmin_of(p); }
     float y = h * mult;                       /* h x s of Eq. 1 */
     if (c->rounding == 1) {
-        /* stochastic rounding (extension): floor(y + u), u uniform in [0, 1): up with probability frac(y) */
+        /* stochastic rounding (extension): floor(y + u), u uniform over 256 values in (0, 1): up with probability frac(y) */
         const float t = y + sr_uniform(c, i, k);
         float r = floorf(t);
         const float lo = (float)qmin_of(p), hi = (float)qmax_of(p);

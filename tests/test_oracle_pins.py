@@ -664,7 +664,8 @@ def test_philox_known_answer_vectors():
 
 def test_stochastic_rounding_properties():
     """q is floor or ceil of h x s (inside the range), integers are never moved, the mean over many draws is h x s, the
-    stream depends on (element, iteration, seed) only, and the uniform numbers are 24-bit fractions in [0, 1)."""
+    stream depends on (element, iteration, seed) only, and the added numbers are the 256 cell centres (b + 1/2) / 256,
+    equally likely, one byte of a Philox block of 16 per element."""
     n, s = 1 << 14, 4.0
     kw = dict(bits=8, s=s, s_e=16.0, beta=0.5, reset_period=0, state_fmt=orc.STATE_NONE, grad_dtype=orc.F32, out_dtype=orc.F32)
     cfg = orc.OracleConfig(rounding=1, seed=12345, **kw)
@@ -692,9 +693,18 @@ def test_stochastic_rounding_properties():
     comm3 = orc.new_comm(other, n)
     orc.send_step(other, h, orc.new_state(other, n), comm3, 200)
     assert (orc.unpack_codes(comm3, n, 8) != draws[-1]).mean() > 0.2
-    us = np.array([orc.sr_uniform(cfg, i, 7) for i in range(4096)])
-    assert us.min() >= 0.0 and us.max() < 1.0 and abs(us.mean() - 0.5) < 0.02
-    assert np.array_equal(us * 2 ** 24, np.round(us * 2 ** 24))
+    us = np.array([orc.sr_uniform(cfg, i, 7) for i in range(1 << 16)])
+    assert us.min() > 0.0 and us.max() < 1.0 and abs(us.mean() - 0.5) < 0.005
+    cells = us * 256 - 0.5
+    assert np.array_equal(cells, np.round(cells))                       # cell centres only
+    counts = np.bincount(cells.astype(np.int64), minlength=256)
+    assert counts.min() > 176 and counts.max() < 336                    # 256 expected per cell, 5 sigma
+    # element i takes byte (i mod 4) of word ((i mod 16) / 4) of the block's Philox output
+    for i in (0, 5, 15, 16, 1000003):
+        blk = i >> 4
+        words = orc.philox4x32_10((blk & 0xffffffff, blk >> 32, 7, 0), (12345, 0))
+        b = (int(words[(i >> 2) & 3]) >> (8 * (i & 3))) & 0xff
+        assert orc.sr_uniform(cfg, i, 7) == (b + 0.5) / 256
     # the position inside a bucket matters, not the bucket's partitioning
     cfgp = orc.OracleConfig(rounding=1, seed=12345, num_partitions=4, **kw)
     commp = orc.new_comm(cfgp, n)
