@@ -168,6 +168,7 @@ SendKernel pick_send_mode(int mode, int var) {
         if (var == VAR_LEAN_X) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_LEAN_X>, smem};
         if (var == VAR_LEAN_NR_X && (STATE == ST_INT8 || STATE == ST_Q8COMP))
             return {loco_send_kernel<GRAD, (STATE == ST_INT8 || STATE == ST_Q8COMP) ? STATE : ST_INT8, BITS, MODE_FIXED, VAR_LEAN_NR_X>, smem};
+        if (var == VAR_LEAN_SR) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_LEAN_SR>, smem};
         if (var == VAR_STOCHASTIC) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_STOCHASTIC>, smem};
         return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_GENERAL>, smem};
     }
@@ -343,6 +344,7 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
         if (cfg->rounding == LOCO_ROUND_STOCHASTIC) {
             var = VAR_STOCHASTIC;
             if (st->mode == MODE_BLOCK) st->fast = 0;        // block scales with stochastic rounding: careful routine only
+            else if (st->dq.mode == DEC_FMA && st->de.mode == DEC_FMA) var = VAR_LEAN_SR;
         } else if (st->mode == MODE_BLOCK) {
             var = cfg->clip > 0.0f ? VAR_GENERAL : VAR_LEAN;      // the plain lean variants carry no clipping
         } else {

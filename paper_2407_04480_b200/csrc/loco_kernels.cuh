@@ -127,14 +127,15 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, unsigned k0, unsigned k1
     }
     return c;
 }
-// The four uniform numbers in [0, 1) of bucket elements 4 blk .. 4 blk + 3 at iteration (k_hi, k_lo): top 24 bits of the words.
-__device__ __forceinline__ void sr_uniform4(unsigned long long blk, unsigned k_lo, unsigned k_hi, unsigned seed_lo, unsigned seed_hi,
-                                            float (&u)[4]) {
-    const uint4 r = philox4x32_10(make_uint4(static_cast<unsigned>(blk), static_cast<unsigned>(blk >> 32), k_lo, k_hi), seed_lo, seed_hi);
-    u[0] = __uint2float_rn(r.x >> 8) * 5.9604644775390625e-8f;
-    u[1] = __uint2float_rn(r.y >> 8) * 5.9604644775390625e-8f;
-    u[2] = __uint2float_rn(r.z >> 8) * 5.9604644775390625e-8f;
-    u[3] = __uint2float_rn(r.w >> 8) * 5.9604644775390625e-8f;
+// Stochastic rounding adds (b + 1/2) / 256 to h x s, b = one byte of the Philox block of the element's group of 16:
+// element i of the bucket takes byte (i mod 4) of word ((i mod 16) / 4) of
+// philox(counter = (i/16 low, i/16 high, k low, k high), key = seed).
+__device__ __forceinline__ uint4 sr_block(unsigned long long blk, unsigned k_lo, unsigned k_hi, unsigned seed_lo, unsigned seed_hi) {
+    return philox4x32_10(make_uint4(static_cast<unsigned>(blk), static_cast<unsigned>(blk >> 32), k_lo, k_hi), seed_lo, seed_hi);
+}
+__device__ __forceinline__ float sr_dither(unsigned word, int byte) {
+    const float m = __uint_as_float(__byte_perm(word, 0x4B000000u, 0x7540 + byte));      // 2^23 + b
+    return __fmaf_rn(m, 0.00390625f, -32767.998046875f);                                 // b / 256 + 1 / 512, exact
 }
 
 __device__ __forceinline__ float warp_group_max(float v, int lanes) {
@@ -217,12 +218,12 @@ __device__ __forceinline__ void send_core(const SendParams &P, const float (&g)[
         mult = amax > 0.0f ? __fdiv_rn(hi, amax) : 0.0f;
     }
     float u8[8];
-    if (STOCH) {                                            // i0 is a multiple of 8: two counters
-        float ua[4], ub[4];
-        sr_uniform4(i0 >> 2, P.k_lo, P.k_hi, P.seed_lo, P.seed_hi, ua);
-        sr_uniform4((i0 >> 2) + 1, P.k_lo, P.k_hi, P.seed_lo, P.seed_hi, ub);
+    if (STOCH) {                                            // i0 is a multiple of 8: one half of a block of 16
+        const uint4 r = sr_block(i0 >> 4, P.k_lo, P.k_hi, P.seed_lo, P.seed_hi);
+        const bool upper = ((i0 >> 3) & 1ull) != 0ull;
+        const unsigned w0 = upper ? r.z : r.x, w1 = upper ? r.w : r.y;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) { u8[j] = ua[j]; u8[4 + j] = ub[j]; }
+        for (int j = 0; j < 4; ++j) { u8[j] = sr_dither(w0, j); u8[4 + j] = sr_dither(w1, j); }
     }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
@@ -676,14 +677,16 @@ __global__ void loco_division_selfcheck_kernel(unsigned long long *mismatch) {
 // VAR_GENERAL: the forms are chosen per call at run time (scalar code) and statistics may be collected.
 // VAR_STOCHASTIC: VAR_GENERAL with stochastic rounding of the gradient codes (extension; global scale only).
 // VAR_LEAN_X / VAR_LEAN_NR_X: the lean forms plus what a call may ask for on top (statistics, clipping of g).
-enum : int { VAR_LEAN = 0, VAR_LEAN_NR = 1, VAR_GENERAL = 2, VAR_STOCHASTIC = 3, VAR_LEAN_X = 4, VAR_LEAN_NR_X = 5 };
-__host__ __device__ constexpr bool var_is_lean(int var) { return var == VAR_LEAN || var == VAR_LEAN_NR || var == VAR_LEAN_X || var == VAR_LEAN_NR_X; }
+// VAR_LEAN_SR: VAR_LEAN_X with stochastic rounding.
+enum : int { VAR_LEAN = 0, VAR_LEAN_NR = 1, VAR_GENERAL = 2, VAR_STOCHASTIC = 3, VAR_LEAN_X = 4, VAR_LEAN_NR_X = 5, VAR_LEAN_SR = 6 };
+__host__ __device__ constexpr bool var_is_lean(int var) { return var == VAR_LEAN || var == VAR_LEAN_NR || var == VAR_LEAN_X || var == VAR_LEAN_NR_X || var == VAR_LEAN_SR; }
 __host__ __device__ constexpr bool var_has_extras(int var) { return var != VAR_LEAN && var != VAR_LEAN_NR; }
+__host__ __device__ constexpr bool var_is_sr(int var) { return var == VAR_STOCHASTIC || var == VAR_LEAN_SR; }
 
 // dec(e; s_e) of a pair from the magic floats m2 = kMagic + 128 + e
 template <int VAR>
 __device__ __forceinline__ f32x2 dec_state2(const SendConsts &K, f32x2 m2, float emagic, int de_mode) {
-    if (VAR == VAR_LEAN || VAR == VAR_LEAN_X) return ffma2(m2, dup2(K.de_a), dup2(K.de_b));
+    if (VAR == VAR_LEAN || VAR == VAR_LEAN_X || VAR == VAR_LEAN_SR) return ffma2(m2, dup2(K.de_a), dup2(K.de_b));
     if (VAR == VAR_LEAN_NR || VAR == VAR_LEAN_NR_X) {
         const f32x2 e2 = fadd2(m2, dup2(-emagic));                   // the codes, exact
         const f32x2 inv2 = dup2(K.inv_se);
@@ -813,17 +816,19 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     unsigned mb[16];
     f32x2 en2[8];
     const f32x2 mult2 = dup2(mult), qmagic2 = dup2(qmagic), omb2 = dup2(K.omb), beta2 = dup2(K.beta);
+    uint4 rnd = make_uint4(0u, 0u, 0u, 0u);                // the lane's 16 elements are one block of the Philox stream
+    if (var_is_sr(VAR))
+        rnd = sr_block((L.elem0 + static_cast<unsigned long long>(wrow) * kWide) >> 4, K.k_lo, K.k_hi, K.seed_lo, K.seed_hi);
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
         float y0, y1;
         unpk2(fmul2(h2[k], mult2), y0, y1);
         float t0 = y0, t1 = y1;
         bool sat0 = false, sat1 = false;
-        if (VAR == VAR_STOCHASTIC) {                       // floor(y + u): up with probability frac(y)
-            float u[4];
-            sr_uniform4((L.elem0 + static_cast<unsigned long long>(wrow) * kWide + 2 * (k & ~1)) >> 2, K.k_lo, K.k_hi, K.seed_lo, K.seed_hi, u);
-            t0 = floorf(__fadd_rn(y0, u[2 * (k & 1)]));
-            t1 = floorf(__fadd_rn(y1, u[2 * (k & 1) + 1]));
+        if (var_is_sr(VAR)) {                       // floor(y + u): up with probability frac(y)
+            const unsigned word = (k >> 1) == 0 ? rnd.x : ((k >> 1) == 1 ? rnd.y : ((k >> 1) == 2 ? rnd.z : rnd.w));
+            t0 = floorf(__fadd_rn(y0, sr_dither(word, 2 * (k & 1))));
+            t1 = floorf(__fadd_rn(y1, sr_dither(word, 2 * (k & 1) + 1)));
             sat0 = t0 < lo || t0 > hi;
             sat1 = t1 < lo || t1 > hi;
         }
@@ -840,7 +845,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
                      dec_fast(__uint_as_float(mb[2 * k + 1]), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s));
         }
         if (MODE != MODE_BLOCK && EXTRAS && stats) {
-            if (VAR == VAR_STOCHASTIC) {
+            if (var_is_sr(VAR)) {
                 saturated += (sat0 ? 1u : 0u) + (sat1 ? 1u : 0u);
             } else {
                 if (y0 >= hi + 0.5f || y0 < lo - 0.5f) saturated += 1u;
@@ -991,8 +996,8 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_con
             if (stage_wrow < full_wide) stage(stage_off, stage_wrow);
             cp_async_commit();                 // one group per iteration, empty near the end
             if (!send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, wrow, lane, stats, saturated)) {
-                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, VAR == VAR_STOCHASTIC>(P, part, static_cast<unsigned long long>(wrow) * kWide, lane);
-                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, VAR == VAR_STOCHASTIC>(P, part, static_cast<unsigned long long>(wrow) * kWide + kRow, lane);
+                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, var_is_sr(VAR)>(P, part, static_cast<unsigned long long>(wrow) * kWide, lane);
+                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, var_is_sr(VAR)>(P, part, static_cast<unsigned long long>(wrow) * kWide + kRow, lane);
             }
             slot_off = slot_off + R::kSlotStride == R::kBytes ? 0u : slot_off + R::kSlotStride;
             stage_off = stage_off + R::kSlotStride == R::kBytes ? 0u : stage_off + R::kSlotStride;
@@ -1001,7 +1006,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_con
         }
     }
     for (unsigned r = first_careful + warp; r < rows; r += nwarps)
-        careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, VAR == VAR_STOCHASTIC>(P, part, static_cast<unsigned long long>(r) * kRow, lane);
+        careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, var_is_sr(VAR)>(P, part, static_cast<unsigned long long>(r) * kRow, lane);
     // each careful call adds at most 8 saturated codes and 2^31 per row with a non-finite value; the 64-bit
     // sum keeps the flag apart from the count
     const unsigned nonfinite = (careful_acc >> 31) != 0ull ? 1u : 0u;

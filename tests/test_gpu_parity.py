@@ -391,6 +391,17 @@ def test_stochastic_rounding(mode, fmt, bits):
         assert_reduced_equal(got, want, False)
 
 
+@pytest.mark.parametrize("s,s_e", [(2.0 ** 9, 6 * 2.0 ** 9), (3000.0, 12000.0)])
+def test_stochastic_rounding_other_decompressor_forms(s, s_e):
+    """Scales for which the state decompressor is the Newton-Raphson form or the division itself: stochastic rounding then
+    runs in the kernel variant that chooses the forms per call."""
+    n = 90_007
+    for fmt in (loco.STATE_INT8, loco.STATE_FP32_Q8COMP):
+        gcfg, ocfg = both_configs(bits=4, s=s, s_e=s_e, beta=0.5, reset_period=0, state_fmt=fmt, grad_dtype=loco.BF16,
+                                  out_dtype=loco.F32, num_partitions=2, rounding=1, seed=99)
+        run_steps(gcfg, ocfg, n, 3, 2e-3, seed=19, k0=2)
+
+
 def test_stochastic_rounding_differs_from_nearest_and_between_seeds():
     n = 1 << 16
     g = inputs.gaussian(n, 2e-3, seed=18, dtype=torch.bfloat16, device="cuda")
