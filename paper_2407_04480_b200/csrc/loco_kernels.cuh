@@ -706,6 +706,10 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     constexpr float lo = QRange<BITS>::lo, hi = QRange<BITS>::hi, qmagic = kMagic + QRange<BITS>::off;
     constexpr float emagic = kMagic + 128.0f;
     constexpr bool kStateF32 = (STATE == ST_FP32 || STATE == ST_Q8COMP);
+    // With the 8-bit state (or none) everything stored is a code or a scale, which the sign of a zero cannot change: the
+    // products of Eq. 5 may then be taken as fma(a, b, +0) (the rounded product up to the sign of zero) and summed with
+    // a packed add; with an fp32 state the sign of a zero is stored, so there the sum stays scalar (see fadd2_after_mul).
+    constexpr bool kSignFree = !kStateF32;
     constexpr int GW = WideIn<GRAD, STATE>::GW, EW = WideIn<GRAD, STATE>::EW;
     constexpr bool LEAN = var_is_lean(VAR), EXTRAS = var_has_extras(VAR);
     const int dq_mode = LEAN ? DEC_FMA : K.dq_mode, de_mode = K.de_mode;
@@ -771,7 +775,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             const float m0 = __uint_as_float(__byte_perm(x, kMagicBits, 0x7650 + 2 * (k & 1)));     // kMagic + 128 + e
             const float m1 = __uint_as_float(__byte_perm(x, kMagicBits, 0x7651 + 2 * (k & 1)));
             if (MODE == MODE_BLOCK) {
-                c2 = fmul2(fadd2(pk2(m0, m1), dup2(-emagic)), dup2(in.sscale));
+                c2 = fmul2_pz(fadd2(pk2(m0, m1), dup2(-emagic)), dup2(in.sscale));   // kSignFree holds here
             } else {
                 c2 = dec_state2<VAR>(K, pk2(m0, m1), emagic, de_mode);
             }
@@ -791,7 +795,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             prev2[k] = zero2;
         }
         // g + 0 changes at most the sign of a zero, never a code; in block mode c is a product
-        h2[k] = (STATE == ST_NONE) ? g2[k] : ((MODE == MODE_BLOCK && STATE == ST_INT8) ? fadd2_after_mul(g2[k], c2) : fadd2(g2[k], c2));
+        h2[k] = (STATE == ST_NONE) ? g2[k] : fadd2(g2[k], c2);
     }
 
     // ---- block scale (extension): absmax of the block's h over the lanes that share it ---------------------------
@@ -837,7 +841,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         mb[2 * k + 1] = static_cast<unsigned>(m2 >> 32);
         f32x2 d2;
         if (MODE == MODE_BLOCK) {
-            d2 = fmul2(fadd2(m2, dup2(-qmagic)), dup2(scale));
+            d2 = fmul2_pz(fadd2(m2, dup2(-qmagic)), dup2(scale));          // q is never -0 and a non-zero q times a block scale never underflows
         } else if (LEAN) {
             d2 = ffma2(m2, dup2(K.dq_a), dup2(K.dq_b));
         } else {
@@ -852,8 +856,10 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
                 if (y1 >= hi + 0.5f || y1 < lo - 0.5f) saturated += 1u;
             }
         }
-        const f32x2 delta2 = (MODE == MODE_BLOCK) ? fsub2_after_mul(h2[k], d2) : fsub2(h2[k], d2);
-        en2[k] = (STATE == ST_NONE) ? zero2 : fadd2_after_mul(fmul2(omb2, prev2[k]), fmul2(beta2, delta2));
+        const f32x2 delta2 = fsub2(h2[k], d2);
+        en2[k] = (STATE == ST_NONE) ? zero2
+                 : (kSignFree ? fadd2(fmul2_pz(omb2, prev2[k]), fmul2_pz(beta2, delta2))
+                              : fadd2_after_mul(fmul2(omb2, prev2[k]), fmul2(beta2, delta2)));
     }
     uint8_t *cdst = L.codes + static_cast<size_t>(wrow) * (kWide * BITS / 8);
     if (BITS == 4) {
