@@ -828,13 +828,10 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         float y0, y1;
         unpk2(fmul2(h2[k], mult2), y0, y1);
         float t0 = y0, t1 = y1;
-        bool sat0 = false, sat1 = false;
         if (var_is_sr(VAR)) {                       // floor(y + u): up with probability frac(y)
             const unsigned word = (k >> 1) == 0 ? rnd.x : ((k >> 1) == 1 ? rnd.y : ((k >> 1) == 2 ? rnd.z : rnd.w));
             t0 = floorf(__fadd_rn(y0, sr_dither(word, 2 * (k & 1))));
             t1 = floorf(__fadd_rn(y1, sr_dither(word, 2 * (k & 1) + 1)));
-            sat0 = t0 < lo || t0 > hi;
-            sat1 = t1 < lo || t1 > hi;
         }
         const f32x2 m2 = fadd2(pk2(fminf(fmaxf(t0, lo), hi), fminf(fmaxf(t1, lo), hi)), qmagic2);   // kMagic + 2^(p-1) + q
         mb[2 * k] = static_cast<unsigned>(m2);
@@ -850,7 +847,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         }
         if (MODE != MODE_BLOCK && EXTRAS && stats) {
             if (var_is_sr(VAR)) {
-                saturated += (sat0 ? 1u : 0u) + (sat1 ? 1u : 0u);
+                saturated += ((t0 < lo || t0 > hi) ? 1u : 0u) + ((t1 < lo || t1 > hi) ? 1u : 0u);
             } else {
                 if (y0 >= hi + 0.5f || y0 < lo - 0.5f) saturated += 1u;
                 if (y1 >= hi + 0.5f || y1 < lo - 0.5f) saturated += 1u;
