@@ -428,6 +428,7 @@ def sweep(args, device):
             return
         base = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=512, state_fmt=2,
                     grad_dtype=1, out_dtype=1, num_partitions=8)
+        one_part = kw.pop("one_part", False)            # only part 3 of 8: what one rank averages after the exchange
         base.update(kw)
         cfg = loco.Config(**base)
         osz = 2 if cfg.out_dtype == loco.BF16 else 4
@@ -449,8 +450,16 @@ def sweep(args, device):
                 packed.append([torch.randint(0, 256, (max(pb, 16),), dtype=torch.uint8, device=device, generator=gen) for _ in range(workers)])
         outs = [torch.empty(n, dtype=torch.bfloat16 if osz == 2 else torch.float32, device=device) for _ in range(nsets)]
         torch.cuda.synchronize()
-        us = _time_launches(lambda i, st: loco.loco_unpack_dequant_reduce(cfg, packed[i], n, outs[i], stream=st),
-                            nsets, max(12, min(200, 4 * nsets)), streams)
+        if one_part:
+            stride = loco.loco_partition_bytes(cfg, n)
+            slots = [[b[3 * stride:4 * stride] for b in bufs] for bufs in packed]
+            us = _time_launches(lambda i, st: loco.loco_unpack_dequant_reduce(cfg, slots[i], n, outs[i], first_partition=3,
+                                                                                partition_count=1, stream=st),
+                                nsets, max(12, min(200, 4 * nsets)), streams)
+            n = loco.loco_partition_elems(cfg, n, 3)        # elements this launch produces
+        else:
+            us = _time_launches(lambda i, st: loco.loco_unpack_dequant_reduce(cfg, packed[i], n, outs[i], stream=st),
+                                nsets, max(12, min(200, 4 * nsets)), streams)
         bpe = workers * cfg.bits / 8 + osz + (workers * 4.0 / cfg.block_size if cfg.scale_mode == 1 else 0.0)
         gbs = bpe * n / us / 1e3
         rows.append(dict(kernel="reduce", case=label, n=n, workers=workers, bytes_per_elem=round(bpe, 3), us=round(us, 2),
@@ -513,6 +522,8 @@ def sweep(args, device):
                 reduce_case("%d bit, %s out, fixed" % (bits, "bf16" if od else "fp32"), M, N, bits=bits, out_dtype=od)
     reduce_case("4 bit, bf16 out, fixed, s = 3000 (generic path)", M, 8, s=3000.0)
     reduce_case("4 bit, bf16 out, fixed, 3 workers (division by 3)", M, 3)
+    reduce_case("4 bit, bf16 out, fixed, one part of 8 of a 25M-element bucket (a rank's share after the exchange)", M, 8, one_part=True)
+    reduce_case("4 bit, bf16 out, fixed, one part of 8 of a 200M-element bucket", 8 * M, 8, one_part=True)
     reduce_case("4 bit, bf16 out, block-256 absmax", M, 8, scale_mode=1)
     reduce_case("4 bit, bf16 out, block-32 absmax", M, 8, scale_mode=1, block_size=32)
     reduce_case("8 bit, bf16 out, block-256 absmax, 1 worker (Zero++-style weight payload)", M, 1, bits=8, scale_mode=1)
