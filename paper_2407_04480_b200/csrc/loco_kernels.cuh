@@ -419,23 +419,19 @@ __device__ __forceinline__ f32x2 fsub2(f32x2 a, f32x2 b) { f32x2 d; asm("sub.rn.
 __device__ __forceinline__ f32x2 fmul2(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 __device__ __forceinline__ f32x2 ffma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
 // The assembler contracts a packed multiply that feeds a packed add or subtract into one packed FMA even
-// though both carry an explicit rounding mode (seen as single-rounded results on sm_100a, CUDA 12.9).  Where
-// Algorithm 1 rounds the product and the sum separately, the sum is therefore taken with scalar
-// instructions, which are never contracted.
+// though both carry an explicit rounding mode (seen as single-rounded results on sm_100a, CUDA 12.9; the same
+// happens when the product is written fma(a, b, -0)).  Where Algorithm 1 rounds the product and the sum
+// separately there are two ways out: the sum with scalar instructions, which are never contracted
+// (fadd2_after_mul), or the product as fma(a, b, +0) (fmul2_pz), where the sign of a zero does not matter.
 __device__ __forceinline__ f32x2 fadd2_after_mul(f32x2 a, f32x2 b) {
     float a0, a1, b0, b1;
     unpk2(a, a0, a1);
     unpk2(b, b0, b1);
     return pk2(__fadd_rn(a0, b0), __fadd_rn(a1, b1));
 }
-__device__ __forceinline__ f32x2 fsub2_after_mul(f32x2 a, f32x2 b) {
-    float a0, a1, b0, b1;
-    unpk2(a, a0, a1);
-    unpk2(b, b0, b1);
-    return pk2(__fsub_rn(a0, b0), __fsub_rn(a1, b1));
-}
-// For a running sum that starts at +0 the sign of a zero product never shows (acc is never -0), so there the product
-// may be taken as fma(a, b, +0): the rounded product up to the sign of zero, which no later add can be contracted with.
+// fma(a, b, +0) is the rounded product except that a product of -0 comes out as +0, and no later add can be contracted
+// with it.  Usable where that sign cannot show: in a running sum that starts at +0 (such a sum is never -0), and where
+// everything computed from the result is stored as integer codes or as scales taken from magnitudes.
 __device__ __forceinline__ f32x2 fmul2_pz(f32x2 a, f32x2 b) {
     f32x2 d;
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(0ull));
