@@ -373,6 +373,29 @@ def test_zero_plus_plus_style_weight_payload():
     assert bool(((back - x).abs() <= 0.5 * step * 1.001 + x.abs() * 2.0 ** -8).all())
 
 
+# ---------------------------------------------------------------- a long horizon: 100 iterations, several resets
+
+@pytest.mark.parametrize("mode,fmt,rounding", [(loco.SCALE_FIXED, loco.STATE_INT8, 0), (loco.SCALE_FIXED, loco.STATE_FP32, 0),
+                                               (loco.SCALE_BLOCK_ABSMAX, loco.STATE_INT8, 0), (loco.SCALE_FIXED, loco.STATE_INT8, 1)])
+def test_hundred_iterations(mode, fmt, rounding):
+    """100 consecutive iterations on one bucket (the iteration count the Llama-2-7B configuration names), error state carried
+    from step to step on both sides, reset every 32 iterations: codes, scales and state compared around the resets and at the
+    end -- a single differing state code anywhere on the way would show in what follows."""
+    n = 400_003
+    gcfg, ocfg = both_configs(bits=4, scale_mode=mode, block_size=128, s=2.0 ** 13, s_e=2.0 ** 15, beta=0.5, reset_period=32,
+                              state_fmt=fmt, grad_dtype=loco.BF16, out_dtype=loco.BF16, num_partitions=8, rounding=rounding,
+                              seed=7)
+    w = Worker(gcfg, ocfg, n)
+    check_at = {0, 1, 2, 31, 32, 33, 63, 64, 65, 98, 99}
+    for k in range(100):
+        g = inputs.gaussian(n, 1e-4, seed=41, worker=0, step=k, dtype=torch.bfloat16, device="cuda")
+        w.step(grad_bits(g), k)
+        if k in check_at:
+            w.compare("iteration %d" % k)
+    got, want = reduce_both(gcfg, ocfg, n, [w, w, w])
+    assert_reduced_equal(got, want, True)
+
+
 # ---------------------------------------------------------------- stochastic rounding on the shared Philox stream
 
 @pytest.mark.parametrize("mode", [loco.SCALE_FIXED, loco.SCALE_BLOCK_ABSMAX])
