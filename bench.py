@@ -303,13 +303,24 @@ def run_exchange(args, rank: int, world: int, device, config):
     grad = torch.empty(total, dtype=torch.bfloat16, device=device)
     for lo, hi in buckets:
         grad[lo:hi] = inputs.layout_slice(layout, lo, hi, scales, 1e-4, seed=1, worker=rank, step=0, device=device)
-    transport = exchange.Transport(cfg, BUCKET, kind=args.exchange, device=device)
-    exs = [exchange.BucketExchange(cfg, hi - lo, shared=transport) for lo, hi in buckets]
-    shard = torch.empty(max(e.shard_elems() for e in exs), dtype=torch.bfloat16, device=device)
+    if args.exchange == "reduce_scatter_bf16":
+        # the uncompressed baseline: every bucket padded to a multiple of the group size and reduce-scattered as it is
+        padded = [-(-(hi - lo) // world) * world for lo, hi in buckets]
+        stage = torch.zeros(max(padded), dtype=torch.bfloat16, device=device)
+        shard = torch.empty(max(padded) // world, dtype=torch.bfloat16, device=device)
 
-    def step(k):
-        for e, (lo, hi) in zip(exs, buckets):
-            e.step(grad[lo:hi], k, shard)
+        def step(k):
+            for (lo, hi), m in zip(buckets, padded):
+                stage[:hi - lo].copy_(grad[lo:hi])
+                dist.reduce_scatter_tensor(shard[:m // world], stage[:m], op=dist.ReduceOp.AVG)
+    else:
+        transport = exchange.Transport(cfg, BUCKET, kind=args.exchange, device=device)
+        exs = [exchange.BucketExchange(cfg, hi - lo, shared=transport) for lo, hi in buckets]
+        shard = torch.empty(max(e.shard_elems() for e in exs), dtype=torch.bfloat16, device=device)
+
+        def step(k):
+            for e, (lo, hi) in zip(exs, buckets):
+                e.step(grad[lo:hi], k, shard)
 
     for k in range(max(3, args.warmup)):
         step(k)
@@ -335,7 +346,9 @@ def run_exchange(args, rank: int, world: int, device, config):
         config = dict(config, exchange=args.exchange, streams=1, workers_on_reduce_side=world,
                       workload=config["workload"].split(":")[0] + ": %d bf16 buckets per rank; per bucket: send pass, exchange "
                       "of %d parts between the ranks, average of this rank's part" % (len(buckets), world))
-        print(json.dumps({"metric": METRIC + " -- with the real exchange", "value": world * 2 * total / (step_ms * 1e-3) / 1e9,
+        suffix = (" -- uncompressed bf16 NCCL reduce-scatter of the same buckets (what the method replaces; none of this "
+                  "library's kernels)") if args.exchange == "reduce_scatter_bf16" else " -- with the real exchange"
+        print(json.dumps({"metric": METRIC + suffix, "value": world * 2 * total / (step_ms * 1e-3) / 1e9,
                           "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
                           "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                           "dtype": "f32", "data": "synthetic", "config": config, "clocks": clocks, "e2e": None,
@@ -553,10 +566,12 @@ def main():
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the bench line: the size / type / width / worker-count table (one JSON line per case, then markdown)")
     ap.add_argument("--sweep-filter", default="", help="with --sweep: only the cases whose 'kernel: label' contains this text")
-    ap.add_argument("--exchange", choices=("none", "collective", "peer_store"), default="none",
+    ap.add_argument("--exchange", choices=("none", "collective", "peer_store", "reduce_scatter_bf16"), default="none",
                     help="none (default): every rank runs the two passes on its own buckets, no data-path collective; "
                          "collective / peer_store: the real exchange of Sec. 3.3 between the ranks (NCCL all-to-all, or the "
-                         "send kernel storing into the peers' receive slots), each rank reducing its own shard")
+                         "send kernel storing into the peers' receive slots), each rank reducing its own shard; "
+                         "reduce_scatter_bf16: what the method replaces -- NCCL reduce-scatter (average) of the uncompressed bf16 "
+                         "buckets, none of this library's kernels, for comparison on the same buckets")
     ap.add_argument("--streams", type=int, default=2,
                     help="streams the per-bucket launches of a phase are spread over (1 = strictly one after the other)")
     args = ap.parse_args()
