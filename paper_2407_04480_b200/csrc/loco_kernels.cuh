@@ -821,15 +821,24 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         rnd = sr_block((L.elem0 + static_cast<unsigned long long>(wrow) * kWide) >> 4, K.k_lo, K.k_hi, K.seed_lo, K.seed_hi);
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
-        float y0, y1;
-        unpk2(fmul2(h2[k], mult2), y0, y1);
-        float t0 = y0, t1 = y1;
-        if (var_is_sr(VAR)) {                       // floor(y + u): up with probability frac(y)
-            const unsigned word = (k >> 1) == 0 ? rnd.x : ((k >> 1) == 1 ? rnd.y : ((k >> 1) == 2 ? rnd.z : rnd.w));
-            t0 = floorf(__fadd_rn(y0, sr_dither(word, 2 * (k & 1))));
-            t1 = floorf(__fadd_rn(y1, sr_dither(word, 2 * (k & 1) + 1)));
+        float y0 = 0.0f, y1 = 0.0f, t0 = 0.0f, t1 = 0.0f;
+        f32x2 m2;                                                                                    // kMagic + 2^(p-1) + q
+        if (MODE == MODE_BLOCK && !var_is_sr(VAR)) {
+            // |h| <= amax and mult = fl(qmax / amax), so |h x mult| <= qmax (1 + 2^-22): the nearest integer is inside the
+            // range and the clamp of Eq. 1 has nothing to do.  The product as fma(h, mult, +0), so that the add of the
+            // magic constant cannot be contracted with it (the sign of a zero product does not reach the sum).
+            m2 = fadd2(fmul2_pz(h2[k], mult2), qmagic2);
+        } else {
+            unpk2(fmul2(h2[k], mult2), y0, y1);
+            t0 = y0;
+            t1 = y1;
+            if (var_is_sr(VAR)) {                   // floor(y + u): up with probability frac(y)
+                const unsigned word = (k >> 1) == 0 ? rnd.x : ((k >> 1) == 1 ? rnd.y : ((k >> 1) == 2 ? rnd.z : rnd.w));
+                t0 = floorf(__fadd_rn(y0, sr_dither(word, 2 * (k & 1))));
+                t1 = floorf(__fadd_rn(y1, sr_dither(word, 2 * (k & 1) + 1)));
+            }
+            m2 = fadd2(pk2(fminf(fmaxf(t0, lo), hi), fminf(fmaxf(t1, lo), hi)), qmagic2);
         }
-        const f32x2 m2 = fadd2(pk2(fminf(fmaxf(t0, lo), hi), fminf(fmaxf(t1, lo), hi)), qmagic2);   // kMagic + 2^(p-1) + q
         mb[2 * k] = static_cast<unsigned>(m2);
         mb[2 * k + 1] = static_cast<unsigned>(m2 >> 32);
         f32x2 d2;
