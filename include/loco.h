@@ -210,6 +210,35 @@ int loco_unpack_dequant_reduce_adam(const loco_config_t *cfg, const void *const 
                                     const loco_adam_t *adam, float *d_m, float *d_v, float *d_theta,
                                     void *d_grad_out, void *stream);
 
+/* ---- several buckets per call -----------------------------------------------------------------
+ * (No counterpart in the paper: a convenience of the library.)  Algorithm 1 is applied bucket by bucket, and a
+ * bucket of the usual size is a kernel of 15-30 microseconds, a third of which is start-up and tail when the
+ * kernels of a stream run strictly one after the other.  These two calls do what `count` single-bucket calls on
+ * `stream` would do -- same kernels, same results, everything ordered after the work `stream` already holds and
+ * before whatever is enqueued on it next -- but issue the launches alternately on two streams that the library
+ * owns, so that one bucket's tail overlaps the next bucket's start-up.
+ *   - The buckets of one call must be independent of each other (distinct states and buffers), as they run
+ *     concurrently.  All of them belong to the current device.
+ *   - The first such call on a device creates two non-blocking streams and three events there (driver objects;
+ *     no device memory), kept until the process exits; make it outside any stream capture.  Later calls only
+ *     record and wait on those events and launch; they may be captured into a CUDA graph like the single calls.
+ *   - Calls on one device are serialised on the host while they enqueue their work (they share the events).
+ * If one bucket's launch is refused the others are still issued, the streams are joined, and the first error is
+ * returned.  count = 0 does nothing.  Errors: as for the single-bucket calls, ARG for null arrays or entries.
+ */
+
+/* loco_compensate_quantize_pack for buckets i < count: states[i], d_grads[i], d_comms[i] (HOST arrays of count
+ * entries each), all at iteration step_k. */
+int loco_compensate_quantize_pack_multi(loco_state_t *const *states, const void *const *d_grads,
+                                        void *const *d_comms, int32_t count, int64_t step_k, void *stream);
+
+/* loco_unpack_dequant_reduce over all parts (first_partition 0, partition_count num_partitions) for buckets
+ * i < count: d_packed[i] is bucket i's HOST array of num_workers DEVICE pointers, n[i] its length, d_outs[i] its
+ * output (HOST arrays of count entries). */
+int loco_unpack_dequant_reduce_multi(const loco_config_t *cfg, const void *const *const *d_packed,
+                                     int32_t num_workers, const uint64_t *n, void *const *d_outs, int32_t count,
+                                     void *stream);
+
 /* ---- host-buffer variants ------------------------------------------------------------------
  * The same two passes for callers whose gradient and communication buffers live in HOST memory
  * (pinned memory makes the copies asynchronous).  Each call enqueues, on `stream`: the

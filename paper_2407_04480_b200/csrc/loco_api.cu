@@ -642,6 +642,90 @@ int loco_unpack_dequant_reduce_adam(const loco_config_t *cfg, const void *const 
                          d_theta, stream);
 }
 
+}  // extern "C"
+
+namespace {
+
+// Two streams and three events per device, owned by the library, over which the multi-bucket calls spread their launches:
+// fork from the caller's stream, alternate, join back.  Created on a device's first multi-bucket call, kept until exit.
+struct SideStreams {
+    cudaStream_t s[2] = {nullptr, nullptr};
+    cudaEvent_t fork = nullptr, join[2] = {nullptr, nullptr};
+    bool ready = false;
+    std::mutex in_use;          // one fork / launch / join sequence at a time: the events are shared
+};
+
+int side_streams(SideStreams **out) {
+    static SideStreams per_device[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return LOCO_ERR_CUDA; }
+    std::lock_guard<std::mutex> lock(mu);
+    SideStreams &S = per_device[dev];
+    if (!S.ready) {
+        bool ok = cudaEventCreateWithFlags(&S.fork, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < 2 && ok; ++i)
+            ok = cudaStreamCreateWithFlags(&S.s[i], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&S.join[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) { cudaGetLastError(); return LOCO_ERR_CUDA; }
+        S.ready = true;
+    }
+    *out = &S;
+    return LOCO_OK;
+}
+
+// Run launch(i, stream_i) for i < count with the launches alternating between the two side streams, all of them after
+// what `stream` holds now and all of them before what is enqueued on `stream` next.
+template <typename Launch>
+int fan_out(int32_t count, void *stream, Launch launch) {
+    SideStreams *S = nullptr;
+    int rc = side_streams(&S);
+    if (rc != LOCO_OK) return rc;
+    cudaStream_t user = static_cast<cudaStream_t>(stream);
+    std::lock_guard<std::mutex> lock(S->in_use);
+    if (cudaEventRecord(S->fork, user) != cudaSuccess) { cudaGetLastError(); return LOCO_ERR_CUDA; }
+    const int used = count > 1 ? 2 : 1;
+    for (int i = 0; i < used; ++i)
+        if (cudaStreamWaitEvent(S->s[i], S->fork, 0) != cudaSuccess) { cudaGetLastError(); return LOCO_ERR_CUDA; }
+    for (int32_t i = 0; i < count; ++i) {
+        const int r = launch(i, static_cast<void *>(S->s[i & 1]));
+        if (r != LOCO_OK && rc == LOCO_OK) rc = r;            // the join below still happens
+    }
+    for (int i = 0; i < used; ++i) {
+        if (cudaEventRecord(S->join[i], S->s[i]) != cudaSuccess || cudaStreamWaitEvent(user, S->join[i], 0) != cudaSuccess) {
+            cudaGetLastError();
+            if (rc == LOCO_OK) rc = LOCO_ERR_CUDA;
+        }
+    }
+    return rc;
+}
+
+}  // namespace
+
+extern "C" {
+
+int loco_compensate_quantize_pack_multi(loco_state_t *const *states, const void *const *d_grads, void *const *d_comms,
+                                        int32_t count, int64_t step_k, void *stream) {
+    if (count < 0 || (count > 0 && (!states || !d_grads || !d_comms))) return LOCO_ERR_ARG;
+    if (count == 0) return LOCO_OK;
+    for (int32_t i = 0; i < count; ++i)
+        if (!states[i]) return LOCO_ERR_ARG;
+    return fan_out(count, stream, [&](int32_t i, void *s) {
+        return loco_compensate_quantize_pack(states[i], d_grads[i], d_comms[i], step_k, s);
+    });
+}
+
+int loco_unpack_dequant_reduce_multi(const loco_config_t *cfg, const void *const *const *d_packed, int32_t num_workers,
+                                     const uint64_t *n, void *const *d_outs, int32_t count, void *stream) {
+    if (count < 0 || (count > 0 && (!cfg || !d_packed || !n || !d_outs))) return LOCO_ERR_ARG;
+    if (count == 0) return LOCO_OK;
+    const int rc = check_config(cfg);
+    if (rc != LOCO_OK) return rc;
+    return fan_out(count, stream, [&](int32_t i, void *s) {
+        return loco_unpack_dequant_reduce(cfg, d_packed[i], num_workers, n[i], 0, cfg->num_partitions, d_outs[i], s);
+    });
+}
+
 uint64_t loco_send_host_workspace_bytes(const loco_config_t *cfg, uint64_t n) {
     if (!layout_ok(cfg) || n == 0) return 0;
     const uint64_t gbytes = round_up(n * (cfg->grad_dtype == LOCO_BF16 ? 2u : 4u), 256);

@@ -31,7 +31,8 @@ EXPORTS = ("loco_state_bytes", "loco_packed_bytes", "loco_partition_bytes", "loc
            "loco_send_host_workspace_bytes", "loco_reduce_host_workspace_bytes",
            "loco_compensate_quantize_pack_host", "loco_unpack_dequant_reduce_host",
            "loco_unpack_dequant_reduce_host_noalloc", "loco_selfcheck_block_division",
-           "loco_unpack_dequant_reduce_adam", "loco_compensate_quantize_pack_scatter")
+           "loco_unpack_dequant_reduce_adam", "loco_compensate_quantize_pack_scatter",
+           "loco_compensate_quantize_pack_multi", "loco_unpack_dequant_reduce_multi")
 NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
@@ -115,6 +116,10 @@ def lib() -> C.CDLL:
         L.loco_reduce_host_workspace_bytes.argtypes = [cp, u64, i32, i32]
         L.loco_compensate_quantize_pack_scatter.restype = C.c_int
         L.loco_compensate_quantize_pack_scatter.argtypes = [vp, vp, vp, i64, vp]
+        L.loco_compensate_quantize_pack_multi.restype = C.c_int
+        L.loco_compensate_quantize_pack_multi.argtypes = [vp, vp, vp, C.c_int32, i64, vp]
+        L.loco_unpack_dequant_reduce_multi.restype = C.c_int
+        L.loco_unpack_dequant_reduce_multi.argtypes = [vp, vp, C.c_int32, vp, vp, C.c_int32, vp]
         L.loco_compensate_quantize_pack_host.restype = C.c_int
         L.loco_compensate_quantize_pack_host.argtypes = [vp, vp, vp, vp, u64, i64, vp]
         L.loco_unpack_dequant_reduce_host.restype = C.c_int
@@ -271,6 +276,55 @@ def loco_unpack_dequant_reduce(cfg: Config, packed: Sequence, n: int, out: torch
     _check(lib().loco_unpack_dequant_reduce(C.byref(cfg.c()), ptrs, len(packed), n, first_partition,
                                             partition_count, _dev_ptr(out), _stream_ptr(stream)),
            "loco_unpack_dequant_reduce")
+
+
+class MultiSend:
+    """Argument tables of loco_compensate_quantize_pack_multi, marshalled once for a fixed set of buckets."""
+
+    def __init__(self, states: Sequence[State], grads: Sequence[torch.Tensor], comms: Sequence[torch.Tensor]):
+        if not (len(states) == len(grads) == len(comms)):
+            raise ValueError("one gradient and one communication buffer per state are needed")
+        for st, g, c in zip(states, grads, comms):
+            want = torch.bfloat16 if st.cfg.grad_dtype == BF16 else torch.float32
+            if g.dtype != want or g.numel() != st.n:
+                raise ValueError("gradient must be %s with %d elements" % (want, st.n))
+            if c.dtype != torch.uint8 or c.numel() < loco_packed_bytes(st.cfg, st.n):
+                raise ValueError("communication buffer too small or not uint8")
+        self.keep = (list(states), list(grads), list(comms))
+        self.count = len(states)
+        self.h = (C.c_void_p * self.count)(*[st.handle.value for st in states])
+        self.g = (C.c_void_p * self.count)(*[_dev_ptr(g) for g in grads])
+        self.c = (C.c_void_p * self.count)(*[_dev_ptr(c) for c in comms])
+
+
+def loco_compensate_quantize_pack_multi(ms: MultiSend, step_k: int, stream=None) -> None:
+    """The send pass for all buckets of ms, their launches overlapped on the library's two streams."""
+    _check(lib().loco_compensate_quantize_pack_multi(ms.h, ms.g, ms.c, ms.count, step_k, _stream_ptr(stream)),
+           "loco_compensate_quantize_pack_multi")
+
+
+class MultiReduce:
+    """Argument tables of loco_unpack_dequant_reduce_multi for a fixed set of buckets (whole buckets, all parts)."""
+
+    def __init__(self, cfg: Config, packed: Sequence[Sequence], ns: Sequence[int], outs: Sequence[torch.Tensor]):
+        if not (len(packed) == len(ns) == len(outs)) or any(len(p) != len(packed[0]) for p in packed):
+            raise ValueError("one list of worker buffers, one length and one output per bucket are needed")
+        want = torch.bfloat16 if cfg.out_dtype == BF16 else torch.float32
+        for n, o in zip(ns, outs):
+            if o.dtype != want or o.numel() < n:
+                raise ValueError("output must be %s with at least %d elements" % (want, n))
+        self.cfg, self.count, self.workers = cfg, len(ns), len(packed[0]) if packed else 0
+        self.keep = (list(packed), list(outs))
+        self.rows = [(C.c_void_p * self.workers)(*[p if isinstance(p, int) else _dev_ptr(p) for p in row]) for row in packed]
+        self.p = (C.c_void_p * self.count)(*[C.cast(r, C.c_void_p).value for r in self.rows])
+        self.n = (C.c_uint64 * self.count)(*ns)
+        self.o = (C.c_void_p * self.count)(*[_dev_ptr(o) for o in outs])
+
+
+def loco_unpack_dequant_reduce_multi(mr: MultiReduce, stream=None) -> None:
+    """The receive pass for all buckets of mr, their launches overlapped on the library's two streams."""
+    _check(lib().loco_unpack_dequant_reduce_multi(C.byref(mr.cfg.c()), mr.p, mr.workers, mr.n, mr.o, mr.count,
+                                                  _stream_ptr(stream)), "loco_unpack_dequant_reduce_multi")
 
 
 def loco_last_status(st: State, stream=None):
