@@ -573,7 +573,8 @@ def main():
                          "reduce_scatter_bf16: what the method replaces -- NCCL reduce-scatter (average) of the uncompressed bf16 "
                          "buckets, none of this library's kernels, for comparison on the same buckets")
     ap.add_argument("--streams", type=int, default=2,
-                    help="streams the per-bucket launches of a phase are spread over (1 = strictly one after the other)")
+                    help="2 (default): each phase is one multi-bucket call of the library on one stream (the library overlaps "
+                         "consecutive launches on two streams of its own); 1: single-bucket calls strictly one after the other")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -581,7 +582,9 @@ def main():
     cores = os.cpu_count() or 1
     config = {"workload": "llama2-7b: 270 bf16 buckets of 25M elements (6,738,415,616): one worker's send pass per bucket, then the 8-worker reduce of the bucket",
               "bits": 4, "scale": "fixed s=2^14, s_e=4s (Eq. 1)", "beta": 0.5, "T_c": 512, "state": "int8",
-              "workers_on_reduce_side": WORKERS, "out": "bf16", "streams": args.streams,
+              "workers_on_reduce_side": WORKERS, "out": "bf16",
+              "streams": ("1 caller stream; loco_*_multi calls overlap consecutive buckets on the library's 2 streams"
+                          if args.streams > 1 and not args.no_graph else "1, single-bucket calls one after the other"),
               "l2": "inputs larger than L2: each step streams ~70 GB once, no reuse between launches"}
 
     if args.impl == "reference":
@@ -646,10 +649,23 @@ def main():
     else:
         side = [torch.cuda.Stream(device=device) for _ in range(args.streams)] if args.streams > 1 else None
         g_send, g_reduce = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g_send):
-            wl.send_phase(100, side)
-        with torch.cuda.graph(g_reduce):
-            wl.reduce_phase(side)
+        if args.streams > 1:
+            # the library's multi-bucket calls, issued on this one stream: they alternate the launches over two streams of
+            # the library's own and join them back, so that a bucket's tail overlaps the next bucket's start-up
+            ms = loco.MultiSend(wl.states, wl.grads, wl.comms)
+            mr = loco.MultiReduce(wl.cfg, wl.packed, [hi - lo for lo, hi in wl.buckets], wl.outs)
+            loco.loco_compensate_quantize_pack_multi(ms, 100)       # first call outside capture: creates the library's streams
+            loco.loco_unpack_dequant_reduce_multi(mr)
+            torch.cuda.synchronize()
+            with torch.cuda.graph(g_send):
+                loco.loco_compensate_quantize_pack_multi(ms, 100)
+            with torch.cuda.graph(g_reduce):
+                loco.loco_unpack_dequant_reduce_multi(mr)
+        else:
+            with torch.cuda.graph(g_send):
+                wl.send_phase(100, None)
+            with torch.cuda.graph(g_reduce):
+                wl.reduce_phase(None)
     for k in range(max(3, args.warmup)):
         g_send.replay()
         g_reduce.replay()
@@ -744,8 +760,10 @@ def main():
     peak, peak_kind = measured_peak()
     send_gbs = wl.send_bytes / (send_ms * 1e-3) / 1e9
     recv_gbs = wl.recv_bytes / (recv_ms * 1e-3) / 1e9
-    how = ("CUDA events around this kernel's phase of every timed step / launches in it; the launches of a phase "
-           "alternate between %d streams, so a kernel's start-up and tail overlap its neighbour" % max(1, args.streams))
+    how = ("CUDA events around this kernel's phase of every timed step / launches in it; " +
+           ("a phase is one multi-bucket call of the library on one stream, which alternates the launches between two streams of "
+            "its own, so a kernel's start-up and tail overlap its neighbour" if args.streams > 1 and not args.no_graph else
+            "every launch strictly after the previous one"))
     roof_send = {"kernel": "loco_send_kernel<bf16 g, int8 state, 4 bit, fixed scale>", "bound": "hbm",
                  "achieved": send_gbs, "peak": peak, "peak_kind": "%s HBM copy bandwidth" % peak_kind, "unit": "GB/s",
                  "frac": send_gbs / peak, "frac_of_nominal_8TBps": send_gbs / 8000.0, "traffic": SEND_DRAM_BYTES_PER_LAUNCH,
