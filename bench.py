@@ -573,8 +573,8 @@ def main():
                          "reduce_scatter_bf16: what the method replaces -- NCCL reduce-scatter (average) of the uncompressed bf16 "
                          "buckets, none of this library's kernels, for comparison on the same buckets")
     ap.add_argument("--streams", type=int, default=2,
-                    help="2 (default): each phase is one multi-bucket call of the library on one stream (the library overlaps "
-                         "consecutive launches on two streams of its own); 1: single-bucket calls strictly one after the other")
+                    help="2 or more (default): each phase is one multi-bucket call of the library on one stream (the library overlaps "
+                         "consecutive launches on streams of its own); 1: single-bucket calls strictly one after the other")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -583,7 +583,7 @@ def main():
     config = {"workload": "llama2-7b: 270 bf16 buckets of 25M elements (6,738,415,616): one worker's send pass per bucket, then the 8-worker reduce of the bucket",
               "bits": 4, "scale": "fixed s=2^14, s_e=4s (Eq. 1)", "beta": 0.5, "T_c": 512, "state": "int8",
               "workers_on_reduce_side": WORKERS, "out": "bf16",
-              "streams": ("1 caller stream; loco_*_multi calls overlap consecutive buckets on the library's 2 streams"
+              "streams": ("1 caller stream; loco_*_multi calls overlap consecutive buckets on the library's 3 streams"
                           if args.streams > 1 and not args.no_graph else "1, single-bucket calls one after the other"),
               "l2": "inputs larger than L2: each step streams ~70 GB once, no reuse between launches"}
 
@@ -650,7 +650,7 @@ def main():
         side = [torch.cuda.Stream(device=device) for _ in range(args.streams)] if args.streams > 1 else None
         g_send, g_reduce = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
         if args.streams > 1:
-            # the library's multi-bucket calls, issued on this one stream: they alternate the launches over two streams of
+            # the library's multi-bucket calls, issued on this one stream: they take three streams of
             # the library's own and join them back, so that a bucket's tail overlaps the next bucket's start-up
             ms = loco.MultiSend(wl.states, wl.grads, wl.comms)
             mr = loco.MultiReduce(wl.cfg, wl.packed, [hi - lo for lo, hi in wl.buckets], wl.outs)
@@ -761,7 +761,7 @@ def main():
     send_gbs = wl.send_bytes / (send_ms * 1e-3) / 1e9
     recv_gbs = wl.recv_bytes / (recv_ms * 1e-3) / 1e9
     how = ("CUDA events around this kernel's phase of every timed step / launches in it; " +
-           ("a phase is one multi-bucket call of the library on one stream, which alternates the launches between two streams of "
+           ("a phase is one multi-bucket call of the library on one stream, which spreads the launches over three streams of "
             "its own, so a kernel's start-up and tail overlap its neighbour" if args.streams > 1 and not args.no_graph else
             "every launch strictly after the previous one"))
     roof_send = {"kernel": "loco_send_kernel<bf16 g, int8 state, 4 bit, fixed scale>", "bound": "hbm",

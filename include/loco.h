@@ -215,11 +215,11 @@ int loco_unpack_dequant_reduce_adam(const loco_config_t *cfg, const void *const 
  * bucket of the usual size is a kernel of 15-30 microseconds, a third of which is start-up and tail when the
  * kernels of a stream run strictly one after the other.  These two calls do what `count` single-bucket calls on
  * `stream` would do -- same kernels, same results, everything ordered after the work `stream` already holds and
- * before whatever is enqueued on it next -- but issue the launches alternately on two streams that the library
- * owns, so that one bucket's tail overlaps the next bucket's start-up.
+ * before whatever is enqueued on it next -- but issue the launches in turn on three streams that the library
+ * owns, so that one bucket's tail overlaps the start-up of the next ones.
  *   - The buckets of one call must be independent of each other (distinct states and buffers), as they run
  *     concurrently.  All of them belong to the current device.
- *   - The first such call on a device creates two non-blocking streams and three events there (driver objects;
+ *   - The first such call on a device creates three non-blocking streams and four events there (driver objects;
  *     no device memory), kept until the process exits; make it outside any stream capture.  Later calls only
  *     record and wait on those events and launch; they may be captured into a CUDA graph like the single calls.
  *   - Calls on one device are serialised on the host while they enqueue their work (they share the events).

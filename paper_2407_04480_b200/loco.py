@@ -298,7 +298,7 @@ class MultiSend:
 
 
 def loco_compensate_quantize_pack_multi(ms: MultiSend, step_k: int, stream=None) -> None:
-    """The send pass for all buckets of ms, their launches overlapped on the library's two streams."""
+    """The send pass for all buckets of ms, their launches overlapped on the library's own streams."""
     _check(lib().loco_compensate_quantize_pack_multi(ms.h, ms.g, ms.c, ms.count, step_k, _stream_ptr(stream)),
            "loco_compensate_quantize_pack_multi")
 
@@ -322,7 +322,7 @@ class MultiReduce:
 
 
 def loco_unpack_dequant_reduce_multi(mr: MultiReduce, stream=None) -> None:
-    """The receive pass for all buckets of mr, their launches overlapped on the library's two streams."""
+    """The receive pass for all buckets of mr, their launches overlapped on the library's own streams."""
     _check(lib().loco_unpack_dequant_reduce_multi(C.byref(mr.cfg.c()), mr.p, mr.workers, mr.n, mr.o, mr.count,
                                                   _stream_ptr(stream)), "loco_unpack_dequant_reduce_multi")
 
