@@ -48,8 +48,8 @@ SEND_BYTES_PER_ELEM = 2 + 1 + 1 + 0.5
 # dram__bytes_read.sum + dram__bytes_write.sum per launch (one 25M-element bucket) from the ncu captures summarised under
 # profiles/.  Reads equal the algorithmic reads; most written lines are still in the 126 MB L2 when a lone launch ends,
 # so the DRAM write counter of a single captured launch is far below the algorithmic 37.5 / 50 MB.
-SEND_DRAM_BYTES_PER_LAUNCH = 75.03e6 + 3.04e6
-REDUCE_DRAM_BYTES_PER_LAUNCH = 100.03e6 + 14.39e6
+SEND_DRAM_BYTES_PER_LAUNCH = 75.03e6 + 2.53e6
+REDUCE_DRAM_BYTES_PER_LAUNCH = 100.03e6 + 14.24e6
 
 
 def measured_peak():
