@@ -393,7 +393,8 @@ def sweep(args, device):
     unless the row says so."""
     from paper_2407_04480_b200 import inputs, loco
     peak, peak_kind = measured_peak()
-    streams = [torch.cuda.Stream(device=device) for _ in range(max(1, args.streams))]
+    # launches alternate between three streams, as the library's multi-bucket calls issue them (one stream with --streams 1)
+    streams = [torch.cuda.Stream(device=device) for _ in range(3 if args.streams > 1 else 1)]
     rows = []
     budget = 6 << 30                    # device bytes per case
 
