@@ -9,7 +9,30 @@
 #include <mutex>
 #include <new>
 
-#include "loco_kernels.cuh"
+#include "loco_dispatch.h"
+
+namespace loco {
+
+// mismatch[0]: amax / c, mismatch[1]: c / amax, over all positive finite floats, for c = 1, 7, 127
+__global__ void loco_division_selfcheck_kernel(unsigned long long *mismatch) {
+    const float cs[3] = {1.0f, 7.0f, 127.0f};
+    unsigned long long bad0 = 0, bad1 = 0;
+    for (unsigned long long b = blockIdx.x * static_cast<unsigned long long>(blockDim.x) + threadIdx.x + 1; b <= 0x7f7fffffull;
+         b += static_cast<unsigned long long>(gridDim.x) * blockDim.x) {
+        const float a = __uint_as_float(static_cast<unsigned>(b));
+#pragma unroll
+        for (int i = 0; i < 3; ++i) {
+            const float c = cs[i];
+            if (__float_as_uint(div_by_qmax(a, c, __frcp_rn(c))) != __float_as_uint(__fdiv_rn(a, c))) ++bad0;
+            if (__float_as_uint(qmax_over(c, a)) != __float_as_uint(__fdiv_rn(c, a))) ++bad1;
+            if (in_midrange(a) && __float_as_uint(qmax_over_midrange(c, a)) != __float_as_uint(__fdiv_rn(c, a))) ++bad1;
+        }
+    }
+    if (bad0) atomicAdd(mismatch, bad0);
+    if (bad1) atomicAdd(mismatch + 1, bad1);
+}
+
+}  // namespace loco
 
 namespace {
 
@@ -153,89 +176,19 @@ int num_sms() {
     return sms;
 }
 
-// ---- send dispatch -----------------------------------------------------------------------
-
-using SendFn = void (*)(const SendParams);
-struct SendKernel { SendFn fn; int smem_bytes; };
-
-template <int GRAD, int STATE, int BITS>
-SendKernel pick_send_mode(int mode, int var) {
-    if (mode == MODE_FIXED) {
-        const int smem = Ring<GRAD, STATE, MODE_FIXED>::kBytes;
-        if (var == VAR_LEAN) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_LEAN>, smem};
-        if (var == VAR_LEAN_NR && (STATE == ST_INT8 || STATE == ST_Q8COMP))
-            return {loco_send_kernel<GRAD, (STATE == ST_INT8 || STATE == ST_Q8COMP) ? STATE : ST_INT8, BITS, MODE_FIXED, VAR_LEAN_NR>, smem};
-        if (var == VAR_LEAN_X) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_LEAN_X>, smem};
-        if (var == VAR_LEAN_NR_X && (STATE == ST_INT8 || STATE == ST_Q8COMP))
-            return {loco_send_kernel<GRAD, (STATE == ST_INT8 || STATE == ST_Q8COMP) ? STATE : ST_INT8, BITS, MODE_FIXED, VAR_LEAN_NR_X>, smem};
-        if (var == VAR_LEAN_SR) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_LEAN_SR>, smem};
-        if (var == VAR_STOCHASTIC) return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_STOCHASTIC>, smem};
-        return {loco_send_kernel<GRAD, STATE, BITS, MODE_FIXED, VAR_GENERAL>, smem};
-    }
-    if (STATE == ST_Q8COMP) return {nullptr, 0};                // Q8COMP exists for the global scales only
-    constexpr int ST = (STATE == ST_Q8COMP ? ST_FP32 : STATE);
-    if (var == VAR_GENERAL) return {loco_send_kernel<GRAD, ST, BITS, MODE_BLOCK, VAR_GENERAL>, Ring<GRAD, ST, MODE_BLOCK>::kBytes};
-    if (var == VAR_STOCHASTIC) return {loco_send_kernel<GRAD, ST, BITS, MODE_BLOCK, VAR_STOCHASTIC>, Ring<GRAD, ST, MODE_BLOCK>::kBytes};
-    return {loco_send_kernel<GRAD, ST, BITS, MODE_BLOCK, VAR_LEAN>, Ring<GRAD, ST, MODE_BLOCK>::kBytes};
-}
-template <int GRAD, int STATE>
-SendKernel pick_send_bits(int bits, int mode, int var) {
-    switch (bits) {
-    case 2: return pick_send_mode<GRAD, STATE, 2>(mode, var);
-    case 4: return pick_send_mode<GRAD, STATE, 4>(mode, var);
-    default: return pick_send_mode<GRAD, STATE, 8>(mode, var);
-    }
-}
-template <int GRAD>
-SendKernel pick_send_state(int state, int bits, int mode, int var) {
-    switch (state) {
-    case LOCO_STATE_INT8: return pick_send_bits<GRAD, ST_INT8>(bits, mode, var);
-    case LOCO_STATE_FP32: return pick_send_bits<GRAD, ST_FP32>(bits, mode, var);
-    case LOCO_STATE_NONE: return pick_send_bits<GRAD, ST_NONE>(bits, mode, var);
-    default: return pick_send_bits<GRAD, ST_Q8COMP>(bits, mode, var);
-    }
-}
 SendKernel pick_send(const loco_config_t *c, int mode, int var) {
-    return c->grad_dtype == LOCO_BF16 ? pick_send_state<GRAD_BF16>(c->state_fmt, c->bits, mode, var)
-                                      : pick_send_state<GRAD_F32>(c->state_fmt, c->bits, mode, var);
-}
-
-// ---- reduce dispatch ---------------------------------------------------------------------
-
-using ReduceFn = void (*)(const ReduceParams);
-struct ReduceKernel { ReduceFn fn; int smem_bytes; };     // smem_bytes: the kernel's cp.async ring (0: none)
-
-template <int OUT, int BITS>
-ReduceKernel pick_reduce_path(int mode, int path, bool adam) {
-    if (adam) {
-        if (mode != MODE_FIXED) return {loco_reduce_adam_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>, 0};
-        switch (path) {
-        case PATH_INT: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_INT>, 0};
-        case PATH_MUL: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, 0};
-        case PATH_NEWTON: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON>, 0};
-        default: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE>, 0};
-        }
-    }
-    if (mode != MODE_FIXED) return {loco_reduce_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>, static_cast<int>(RecvRing<BITS, MODE_BLOCK>::kCtaBytes)};
-    const int smem = static_cast<int>(RecvRing<BITS, MODE_FIXED>::kCtaBytes);
-    switch (path) {
-    case PATH_INT: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_INT>, smem};
-    case PATH_MUL: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, smem};
-    case PATH_NEWTON: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON>, smem};
-    default: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE>, smem};
+    const bool bf = c->grad_dtype == LOCO_BF16;
+    switch (c->state_fmt) {
+    case LOCO_STATE_INT8: return bf ? pick_send_g1_s0(c->bits, mode, var) : pick_send_g0_s0(c->bits, mode, var);
+    case LOCO_STATE_FP32: return bf ? pick_send_g1_s1(c->bits, mode, var) : pick_send_g0_s1(c->bits, mode, var);
+    case LOCO_STATE_NONE: return bf ? pick_send_g1_s2(c->bits, mode, var) : pick_send_g0_s2(c->bits, mode, var);
+    default: return bf ? pick_send_g1_s3(c->bits, mode, var) : pick_send_g0_s3(c->bits, mode, var);
     }
 }
-template <int OUT>
-ReduceKernel pick_reduce_bits(int bits, int mode, int path, bool adam) {
-    switch (bits) {
-    case 2: return pick_reduce_path<OUT, 2>(mode, path, adam);
-    case 4: return pick_reduce_path<OUT, 4>(mode, path, adam);
-    default: return pick_reduce_path<OUT, 8>(mode, path, adam);
-    }
-}
+
 ReduceKernel pick_reduce(const loco_config_t *c, int mode, int path, bool adam) {
-    return c->out_dtype == LOCO_BF16 ? pick_reduce_bits<GRAD_BF16>(c->bits, mode, path, adam)
-                                     : pick_reduce_bits<GRAD_F32>(c->bits, mode, path, adam);
+    if (c->out_dtype == LOCO_BF16) return adam ? pick_reduce_o1_a1(c->bits, mode, path) : pick_reduce_o1_a0(c->bits, mode, path);
+    return adam ? pick_reduce_o0_a1(c->bits, mode, path) : pick_reduce_o0_a0(c->bits, mode, path);
 }
 
 unsigned grid_x_for(uint64_t rows_per_partition, int partitions, int ctas_per_sm) {

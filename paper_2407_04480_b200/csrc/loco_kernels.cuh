@@ -646,25 +646,6 @@ __device__ __forceinline__ float group_max16(float v, int lanes) {
     return v;
 }
 
-// mismatch[0]: amax / c, mismatch[1]: c / amax, over all positive finite floats, for c = 1, 7, 127
-__global__ void loco_division_selfcheck_kernel(unsigned long long *mismatch) {
-    const float cs[3] = {1.0f, 7.0f, 127.0f};
-    unsigned long long bad0 = 0, bad1 = 0;
-    for (unsigned long long b = blockIdx.x * static_cast<unsigned long long>(blockDim.x) + threadIdx.x + 1; b <= 0x7f7fffffull;
-         b += static_cast<unsigned long long>(gridDim.x) * blockDim.x) {
-        const float a = __uint_as_float(static_cast<unsigned>(b));
-#pragma unroll
-        for (int i = 0; i < 3; ++i) {
-            const float c = cs[i];
-            if (__float_as_uint(div_by_qmax(a, c, __frcp_rn(c))) != __float_as_uint(__fdiv_rn(a, c))) ++bad0;
-            if (__float_as_uint(qmax_over(c, a)) != __float_as_uint(__fdiv_rn(c, a))) ++bad1;
-            if (in_midrange(a) && __float_as_uint(qmax_over_midrange(c, a)) != __float_as_uint(__fdiv_rn(c, a))) ++bad1;
-        }
-    }
-    if (bad0) atomicAdd(mismatch, bad0);
-    if (bad1) atomicAdd(mismatch + 1, bad1);
-}
-
 // One wide row.  Returns false (and stores nothing) if some lane of the warp met a value that the fast
 // arithmetic does not cover (NaN, +-Inf, or a magnitude that could overflow): the caller then redoes the row
 // with the careful routine.

@@ -1,0 +1,45 @@
+// Instantiations of the receive kernels for one output type, with or without the fused Adam-family step, chosen with
+// -DLOCO_TU_OUT=<GRAD_*> -DLOCO_TU_ADAM=0|1; see loco_dispatch.h.
+#include "loco_dispatch.h"
+
+#if !defined(LOCO_TU_OUT) || !defined(LOCO_TU_ADAM)
+#error "compile with -DLOCO_TU_OUT=0|1 -DLOCO_TU_ADAM=0|1"
+#endif
+
+namespace loco {
+
+namespace {
+
+template <int OUT, int BITS>
+ReduceKernel pick_reduce_path(int mode, int path) {
+#if LOCO_TU_ADAM
+    if (mode != MODE_FIXED) return {loco_reduce_adam_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>, 0};
+    switch (path) {
+    case PATH_INT: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_INT>, 0};
+    case PATH_MUL: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, 0};
+    case PATH_NEWTON: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON>, 0};
+    default: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE>, 0};
+    }
+#else
+    if (mode != MODE_FIXED) return {loco_reduce_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>, static_cast<int>(RecvRing<BITS, MODE_BLOCK>::kCtaBytes)};
+    const int smem = static_cast<int>(RecvRing<BITS, MODE_FIXED>::kCtaBytes);
+    switch (path) {
+    case PATH_INT: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_INT>, smem};
+    case PATH_MUL: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, smem};
+    case PATH_NEWTON: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON>, smem};
+    default: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE>, smem};
+    }
+#endif
+}
+
+}  // namespace
+
+ReduceKernel LOCO_REDUCE_TU_NAME(LOCO_TU_OUT, LOCO_TU_ADAM)(int bits, int mode, int path) {
+    switch (bits) {
+    case 2: return pick_reduce_path<LOCO_TU_OUT, 2>(mode, path);
+    case 4: return pick_reduce_path<LOCO_TU_OUT, 4>(mode, path);
+    default: return pick_reduce_path<LOCO_TU_OUT, 8>(mode, path);
+    }
+}
+
+}  // namespace loco
