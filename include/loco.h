@@ -99,9 +99,14 @@ typedef struct {
                                 experiments; the paper states no threshold); 0 = off.  +-Inf becomes
                                 +-clip, NaN stays NaN                                             */
     int32_t rounding;        /* loco_rounding_t: 0 = nearest integer as Eq. 1 states (the paper), 1 =
-                                stochastic rounding, an extension: floor(h x s + u), u uniform in
-                                [0, 1) from Philox4x32-10 with counter (element/4, iteration) and key
-                                `seed`; word element%4, top 24 bits                               */
+                                stochastic rounding, an extension: q = clamp(floor(h x s + u)) with
+                                u = (b + 1/2) / 256, one fp32 add, where for element i of the bucket at
+                                iteration k the byte b is byte (i mod 4), least significant first, of
+                                output word ((i mod 16) / 4) of Philox4x32-10 with the 4-word counter
+                                (floor(i/16) low 32 bits, floor(i/16) high 32 bits, k low, k high) and
+                                the 2-word key (seed_lo, seed_hi): 16 elements share one Philox block,
+                                256 equally likely values of u at the centres of their cells.  Not
+                                available with bits = 1                                           */
     uint32_t seed_lo, seed_hi; /* key of that stream (ignored with rounding 0)                      */
 } loco_config_t;
 

@@ -44,6 +44,12 @@
  *     parameter (0 = off), applied to g before step 1;
  *   - stochastic rounding (not in the paper, which rounds to nearest): floor(h x s + u) with u from a
  *     Philox4x32-10 stream keyed by a seed and indexed by (element, iteration), so that it can be reproduced anywhere;
+ *   - 1-bit LoCo (the paper names it in the GPT-2 experiment and never defines it; Eq. 1 with p = 1 would give the
+ *     range {-1, 0}): bits = 1 sends the sign, q = -1 if h < 0 else +1 (so +-0 and NaN give +1), one wire bit per
+ *     element (1 = negative), and d = q / s with the global scale, or d = q x (mean |h| of the block) with block
+ *     scales -- the magnitude that minimises the squared error of a sign code; that mean is taken in fp32 by
+ *     pairwise (balanced binary tree) summation over the block's B positions, absent and non-finite elements
+ *     entering as 0, divided by the number of elements of the block that exist.  Steps 2 (Eq. 5, Eq. 7) unchanged;
  *   - Eq. 8 is summed in worker order in fp32, then divided by (float)N;
  *   - the Adam-family step is taken exactly as printed (no bias correction, delta inside the root), with
  *     eta_k = eta / sqrt(v_k + delta) evaluated as one square root and one division.
@@ -57,9 +63,13 @@
  * the packing, and a hand-worked example (tests/golden/); for the fused Adam-family step: the sign-update special
  * case (beta1 = beta2 = 1, delta = 0), the closed form of the moments under a constant gradient, a zero gradient,
  * agreement with the textbook formulas in float64, and a hand-worked dyadic example.
- * Unpinned by anything in the paper: the value of beta, the block size and the
- * block-scaled variant as a whole ("parity unpinned" for SCALE_BLOCK_ABSMAX:
- * it is pinned only by the invariants that do not depend on the scale rule).
+ * The block-scaled 8-bit state (scale rule amax/127, largest code 127, half-step bound, reset, Lemma 1's identity in
+ * its 8-bit form) and the bf16 conversions (against an independent conversion, ties, NaN, Inf, denormals) have
+ * pins of their own; the 1-bit compressor is pinned by its optimality on brute-forced blocks, the order of its
+ * pairwise sum on a hand-worked block, Lemma 1's identity and the packing of all 256 bytes.
+ * Unpinned by anything in the paper: the value of beta, the block size, the
+ * block-scaled variant as a whole and the 1-bit compressor ("parity unpinned" for SCALE_BLOCK_ABSMAX and
+ * for bits = 1: they are pinned only by what the mathematics fixes once the reading is chosen).
  */
 #include <math.h>
 #include <stdint.h>
@@ -73,7 +83,7 @@ enum { ORC_FLAG_NONFINITE = 1u };
 
 /* Algorithm 1's inputs (s, s_e, T_c, beta) plus the storage choices. */
 typedef struct {
-    int32_t bits;           /* p of Eq. 1 for the gradient codes: 2, 4 or 8 */
+    int32_t bits;           /* p of Eq. 1 for the gradient codes: 2, 4 or 8; 1 = sign code (1-bit LoCo) */
     int32_t scale_mode;     /* ORC_SCALE_* */
     int32_t block_size;     /* B, BLOCK_ABSMAX only */
     float   s;              /* Eq. 1 / Eq. 3 */
@@ -149,6 +159,8 @@ static uint16_t f32_to_bf16_rne(float f) {
 }
 uint16_t orc_f32_to_bf16(float f) { return f32_to_bf16_rne(f); }
 float orc_bf16_to_f32(uint16_t b) { return bf16_to_f32(b); }
+void orc_f32_to_bf16_array(const float *f, uint64_t n, uint16_t *b) { for (uint64_t i = 0; i < n; ++i) b[i] = f32_to_bf16_rne(f[i]); }
+void orc_bf16_to_f32_array(const uint16_t *b, uint64_t n, float *f) { for (uint64_t i = 0; i < n; ++i) f[i] = bf16_to_f32(b[i]); }
 
 /* ---------- Eq. 1 ---------- */
 static int32_t qmin_of(int p) { return -(1 << (p - 1)); }
@@ -177,7 +189,7 @@ static uint64_t round_up(uint64_t x, uint64_t m) { return (x + m - 1) / m * m; }
 
 static int config_ok(const orc_config *c) {
     if (!c) return 0;
-    if (c->bits != 2 && c->bits != 4 && c->bits != 8) return 0;
+    if (c->bits != 1 && c->bits != 2 && c->bits != 4 && c->bits != 8) return 0;
     if (c->scale_mode != ORC_SCALE_FIXED && c->scale_mode != ORC_SCALE_BLOCK_ABSMAX) return 0;
     if (c->scale_mode == ORC_SCALE_BLOCK_ABSMAX) {
         int b = c->block_size;
@@ -196,6 +208,7 @@ static int config_ok(const orc_config *c) {
     if (c->num_partitions < 1) return 0;
     if (!(c->clip >= 0.0f) || !isfinite(c->clip)) return 0;
     if (c->rounding != 0 && c->rounding != 1) return 0;
+    if (c->bits == 1 && c->rounding != 0) return 0;       /* a sign code has nothing to round */
     return 1;
 }
 
@@ -251,6 +264,7 @@ uint64_t orc_state_bytes(const orc_config *c, uint64_t n) {
 
 /* Write the p-bit two's-complement field of element `o` of a partition's code area. */
 static void put_code(uint8_t *codes, uint64_t o, int p, int32_t q) {
+    if (p == 1) q = q < 0 ? 1 : 0;           /* sign code: the wire bit is 1 for -1, 0 for +1 */
     int per = 8 / p;
     uint64_t byte = o / (uint64_t)per;
     int shift = (int)(o % (uint64_t)per) * p;
@@ -263,6 +277,7 @@ static int32_t get_code(const uint8_t *codes, uint64_t o, int p) {
     uint64_t byte = o / (uint64_t)per;
     int shift = (int)(o % (uint64_t)per) * p;
     int32_t v = (int32_t)((codes[byte] >> shift) & ((1u << p) - 1u));
+    if (p == 1) return v ? -1 : 1;            /* sign code */
     if (v >= (1 << (p - 1))) v -= (1 << p);
     return v;
 }
@@ -288,6 +303,11 @@ static float load_grad(const orc_config *c, const void *grad, uint64_t i) {
  * Returns the code; *err0 is set when the element's compression error is defined as 0. */
 static int32_t quantise(const orc_config *c, uint64_t i, int64_t k, float h, float mult, int p, int *err0, uint64_t *status) {
     *err0 = 0;
+    if (p == 1) {
+        /* 1-bit LoCo: the sign, q in {+1, -1}; the compression error of a non-finite element is taken as 0 */
+        if (isnan(h) || isinf(h)) { *err0 = 1; status[0] |= ORC_FLAG_NONFINITE; }
+        return h < 0.0f ? -1 : 1;
+    }
     if (isnan(h)) { *err0 = 1; status[0] |= ORC_FLAG_NONFINITE; return 0; }
     if (isinf(h)) { *err0 = 1; status[0] |= ORC_FLAG_NONFINITE; return h > 0 ? qmax_of(p) : qmin_of(p); }
     float y = h * mult;                       /* h x s of Eq. 1 */
@@ -308,6 +328,14 @@ static int32_t quantise(const orc_config *c, uint64_t i, int64_t k, float h, flo
     return q;
 }
 
+/* Pairwise summation in fp32: the sum of a[0..len) is the sum of its first half plus the sum of its second half,
+ * len a power of two. */
+static float pairwise_sum(const float *a, uint64_t len) {
+    if (len == 1) return a[0];
+    return pairwise_sum(a, len / 2) + pairwise_sum(a + len / 2, len / 2);
+}
+float orc_pairwise_sum(const float *a, uint64_t len) { return pairwise_sum(a, len); }
+
 /*
  * One LoCo send step for one worker and one bucket (Algorithm 1, steps 1 and 2),
  * followed by packing the codes into the partitioned communication buffer.
@@ -317,7 +345,9 @@ static int32_t quantise(const orc_config *c, uint64_t i, int64_t k, float h, flo
  *   comm   communication buffer of orc_packed_bytes(); code and scale areas are
  *          fully written, bytes past them inside a stride are left alone
  *   k      the paper's 0-based iteration counter
- *   status [0] flag bits (or-ed in), [1] count of saturated gradient codes (added to)
+ *   status [0] flag bits (or-ed in), [1] count of saturated gradient codes (added to), [2] count of saturated
+ *          8-bit error codes (added to): elements whose e~ x s_e has its nearest integer outside [-128, 127], the
+ *          clamp of Eq. 7 (global s_e only; a block-scaled state cannot saturate)
  * Returns 0, or -1 on a bad configuration.
  */
 int orc_send_step(const orc_config *cfg, uint64_t n, const void *grad, void *state,
@@ -334,7 +364,7 @@ int orc_send_step(const orc_config *cfg, uint64_t n, const void *grad, void *sta
     const float beta = cfg->beta;
     const float omb = 1.0f - beta;            /* (1 - beta) of Eq. 5, rounded once */
     const int reset = cfg->reset_period > 0 && (k % (int64_t)cfg->reset_period) == 0;   /* Eq. 7 */
-    uint64_t st_local[2] = {0, 0};
+    uint64_t st_local[3] = {0, 0, 0};
     if (!status) status = st_local;
 
     int8_t *e8 = (int8_t *)state;                              /* STATE_INT8 codes */
@@ -351,7 +381,8 @@ int orc_send_step(const orc_config *cfg, uint64_t n, const void *grad, void *sta
     float *cb = (float *)malloc(sizeof(float) * B);
     float *pb = (float *)malloc(sizeof(float) * B);
     float *nb = (float *)malloc(sizeof(float) * B);
-    if (!hb || !cb || !pb || !nb) { free(hb); free(cb); free(pb); free(nb); return -1; }
+    float *ab = (float *)malloc(sizeof(float) * B);
+    if (!hb || !cb || !pb || !nb || !ab) { free(hb); free(cb); free(pb); free(nb); free(ab); return -1; }
 
     for (uint64_t b0 = 0; b0 < n; b0 += B) {
         const uint64_t len = (b0 + B <= n) ? B : n - b0;
@@ -372,7 +403,11 @@ int orc_send_step(const orc_config *cfg, uint64_t n, const void *grad, void *sta
                 break;
             case ORC_STATE_FP32_Q8COMP:
                 prev = ef[i];
-                c = (float)round_pbit(prev * cfg->s_e, 8) / cfg->s_e;
+                {
+                    const float ye = prev * cfg->s_e, re = rintf(ye);
+                    if (re < -128.0f || re > 127.0f) status[2] += 1;
+                    c = (float)round_pbit(ye, 8) / cfg->s_e;
+                }
                 break;
             default:
                 c = 0.0f;
@@ -385,7 +420,12 @@ int orc_send_step(const orc_config *cfg, uint64_t n, const void *grad, void *sta
 
         /* scale of the block (extension); the paper's s otherwise */
         float mult = cfg->s, scale = 0.0f;
-        if (!fixed) {
+        if (!fixed && p == 1) {
+            /* sign code: the block's magnitude is the mean of |h| (pairwise sum over the B positions / elements that exist) */
+            for (uint64_t t = 0; t < B; ++t) ab[t] = (t < len && isfinite(hb[t])) ? fabsf(hb[t]) : 0.0f;
+            scale = pairwise_sum(ab, B) / (float)len;
+            mult = 0.0f;
+        } else if (!fixed) {
             float amax = 0.0f;
             for (uint64_t t = 0; t < len; ++t)
                 if (isfinite(hb[t]) && fabsf(hb[t]) > amax) amax = fabsf(hb[t]);
@@ -436,13 +476,16 @@ int orc_send_step(const orc_config *cfg, uint64_t n, const void *grad, void *sta
                 emult = amax > 0.0f ? 127.0f / amax : 0.0f;
                 e8_scale[blk] = escale;
             }
-            for (uint64_t t = 0; t < len; ++t)
-                e8[b0 + t] = (int8_t)round_pbit(nb[t] * emult, 8);   /* compressor(e~; s_e, 8) */
+            for (uint64_t t = 0; t < len; ++t) {
+                const float ye = nb[t] * emult, re = rintf(ye);
+                if (fixed && (re < -128.0f || re > 127.0f)) status[2] += 1;     /* the clamp of Eq. 7 acts */
+                e8[b0 + t] = (int8_t)round_pbit(ye, 8);                          /* compressor(e~; s_e, 8) */
+            }
         } else {
             for (uint64_t t = 0; t < len; ++t) ef[b0 + t] = nb[t];
         }
     }
-    free(hb); free(cb); free(pb); free(nb);
+    free(hb); free(cb); free(pb); free(nb); free(ab);
     return 0;
 }
 

@@ -108,10 +108,16 @@ def lib():
         L.orc_philox4x32_10.argtypes = [vp, vp, vp]
         L.orc_sr_uniform.restype = C.c_float
         L.orc_sr_uniform.argtypes = [cp, u64, i64]
+        L.orc_pairwise_sum.restype = C.c_float
+        L.orc_pairwise_sum.argtypes = [vp, u64]
         L.orc_f32_to_bf16.restype = C.c_uint16
         L.orc_f32_to_bf16.argtypes = [C.c_float]
         L.orc_bf16_to_f32.restype = C.c_float
         L.orc_bf16_to_f32.argtypes = [C.c_uint16]
+        L.orc_f32_to_bf16_array.restype = None
+        L.orc_f32_to_bf16_array.argtypes = [vp, u64, vp]
+        L.orc_bf16_to_f32_array.restype = None
+        L.orc_bf16_to_f32_array.argtypes = [vp, u64, vp]
         _lib = L
     return _lib
 
@@ -159,8 +165,19 @@ def unpack_codes(b: np.ndarray, n: int, p: int) -> np.ndarray:
 
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
-    f = lib().orc_f32_to_bf16
-    return np.array([f(float(v)) for v in np.asarray(x, dtype=np.float32).ravel()], dtype=np.uint16)
+    """The oracle's fp32 -> bf16 conversion (round to nearest, ties to even), elementwise, as bit patterns."""
+    x = np.ascontiguousarray(np.asarray(x, dtype=np.float32).ravel())
+    out = np.empty(x.size, dtype=np.uint16)
+    lib().orc_f32_to_bf16_array(_ptr(x), x.size, _ptr(out))
+    return out
+
+
+def bf16_bits_to_f32(b: np.ndarray) -> np.ndarray:
+    """The oracle's bf16 -> fp32 widening, elementwise."""
+    b = np.ascontiguousarray(np.asarray(b, dtype=np.uint16).ravel())
+    out = np.empty(b.size, dtype=np.float32)
+    lib().orc_bf16_to_f32_array(_ptr(b), b.size, _ptr(out))
+    return out
 
 
 def new_state(cfg: OracleConfig, n: int) -> np.ndarray:
@@ -173,11 +190,11 @@ def new_comm(cfg: OracleConfig, n: int, fill: int = 0) -> np.ndarray:
 
 
 def send_step(cfg: OracleConfig, grad: np.ndarray, state: np.ndarray, comm: np.ndarray, k: int,
-              trace: bool = False):
+              trace: bool = False, full_status: bool = False):
     """Algorithm 1 steps 1-2 for one worker; updates state and comm in place.
 
-    grad is float32, or uint16 holding bf16 bit patterns.  Returns (flags, n_saturated)
-    and, when trace is set, a dict of the per-element intermediates.
+    grad is float32, or uint16 holding bf16 bit patterns.  Returns (flags, n_saturated) -- with full_status
+    (flags, n_saturated, n_saturated_state) -- and, when trace is set, a dict of the per-element intermediates.
     """
     n = grad.size
     if cfg.grad_dtype == BF16:
@@ -186,7 +203,7 @@ def send_step(cfg: OracleConfig, grad: np.ndarray, state: np.ndarray, comm: np.n
         assert grad.dtype == np.float32
     assert state.dtype == np.uint8 and state.size >= state_bytes(cfg, n)
     assert comm.dtype == np.uint8 and comm.size >= packed_bytes(cfg, n)
-    status = np.zeros(2, dtype=np.uint64)
+    status = np.zeros(3, dtype=np.uint64)
     tr = None
     rec = None
     if trace:
@@ -199,7 +216,7 @@ def send_step(cfg: OracleConfig, grad: np.ndarray, state: np.ndarray, comm: np.n
                              C.byref(tr) if tr is not None else None, _ptr(status))
     if rc != 0:
         raise ValueError("oracle: bad configuration")
-    out = (int(status[0]), int(status[1]))
+    out = (int(status[0]), int(status[1]), int(status[2])) if full_status else (int(status[0]), int(status[1]))
     return (out, rec) if trace else out
 
 
@@ -250,6 +267,13 @@ def philox4x32_10(ctr, key) -> np.ndarray:
     out = np.zeros(4, dtype=np.uint32)
     lib().orc_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
     return out
+
+
+def pairwise_sum(a: np.ndarray) -> float:
+    """fp32 pairwise (balanced binary tree) sum of a power-of-two number of values."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    assert a.size > 0 and a.size & (a.size - 1) == 0
+    return float(lib().orc_pairwise_sum(_ptr(a), a.size))
 
 
 def sr_uniform(cfg: OracleConfig, i: int, k: int) -> float:

@@ -150,9 +150,9 @@ def test_hand_worked_example():
     state, comm = orc.new_state(cfg, n), orc.new_comm(cfg, n)
     comms = []
     for k, tag in ((1, "1"), (2, "2")):
-        (flags, sat), tr = orc.send_step(cfg, f("g" + tag), state, comm, k, trace=True)
+        (flags, sat, ssat), tr = orc.send_step(cfg, f("g" + tag), state, comm, k, trace=True, full_status=True)
         nxt = str(k + 1)
-        assert flags == 0 and sat == int(G["sat" + tag][0])
+        assert flags == 0 and sat == int(G["sat" + tag][0]) and ssat == int(G["ssat" + tag][0])
         assert np.array_equal(tr["h"], f("h" + tag))
         assert np.array_equal(tr["q"], f("q" + tag).astype(np.int32))
         assert np.array_equal(tr["d"], f("d" + tag))
@@ -711,3 +711,247 @@ def test_stochastic_rounding_properties():
     orc.send_step(cfgp, h, orc.new_state(cfgp, n), commp, 200)
     qp = np.concatenate([orc.unpack_codes(c, orc.partition_elems(cfgp, n, j), 8) for j, (c, _) in enumerate(orc.comm_views(cfgp, n, commp))])
     assert np.array_equal(qp, draws[-1])
+
+
+# ---------------------------------------------------------------- Eq. 7's clamp: saturated 8-bit error codes
+
+def test_state_clamp_hand_worked_example():
+    """tests/golden/eq7_clamp_worked_example.txt: error codes whose nearest integer leaves [-128, 127] are clamped
+    (Eq. 7 compresses with the 8-bit compressor of Eq. 1) and counted; the ties 127.5 and -128.5 fall on either side."""
+    G = load_golden("eq7_clamp_worked_example.txt")
+    f = lambda k: np.array([float(v) for v in G[k]], dtype=np.float32)
+    for fmt in (orc.STATE_INT8, orc.STATE_FP32_Q8COMP):
+        cfg = OracleConfig(bits=int(G["p"][0]), s=float(G["s"][0]), s_e=float(G["s_e"][0]), beta=float(G["beta"][0]),
+                           reset_period=0, state_fmt=fmt)
+        state, comm = orc.new_state(cfg, 6), orc.new_comm(cfg, 6)
+        (flags, sat, ssat), tr = orc.send_step(cfg, f("g1"), state, comm, 1, trace=True, full_status=True)
+        assert flags == 0 and sat == int(G["sat1"][0])
+        assert np.array_equal(tr["q"], f("q1").astype(np.int32)) and np.array_equal(tr["d"], f("d1"))
+        assert np.array_equal(tr["e_new"], f("et2"))
+        if fmt == orc.STATE_INT8:
+            assert ssat == int(G["ssat1"][0])
+            assert np.array_equal(state[:6].view(np.int8), f("e2").astype(np.int8))
+        else:
+            # the fp32 error is kept; its 8-bit image is formed (and its clamp counted) when it is next used
+            assert ssat == 0
+            (_, _, ssat2), tr2 = orc.send_step(cfg, np.zeros(6, np.float32), state, comm, 2, trace=True, full_status=True)
+            assert ssat2 == int(G["ssat1"][0])
+            assert np.array_equal(tr2["c"], f("e2") / np.float32(16))
+
+
+# ---------------------------------------------------------------- block-scaled 8-bit error state (extension)
+
+@pytest.mark.parametrize("B", [32, 256, 1024])
+@pytest.mark.parametrize("p", [4, 8])
+def test_block_scaled_int8_state(B, p):
+    """The 8-bit error state with one scale per block (no counterpart in the paper; Eq. 7's 8-bit compression with the
+    global s_e replaced by 127 / amax of the block).  What the mathematics fixes: the stored scale is fl(amax / 127),
+    the largest code of a non-zero block is 127 in magnitude, |e~ - e x scale| <= scale / 2, a zero block and a
+    reset give scale 0 and codes 0, the next iteration compensates with e x scale, and Lemma 1's identity holds in
+    its 8-bit form d - g = (e^_k - e~_{k+1}) / beta with e^_k = e_k x scale_k."""
+    n = 5 * B + B // 2 + 3                       # five whole blocks, one ragged
+    beta = 0.5
+    cfg = OracleConfig(bits=p, scale_mode=orc.SCALE_BLOCK_ABSMAX, block_size=B, beta=beta, reset_period=3,
+                       state_fmt=orc.STATE_INT8)
+    nblk = (n + B - 1) // B
+    state, comm = orc.new_state(cfg, n), orc.new_comm(cfg, n)
+    codes_v, scales_v = orc.state_views(cfg, n, state)
+    prev_codes, prev_scales = codes_v.copy(), scales_v.copy()
+    assert not prev_codes.any() and not prev_scales.any()
+    for k in range(1, 7):                        # k = 3 and k = 6 reset
+        g = RNG.normal(0, 1e-3, n).astype(np.float32)
+        g[2 * B:3 * B] = 0                       # block 2 never carries anything
+        (_, _), tr = orc.send_step(cfg, g, state, comm, k, trace=True)
+        # step 1 compensated with the stored image of the previous error: one product per element
+        want_c = prev_codes.astype(np.float32) * np.repeat(prev_scales, B)[:n]
+        assert np.array_equal(tr["c"], want_c)
+        assert np.array_equal(tr["h"], g + want_c)
+        # Lemma 1, 8-bit form
+        lhs = tr["d"].astype(np.float64) - g.astype(np.float64)
+        rhs = (tr["c"].astype(np.float64) - tr["e_new"].astype(np.float64)) / beta
+        assert np.allclose(lhs, rhs, rtol=0, atol=1e-9)
+        if k % 3 == 0:
+            assert not codes_v.any() and not scales_v.any()
+        else:
+            for b in range(nblk):
+                blk = slice(b * B, min((b + 1) * B, n))
+                en = tr["e_new"][blk]
+                amax = np.abs(en).max()
+                assert scales_v[b].view(np.uint32) == (np.float32(amax) / np.float32(127)).view(np.uint32)
+                if amax == 0:
+                    assert scales_v[b] == 0 and not codes_v[blk].any()
+                    continue
+                e = codes_v[blk].astype(np.float64)
+                assert np.abs(e).max() == 127
+                # en x fl(127 / amax) is rounded once before the nearest-integer step: a few ulps of slack
+                assert np.all(np.abs(en.astype(np.float64) - e * float(scales_v[b])) <= float(scales_v[b]) * (0.5 + 1e-4))
+            assert scales_v[2] == 0 and not codes_v[2 * B:3 * B].any()
+        prev_codes, prev_scales = codes_v.copy(), scales_v.copy()
+
+
+def test_block_scaled_int8_state_detects_a_wrong_divisor():
+    """The pin above has teeth: codes formed with 128 / amax (a plausible slip) against the stored scale amax / 127
+    break the half-step bound."""
+    en = RNG.normal(0, 1e-3, 256).astype(np.float32)
+    amax = np.abs(en).max()
+    scale = float(np.float32(amax) / np.float32(127))
+    wrong = np.rint(en * (np.float32(128) / amax)).clip(-128, 127).astype(np.float64)
+    right = np.rint(en * (np.float32(127) / amax)).clip(-128, 127).astype(np.float64)
+    assert np.all(np.abs(en - right * scale) <= scale * (0.5 + 1e-4))
+    assert np.any(np.abs(en - wrong * scale) > scale * (0.5 + 1e-4))
+
+
+# ---------------------------------------------------------------- bf16 conversions
+
+def _torch_bf16_bits(x: np.ndarray) -> np.ndarray:
+    return torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+
+def test_bf16_conversions_against_an_independent_conversion():
+    """bf16 is the upper half of binary32; conversion to it rounds to nearest, ties to even.  Checked against PyTorch's
+    own conversion on ties, +-0, denormals, the largest finite values, +-Inf, NaN and a million random bit patterns."""
+    special = np.array([0x00000000, 0x80000000, 0x00000001, 0x80000001, 0x00008000, 0x00018000, 0x00007fff, 0x0000ffff,
+                        0x3f808000, 0x3f818000, 0x3f807fff, 0x3f808001, 0x3f817fff, 0x3f818001,      # ties and their neighbours
+                        0x7f7fffff, 0xff7fffff, 0x7f7f7fff, 0x7f7f8000, 0x7f7f8001,                  # largest finite: rounds to Inf
+                        0x7f800000, 0xff800000, 0x007fffff, 0x00800000, 0x807fffff], dtype=np.uint32)
+    rnd = RNG.integers(0, 2 ** 32, 1_000_000, dtype=np.uint64).astype(np.uint32)
+    words = np.concatenate([special, rnd])
+    x = words.view(np.float32)
+    got = orc.f32_to_bf16_bits(x)
+    want = _torch_bf16_bits(x)
+    nan = np.isnan(x)
+    assert np.array_equal(got[~nan], want[~nan])
+    # a NaN stays a NaN (its payload is not part of the contract)
+    assert np.all((got[nan] & 0x7f80) == 0x7f80) and np.all((got[nan] & 0x007f) != 0)
+    # ties-to-even spelled out: 1 + 2^-8 -> 1 (even), 1 + 3 * 2^-8 -> 1 + 2^-6
+    assert list(orc.f32_to_bf16_bits(np.array([0x3f808000, 0x3f818000], np.uint32).view(np.float32))) == [0x3f80, 0x3f82]
+    # widening is exact and inverts the narrowing on every bf16 value
+    allb = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    wide = orc.bf16_bits_to_f32(allb)
+    assert np.array_equal(wide.view(np.uint32), allb.astype(np.uint32) << 16)
+    fin = ~np.isnan(wide)
+    assert np.array_equal(orc.f32_to_bf16_bits(wide[fin]), allb[fin])
+    assert np.array_equal(wide[fin], torch.from_numpy(allb[fin].view(np.int16)).view(torch.bfloat16).float().numpy())
+
+
+def test_bf16_gradient_is_the_widened_value_and_bf16_output_is_the_rounded_mean():
+    """A bf16 gradient enters Algorithm 1 as the fp32 number it denotes; a bf16 output is the fp32 result of Eq. 8
+    rounded once (checked with PyTorch's conversion, not the oracle's)."""
+    n = 4099
+    kw = dict(bits=4, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=0, num_partitions=3)
+    cb, cf = OracleConfig(grad_dtype=orc.BF16, **kw), OracleConfig(grad_dtype=orc.F32, **kw)
+    sb, sf = orc.new_state(cb, n), orc.new_state(cf, n)
+    comms_b, comms_f = [], []
+    for k in range(1, 4):
+        gb = _torch_bf16_bits(RNG.normal(0, 1e-3, n).astype(np.float32))
+        gf = torch.from_numpy(gb.view(np.int16)).view(torch.bfloat16).float().numpy()
+        mb, mf = orc.new_comm(cb, n), orc.new_comm(cf, n)
+        assert orc.send_step(cb, gb, sb, mb, k) == orc.send_step(cf, gf, sf, mf, k)
+        assert np.array_equal(mb, mf) and np.array_equal(sb, sf)
+        comms_b.append(mb)
+        comms_f.append(mf)
+    o32 = orc.reduce(cf, n, comms_f)
+    o16 = orc.reduce(OracleConfig(grad_dtype=orc.F32, out_dtype=orc.BF16, **kw), n, comms_f)
+    assert np.array_equal(o16, _torch_bf16_bits(o32))
+
+
+# ---------------------------------------------------------------- 1-bit LoCo (sign code; named in the paper, not defined)
+
+def test_one_bit_code_is_the_sign():
+    """Reading for bits = 1: q = -1 if h < 0 else +1 (so +-0 -> +1), wire bit 1 for -1, d = q / s, eight codes per
+    byte with element i at bit i mod 8; Eq. 8 then averages +-1/s."""
+    s = 8.0
+    cfg = OracleConfig(bits=1, s=s, s_e=4 * s, beta=1.0, reset_period=0, state_fmt=orc.STATE_FP32)
+    g = np.array([0.5, -0.5, 0.0, -0.0, 1e-30, -1e-30, 3.0, -7.0, 0.125, -0.125], dtype=np.float32)
+    state, comm = orc.new_state(cfg, g.size), orc.new_comm(cfg, g.size, fill=0xEE)
+    (flags, sat), tr = orc.send_step(cfg, g, state, comm, 1, trace=True)
+    assert flags == 0 and sat == 0
+    assert list(tr["q"]) == [1, -1, 1, 1, 1, -1, 1, -1, 1, -1]
+    assert np.array_equal(tr["d"], tr["q"].astype(np.float32) / np.float32(s))
+    assert comm[0] == 0b10100010 and comm[1] == 0b00000010        # bits 1, 5, 7 and bit 9
+    # beta = 1: classic error feedback, e~ = h - sign(h) / s
+    assert np.array_equal(state.view(np.float32)[:g.size], g - tr["d"])
+    # idempotent: the dequantised vector compresses to the same codes
+    comm2 = orc.new_comm(cfg, g.size)
+    (_, _), tr2 = orc.send_step(cfg, tr["d"], orc.new_state(cfg, g.size), comm2, 1, trace=True)
+    assert np.array_equal(tr2["q"], tr["q"]) and np.array_equal(tr2["d"], tr["d"])
+    # Eq. 8 over 3 workers holding q, q and -q: (q + q - q) / (3 s)
+    gneg = np.where(tr["q"] > 0, -1.0, 1.0).astype(np.float32)
+    comm3 = orc.new_comm(cfg, g.size)
+    orc.send_step(cfg, gneg, orc.new_state(cfg, g.size), comm3, 1)
+    got = orc.reduce(cfg, g.size, [comm, comm, comm3])
+    want = ((tr["d"] + tr["d"]) - tr["d"]) / np.float32(3)
+    assert np.array_equal(got, want)
+
+
+def test_one_bit_packing_all_byte_values():
+    """Brute force over all 256 bytes: bit i of a byte is element i, 1 meaning -1."""
+    for b in range(256):
+        q = orc.unpack_codes(np.array([b], np.uint8), 8, 1)
+        assert list(q) == [(-1 if (b >> i) & 1 else 1) for i in range(8)]
+        assert orc.pack_codes(q, 1)[0] == b
+
+
+def test_one_bit_block_scale_is_the_pairwise_mean_of_magnitudes():
+    """With block scales the magnitude sent for a block is the mean of |h| -- the value that minimises the squared
+    error sum (h - q mu)^2 of a sign code -- formed by pairwise summation in fp32 over the block's positions."""
+    B = 32
+    cfg = OracleConfig(bits=1, scale_mode=orc.SCALE_BLOCK_ABSMAX, block_size=B, beta=0.5, reset_period=0,
+                       state_fmt=orc.STATE_FP32)
+    # (a) the order of the sum, on values where it shows: sequential summation would lose the three 2^-24
+    g = np.zeros(2 * B + 5, dtype=np.float32)
+    g[0], g[1], g[2], g[3] = 1.0, -(2.0 ** -24), 2.0 ** -24, -(2.0 ** -24)
+    g[B:2 * B] = np.arange(1, B + 1, dtype=np.float32) * np.where(np.arange(B) % 2, -1, 1)   # 1, -2, 3, ...: exact sum 528
+    g[2 * B:] = [4.0, -1.0, 0.5, -0.25, 0.25]                                                # ragged block: 6 / 5
+    state, comm = orc.new_state(cfg, g.size), orc.new_comm(cfg, g.size)
+    (_, _), tr = orc.send_step(cfg, g, state, comm, 1, trace=True)
+    _, scales = orc.comm_views(cfg, g.size, comm)[0]
+    # (1 + 2^-24) rounds to 1 (tie to even); (2^-24 + 2^-24) = 2^-23; 1 + 2^-23 is representable; / 32 is exact
+    assert scales[0] == np.float32((1.0 + 2.0 ** -23) / 32)
+    assert scales[1] == np.float32(528.0 / 32) and scales[2] == np.float32(6.0) / np.float32(5.0)
+    assert np.array_equal(tr["d"], np.where(g < 0, -1, 1).astype(np.float32) * np.repeat(scales, B)[:g.size])
+    # (b) optimality, brute force on a tiny block: no magnitude on a fine grid beats the one sent
+    h = RNG.normal(0, 1e-3, B).astype(np.float32)
+    comm = orc.new_comm(cfg, B)
+    orc.send_step(cfg, h, orc.new_state(cfg, B), comm, 1)
+    mu = float(orc.comm_views(cfg, B, comm)[0][1][0])
+    a = np.abs(h.astype(np.float64))
+    loss = lambda m: float(((a - m) ** 2).sum())
+    grid = np.linspace(0.0, 2 * a.max(), 4001)
+    assert all(loss(mu) <= loss(m) + 1e-18 for m in grid)
+    assert abs(mu - a.mean()) <= 6 * 2.0 ** -24 * a.mean()         # log2(32) + 1 roundings
+    # (c) pairwise summation is exact whenever no partial sum needs rounding, and within log2(B) ulps otherwise
+    d = dyadic(1024, 10, 2.0 ** -20)
+    assert orc.pairwise_sum(np.abs(d)) == float(np.abs(d.astype(np.float64)).sum())
+    r = np.abs(RNG.normal(0, 1, 4096)).astype(np.float32)
+    assert abs(orc.pairwise_sum(r) - float(r.astype(np.float64).sum())) <= 12 * 2.0 ** -24 * float(r.sum())
+
+
+@pytest.mark.parametrize("mode,fmt", [(orc.SCALE_FIXED, orc.STATE_FP32), (orc.SCALE_FIXED, orc.STATE_INT8),
+                                      (orc.SCALE_BLOCK_ABSMAX, orc.STATE_FP32), (orc.SCALE_BLOCK_ABSMAX, orc.STATE_INT8)])
+def test_one_bit_keeps_lemma_1_identity(mode, fmt):
+    """Lemma 1's identity d - g = (e^_k - e~_{k+1}) / beta does not depend on the compressor: it holds for the sign code."""
+    n, beta = 777, 0.25
+    cfg = OracleConfig(bits=1, scale_mode=mode, block_size=64, s=2.0 ** 9, s_e=2.0 ** 13, beta=beta, reset_period=0,
+                       state_fmt=fmt)
+    state, comm = orc.new_state(cfg, n), orc.new_comm(cfg, n)
+    for k in range(1, 5):
+        g = RNG.normal(0, 1e-3, n).astype(np.float32)
+        (_, _), tr = orc.send_step(cfg, g, state, comm, k, trace=True)
+        assert set(np.unique(tr["q"])) <= {-1, 1}
+        lhs = tr["d"].astype(np.float64) - g.astype(np.float64)
+        rhs = (tr["c"].astype(np.float64) - tr["e_new"].astype(np.float64)) / beta
+        assert np.allclose(lhs, rhs, rtol=0, atol=1e-9)
+    with pytest.raises(ValueError):
+        orc.send_step(dataclasses.replace(cfg, rounding=1), g, state, comm, 1)     # a sign code has nothing to round
+
+
+def test_one_bit_non_finite_inputs():
+    cfg = OracleConfig(bits=1, s=2.0 ** 10, s_e=2.0 ** 12, beta=0.5, reset_period=0, state_fmt=orc.STATE_FP32)
+    g = np.array([np.nan, np.inf, -np.inf, 1e-3], dtype=np.float32)
+    state, comm = orc.new_state(cfg, 4), orc.new_comm(cfg, 4)
+    (flags, sat), tr = orc.send_step(cfg, g, state, comm, 1, trace=True)
+    assert flags & orc.FLAG_NONFINITE and sat == 0
+    assert list(tr["q"]) == [1, 1, -1, 1]
+    e = state.view(np.float32)[:4]
+    assert e[0] == 0 and e[1] == 0 and e[2] == 0 and np.isfinite(e).all()
