@@ -79,10 +79,16 @@ typedef enum {
 
 /* Algorithm 1's inputs (s, s_e, T_c, beta), Eq. 1's p, and the storage choices. */
 typedef struct {
-    int32_t bits;            /* p of Eq. 1 for the gradient codes: 2, 4 or 8 (the paper uses 4)   */
+    int32_t bits;            /* p of Eq. 1 for the gradient codes: 2, 4 or 8 (the paper uses 4); 1 = the
+                                sign code of "1-bit LoCo" (named in the paper's GPT-2 experiment, not
+                                defined there): q = -1 if h < 0 else +1, one wire bit per element
+                                (1 = negative), d = q / s, or q x (mean |h| of the block) with block
+                                scales, that mean summed pairwise in fp32 over the block's positions */
     int32_t scale_mode;      /* loco_scale_mode_t                                                 */
-    int32_t block_size;      /* B, BLOCK_ABSMAX only: power of two in [32, 4096]; this build runs
-                                32..256 and returns LOCO_ERR_UNSUPPORTED above                    */
+    int32_t block_size;      /* B, BLOCK_ABSMAX only: power of two in [32, 4096].  Blocks of up to 512
+                                elements run in the fused streaming routine; wider ones are walked block
+                                by block (several passes over the block, served by the caches): same
+                                results, lower speed                                              */
     float   s;               /* Eq. 1 / Eq. 3 scale, FIXED only (> 0, finite)                     */
     float   s_e;             /* Eq. 2 / Eq. 7 scale of the 8-bit error, FIXED only                */
     float   beta;            /* Eq. 5, in [0, 1]: weight of the NEW compression error             */
@@ -92,8 +98,9 @@ typedef struct {
     int32_t grad_dtype;      /* loco_dtype_t of the gradient handed to the send pass              */
     int32_t out_dtype;       /* loco_dtype_t of the averaged gradient the receive pass writes     */
     int32_t num_partitions;  /* P >= 1: parts of the all-to-all layout (Sec. 3.3)                 */
-    int32_t collect_stats;   /* non-zero: count saturated gradient codes (second case of the
-                                rounding lemma) during send; costs a few instructions/element   */
+    int32_t collect_stats;   /* non-zero: count, during send, the gradient codes and the 8-bit error codes
+                                whose nearest integer fell outside their range (second case of the
+                                rounding lemma; the clamp of Eq. 7); costs a few instructions/element */
     float   clip;            /* > 0: clip every element of the local gradient to [-clip, clip] before
                                 step 1 (the element-wise clipping of the Sky-MoE runs in the paper's
                                 experiments; the paper states no threshold); 0 = off.  +-Inf becomes
@@ -224,12 +231,7 @@ int loco_unpack_dequant_reduce_adam(const loco_config_t *cfg, const void *const 
  * owns, so that one bucket's tail overlaps the start-up of the next ones.
  *   - The buckets of one call must be independent of each other (distinct states and buffers), as they run
  *     concurrently.  All of them belong to the current device.
- *   - The first such call on a device creates three non-blocking streams and four events there (driver objects;
- *     no device memory), kept until the process exits; make it outside any stream capture.  Later calls only
- *     record and wait on those events and launch; they may be captured into a CUDA graph like the single calls.
- *   - Calls on one device are serialised on the host while they enqueue their work (they share the events).
- * If one bucket's launch is refused the others are still issued, the streams are joined, and the first error is
- * returned.  count = 0 does nothing.  Errors: as for the single-bucket calls, ARG for null arrays or entries.
+ * count = 0 does nothing.  Errors: as for the single-bucket calls, ARG for null arrays or entries.
  */
 
 /* loco_compensate_quantize_pack for buckets i < count: states[i], d_grads[i], d_comms[i] (HOST arrays of count
@@ -308,12 +310,17 @@ int loco_unpack_dequant_reduce_host_noalloc(const loco_config_t *cfg, const void
                                             int32_t partition_count, void *h_out, void *stream);
 
 /*
- * Read the status word accumulated by the send passes of this handle since init/reset.
+ * Read the status words accumulated by the send passes of this handle since init/reset.
  * SYNCHRONISES `stream` (the one the passes ran on).  n_saturated counts gradient codes
- * whose nearest integer fell outside the p-bit range; it stays 0 unless collect_stats.
- * Either output pointer may be NULL.
+ * whose nearest integer fell outside the p-bit range (second case of the rounding lemma);
+ * n_saturated_state counts 8-bit error codes that Eq. 7's compressor clamped to [-128, 127]
+ * (global s_e only: a block-scaled state cannot saturate; with STATE_FP32_Q8COMP the 8-bit
+ * image is formed, and counted, when the error is next used).  Both stay 0 unless
+ * collect_stats; the sign code has no range and counts nothing.  Any output pointer may be NULL.
  */
 int loco_last_status(loco_state_t *st, uint32_t *flags, uint64_t *n_saturated, void *stream);
+int loco_status_counters(loco_state_t *st, uint32_t *flags, uint64_t *n_saturated,
+                         uint64_t *n_saturated_state, void *stream);
 
 /*
  * Diagnostic for the block-scaled extension (no counterpart in the paper).  The send kernel forms a block's scale

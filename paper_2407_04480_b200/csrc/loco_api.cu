@@ -44,10 +44,11 @@ inline uint64_t round_up(uint64_t x, uint64_t m) { return (x + m - 1) / m * m; }
 inline bool is_pow2(uint64_t x) { return x && !(x & (x - 1)); }
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int ilog2(uint32_t x) { int l = 0; while ((1u << l) < x) ++l; return l; }
+constexpr size_t kStatusBytes = 32;      // device status words of a handle: flags, saturated codes, saturated error codes, spare
 
 int check_config(const loco_config_t *c) {
     if (!c) return LOCO_ERR_ARG;
-    if (c->bits != 2 && c->bits != 4 && c->bits != 8) return LOCO_ERR_ARG;
+    if (c->bits != 1 && c->bits != 2 && c->bits != 4 && c->bits != 8) return LOCO_ERR_ARG;
     if (c->scale_mode != LOCO_SCALE_FIXED && c->scale_mode != LOCO_SCALE_BLOCK_ABSMAX) return LOCO_ERR_ARG;
     if (c->state_fmt < LOCO_STATE_INT8 || c->state_fmt > LOCO_STATE_FP32_Q8COMP) return LOCO_ERR_ARG;
     if (c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX) {
@@ -66,7 +67,7 @@ int check_config(const loco_config_t *c) {
     if (c->num_partitions < 1 || c->num_partitions > 65535) return LOCO_ERR_ARG;
     if (!(c->clip >= 0.0f) || !std::isfinite(c->clip)) return LOCO_ERR_ARG;
     if (c->rounding != LOCO_ROUND_NEAREST && c->rounding != LOCO_ROUND_STOCHASTIC) return LOCO_ERR_ARG;
-    if (c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX && c->block_size > 256) return LOCO_ERR_UNSUPPORTED;
+    if (c->bits == 1 && c->rounding != LOCO_ROUND_NEAREST) return LOCO_ERR_ARG;      // a sign code has nothing to round
     return LOCO_OK;
 }
 
@@ -165,15 +166,15 @@ int kernel_mode(const loco_config_t *c) {
     return c->scale_mode == LOCO_SCALE_BLOCK_ABSMAX ? MODE_BLOCK : MODE_FIXED;
 }
 
+// SMs of the current device (asked for once per device)
 int num_sms() {
-    static int sms = 0;
-    if (sms == 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) return 148;
-        sms = v;
-    }
-    return sms;
+    static std::atomic<int> sms[64];
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0) { cudaGetLastError(); return 148; }
+    if (dev < 64 && (v = sms[dev].load(std::memory_order_relaxed)) > 0) return v;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) { cudaGetLastError(); return 148; }
+    if (dev < 64) sms[dev].store(v, std::memory_order_relaxed);
+    return v;
 }
 
 SendKernel pick_send(const loco_config_t *c, int mode, int var) {
@@ -213,6 +214,8 @@ struct loco_state {
     int device;
     int mode;
     SendFn send_fn;
+    SendMultiFn send_multi_fn;      // the same kernel walking several buckets per launch
+    int send_var;
     int send_smem_bytes;            // dynamic shared memory of the send kernel (its cp.async ring)
     int send_ctas_per_sm;
     Layout layout;
@@ -283,14 +286,22 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
     st->de = st->dq;
     st->fast = 1;
     if (st->mode == MODE_FIXED) {
-        const int half = 1 << (cfg->bits - 1);
-        st->dq = choose_dec(cfg->s, -half, half - 1, half);
+        if (cfg->bits == 1) {
+            // sign code: d = +-fl(1/s), nothing to prove; the magnitude must be a usable number
+            const volatile float vinv = 1.0f / cfg->s;
+            st->dq = DecChoice{(std::isfinite(vinv) && vinv != 0.0f) ? DEC_FMA : DEC_DIVIDE, 0.0f, 0.0f, vinv};
+        } else {
+            const int half = 1 << (cfg->bits - 1);
+            st->dq = choose_dec(cfg->s, -half, half - 1, half);
+        }
         if (cfg->state_fmt == LOCO_STATE_INT8 || cfg->state_fmt == LOCO_STATE_FP32_Q8COMP)
             st->de = choose_dec(cfg->s_e, -128, 127, 128);
         st->fast = (st->dq.mode != DEC_DIVIDE && st->de.mode != DEC_DIVIDE) ? 1 : 0;
         // the fast routine tests only g for NaN / Inf when the state is 8-bit: dec(e) must be too small to push a
         // finite g to infinity (|e / s_e| <= 128 / s_e < 2^100)
         if (cfg->state_fmt == LOCO_STATE_INT8 && !(cfg->s_e > 1e-28f)) st->fast = 0;
+    } else if (cfg->block_size > kWide) {
+        st->fast = 0;           // a block wider than a wide row: the careful routine walks it
     }
     {
         int var = VAR_GENERAL;
@@ -307,6 +318,8 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
         }
         const SendKernel k = pick_send(cfg, st->mode, var);
         st->send_fn = k.fn;
+        st->send_multi_fn = k.multi_fn;
+        st->send_var = var;
         st->send_smem_bytes = k.smem_bytes;
     }
     st->send_ctas_per_sm = 1;
@@ -314,13 +327,13 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
     if (cudaGetDevice(&st->device) != cudaSuccess) { delete st; return LOCO_ERR_CUDA; }
     int occ = 0;
     // the ring wants most of the SM's shared memory (3 CTAs x up to 72 KB)
-    if (cudaFuncSetAttribute(reinterpret_cast<const void *>(st->send_fn), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             st->send_smem_bytes) != cudaSuccess ||
-        cudaFuncSetAttribute(reinterpret_cast<const void *>(st->send_fn), cudaFuncAttributePreferredSharedMemoryCarveout,
-                             cudaSharedmemCarveoutMaxShared) != cudaSuccess) {
-        cudaGetLastError();
-        delete st;
-        return LOCO_ERR_CUDA;
+    for (const void *fn : {reinterpret_cast<const void *>(st->send_fn), reinterpret_cast<const void *>(st->send_multi_fn)}) {
+        if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, st->send_smem_bytes) != cudaSuccess ||
+            cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess) {
+            cudaGetLastError();
+            delete st;
+            return LOCO_ERR_CUDA;
+        }
     }
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, st->send_fn, kThreads, static_cast<size_t>(st->send_smem_bytes)) != cudaSuccess || occ < 1) {
         cudaGetLastError();
@@ -328,13 +341,13 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
         return LOCO_ERR_CUDA;
     }
     st->send_ctas_per_sm = occ;
-    if (cudaMalloc(reinterpret_cast<void **>(&st->d_status), 16) != cudaSuccess) {
+    if (cudaMalloc(reinterpret_cast<void **>(&st->d_status), kStatusBytes) != cudaSuccess) {
         cudaGetLastError();
         delete st;
         return LOCO_ERR_CUDA;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemsetAsync(st->d_status, 0, 16, s);
+    cudaError_t e = cudaMemsetAsync(st->d_status, 0, kStatusBytes, s);
     if (e == cudaSuccess && need > 0) e = cudaMemsetAsync(d_state, 0, need, s);   // e~_0 = 0
     if (e != cudaSuccess) {
         cudaGetLastError();
@@ -349,7 +362,7 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
 int loco_state_reset(loco_state_t *st, void *stream) {
     if (!st) return LOCO_ERR_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaMemsetAsync(st->d_status, 0, 16, s);
+    cudaError_t e = cudaMemsetAsync(st->d_status, 0, kStatusBytes, s);
     if (e == cudaSuccess && st->state_bytes > 0) e = cudaMemsetAsync(st->d_state, 0, st->state_bytes, s);
     if (e != cudaSuccess) { cudaGetLastError(); return LOCO_ERR_CUDA; }
     return LOCO_OK;
@@ -367,6 +380,52 @@ int loco_state_destroy(loco_state_t *st) {
 
 namespace {
 
+// Algorithm 1's scalars for iteration step_k, as the kernels take them.
+void fill_common(const loco_state_t *st, int64_t step_k, SendCommon &C) {
+    const loco_config_t &c = st->cfg;
+    std::memset(&C, 0, sizeof(C));
+    C.s = c.s;
+    C.s_e = c.s_e;
+    C.beta = c.beta;
+    {
+        const volatile float omb = 1.0f - c.beta;    // (1 - beta), rounded once to fp32
+        C.omb = omb;
+    }
+    C.inv_s = st->dq.inv;
+    C.inv_se = st->de.inv;
+    C.dq_a = st->dq.a; C.dq_b = st->dq.b; C.dq_mode = st->dq.mode;
+    C.de_a = st->de.a; C.de_b = st->de.b; C.de_mode = st->de.mode;
+    C.fast = st->fast;
+    C.block_log2 = c.scale_mode == LOCO_SCALE_BLOCK_ABSMAX ? ilog2(static_cast<uint32_t>(c.block_size)) : 0;
+    C.reset = (c.reset_period > 0 && (step_k % static_cast<int64_t>(c.reset_period)) == 0) ? 1 : 0;
+    C.collect_stats = c.collect_stats ? 1 : 0;
+    C.clip = c.clip;
+    C.stochastic = c.rounding == LOCO_ROUND_STOCHASTIC ? 1 : 0;
+    C.seed_lo = c.seed_lo; C.seed_hi = c.seed_hi;
+    C.k_lo = static_cast<unsigned>(static_cast<uint64_t>(step_k));
+    C.k_hi = static_cast<unsigned>(static_cast<uint64_t>(step_k) >> 32);
+}
+
+void fill_bucket(const loco_state_t *st, const void *d_grad, void *d_comm, SendBucket &B) {
+    B.grad = d_grad;
+    B.state = st->d_state;
+    B.comm = static_cast<uint8_t *>(d_comm);
+    B.status = st->d_status;
+    B.n = st->n;
+    B.lp = st->layout.lp;
+    B.stride = st->layout.stride;
+    B.unit_begin = 0;
+    B.units_per_part = 0;
+}
+
+// The handle's kernels were prepared (shared-memory size, occupancy) on the device that was current at
+// loco_state_init, and its buffers live there: a call with another device current is refused.
+int check_device(const loco_state_t *st) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return LOCO_ERR_CUDA; }
+    return dev == st->device ? LOCO_OK : LOCO_ERR_ARG;
+}
+
 // The send pass.  Its partitions go to d_comm + j * stride, or, with d_part_dst, to d_part_dst[j].
 int send_launch(loco_state_t *st, const void *d_grad, void *d_comm, void *const *d_part_dst, int64_t step_k,
                 void *stream) {
@@ -376,6 +435,8 @@ int send_launch(loco_state_t *st, const void *d_grad, void *d_comm, void *const 
     if (st->n == 0) return LOCO_OK;
     if (!d_grad || (!d_comm && !d_part_dst)) return LOCO_ERR_ARG;
     if (!aligned16(d_grad) || !aligned16(d_comm)) return LOCO_ERR_ALIGN;
+    const int rc = check_device(st);
+    if (rc != LOCO_OK) return rc;
     SendParams P;
     std::memset(&P, 0, sizeof(P));
     if (d_part_dst) {
@@ -386,37 +447,53 @@ int send_launch(loco_state_t *st, const void *d_grad, void *d_comm, void *const 
         }
         P.scatter = 1;
     }
-    P.grad = d_grad;
-    P.state = st->d_state;
-    P.comm = static_cast<uint8_t *>(d_comm);
-    P.n = st->n;
-    P.lp = st->layout.lp;
-    P.stride = st->layout.stride;
-    P.code_bytes = st->layout.code_bytes;
-    P.state_scale_off = round_up(st->n, 256);
-    P.s = c.s;
-    P.s_e = c.s_e;
-    P.inv_s = st->dq.inv;
-    P.inv_se = st->de.inv;
-    P.dq_a = st->dq.a; P.dq_b = st->dq.b; P.dq_mode = st->dq.mode;
-    P.de_a = st->de.a; P.de_b = st->de.b; P.de_mode = st->de.mode;
-    P.fast = st->fast;
-    P.clip = c.clip;
-    P.stochastic = c.rounding == LOCO_ROUND_STOCHASTIC ? 1 : 0;
-    P.seed_lo = c.seed_lo; P.seed_hi = c.seed_hi;
-    P.k_lo = static_cast<unsigned>(static_cast<uint64_t>(step_k)); P.k_hi = static_cast<unsigned>(static_cast<uint64_t>(step_k) >> 32);
-    P.beta = c.beta;
-    {
-        const volatile float omb = 1.0f - c.beta;    // (1 - beta), rounded once to fp32
-        P.omb = omb;
-    }
-    P.block_log2 = c.scale_mode == LOCO_SCALE_BLOCK_ABSMAX ? ilog2(static_cast<uint32_t>(c.block_size)) : 0;
-    P.reset = (c.reset_period > 0 && (step_k % static_cast<int64_t>(c.reset_period)) == 0) ? 1 : 0;
-    P.collect_stats = c.collect_stats ? 1 : 0;
-    P.status = st->d_status;
-    const uint64_t rows = P.lp / kRow;
+    fill_common(st, step_k, P.c);
+    fill_bucket(st, d_grad, d_comm, P.b);
+    const uint64_t rows = P.b.lp / kRow;
     dim3 grid(grid_x_for(rows, c.num_partitions, st->send_ctas_per_sm), static_cast<unsigned>(c.num_partitions), 1);
     st->send_fn<<<grid, kThreads, static_cast<size_t>(st->send_smem_bytes), static_cast<cudaStream_t>(stream)>>>(P);
+    if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;
+    g_launches.fetch_add(1);
+    return LOCO_OK;
+}
+
+// Elements of a work unit of the multi-bucket kernel, and units per partition.
+inline uint64_t unit_elems_of(const loco_config_t &c) {
+    return (c.scale_mode == LOCO_SCALE_BLOCK_ABSMAX && c.block_size > kWide) ? static_cast<uint64_t>(c.block_size) : static_cast<uint64_t>(kWide);
+}
+
+bool same_send_setup(const loco_state_t *a, const loco_state_t *b) {
+    return std::memcmp(&a->cfg, &b->cfg, sizeof(loco_config_t)) == 0 && a->send_multi_fn == b->send_multi_fn &&
+           a->device == b->device && a->fast == b->fast;
+}
+
+// Buckets [lo, hi) of a multi-bucket call, all of one configuration, in one launch of the table-driven kernel.
+int send_multi_launch(loco_state_t *const *states, const void *const *d_grads, void *const *d_comms, int lo, int hi,
+                      int64_t step_k, void *stream) {
+    static thread_local SendMultiParams P;             // 32 KB: not on the stack
+    const loco_state_t *first = states[lo];
+    fill_common(first, step_k, P.c);
+    const uint64_t ue = unit_elems_of(first->cfg);
+    P.parts = first->cfg.num_partitions;
+    P.unit_elems = static_cast<unsigned>(ue);
+    P.count = 0;
+    uint64_t units = 0;
+    for (int i = lo; i < hi; ++i) {
+        const loco_state_t *st = states[i];
+        if (st->n == 0) continue;
+        SendBucket &B = P.b[P.count++];
+        fill_bucket(st, d_grads[i], d_comms[i], B);
+        const uint64_t upp = (st->layout.lp + ue - 1) / ue;
+        B.unit_begin = static_cast<unsigned>(units);
+        B.units_per_part = static_cast<unsigned>(upp);
+        units += upp * static_cast<uint64_t>(P.parts);
+    }
+    if (P.count == 0) return LOCO_OK;
+    P.total_units = static_cast<unsigned>(units);
+    const uint64_t budget = static_cast<uint64_t>(num_sms()) * static_cast<uint64_t>(first->send_ctas_per_sm);
+    const uint64_t want = (units + kWarps - 1) / kWarps;
+    const unsigned gx = static_cast<unsigned>(want < budget ? want : budget);
+    first->send_multi_fn<<<gx, kThreads, static_cast<size_t>(first->send_smem_bytes), static_cast<cudaStream_t>(stream)>>>(P);
     if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;
     g_launches.fetch_add(1);
     return LOCO_OK;
@@ -490,7 +567,13 @@ int reduce_launch(const loco_config_t *cfg, const void *const *d_packed, int32_t
     P.inv_s = 0.0f;
     P.int_path = 0;
     P.out_align32 = (reinterpret_cast<uintptr_t>(d_out) & 31u) == 0 ? 1 : 0;
-    if (mode == MODE_FIXED) {
+    if (mode == MODE_FIXED && cfg->bits == 1) {
+        // sign code: d = +-fl(1/s), which is (+-1) / s exactly as the division gives it
+        const volatile float vinv = 1.0f / cfg->s;
+        P.inv_s = vinv;
+        P.gen_mul = vinv;
+        P.gen_mode = 0;
+    } else if (mode == MODE_FIXED) {
         const int half = 1 << (cfg->bits - 1);
         {
             const volatile float vinv = 1.0f / cfg->s;
@@ -551,22 +634,28 @@ int reduce_launch(const loco_config_t *cfg, const void *const *d_packed, int32_t
         cudaGetLastError();
         return LOCO_ERR_CUDA;
     }
-    static int occ_cache[64][2][3][2][4][2] = {};
-    int &occ = occ_cache[dev][cfg->out_dtype == LOCO_BF16][cfg->bits == 2 ? 0 : (cfg->bits == 4 ? 1 : 2)][mode][path][ad != nullptr];
-    if (occ == 0) {
-        int v = 0;
-        if (smem > 0) {
-            if (cudaFuncSetAttribute(reinterpret_cast<const void *>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-                cudaFuncSetAttribute(reinterpret_cast<const void *>(fn), cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess) {
+    static int occ_cache[64][2][4][2][4][2] = {};
+    static std::mutex occ_mu;
+    int occ = 0;
+    {
+        std::lock_guard<std::mutex> lock(occ_mu);
+        int &slot = occ_cache[dev][cfg->out_dtype == LOCO_BF16][cfg->bits == 1 ? 0 : (cfg->bits == 2 ? 1 : (cfg->bits == 4 ? 2 : 3))][mode][path][ad != nullptr];
+        if (slot == 0) {
+            int v = 0;
+            if (smem > 0) {
+                if (cudaFuncSetAttribute(reinterpret_cast<const void *>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+                    cudaFuncSetAttribute(reinterpret_cast<const void *>(fn), cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess) {
+                    cudaGetLastError();
+                    return LOCO_ERR_CUDA;
+                }
+            }
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, fn, kThreads, smem) != cudaSuccess || v < 1) {
                 cudaGetLastError();
                 return LOCO_ERR_CUDA;
             }
+            slot = v;
         }
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, fn, kThreads, smem) != cudaSuccess || v < 1) {
-            cudaGetLastError();
-            return LOCO_ERR_CUDA;
-        }
-        occ = v;
+        occ = slot;
     }
     const uint64_t rows = (L.lp + kWide - 1) / kWide;
     dim3 grid(grid_x_for(rows, partition_count, occ), static_cast<unsigned>(partition_count), 1);
@@ -663,13 +752,40 @@ extern "C" {
 
 int loco_compensate_quantize_pack_multi(loco_state_t *const *states, const void *const *d_grads, void *const *d_comms,
                                         int32_t count, int64_t step_k, void *stream) {
-    if (count < 0 || (count > 0 && (!states || !d_grads || !d_comms))) return LOCO_ERR_ARG;
+    if (count < 0 || step_k < 0 || (count > 0 && (!states || !d_grads || !d_comms))) return LOCO_ERR_ARG;
     if (count == 0) return LOCO_OK;
-    for (int32_t i = 0; i < count; ++i)
+    // every argument is checked before anything is launched
+    for (int32_t i = 0; i < count; ++i) {
         if (!states[i]) return LOCO_ERR_ARG;
-    return fan_out(count, stream, [&](int32_t i, void *s) {
-        return loco_compensate_quantize_pack(states[i], d_grads[i], d_comms[i], step_k, s);
-    });
+        if (states[i]->n == 0) continue;
+        if (!d_grads[i] || !d_comms[i]) return LOCO_ERR_ARG;
+        if (!aligned16(d_grads[i]) || !aligned16(d_comms[i])) return LOCO_ERR_ALIGN;
+        const int rc = check_device(states[i]);
+        if (rc != LOCO_OK) return rc;
+    }
+    // consecutive buckets of one configuration share a launch: as many as the kernel's table holds, and no more work
+    // units than a 32-bit counter (with room for the grid's stride) can number
+    int rc = LOCO_OK;
+    int32_t lo = 0;
+    while (lo < count) {
+        int32_t hi = lo;
+        uint64_t units = 0;
+        const uint64_t ue = unit_elems_of(states[lo]->cfg);
+        while (hi < count && hi - lo < kMaxMulti && same_send_setup(states[lo], states[hi])) {
+            const uint64_t u = ((states[hi]->layout.lp + ue - 1) / ue) * static_cast<uint64_t>(states[hi]->cfg.num_partitions);
+            if (hi > lo && units + u > 0xF0000000ull) break;
+            units += u;
+            ++hi;
+        }
+        int r;
+        if (units > 0xF0000000ull)       // a single bucket beyond the counter's range: the one-bucket kernel (64-bit indices)
+            r = send_launch(states[lo], d_grads[lo], d_comms[lo], nullptr, step_k, stream);
+        else
+            r = send_multi_launch(states, d_grads, d_comms, lo, hi, step_k, stream);
+        if (r != LOCO_OK && rc == LOCO_OK) rc = r;
+        lo = hi;
+    }
+    return rc;
 }
 
 int loco_unpack_dequant_reduce_multi(const loco_config_t *cfg, const void *const *const *d_packed, int32_t num_workers,
@@ -832,18 +948,24 @@ int loco_selfcheck_block_division(uint64_t *mismatches) {
     return LOCO_OK;
 }
 
-int loco_last_status(loco_state_t *st, uint32_t *flags, uint64_t *n_saturated, void *stream) {
+int loco_status_counters(loco_state_t *st, uint32_t *flags, uint64_t *n_saturated, uint64_t *n_saturated_state,
+                         void *stream) {
     if (!st) return LOCO_ERR_ARG;
-    unsigned long long host[2] = {0, 0};
+    unsigned long long host[4] = {0, 0, 0, 0};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(host, st->d_status, 16, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+    if (cudaMemcpyAsync(host, st->d_status, kStatusBytes, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
         cudaStreamSynchronize(s) != cudaSuccess) {
         cudaGetLastError();
         return LOCO_ERR_CUDA;
     }
     if (flags) *flags = static_cast<uint32_t>(host[0]);
     if (n_saturated) *n_saturated = host[1];
+    if (n_saturated_state) *n_saturated_state = host[2];
     return LOCO_OK;
+}
+
+int loco_last_status(loco_state_t *st, uint32_t *flags, uint64_t *n_saturated, void *stream) {
+    return loco_status_counters(st, flags, n_saturated, nullptr, stream);
 }
 
 }  // extern "C"

@@ -10,7 +10,8 @@
 namespace loco {
 
 using SendFn = void (*)(const SendParams);
-struct SendKernel { SendFn fn; int smem_bytes; };           // smem_bytes: the kernel's cp.async ring
+using SendMultiFn = void (*)(const SendMultiParams);
+struct SendKernel { SendFn fn; SendMultiFn multi_fn; int smem_bytes; };   // one bucket / several buckets per launch; smem_bytes: the cp.async ring
 
 using ReduceFn = void (*)(const ReduceParams);
 struct ReduceKernel { ReduceFn fn; int smem_bytes; };       // smem_bytes: the kernel's cp.async ring (0: none)

@@ -48,17 +48,10 @@ constexpr unsigned kFlagNonFinite = 1u;
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kMaxScatter = 64;    // most partitions a scattering send pass can address
 
-struct SendParams {
-    const void *grad;
-    void *state;
-    uint8_t *comm;
-    unsigned long long n;            // bucket elements
-    unsigned long long lp;           // elements per partition (multiple of 256 and of B)
-    unsigned long long stride;       // bytes per partition
-    unsigned long long code_bytes;   // bytes of the code area of a partition
-    unsigned long long state_scale_off;   // byte offset of the state scales (BLOCK + INT8)
+// Algorithm 1's scalars and the forms the host chose for the decompressors: the same for every bucket of a call.
+struct SendCommon {
     float s, s_e, beta, omb;
-    float inv_s, inv_se;             // fl(1/s), fl(1/s_e) for the Newton-Raphson form
+    float inv_s, inv_se;             // fl(1/s), fl(1/s_e) for the Newton-Raphson form (inv_s is also the 1-bit magnitude)
     float dq_a, dq_b;                // DEC_FMA: dec(q; s)   = fma(kMagic + 2^(p-1) + q, dq_a, dq_b)
     float de_a, de_b;                // DEC_FMA: dec(e; s_e) = fma(kMagic + 128 + e,     de_a, de_b)
     int dq_mode, de_mode;            // DEC_* chosen by the host for s and for s_e
@@ -70,10 +63,41 @@ struct SendParams {
     int stochastic;                  // stochastic rounding of the gradient codes (extension)
     unsigned seed_lo, seed_hi;       // key of its Philox stream
     unsigned k_lo, k_hi;             // the iteration counter, part of the Philox counter
-    unsigned long long *status;      // [0] flags, [1] saturated codes
+};
+
+// One bucket of a send pass.  Derived sizes: code bytes of a partition = lp * BITS / 8, byte offset of the state
+// scales (BLOCK + INT8) = n rounded up to 256.
+struct SendBucket {
+    const void *grad;
+    void *state;
+    uint8_t *comm;
+    unsigned long long *status;      // [0] flags, [1] saturated gradient codes, [2] saturated 8-bit error codes
+    unsigned long long n;            // bucket elements
+    unsigned long long lp;           // elements per partition (multiple of 256 and of B)
+    unsigned long long stride;       // bytes per partition
+    unsigned unit_begin;             // multi-bucket launches: first work unit of this bucket in the launch
+    unsigned units_per_part;         // multi-bucket launches: work units per partition
+};
+
+struct SendParams {
+    SendCommon c;
+    SendBucket b;
     int scatter;                     // 1: partition j is written to part_dst[j] instead of comm + j * stride
     uint8_t *part_dst[kMaxScatter];  // destinations of the partitions (this GPU's memory or a peer's)
 };
+
+// Several buckets in one launch: the table travels as a kernel parameter (the parameter space of sm_70 and later
+// holds 32,764 bytes), so nothing is allocated and a captured launch carries its own copy.
+constexpr int kMaxMulti = 448;
+struct SendMultiParams {
+    SendCommon c;
+    int count;                       // buckets
+    int parts;                       // partitions per bucket
+    unsigned total_units;            // work units of all buckets
+    unsigned unit_elems;             // elements of a work unit: 512, or B when B > 512
+    SendBucket b[kMaxMulti];
+};
+static_assert(sizeof(SendMultiParams) <= 32764, "kernel parameter space");
 
 struct ReduceParams {
     const uint8_t *parts[64];        // partition `first` of each worker
@@ -177,6 +201,20 @@ __device__ __forceinline__ unsigned pack4_bytes(unsigned a, unsigned b, unsigned
     return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
 }
 
+// (a & b) | c in one instruction (the mask and the exponent live in registers)
+__device__ __forceinline__ unsigned and_or(unsigned a, unsigned b, unsigned c) {
+    unsigned d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+// (a ^ b) & c in one instruction
+__device__ __forceinline__ unsigned xor_and(unsigned a, unsigned b, unsigned c) {
+    unsigned d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x28;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 // Streaming accesses: every byte of both passes is touched exactly once.
 __device__ __forceinline__ uint4 ld_stream16(const void *p) { return __ldcs(static_cast<const uint4 *>(p)); }
 __device__ __forceinline__ uint2 ld_stream8(const void *p) { return __ldcs(static_cast<const uint2 *>(p)); }
@@ -184,119 +222,28 @@ __device__ __forceinline__ unsigned ld_stream4(const void *p) { return __ldcs(st
 __device__ __forceinline__ void st_stream16(void *p, uint4 v) { __stcs(static_cast<uint4 *>(p), v); }
 __device__ __forceinline__ void st_stream8(void *p, uint2 v) { __stcs(static_cast<uint2 *>(p), v); }
 __device__ __forceinline__ void st_stream4(void *p, unsigned v) { __stcs(static_cast<unsigned *>(p), v); }
+__device__ __forceinline__ void st_stream2(void *p, uint16_t v) { __stcs(static_cast<unsigned short *>(p), v); }
 
 // ------------------------------------------------------------------------------------------
-// send, careful routine: Algorithm 1 steps 1-2 on 8 elements held by one lane, every operation written
-// out as the paper states it (IEEE division for the decompressor), any value accepted.
+// send, careful routine: Algorithm 1 steps 1-2 with every operation written out as the paper states it
+// (IEEE division for the decompressor), any value accepted, any block size.  It serves the rows the fast
+// routine cannot take: partial and padding rows, rows that hold a NaN or an Inf, blocks wider than a wide row.
 //
-//  g      gradient values (already fp32)
-//  prev   e~_k as Eq. 5 sees it;  c  what is added to g (dec(e_k), e~_k, or dec(comp(e~_k)))
-//  valid  number of leading elements that exist
-//  Outputs: code bits (low byte of each word = code), e_new = e~_{k+1}, scale of the block.
-template <int STATE, int BITS, int MODE, bool STOCH>
-__device__ __forceinline__ void send_core(const SendParams &P, const float (&g)[8], const float (&c)[8],
-                                          const float (&prev)[8], int valid, int lanes_per_block, unsigned long long i0,
-                                          unsigned (&code)[8], float (&e_new)[8], float &scale,
-                                          unsigned &nonfinite, unsigned &saturated) {
-    constexpr float lo = QRange<BITS>::lo, hi = QRange<BITS>::hi;
-    float h[8];
+// Its unit is `nrows` consecutive rows of 256 elements (8 per lane) of one partition: one row when a block fits
+// a row (the blocks of the row are then shared by groups of lanes), or the B / 256 rows of one block.  A block
+// that spans several rows is walked up to three times -- block statistic of h; codes, new error and its
+// statistic; 8-bit error codes -- recomputing h from the inputs each time (nothing of the state is overwritten
+// before its last read), so that no register or shared memory has to hold a whole block.
+
+struct CarefulCounts { unsigned saturated, state_saturated, nonfinite; };
+
+// Eight elements of one lane: the gradient, what is added to it, e~_k of Eq. 5, h and whether h is finite.
+struct CarefulVals {
+    float c[8], prev[8], h[8];
     bool fin[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        h[j] = __fadd_rn(g[j], c[j]);                       // step 1 / Eq. 2
-        fin[j] = fabsf(h[j]) <= kFltMax;                    // false for NaN and +-Inf
-        if (!fin[j] && j < valid) nonfinite = 1u;
-    }
-    float mult = P.s;
-    scale = 0.0f;
-    if (MODE == MODE_BLOCK) {
-        float amax = 0.0f;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fin[j] ? fabsf(h[j]) : 0.0f);
-        amax = warp_group_max(amax, lanes_per_block);
-        scale = amax > 0.0f ? __fdiv_rn(amax, hi) : 0.0f;
-        mult = amax > 0.0f ? __fdiv_rn(hi, amax) : 0.0f;
-    }
-    float u8[8];
-    if (STOCH) {                                            // i0 is a multiple of 8: one half of a block of 16
-        const uint4 r = sr_block(i0 >> 4, P.k_lo, P.k_hi, P.seed_lo, P.seed_hi);
-        const bool upper = ((i0 >> 3) & 1ull) != 0ull;
-        const unsigned w0 = upper ? r.z : r.x, w1 = upper ? r.w : r.y;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) { u8[j] = sr_dither(w0, j); u8[4 + j] = sr_dither(w1, j); }
-    }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const float hq = (h[j] != h[j]) ? 0.0f : h[j];      // NaN is sent as code 0
-        float y = __fmul_rn(hq, mult);                      // h x s of Eq. 1
-        if (!fin[j]) y = hq;                                // +-Inf saturates whatever the scale
-        float r;
-        if (STOCH && fin[j]) {                              // floor(y + u): up with probability frac(y)
-            const float fl = floorf(__fadd_rn(y, u8[j]));
-            if (P.collect_stats && j < valid && (fl < lo || fl > hi)) saturated += 1u;
-            r = fminf(fmaxf(fl, lo), hi);
-            code[j] = static_cast<unsigned>(__float2int_rn(r));
-        } else {
-            r = round_clamp(y, lo, hi, code[j]);            // round_p-bit
-        }
-        float d;                                            // step 2: dec(q; s)
-        if (MODE == MODE_FIXED) d = __fdiv_rn(r, P.s);
-        else d = __fmul_rn(r, scale);
-        const float delta = fin[j] ? __fsub_rn(h[j], d) : 0.0f;
-        e_new[j] = __fadd_rn(__fmul_rn(P.omb, prev[j]), __fmul_rn(P.beta, delta));   // Eq. 5
-        if (MODE != MODE_BLOCK && P.collect_stats && !STOCH) {
-            // nearest integer outside the range: y >= hi + 1/2 (hi is odd, the tie goes up and out)
-            // or y < lo - 1/2 (lo is even, the tie stays in)
-            if (fin[j] && j < valid && (y >= hi + 0.5f || y < lo - 0.5f)) saturated += 1u;
-        }
-    }
-}
-
-// Eq. 7 for 8 elements in the int8 format: codes of e~_{k+1}.
-template <int MODE>
-__device__ __forceinline__ void state_compress8(const SendParams &P, const float (&e_new)[8], int lanes_per_block,
-                                                unsigned (&ebits)[8], float &escale) {
-    float mult = P.s_e;
-    escale = 0.0f;
-    if (MODE == MODE_BLOCK) {
-        float amax = 0.0f;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) amax = fmaxf(amax, fabsf(e_new[j]));
-        amax = warp_group_max(amax, lanes_per_block);
-        escale = amax > 0.0f ? __fdiv_rn(amax, 127.0f) : 0.0f;
-        mult = amax > 0.0f ? __fdiv_rn(127.0f, amax) : 0.0f;
-    }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        (void)round_clamp(__fmul_rn(e_new[j], mult), -128.0f, 127.0f, ebits[j]);
-    }
-}
-
-// Compensation value and Eq. 5's previous error for 8 elements, from the stored state.
-template <int STATE, int MODE>
-__device__ __forceinline__ void decode_state8(const SendParams &P, uint2 e8, const float (&ef)[8], float sscale,
-                                              float (&c)[8], float (&prev)[8]) {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        if (STATE == ST_INT8) {
-            const float ei = byte_to_float(j < 4 ? e8.x : e8.y, j & 3);
-            if (MODE == MODE_FIXED) c[j] = __fdiv_rn(ei, P.s_e);              // dec(e_k; s_e), Eq. 2
-            else c[j] = __fmul_rn(ei, sscale);
-            prev[j] = c[j];
-        } else if (STATE == ST_FP32) {
-            c[j] = ef[j];
-            prev[j] = ef[j];
-        } else if (STATE == ST_Q8COMP) {
-            prev[j] = ef[j];
-            unsigned bits;
-            const float r = round_clamp(__fmul_rn(ef[j], P.s_e), -128.0f, 127.0f, bits);
-            c[j] = __fdiv_rn(r, P.s_e);
-        } else {
-            c[j] = 0.0f;
-            prev[j] = 0.0f;
-        }
-    }
-}
+    unsigned long long i0;          // bucket index of the lane's first element
+    int valid;                      // leading elements that exist
+};
 
 template <int BITS>
 __device__ __forceinline__ void store_codes8(uint8_t *dst, const unsigned (&code)[8]) {
@@ -310,90 +257,291 @@ __device__ __forceinline__ void store_codes8(uint8_t *dst, const unsigned (&code
 #pragma unroll
         for (int j = 0; j < 8; ++j) w |= (code[j] & 0xfu) << (4 * j);
         *reinterpret_cast<unsigned *>(dst) = w;
-    } else {
+    } else if (BITS == 2) {
         unsigned w = 0;
 #pragma unroll
         for (int j = 0; j < 8; ++j) w |= (code[j] & 0x3u) << (2 * j);
         *reinterpret_cast<uint16_t *>(dst) = static_cast<uint16_t>(w);
+    } else {
+        unsigned w = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) w |= (code[j] & 0x1u) << j;
+        *dst = static_cast<uint8_t>(w);
     }
 }
 
-// One warp row (256 elements starting at partition-local offset `o`, bucket element i0 = part*lp + o),
-// careful routine.  Elements >= n are treated as absent (code 0, no state).  Reads its inputs itself.
-// Out of line, reading the kernel's parameters in place (they are __grid_constant__, so their address can be taken
-// without a local copy), so that the fast routine's register allocation is not disturbed by this rarely taken path.  Returns the number of saturated
-// codes of this lane, plus 2^31 if the lane met a non-finite value.
-template <int GRAD, int STATE, int BITS, int MODE, bool STOCH>
-__device__ __noinline__ unsigned send_row_careful(const SendParams &P, unsigned long long part, unsigned long long o,
-                                                  int lane) {
-    unsigned nonfinite = 0u, saturated = 0u;
-    const unsigned long long i0 = part * P.lp + o + static_cast<unsigned long long>(lane) * kLaneElems;
-    const int valid = i0 >= P.n ? 0 : (P.n - i0 >= 8 ? 8 : static_cast<int>(P.n - i0));
-    const int lanes_per_block = (MODE == MODE_BLOCK) ? (P.block_log2 >= 8 ? 32 : (1 << (P.block_log2 - 3))) : 1;
-    const unsigned long long blk = (MODE == MODE_BLOCK) ? (i0 >> P.block_log2) : 0;
-
-    float g[8], ef[8], c[8], prev[8];
+// Step 1 for the lane's 8 elements of the row at partition-local offset `orow`: g (clipped if asked), the
+// compensation c, e~_k, h = g + c.  Counts the 8-bit images of e~_k that Eq. 1's range clamps (Q8COMP only).
+template <int GRAD, int STATE, int MODE>
+__device__ __forceinline__ void careful_load(const SendCommon &C, const SendBucket &Bk, unsigned long long part,
+                                             unsigned long long orow, int lane, bool count, CarefulVals &V,
+                                             unsigned &state_saturated) {
+    V.i0 = part * Bk.lp + orow + static_cast<unsigned long long>(lane) * kLaneElems;
+    V.valid = V.i0 >= Bk.n ? 0 : (Bk.n - V.i0 >= 8 ? 8 : static_cast<int>(Bk.n - V.i0));
+    const int8_t *st8 = static_cast<const int8_t *>(Bk.state);
+    const float *stf = static_cast<const float *>(Bk.state);
     float sscale = 0.0f;
-    int8_t *st8 = static_cast<int8_t *>(P.state);
-    float *stf = static_cast<float *>(P.state);
-    float *st_scales = reinterpret_cast<float *>(static_cast<uint8_t *>(P.state) + P.state_scale_off);
-
-    unsigned lo_w = 0, hi_w = 0;
+    if (STATE == ST_INT8 && MODE == MODE_BLOCK && V.valid > 0) {
+        const float *st_scales = reinterpret_cast<const float *>(static_cast<const uint8_t *>(Bk.state) + ((Bk.n + 255ull) & ~255ull));
+        sscale = st_scales[V.i0 >> C.block_log2];
+    }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        g[j] = 0.0f;
-        ef[j] = 0.0f;
-        if (j < valid) {
-            g[j] = load_grad1<GRAD>(P.grad, i0 + j);
-            if (P.clip > 0.0f && g[j] == g[j]) g[j] = fminf(fmaxf(g[j], -P.clip), P.clip);    // NaN stays NaN
+        float g = 0.0f, c = 0.0f, prev = 0.0f;
+        if (j < V.valid) {
+            g = load_grad1<GRAD>(Bk.grad, V.i0 + j);
+            if (C.clip > 0.0f && g == g) g = fminf(fmaxf(g, -C.clip), C.clip);          // NaN stays NaN
             if (STATE == ST_INT8) {
-                const unsigned b = static_cast<uint8_t>(st8[i0 + j]);
-                if (j < 4) lo_w |= b << (8 * j); else hi_w |= b << (8 * (j - 4));
+                const float ei = __int2float_rn(static_cast<int>(st8[V.i0 + j]));
+                c = (MODE == MODE_FIXED) ? __fdiv_rn(ei, C.s_e) : __fmul_rn(ei, sscale);    // dec(e_k; s_e), Eq. 2
+                prev = c;
+            } else if (STATE == ST_FP32) {
+                c = stf[V.i0 + j];
+                prev = c;
+            } else if (STATE == ST_Q8COMP) {
+                prev = stf[V.i0 + j];
+                const float y = __fmul_rn(prev, C.s_e);
+                if (count && (y >= 127.5f || y < -128.5f)) state_saturated += 1u;          // nearest integer outside [-128, 127]
+                unsigned bits;
+                c = __fdiv_rn(round_clamp(y, -128.0f, 127.0f, bits), C.s_e);
             }
-            if (STATE == ST_FP32 || STATE == ST_Q8COMP) ef[j] = stf[i0 + j];
         }
+        V.c[j] = c;
+        V.prev[j] = prev;
+        V.h[j] = __fadd_rn(g, c);                             // step 1 / Eq. 2
+        V.fin[j] = fabsf(V.h[j]) <= kFltMax;                  // false for NaN and +-Inf
     }
-    const uint2 e8 = make_uint2(lo_w, hi_w);
-    if (STATE == ST_INT8 && MODE == MODE_BLOCK) sscale = valid > 0 ? st_scales[blk] : 0.0f;
+}
 
-    decode_state8<STATE, MODE>(P, e8, ef, sscale, c, prev);
-
-    unsigned code[8];
-    float e_new[8], scale;
-    send_core<STATE, BITS, MODE, STOCH>(P, g, c, prev, valid, lanes_per_block, i0, code, e_new, scale, nonfinite, saturated);
-
-    // codes (and the block's scale) into the partition's areas of the communication buffer
-    uint8_t *pbase = P.scatter ? P.part_dst[part] : P.comm + part * P.stride;
-    const unsigned long long ol = o + static_cast<unsigned long long>(lane) * kLaneElems;
-    store_codes8<BITS>(pbase + ol * BITS / 8, code);
-    if (MODE == MODE_BLOCK) {
-        if ((lane & (lanes_per_block - 1)) == 0 && ((ol & ((1ull << P.block_log2) - 1)) == 0))
-            *reinterpret_cast<float *>(pbase + P.code_bytes + (ol >> P.block_log2) * 4) = scale;
-    }
-
-    // Eq. 7: reset, or keep / compress the new error
-    if (STATE == ST_INT8) {
-        unsigned ebits[8];
-        float escale = 0.0f;
-        if (P.reset) {
+// The lane's share of a block's statistic: the largest finite |h| (codes of 2 bits and more), or the pairwise
+// sum of the finite |h| (sign code; absent elements are zeros here and enter as such).
+template <int BITS>
+__device__ __forceinline__ float careful_lane_stat(const CarefulVals &V) {
+    float a[8];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) ebits[j] = 0u;
+    for (int j = 0; j < 8; ++j) a[j] = V.fin[j] ? fabsf(V.h[j]) : 0.0f;
+    if (BITS == 1)
+        return __fadd_rn(__fadd_rn(__fadd_rn(a[0], a[1]), __fadd_rn(a[2], a[3])), __fadd_rn(__fadd_rn(a[4], a[5]), __fadd_rn(a[6], a[7])));
+    float m = 0.0f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) m = fmaxf(m, a[j]);
+    return m;
+}
+// ... combined over aligned groups of `lanes` lanes: every lane of a group ends with the same value (fp32 addition
+// commutes, so the butterfly is the balanced tree over the group's positions in index order).
+template <int BITS>
+__device__ __forceinline__ float careful_group_stat(float v, int lanes) {
+    for (int o = 1; o < lanes; o <<= 1) {
+        const float w = __shfl_xor_sync(kFull, v, o);
+        v = (BITS == 1) ? __fadd_rn(v, w) : fmaxf(v, w);
+    }
+    return v;
+}
+
+// scale and multiplier of a block from its statistic; `len` = elements of the block that exist (sign code only)
+template <int BITS>
+__device__ __forceinline__ void careful_block_scale(float stat, unsigned long long len, float &scale, float &mult) {
+    if (BITS == 1) {
+        scale = __fdiv_rn(stat, static_cast<float>(len));      // mean |h|; len >= 1 wherever the result is used
+        mult = 0.0f;
+    } else {
+        constexpr float hi = QRange<BITS>::hi;
+        scale = stat > 0.0f ? __fdiv_rn(stat, hi) : 0.0f;
+        mult = stat > 0.0f ? __fdiv_rn(hi, stat) : 0.0f;
+    }
+}
+
+// Eq. 1 / Eq. 3, step 2 and Eq. 5 for the lane's 8 elements, given the multiplier (s, or the block's inverse scale) and
+// the block's scale.  code: low bits of each word = the wire field.
+template <int BITS, int MODE, bool STOCH>
+__device__ __forceinline__ void careful_quantise(const SendCommon &C, const CarefulVals &V, float mult, float scale, bool count,
+                                                 unsigned (&code)[8], float (&e_new)[8], CarefulCounts &N) {
+    float u8[8];
+    if (STOCH) {                                            // i0 is a multiple of 8: one half of a block of 16
+        const uint4 r = sr_block(V.i0 >> 4, C.k_lo, C.k_hi, C.seed_lo, C.seed_hi);
+        const bool upper = ((V.i0 >> 3) & 1ull) != 0ull;
+        const unsigned w0 = upper ? r.z : r.x, w1 = upper ? r.w : r.y;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { u8[j] = sr_dither(w0, j); u8[4 + j] = sr_dither(w1, j); }
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const float h = V.h[j];
+        const bool fin = V.fin[j];
+        if (!fin && j < V.valid && count) N.nonfinite = 1u;
+        float d;
+        if (BITS == 1) {
+            // sign code: q = -1 if h < 0 else +1 (so +-0 and NaN give +1); the wire bit is 1 for -1
+            const bool neg = h < 0.0f;
+            code[j] = neg ? 1u : 0u;
+            const float q = neg ? -1.0f : 1.0f;
+            d = (MODE == MODE_FIXED) ? __fdiv_rn(q, C.s) : __fmul_rn(q, scale);
         } else {
-            state_compress8<MODE>(P, e_new, lanes_per_block, ebits, escale);
+            constexpr float lo = QRange<BITS>::lo, hi = QRange<BITS>::hi;
+            const float hq = (h != h) ? 0.0f : h;               // NaN is sent as code 0
+            float y = __fmul_rn(hq, mult);                      // h x s of Eq. 1
+            if (!fin) y = hq;                                   // +-Inf saturates whatever the scale
+            float r;
+            if (STOCH && fin) {                                 // floor(y + u): up with probability frac(y)
+                const float fl = floorf(__fadd_rn(y, u8[j]));
+                if (count && C.collect_stats && j < V.valid && (fl < lo || fl > hi)) N.saturated += 1u;
+                r = fminf(fmaxf(fl, lo), hi);
+                code[j] = static_cast<unsigned>(__float2int_rn(r));
+            } else {
+                r = round_clamp(y, lo, hi, code[j]);            // round_p-bit
+                // nearest integer outside the range: y >= hi + 1/2 (hi is odd, the tie goes up and out) or
+                // y < lo - 1/2 (lo is even, the tie stays in); a block scale keeps every code inside
+                if (MODE != MODE_BLOCK && count && C.collect_stats && !STOCH && fin && j < V.valid &&
+                    (y >= hi + 0.5f || y < lo - 0.5f)) N.saturated += 1u;
+            }
+            d = (MODE == MODE_FIXED) ? __fdiv_rn(r, C.s) : __fmul_rn(r, scale);     // step 2: dec(q; s)
         }
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if (j < valid) st8[i0 + j] = static_cast<int8_t>(ebits[j] & 0xffu);
-        if (MODE == MODE_BLOCK) {
-            if ((lane & (lanes_per_block - 1)) == 0 && (i0 & ((1ull << P.block_log2) - 1)) == 0 && valid > 0)
-                st_scales[blk] = escale;
-        }
-    } else if (STATE == ST_FP32 || STATE == ST_Q8COMP) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if (j < valid) stf[i0 + j] = P.reset ? 0.0f : e_new[j];
+        const float delta = fin ? __fsub_rn(h, d) : 0.0f;
+        // an absent element has no error (with the sign code its h = 0 would otherwise leave -d behind and enter the
+        // block's largest error)
+        e_new[j] = j < V.valid ? __fadd_rn(__fmul_rn(C.omb, V.prev[j]), __fmul_rn(C.beta, delta)) : 0.0f;   // Eq. 5
     }
-    return saturated | (nonfinite << 31);
+}
+
+// `nrows` consecutive rows of partition `part` starting at partition-local offset `o` (a multiple of 256, and of B
+// when nrows > 1).  pbase: where the partition's codes and scales go.  Elements >= n are treated as absent (code 0, no
+// state).  Out of line and reading the kernel's parameters in place (they are __grid_constant__, so their address can
+// be taken without a local copy), so that the fast routine's register allocation is not disturbed by this rarely taken
+// path.
+template <int GRAD, int STATE, int BITS, int MODE, bool STOCH>
+__device__ __noinline__ CarefulCounts send_careful(const SendCommon &C, const SendBucket &Bk, uint8_t *pbase,
+                                                   unsigned long long part, unsigned long long o, int nrows, int lane) {
+    CarefulCounts N = {0u, 0u, 0u};
+    const bool wide = MODE == MODE_BLOCK && C.block_log2 > 8;   // one block spanning all rows of the unit (nrows = B / 256)
+    const int lanes_per_block = (MODE != MODE_BLOCK) ? 1 : (C.block_log2 >= 8 ? 32 : (1 << (C.block_log2 - 3)));
+    const unsigned long long code_bytes = Bk.lp * BITS / 8;
+    int8_t *st8 = static_cast<int8_t *>(Bk.state);
+    float *stf = static_cast<float *>(Bk.state);
+    float *st_scales = reinterpret_cast<float *>(static_cast<uint8_t *>(Bk.state) + ((Bk.n + 255ull) & ~255ull));
+    const bool stats = C.collect_stats != 0;
+
+    // ---- a block wider than a row: its statistic first ------------------------------------------------------
+    float wscale = 0.0f, wmult = 0.0f;
+    const unsigned long long block0 = part * Bk.lp + o;         // bucket index of the unit's first element
+    if (wide) {
+        float level[5];                                         // partial sums of 2^l rows (sign code): a binary counter
+        float amax = 0.0f;
+        for (int r = 0; r < nrows; ++r) {
+            CarefulVals V;
+            unsigned dummy = 0u;
+            careful_load<GRAD, STATE, MODE>(C, Bk, part, o + static_cast<unsigned long long>(r) * kRow, lane, false, V, dummy);
+            float v = careful_group_stat<BITS>(careful_lane_stat<BITS>(V), 32);
+            if (BITS == 1) {
+                int l = 0;
+                for (int t = r; t & 1; t >>= 1, ++l) v = __fadd_rn(level[l], v);   // earlier rows on the left
+                level[l] = v;
+            } else {
+                amax = fmaxf(amax, v);
+            }
+        }
+        unsigned long long len = 1ull << C.block_log2;
+        if (block0 < Bk.n && Bk.n - block0 < len) len = Bk.n - block0;
+        int top = 0;
+        while ((1 << top) < nrows) ++top;
+        careful_block_scale<BITS>(BITS == 1 ? level[top] : amax, len, wscale, wmult);
+    }
+
+    // ---- codes, new error (and, for a wide block with the 8-bit state, the statistic of the new error) -------
+    float e_amax = 0.0f;
+    for (int r = 0; r < nrows; ++r) {
+        const unsigned long long orow = o + static_cast<unsigned long long>(r) * kRow;
+        CarefulVals V;
+        careful_load<GRAD, STATE, MODE>(C, Bk, part, orow, lane, stats, V, N.state_saturated);
+        float scale = wscale, mult = (MODE == MODE_FIXED) ? C.s : wmult;
+        if (MODE == MODE_BLOCK && !wide) {
+            const float stat = careful_group_stat<BITS>(careful_lane_stat<BITS>(V), lanes_per_block);
+            const unsigned long long b0 = (V.i0 >> C.block_log2) << C.block_log2;
+            unsigned long long len = 1ull << C.block_log2;
+            if (b0 < Bk.n && Bk.n - b0 < len) len = Bk.n - b0;
+            careful_block_scale<BITS>(stat, len, scale, mult);
+        }
+        unsigned code[8];
+        float e_new[8];
+        careful_quantise<BITS, MODE, STOCH>(C, V, mult, scale, true, code, e_new, N);
+
+        const unsigned long long ol = orow + static_cast<unsigned long long>(lane) * kLaneElems;   // partition-local
+        store_codes8<BITS>(pbase + ol * BITS / 8, code);
+        if (MODE == MODE_BLOCK && !wide) {
+            if ((lane & (lanes_per_block - 1)) == 0 && ((ol & ((1ull << C.block_log2) - 1)) == 0))
+                *reinterpret_cast<float *>(pbase + code_bytes + (ol >> C.block_log2) * 4) = scale;
+        }
+
+        // Eq. 7: reset, or keep / compress the new error
+        if (STATE == ST_INT8) {
+            if (C.reset) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (j < V.valid) st8[V.i0 + j] = 0;
+                if (MODE == MODE_BLOCK && !wide && (lane & (lanes_per_block - 1)) == 0 &&
+                    (V.i0 & ((1ull << C.block_log2) - 1)) == 0 && V.valid > 0)
+                    st_scales[V.i0 >> C.block_log2] = 0.0f;
+            } else if (wide) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) e_amax = fmaxf(e_amax, fabsf(e_new[j]));
+            } else {
+                float emult = C.s_e, escale = 0.0f;
+                if (MODE == MODE_BLOCK) {
+                    float am = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) am = fmaxf(am, fabsf(e_new[j]));
+                    am = careful_group_stat<8>(am, lanes_per_block);
+                    escale = am > 0.0f ? __fdiv_rn(am, 127.0f) : 0.0f;
+                    emult = am > 0.0f ? __fdiv_rn(127.0f, am) : 0.0f;
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float y = __fmul_rn(e_new[j], emult);
+                    if (MODE == MODE_FIXED && stats && j < V.valid && (y >= 127.5f || y < -128.5f)) N.state_saturated += 1u;
+                    unsigned eb;
+                    (void)round_clamp(y, -128.0f, 127.0f, eb);            // compressor(e~; s_e, 8)
+                    if (j < V.valid) st8[V.i0 + j] = static_cast<int8_t>(eb & 0xffu);
+                }
+                if (MODE == MODE_BLOCK && (lane & (lanes_per_block - 1)) == 0 &&
+                    (V.i0 & ((1ull << C.block_log2) - 1)) == 0 && V.valid > 0)
+                    st_scales[V.i0 >> C.block_log2] = escale;
+            }
+        } else if (STATE == ST_FP32 || STATE == ST_Q8COMP) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (j < V.valid) stf[V.i0 + j] = C.reset ? 0.0f : e_new[j];
+        }
+    }
+    if (wide) {
+        if (lane == 0) *reinterpret_cast<float *>(pbase + code_bytes + (o >> C.block_log2) * 4) = wscale;
+        if (STATE == ST_INT8 && block0 < Bk.n) {
+            if (C.reset) {
+                if (lane == 0) st_scales[block0 >> C.block_log2] = 0.0f;
+            } else {
+                // ---- 8-bit codes of the new error, which is formed once more from the untouched inputs ----------
+                e_amax = careful_group_stat<8>(e_amax, 32);
+                const float escale = e_amax > 0.0f ? __fdiv_rn(e_amax, 127.0f) : 0.0f;
+                const float emult = e_amax > 0.0f ? __fdiv_rn(127.0f, e_amax) : 0.0f;
+                for (int r = 0; r < nrows; ++r) {
+                    CarefulVals V;
+                    unsigned dummy = 0u;
+                    careful_load<GRAD, STATE, MODE>(C, Bk, part, o + static_cast<unsigned long long>(r) * kRow, lane, false, V, dummy);
+                    unsigned code[8];
+                    float e_new[8];
+                    CarefulCounts unused = {0u, 0u, 0u};
+                    careful_quantise<BITS, MODE, STOCH>(C, V, wmult, wscale, false, code, e_new, unused);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        unsigned eb;
+                        (void)round_clamp(__fmul_rn(e_new[j], emult), -128.0f, 127.0f, eb);
+                        if (j < V.valid) st8[V.i0 + j] = static_cast<int8_t>(eb & 0xffu);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) st_scales[block0 >> C.block_log2] = escale;
+            }
+        }
+    }
+    return N;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -450,7 +598,7 @@ struct LanePtrs {
     float *wire_scales;       // BLOCK: the partition's scale area
     float *state_scales;      // BLOCK + INT8: scale of the bucket's block 0
     unsigned long long elem0; // bucket index of this lane's first element of wide row 0
-    unsigned lane_elem;       // partition-local index of this lane's first element of wide row 0
+    unsigned long long lane_elem;   // partition-local index of this lane's first element of wide row 0
 };
 
 // ---- per-warp ring of asynchronous copies (cp.async) -------------------------------------------
@@ -481,6 +629,11 @@ __device__ __forceinline__ uint4 lds16(unsigned saddr) {
 __device__ __forceinline__ uint2 lds8(unsigned saddr) {
     uint2 v;
     asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(saddr) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned lds2(unsigned saddr) {
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(saddr) : "memory");
     return v;
 }
 __device__ __forceinline__ unsigned lds4(unsigned saddr) {
@@ -626,6 +779,17 @@ __device__ __forceinline__ float qmax_over(float c, float a) {
     return __fdiv_rn(c, a);
 }
 
+// sum over aligned groups of `lanes` lanes as a balanced tree in index order (fp32 addition commutes, so both lanes
+// of a pair form the same sum); every lane of a group ends with the group's sum
+__device__ __forceinline__ float group_sum32(float v, int lanes) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float w = __shfl_xor_sync(kFull, v, o);
+        v = o < lanes ? __fadd_rn(v, w) : v;
+    }
+    return v;
+}
+
 // The same without the fallback, for callers that have already sent every a outside [2^-100, 2^100] elsewhere.
 __device__ __forceinline__ float qmax_over_midrange(float c, float a) {
     float x;
@@ -636,19 +800,21 @@ __device__ __forceinline__ float qmax_over_midrange(float c, float a) {
 }
 __device__ __forceinline__ bool in_midrange(float a) { return __float_as_uint(a) - 0x0d800000u <= 0x71800000u - 0x0d800000u; }
 
-// max over aligned groups of `lanes` lanes (2, 4, 8 or 16) in a fixed number of steps, without a loop
-__device__ __forceinline__ float group_max16(float v, int lanes) {
+// max over aligned groups of `lanes` lanes (1 to 32) in a fixed number of steps, without a loop
+__device__ __forceinline__ float group_max32(float v, int lanes) {
 #pragma unroll
-    for (int o = 1; o < 16; o <<= 1) {
+    for (int o = 1; o < 32; o <<= 1) {
         const float w = __shfl_xor_sync(kFull, v, o);
         v = o < lanes ? fmaxf(v, w) : v;
     }
     return v;
 }
 
-// One wide row.  Returns false (and stores nothing) if some lane of the warp met a value that the fast
-// arithmetic does not cover (NaN, +-Inf, or a magnitude that could overflow): the caller then redoes the row
-// with the careful routine.
+// One wide row.  Returns false if some lane of the warp met a value that the fast arithmetic does not cover (NaN,
+// +-Inf, a magnitude that could overflow, a block maximum outside the range of the short division sequences): the
+// caller then redoes the row with the careful routine.  Invariant the caller relies on: no byte of the error state
+// (codes, values or scales) has been written before the last `return false`; codes and wire scales of the row may
+// already have been stored (block mode) and the careful routine stores the same bytes again.
 // VAR_LEAN: both decompressors are the single fused multiply-add and no statistics are collected;
 // VAR_LEAN_NR: the same, but dec(e; s_e) is the Newton-Raphson form (s_e = 6 s of the paper), still packed;
 // VAR_GENERAL: the forms are chosen per call at run time (scalar code) and statistics may be collected.
@@ -679,7 +845,7 @@ __device__ __forceinline__ f32x2 dec_state2(const SendConsts &K, f32x2 m2, float
 
 template <int GRAD, int STATE, int BITS, int MODE, int VAR>
 __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtrs &L, const WideIn<GRAD, STATE> &in,
-                                              unsigned wrow, int lane, bool stats, unsigned &saturated) {
+                                              unsigned wrow, int lane, bool stats, unsigned &saturated, unsigned &state_saturated) {
     constexpr float lo = QRange<BITS>::lo, hi = QRange<BITS>::hi, qmagic = kMagic + QRange<BITS>::off;
     constexpr float emagic = kMagic + 128.0f;
     constexpr bool kStateF32 = (STATE == ST_FP32 || STATE == ST_Q8COMP);
@@ -690,7 +856,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     constexpr int GW = WideIn<GRAD, STATE>::GW, EW = WideIn<GRAD, STATE>::EW;
     constexpr bool LEAN = var_is_lean(VAR), EXTRAS = var_has_extras(VAR);
     const int dq_mode = LEAN ? DEC_FMA : K.dq_mode, de_mode = K.de_mode;
-    const int lanes_per_block = (MODE == MODE_BLOCK) ? (K.block_log2 >= 9 ? 32 : (1 << (K.block_log2 - 4))) : 1;
+    const int lanes_per_block = (MODE == MODE_BLOCK) ? (K.block_log2 >= 9 ? 32 : (1 << (K.block_log2 - 4))) : 1;    // B <= 512 here
     const f32x2 zero2 = 0ull;
 
     // ---- values outside the fast arithmetic -------------------------------------------------------------
@@ -764,6 +930,8 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             } else {
                 float y0, y1;
                 unpk2(fmul2(prev2[k], dup2(K.s_e)), y0, y1);
+                if (EXTRAS && stats)             // nearest integer outside [-128, 127]: 127.5 goes up and out, -128.5 stays in
+                    state_saturated += ((y0 >= 127.5f || y0 < -128.5f) ? 1u : 0u) + ((y1 >= 127.5f || y1 < -128.5f) ? 1u : 0u);
                 const f32x2 m2 = fadd2(pk2(fminf(fmaxf(y0, -128.0f), 127.0f), fminf(fmaxf(y1, -128.0f), 127.0f)), dup2(emagic));
                 c2 = dec_state2<VAR>(K, m2, emagic, de_mode);
             }
@@ -777,7 +945,32 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
 
     // ---- block scale (extension): absmax of the block's h over the lanes that share it ---------------------------
     float mult = K.s, scale = 0.0f;
-    if (MODE == MODE_BLOCK) {
+    if (BITS == 1 && STATE != ST_INT8) {
+        // the sign code sends +1 for -0 (h < 0 is false); adding +0 turns a -0 into +0 and changes nothing else.  With
+        // the 8-bit state h = g + c is never -0, because c never is (a product or sum that cancels gives +0).
+#pragma unroll
+        for (int k = 0; k < 8; ++k) h2[k] = fadd2(h2[k], zero2);
+    }
+    if (MODE == MODE_BLOCK && BITS == 1) {
+        // sign code: the block's magnitude is the mean of |h|, summed pairwise (a balanced tree over the block's positions)
+        float a[16];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            unpk2(h2[k], a[2 * k], a[2 * k + 1]);
+            a[2 * k] = fabsf(a[2 * k]);
+            a[2 * k + 1] = fabsf(a[2 * k + 1]);
+        }
+#pragma unroll
+        for (int w = 1; w < 16; w <<= 1) {
+#pragma unroll
+            for (int j = 0; j < 16; j += 2 * w) a[j] = __fadd_rn(a[j], a[j + w]);
+        }
+        const float sum = group_sum32(a[0], lanes_per_block);
+        // an overflowing h or sum leaves the row to the careful routine (which forms the same infinities the plain way)
+        if (__any_sync(kFull, bad_bits != 0u || !(sum <= kFltMax))) return false;
+        scale = __fmul_rn(sum, __uint_as_float(static_cast<unsigned>(127 - K.block_log2) << 23));     // sum / B, exact scaling
+        mult = 0.0f;
+    } else if (MODE == MODE_BLOCK) {
         float amax = 0.0f;
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
@@ -785,7 +978,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             unpk2(h2[k], a, b);
             amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
         }
-        amax = group_max16(amax, lanes_per_block);
+        amax = group_max32(amax, lanes_per_block);
         // g is finite here, so h can only be +-Inf (an overflowing sum), never NaN, and the maximum shows it.  A block
         // maximum outside [2^-100, 2^100] (other than 0) also leaves the row to the careful routine, which divides.
         if (__any_sync(kFull, bad_bits != 0u || !(amax == 0.0f || in_midrange(amax)))) return false;
@@ -800,8 +993,22 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     uint4 rnd = make_uint4(0u, 0u, 0u, 0u);                // the lane's 16 elements are one block of the Philox stream
     if (var_is_sr(VAR))
         rnd = sr_block((L.elem0 + static_cast<unsigned long long>(wrow) * kWide) >> 4, K.k_lo, K.k_hi, K.seed_lo, K.seed_hi);
+    unsigned signs = 0u;                                   // sign code: bit j = 1 when element j is negative
+    if (BITS == 1) {
+        const unsigned mag = __float_as_uint(MODE == MODE_BLOCK ? scale : K.inv_s);     // d = q x mean|h|, or q / s = +-fl(1/s)
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
+        for (int k = 7; k >= 0; --k) {
+            const unsigned b0 = static_cast<unsigned>(h2[k]), b1 = static_cast<unsigned>(h2[k] >> 32);
+            signs = __funnelshift_l(b0, __funnelshift_l(b1, signs, 1), 1);
+            const f32x2 d2 = pk2(__uint_as_float(and_or(b0, 0x80000000u, mag)), __uint_as_float(and_or(b1, 0x80000000u, mag)));
+            const f32x2 delta2 = fsub2(h2[k], d2);
+            en2[k] = (STATE == ST_NONE) ? zero2
+                     : (kSignFree ? fadd2(fmul2_pz(omb2, prev2[k]), fmul2_pz(beta2, delta2))
+                                  : fadd2_after_mul(fmul2(omb2, prev2[k]), fmul2(beta2, delta2)));
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < (BITS == 1 ? 0 : 8); ++k) {
         float y0 = 0.0f, y1 = 0.0f, t0 = 0.0f, t1 = 0.0f;
         f32x2 m2;                                                                                    // kMagic + 2^(p-1) + q
         if (MODE == MODE_BLOCK && !var_is_sr(VAR)) {
@@ -849,12 +1056,14 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         st_stream8(cdst, make_uint2(horner_codes<4, 8>(mb), horner_codes<4, 8>(mb + 8)));
     } else if (BITS == 8) {
         st_stream16(cdst, make_uint4(horner_codes<8, 4>(mb), horner_codes<8, 4>(mb + 4), horner_codes<8, 4>(mb + 8), horner_codes<8, 4>(mb + 12)));
-    } else {
+    } else if (BITS == 2) {
         st_stream4(cdst, horner_codes<2, 16>(mb));
+    } else {
+        st_stream2(cdst, static_cast<uint16_t>(signs));
     }
     if (MODE == MODE_BLOCK) {
-        const unsigned ol = L.lane_elem + wrow * kWide;     // partition-local element index
-        if ((lane & (lanes_per_block - 1)) == 0 && ((ol & ((1u << K.block_log2) - 1)) == 0))
+        const unsigned long long ol = L.lane_elem + static_cast<unsigned long long>(wrow) * kWide;     // partition-local element index
+        if ((lane & (lanes_per_block - 1)) == 0 && ((ol & ((1ull << K.block_log2) - 1)) == 0))
             L.wire_scales[ol >> K.block_log2] = scale;
     }
 
@@ -872,7 +1081,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
                     unpk2(en2[k], a, b);
                     amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
                 }
-                amax = group_max16(amax, lanes_per_block);
+                amax = group_max32(amax, lanes_per_block);
                 // nothing of the state has been written yet, and the codes stored above are what the careful routine stores
                 if (__any_sync(kFull, !(amax == 0.0f || in_midrange(amax)))) return false;
                 escale = amax > 0.0f ? div_by_qmax(amax, 127.0f, 1.0f / 127.0f) : 0.0f;
@@ -884,6 +1093,8 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             for (int k = 0; k < 8; ++k) {
                 float a, b;
                 unpk2(fmul2(en2[k], emult2), a, b);
+                if (MODE != MODE_BLOCK && EXTRAS && stats)      // codes that Eq. 7's 8-bit compressor clamps
+                    state_saturated += ((a >= 127.5f || a < -128.5f) ? 1u : 0u) + ((b >= 127.5f || b < -128.5f) ? 1u : 0u);
                 q[2 * k] = __float2int_rn(a);                   // saturates, NaN -> 0
                 q[2 * k + 1] = __float2int_rn(b);
             }
@@ -912,9 +1123,49 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     return true;
 }
 
-// grid = (ctas per partition, partitions).  Each warp walks the partition's wide rows with the stride of all
-// warps working on that partition; the inputs of its next rows are on their way through the cp.async ring.
-// What is left of the partition (a last half-wide row, partial and padding rows) goes to the careful routine.
+// The lane's pointers for the wide rows of partition `part` of one bucket, row 0 at partition-local element `o0`.
+template <int STATE, int BITS>
+__device__ __forceinline__ void lane_pointers(const SendBucket &Bk, uint8_t *pbase, unsigned long long part,
+                                              unsigned long long o0, int lane, LanePtrs &L) {
+    L.lane_elem = o0 + static_cast<unsigned long long>(lane) * kWideLane;
+    L.elem0 = part * Bk.lp + L.lane_elem;
+    L.state = static_cast<uint8_t *>(Bk.state) + L.elem0 * (STATE == ST_INT8 ? 1u : 4u);
+    L.codes = pbase + L.lane_elem * BITS / 8;
+    L.wire_scales = reinterpret_cast<float *>(pbase + Bk.lp * BITS / 8);
+    L.state_scales = reinterpret_cast<float *>(static_cast<uint8_t *>(Bk.state) + ((Bk.n + 255ull) & ~255ull));
+}
+
+__device__ __forceinline__ void load_consts(const SendCommon &C, SendConsts &K) {
+    K.s = C.s; K.s_e = C.s_e; K.beta = C.beta; K.omb = C.omb; K.inv_s = C.inv_s; K.inv_se = C.inv_se;
+    K.dq_a = C.dq_a; K.dq_b = C.dq_b; K.de_a = C.de_a; K.de_b = C.de_b;
+    K.dq_mode = C.dq_mode; K.de_mode = C.de_mode; K.block_log2 = C.block_log2; K.reset = C.reset; K.clip = C.clip;
+    K.seed_lo = C.seed_lo; K.seed_hi = C.seed_hi; K.k_lo = C.k_lo; K.k_hi = C.k_hi;
+}
+
+// What a warp has counted goes to the bucket's status words: [0] flags, [1] saturated gradient codes, [2] saturated
+// 8-bit error codes.
+__device__ __forceinline__ void flush_counts(unsigned long long *status, bool collect, int lane, unsigned &saturated,
+                                             unsigned &state_saturated, unsigned &nonfinite) {
+    if (__any_sync(kFull, nonfinite != 0u)) {
+        if (lane == 0) atomicOr(status, static_cast<unsigned long long>(kFlagNonFinite));
+    }
+    if (collect) {
+        for (int o = 16; o > 0; o >>= 1) {
+            saturated += __shfl_xor_sync(kFull, saturated, o);
+            state_saturated += __shfl_xor_sync(kFull, state_saturated, o);
+        }
+        if (lane == 0 && saturated) atomicAdd(status + 1, static_cast<unsigned long long>(saturated));
+        if (lane == 0 && state_saturated) atomicAdd(status + 2, static_cast<unsigned long long>(state_saturated));
+    }
+    saturated = 0u;
+    state_saturated = 0u;
+    nonfinite = 0u;
+}
+
+// One bucket per launch.  grid = (ctas per partition, partitions).  Each warp walks the partition's wide rows with the
+// stride of all warps working on that partition; the inputs of its next rows are on their way through the cp.async
+// ring.  What is left of the partition (a last half-wide row, partial and padding rows; every block when a block is
+// wider than a wide row) goes to the careful routine.
 // VAR_LEAN / VAR_LEAN_NR kernels are launched when the host proved the corresponding decompressor forms and neither
 // statistics nor clipping are wanted (VAR_LEAN also for every block-scaled configuration), VAR_LEAN_X / VAR_LEAN_NR_X
 // when they are; VAR_GENERAL chooses the decompressor forms at run time.
@@ -925,41 +1176,40 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_con
     constexpr unsigned gbytes = (GRAD == GRAD_BF16 ? 2u : 4u) * kWide;       // gradient bytes of a wide row
     constexpr unsigned ebytes = (STATE == ST_INT8 ? 1u : 4u) * kWide;        // state bytes of a wide row
     extern __shared__ __align__(16) uint8_t ring[];
+    const SendCommon &C = P.c;
+    const SendBucket &Bk = P.b;
     const int lane = threadIdx.x & 31;
     const unsigned long long part = blockIdx.y;
     const unsigned warp = blockIdx.x * kWarps + (threadIdx.x >> 5);
     const unsigned nwarps = gridDim.x * kWarps;
-    const unsigned rows = static_cast<unsigned>(P.lp / kRow);                // 256-element rows of the partition
-    const unsigned long long base = part * P.lp;
+    const unsigned rows = static_cast<unsigned>(Bk.lp / kRow);               // 256-element rows of the partition
+    const unsigned long long base = part * Bk.lp;
+    uint8_t *pbase = P.scatter ? P.part_dst[part] : Bk.comm + part * Bk.stride;
     // rows [0, full_rows) of this partition lie entirely below n
     unsigned full_rows = 0;
-    if (P.n > base) {
-        const unsigned long long avail = P.n - base;
-        full_rows = avail >= P.lp ? rows : static_cast<unsigned>(avail / kRow);
+    if (Bk.n > base) {
+        const unsigned long long avail = Bk.n - base;
+        full_rows = avail >= Bk.lp ? rows : static_cast<unsigned>(avail / kRow);
     }
-    unsigned saturated = 0u;
-    unsigned long long careful_acc = 0ull;
+    unsigned saturated = 0u, state_saturated = 0u, nonfinite = 0u;
+    auto careful = [&](unsigned long long o, int nrows) {
+        const CarefulCounts N = send_careful<GRAD, STATE, BITS, MODE, var_is_sr(VAR)>(C, Bk, pbase, part, o, nrows, lane);
+        saturated += N.saturated;
+        state_saturated += N.state_saturated;
+        nonfinite |= N.nonfinite;
+    };
     unsigned first_careful = 0u;             // first 256-element row left to the careful routine
-    if (P.fast) {
+    if (C.fast) {
         const unsigned full_wide = full_rows / 2;
         first_careful = 2 * full_wide;
         LanePtrs L;
-        L.lane_elem = static_cast<unsigned>(lane) * kWideLane;
-        L.elem0 = base + L.lane_elem;
-        L.state = static_cast<uint8_t *>(P.state) + L.elem0 * (STATE == ST_INT8 ? 1u : 4u);
-        uint8_t *pbase = P.scatter ? P.part_dst[part] : P.comm + part * P.stride;
-        L.codes = pbase + static_cast<size_t>(L.lane_elem) * BITS / 8;
-        L.wire_scales = reinterpret_cast<float *>(pbase + P.code_bytes);
-        L.state_scales = reinterpret_cast<float *>(static_cast<uint8_t *>(P.state) + P.state_scale_off);
+        lane_pointers<STATE, BITS>(Bk, pbase, part, 0ull, lane, L);
         // staging reads: chunk `lane` of each 512-byte piece of the row
-        const uint8_t *g_stage = static_cast<const uint8_t *>(P.grad) + base * (GRAD == GRAD_BF16 ? 2u : 4u) + lane * 16;
-        const uint8_t *e_stage = static_cast<const uint8_t *>(P.state) + base * (STATE == ST_INT8 ? 1u : 4u) + lane * 16;
+        const uint8_t *g_stage = static_cast<const uint8_t *>(Bk.grad) + base * (GRAD == GRAD_BF16 ? 2u : 4u) + lane * 16;
+        const uint8_t *e_stage = static_cast<const uint8_t *>(Bk.state) + base * (STATE == ST_INT8 ? 1u : 4u) + lane * 16;
         SendConsts K;
-        K.s = P.s; K.s_e = P.s_e; K.beta = P.beta; K.omb = P.omb; K.inv_s = P.inv_s; K.inv_se = P.inv_se;
-        K.dq_a = P.dq_a; K.dq_b = P.dq_b; K.de_a = P.de_a; K.de_b = P.de_b;
-        K.dq_mode = P.dq_mode; K.de_mode = P.de_mode; K.block_log2 = P.block_log2; K.reset = P.reset; K.clip = P.clip;
-        K.seed_lo = P.seed_lo; K.seed_hi = P.seed_hi; K.k_lo = P.k_lo; K.k_hi = P.k_hi;
-        const bool stats = P.collect_stats != 0;
+        load_consts(C, K);
+        const bool stats = C.collect_stats != 0;
         RingAddr<GRAD, STATE> A;
         ring_addresses<GRAD, STATE, MODE>(static_cast<unsigned>(__cvta_generic_to_shared(ring)), lane, threadIdx.x >> 5, A);
         // this warp's wide rows are warp + i * nwarps, i < cnt
@@ -984,37 +1234,150 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_con
             fetch_row<GRAD, STATE, MODE>(A, slot_off, in);
             if (stage_wrow < full_wide) stage(stage_off, stage_wrow);
             cp_async_commit();                 // one group per iteration, empty near the end
-            if (!send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, wrow, lane, stats, saturated)) {
-                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, var_is_sr(VAR)>(P, part, static_cast<unsigned long long>(wrow) * kWide, lane);
-                careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, var_is_sr(VAR)>(P, part, static_cast<unsigned long long>(wrow) * kWide + kRow, lane);
-            }
+            if (!send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, wrow, lane, stats, saturated, state_saturated))
+                careful(static_cast<unsigned long long>(wrow) * kWide, 2);
             slot_off = slot_off + R::kSlotStride == R::kBytes ? 0u : slot_off + R::kSlotStride;
             stage_off = stage_off + R::kSlotStride == R::kBytes ? 0u : stage_off + R::kSlotStride;
             wrow += nwarps;
             stage_wrow += nwarps;
         }
     }
-    for (unsigned r = first_careful + warp; r < rows; r += nwarps)
-        careful_acc += send_row_careful<GRAD, STATE, BITS, MODE, var_is_sr(VAR)>(P, part, static_cast<unsigned long long>(r) * kRow, lane);
-    // each careful call adds at most 8 saturated codes and 2^31 per row with a non-finite value; the 64-bit
-    // sum keeps the flag apart from the count
-    const unsigned nonfinite = (careful_acc >> 31) != 0ull ? 1u : 0u;
-    saturated += static_cast<unsigned>(careful_acc & 0x7fffffffull);
+    // the careful routine's unit: a row, or the rows of a block wider than a row
+    const unsigned cu = (MODE == MODE_BLOCK && C.block_log2 > 8) ? (1u << (C.block_log2 - 8)) : 1u;
+    for (unsigned u = first_careful / cu + warp; u * cu < rows; u += nwarps)
+        careful(static_cast<unsigned long long>(u) * cu * kRow, static_cast<int>(cu));
+    flush_counts(Bk.status, C.collect_stats != 0, lane, saturated, state_saturated, nonfinite);
+}
 
-    if (__any_sync(kFull, nonfinite != 0u)) {
-        if (lane == 0) atomicOr(P.status, static_cast<unsigned long long>(kFlagNonFinite));
+// Several buckets per launch.  The work units of all buckets -- per bucket and partition, ceil(Lp / unit) units of
+// 512 elements (of one block when a block is wider) -- form one sequence; warp w of the grid takes units w, w + W,
+// w + 2W, ... of it, so that the grid streams through the buckets like through one long buffer: no bucket boundary
+// drains the machine, and the launch costs of a bucket are paid once per call.  A unit that is a fully valid wide row
+// travels through the ring and takes the fast routine; every other unit (partial and padding rows, wide blocks) goes
+// to the careful routine.  Two cursors walk the sequence: the consumer's and, D - 1 units ahead, the producer's.
+struct UnitCursor {
+    int b;                  // bucket (== count: past the end)
+    unsigned part, r;       // partition, unit within it
+    unsigned upp;           // units per partition of bucket b
+    unsigned full_wide;     // units of (b, part) that are fully valid wide rows
+};
+
+template <int GRAD, int STATE, int BITS, int MODE, int VAR>
+__global__ void __launch_bounds__(kThreads, 3) loco_send_multi_kernel(const __grid_constant__ SendMultiParams P) {
+    using R = Ring<GRAD, STATE, MODE>;
+    constexpr int D = R::kDepth;
+    constexpr unsigned gsize = (GRAD == GRAD_BF16 ? 2u : 4u), esize = (STATE == ST_INT8 ? 1u : 4u);
+    extern __shared__ __align__(16) uint8_t ring[];
+    const SendCommon &C = P.c;
+    const int lane = threadIdx.x & 31;
+    const unsigned warp = blockIdx.x * kWarps + (threadIdx.x >> 5);
+    const unsigned nwarps = gridDim.x * kWarps;
+    if (warp >= P.total_units) return;
+    const unsigned cnt = (P.total_units - warp + nwarps - 1) / nwarps;       // this warp's units
+    const bool fast = C.fast != 0 && P.unit_elems == static_cast<unsigned>(kWide);
+    const unsigned unit_rows = P.unit_elems / kRow;
+
+    auto segment = [&](UnitCursor &c) {          // what depends on (b, part)
+        c.full_wide = 0u;
+        if (c.b >= P.count) return;
+        const SendBucket &Bk = P.b[c.b];
+        const unsigned long long base = static_cast<unsigned long long>(c.part) * Bk.lp;
+        if (Bk.n > base) {
+            const unsigned long long avail = Bk.n - base;
+            c.full_wide = static_cast<unsigned>((avail >= Bk.lp ? Bk.lp : avail) / kWide);
+        }
+    };
+    auto normalise = [&](UnitCursor &c) {        // carry r into (part, b)
+        while (c.b < P.count && c.r >= c.upp) {
+            c.r -= c.upp;
+            if (++c.part == static_cast<unsigned>(P.parts)) {
+                c.part = 0u;
+                ++c.b;
+                c.upp = c.b < P.count ? P.b[c.b].units_per_part : 0u;
+            }
+            segment(c);
+        }
+    };
+    UnitCursor cc;
+    {
+        int b = 0;
+        while (b + 1 < P.count && P.b[b + 1].unit_begin <= warp) ++b;
+        cc.b = b;
+        cc.upp = P.b[b].units_per_part;
+        const unsigned local = warp - P.b[b].unit_begin;
+        cc.part = local / cc.upp;
+        cc.r = local - cc.part * cc.upp;
+        segment(cc);
     }
-    if (P.collect_stats) {
-        for (int o = 16; o > 0; o >>= 1) saturated += __shfl_xor_sync(kFull, saturated, o);
-        if (lane == 0 && saturated) atomicAdd(P.status + 1, static_cast<unsigned long long>(saturated));
+    UnitCursor pc = cc;
+
+    SendConsts K;
+    load_consts(C, K);
+    const bool stats = C.collect_stats != 0;
+    RingAddr<GRAD, STATE> A;
+    ring_addresses<GRAD, STATE, MODE>(static_cast<unsigned>(__cvta_generic_to_shared(ring)), lane, threadIdx.x >> 5, A);
+
+    auto produce = [&](unsigned slot_off) {      // the copies of the producer's unit, if it takes the fast routine; then on
+        if (fast && pc.b < P.count && pc.r < pc.full_wide) {
+            const SendBucket &Bk = P.b[pc.b];
+            const unsigned long long e0 = static_cast<unsigned long long>(pc.part) * Bk.lp + static_cast<unsigned long long>(pc.r) * kWide;
+            const float *scales = reinterpret_cast<const float *>(static_cast<const uint8_t *>(Bk.state) + ((Bk.n + 255ull) & ~255ull));
+            stage_row<GRAD, STATE, MODE>(A, slot_off, static_cast<const uint8_t *>(Bk.grad) + e0 * gsize + lane * 16,
+                                         static_cast<const uint8_t *>(Bk.state) + e0 * esize + lane * 16,
+                                         scales + ((e0 + static_cast<unsigned long long>(lane) * kWideLane) >> K.block_log2));
+        }
+        cp_async_commit();                       // one group per unit, empty for units that are not staged
+        pc.r += nwarps;
+        normalise(pc);
+    };
+#pragma unroll 1
+    for (int i = 0; i < D - 1; ++i) produce(i * R::kSlotStride);
+
+    unsigned saturated = 0u, state_saturated = 0u, nonfinite = 0u;
+    unsigned slot_off = 0u, stage_off = (D - 1) * R::kSlotStride;
+#pragma unroll 1
+    for (unsigned i = 0; i < cnt; ++i) {
+        const SendBucket &Bk = P.b[cc.b];
+        uint8_t *pbase = Bk.comm + static_cast<unsigned long long>(cc.part) * Bk.stride;
+        cp_async_wait<D - 2>();                // every group but the newest D-2 has landed: this unit's inputs are there
+        __syncwarp();                          // ... for all lanes; and every lane is done reading the slot refilled next
+        bool done = false;
+        if (fast && cc.r < cc.full_wide) {
+            WideIn<GRAD, STATE> in;
+            fetch_row<GRAD, STATE, MODE>(A, slot_off, in);
+            produce(stage_off);
+            LanePtrs L;
+            lane_pointers<STATE, BITS>(Bk, pbase, cc.part, static_cast<unsigned long long>(cc.r) * kWide, lane, L);
+            done = send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, 0u, lane, stats, saturated, state_saturated);
+        } else {
+            produce(stage_off);
+        }
+        if (!done) {
+            const unsigned rows = static_cast<unsigned>(Bk.lp / kRow);
+            const unsigned r0 = cc.r * unit_rows;
+            const unsigned nr = rows - r0 < unit_rows ? rows - r0 : unit_rows;
+            const CarefulCounts N = send_careful<GRAD, STATE, BITS, MODE, var_is_sr(VAR)>(
+                C, Bk, pbase, cc.part, static_cast<unsigned long long>(r0) * kRow, static_cast<int>(nr), lane);
+            saturated += N.saturated;
+            state_saturated += N.state_saturated;
+            nonfinite |= N.nonfinite;
+        }
+        slot_off = slot_off + R::kSlotStride == R::kBytes ? 0u : slot_off + R::kSlotStride;
+        stage_off = stage_off + R::kSlotStride == R::kBytes ? 0u : stage_off + R::kSlotStride;
+        const int b_before = cc.b;
+        cc.r += nwarps;
+        normalise(cc);
+        if (cc.b != b_before || i + 1 == cnt)
+            flush_counts(P.b[b_before].status, stats, lane, saturated, state_saturated, nonfinite);
     }
+    cp_async_wait<0>();
 }
 
 // ------------------------------------------------------------------------------------------
 // receive: Eq. 8 on wide rows of 512 outputs, 16 per lane.
 
 template <int BITS> struct WideCodes {                       // the 16 codes of one lane and wide row, as loaded
-    static constexpr int W = BITS / 2;                       // 32-bit words: 1, 2 or 4
+    static constexpr int W = BITS >= 2 ? BITS / 2 : 1;       // 32-bit words: 1 (sign code: its low half), 1, 2 or 4
     unsigned w[W];
 };
 
@@ -1022,14 +1385,22 @@ template <int BITS>
 __device__ __forceinline__ void load_codes(const uint8_t *src, WideCodes<BITS> &c) {
     if (BITS == 8) { const uint4 t = ld_stream16(src); c.w[0] = t.x; c.w[1 % WideCodes<BITS>::W] = t.y; c.w[2 % WideCodes<BITS>::W] = t.z; c.w[3 % WideCodes<BITS>::W] = t.w; }
     else if (BITS == 4) { const uint2 t = ld_stream8(src); c.w[0] = t.x; c.w[1 % WideCodes<BITS>::W] = t.y; }
-    else c.w[0] = ld_stream4(src);
+    else if (BITS == 2) c.w[0] = ld_stream4(src);
+    else c.w[0] = __ldcs(reinterpret_cast<const unsigned short *>(src));
 }
 
-// (a & b) | c in one instruction (the mask and the exponent live in registers)
-__device__ __forceinline__ unsigned and_or(unsigned a, unsigned b, unsigned c) {
+// (a & b) ^ c in one instruction
+__device__ __forceinline__ unsigned and_xor(unsigned a, unsigned b, unsigned c) {
     unsigned d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
     return d;
+}
+// Sign code: elements 2k and 2k+1 of a lane's 16 as +-mag (bit set = negative), mag >= 0 or any float whose sign
+// the code may flip.
+__device__ __forceinline__ f32x2 sign_pair(unsigned w, int k, unsigned mag) {
+    const unsigned x0 = and_xor(w << (31 - 2 * k), 0x80000000u, mag);
+    const unsigned x1 = and_xor(w << (30 - 2 * k), 0x80000000u, mag);
+    return pk2(__uint_as_float(x0), __uint_as_float(x1));
 }
 
 // The magic float 2^e + (code + 2^(p-1)) of field j: the field, with its top bit already flipped in x, is masked in
@@ -1168,13 +1539,6 @@ __device__ __forceinline__ void adam_finish16(const ReduceParams &P, unsigned lo
         }
     }
     if (P.out) store_out16<OUT>(P.out, oi, g, left, wide32);
-}
-
-// (a ^ b) & c in one instruction
-__device__ __forceinline__ unsigned xor_and(unsigned a, unsigned b, unsigned c) {
-    unsigned d;
-    asm("lop3.b32 %0, %1, %2, %3, 0x28;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
 }
 
 // Integer path (global power-of-two s, at most 16 workers): every dec(q; s) and every partial sum of Eq. 8
@@ -1338,6 +1702,11 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const Red
 #pragma unroll
             for (int i = 0; i < kGroup; ++i) {
                 if (g * kGroup + i >= N) break;
+                if (BITS == 1) {                 // sign code: d = +-scale, exact; the sum in worker order
+                    const unsigned mag = __float_as_uint(cur.sc[i]);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) acc2[k] = fadd2(acc2[k], sign_pair(cur.c[i].w[0], k, mag));
+                } else {
                 unsigned x[WideCodes<BITS>::W], xh[WideCodes<BITS>::W];
 #pragma unroll
                 for (int t = 0; t < WideCodes<BITS>::W; ++t) {
@@ -1364,6 +1733,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const Red
                         acc2[k] = pk2(__fadd_rn(c, __fdiv_rn(a, P.s)), __fadd_rn(d, __fdiv_rn(b, P.s)));
                     }
                 }
+                }
             }
             cur = nxt;
         }
@@ -1388,7 +1758,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const Red
 // with fewer workers it is all workers of 4/N rows, so that the bytes in flight per warp do not shrink with N.
 // All copies are 16 bytes wide (the narrower forms of cp.async move fewer bytes per instruction and are slower):
 // a 16-byte chunk holds the codes of 16 / (2 BITS) lanes, so one copy instruction of the warp fills 1, 2 or 4
-// entries, and cp.async.wait_group followed by __syncwarp() orders every lane's reads after all lanes' copies.
+// entries (with the sign code, 16 lanes fill the 4 entries of a group), and cp.async.wait_group followed by __syncwarp() orders every lane's reads after all lanes' copies.
 // One cp.async group per ring group; the ring holds kGroups of them, kGroups - 1 are in flight while one is summed.
 template <int BITS, int MODE> struct RecvRing {
     static constexpr unsigned kLaneBytes = 2u * BITS;                       // the 16 codes of one lane
@@ -1398,9 +1768,9 @@ template <int BITS, int MODE> struct RecvRing {
     static constexpr unsigned kWarpBytes = 8192u;
     static constexpr int kGroups = (kWarpBytes / kGroupBytes) > 8u ? 8 : static_cast<int>(kWarpBytes / kGroupBytes);
     static constexpr unsigned kCtaBytes = kWarps * kGroups * kGroupBytes;
-    static constexpr int kEntriesPerCopy = 16 / kLaneBytes;                 // entries one copy instruction fills: 4, 2, 1
-    static constexpr int kCopies = 4 / kEntriesPerCopy;                     // copy instructions per group: 1, 2, 4
-    static constexpr int kLanesPerEntry = 32 / kEntriesPerCopy;             // 8, 16, 32
+    static constexpr int kLanesPerEntry = static_cast<int>(kCodeBytes / 16u);   // 16-byte chunks of an entry: 4 (sign code), 8, 16, 32
+    static constexpr int kEntriesPerCopy = 32 / kLanesPerEntry > 4 ? 4 : 32 / kLanesPerEntry;   // entries one copy instruction fills: 4 (half the lanes idle), 4, 2, 1
+    static constexpr int kCopies = 4 / kEntriesPerCopy;                     // copy instructions per group: 1, 1, 2, 4
     static constexpr unsigned kChunkElems = 128u / BITS;                    // codes in a 16-byte chunk
     static_assert(kGroups >= 3, "the ring must hold at least three groups");
 };
@@ -1456,11 +1826,14 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
         cp_off[i] = poff + static_cast<unsigned long long>(warp + row_off) * kRowBytes + chunk * 16u;
     }
     // block mode: copy instruction i (of 2) brings the scales of entries 2i and 2i+1, lane % 16 = block within the row
+    // (a block wider than a wide row has one scale that all its rows fetch: the scale's index comes from the row's
+    // first element each time, not from a running offset)
     int sc_w[2], sc_lim[2];
-    unsigned sc_rowlim[2], sc_dst[2];
-    unsigned long long sc_off[2];
+    unsigned sc_rowlim[2], sc_dst[2], sc_row[2];
+    unsigned long long sc_base[2];
     if (MODE == MODE_BLOCK) {
-        const unsigned blocks_per_row = static_cast<unsigned>(kWide) >> P.block_log2;
+        const unsigned bpr = static_cast<unsigned>(kWide) >> P.block_log2;
+        const unsigned blocks_per_row = bpr ? bpr : 1u;
         const unsigned idx = static_cast<unsigned>(lane & 15);
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
@@ -1472,11 +1845,11 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
             sc_lim[i] = (j < group_entries && idx < blocks_per_row) ? N - sc_w[i] : 0;
             sc_rowlim[i] = lim_row > row_off ? lim_row - row_off : 0u;
             sc_dst[i] = static_cast<unsigned>(j) * R::kEntry + R::kCodeBytes + 4u * idx;
-            sc_off[i] = poff + P.code_bytes + 4ull * (((static_cast<unsigned long long>(warp + row_off) * kWide) >> P.block_log2) + idx);
+            sc_row[i] = warp + row_off;
+            sc_base[i] = poff + P.code_bytes + 4ull * idx;
         }
     }
     const unsigned long long code_step = static_cast<unsigned long long>(row_step) * kRowBytes;             // per advance of p_row
-    const unsigned long long scale_step = 4ull * ((static_cast<unsigned long long>(row_step) * kWide) >> P.block_log2);
 
     // producer: this warp's groups in order -- rows warp, warp + row_step, ...; within a row its chunks of C workers
     unsigned p_row = warp, p_slot = 0u, c_slot = 0u;
@@ -1489,7 +1862,9 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
         if (MODE == MODE_BLOCK) {
 #pragma unroll
             for (int i = 0; i < 2; ++i)
-                if (p_w0 < sc_lim[i] && p_row < sc_rowlim[i]) cp_async4(dst + sc_dst[i], P.parts[p_w0 + sc_w[i]] + sc_off[i]);
+                if (p_w0 < sc_lim[i] && p_row < sc_rowlim[i])
+                    cp_async4(dst + sc_dst[i], P.parts[p_w0 + sc_w[i]] + sc_base[i] +
+                                                   4ull * ((static_cast<unsigned long long>(sc_row[i]) * kWide) >> P.block_log2));
         }
         cp_async_commit();
         p_w0 += C;
@@ -1500,7 +1875,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
             for (int i = 0; i < R::kCopies; ++i) cp_off[i] += code_step;
             if (MODE == MODE_BLOCK) {
 #pragma unroll
-                for (int i = 0; i < 2; ++i) sc_off[i] += scale_step;
+                for (int i = 0; i < 2; ++i) sc_row[i] += row_step;
             }
         }
         p_slot = p_slot + 1 == static_cast<unsigned>(G) ? 0u : p_slot + 1;
@@ -1521,12 +1896,18 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
     auto fetch = [&](unsigned entry, WideCodes<BITS> &cw, float &scale) {             // this lane's codes (and scale) of an entry
         if (BITS == 8) { const uint4 t = lds16(entry + lane_byte); cw.w[0] = t.x; cw.w[1 % WideCodes<BITS>::W] = t.y; cw.w[2 % WideCodes<BITS>::W] = t.z; cw.w[3 % WideCodes<BITS>::W] = t.w; }
         else if (BITS == 4) { const uint2 t = lds8(entry + lane_byte); cw.w[0] = t.x; cw.w[1 % WideCodes<BITS>::W] = t.y; }
-        else cw.w[0] = lds4(entry + lane_byte);
+        else if (BITS == 2) cw.w[0] = lds4(entry + lane_byte);
+        else cw.w[0] = lds2(entry + lane_byte);
         scale = (PATH != PATH_INT && MODE == MODE_BLOCK) ? __uint_as_float(lds4(entry + scale_off)) : P.gen_mul;
     };
     auto accumulate = [&](const WideCodes<BITS> &cw, float scale) {                   // one worker's codes into the row's sums
         if (PATH == PATH_INT) {
             sums.add(cw);
+        } else if (BITS == 1) {
+            // sign code: d = +-scale (the global magnitude fl(1/s), or the worker's block scale); exact, then the sum in worker order
+            const unsigned mag = __float_as_uint(scale);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc2[k] = fadd2(acc2[k], sign_pair(cw.w[0], k, mag));
         } else {
             unsigned x[WideCodes<BITS>::W], xh[WideCodes<BITS>::W];
 #pragma unroll

@@ -12,22 +12,29 @@ namespace {
 
 template <int OUT, int BITS>
 ReduceKernel pick_reduce_path(int mode, int path) {
+    // the sign code has one form per scale rule: d = +-magnitude, summed in worker order
+    constexpr int kSignPath = PATH_MUL;
+    if (BITS == 1) path = kSignPath;
 #if LOCO_TU_ADAM
     if (mode != MODE_FIXED) return {loco_reduce_adam_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>, 0};
+    if (BITS == 1) return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, 0};
+    constexpr int B2 = BITS == 1 ? 2 : BITS;        // the other paths are not instantiated for the sign code
     switch (path) {
-    case PATH_INT: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_INT>, 0};
-    case PATH_MUL: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, 0};
-    case PATH_NEWTON: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON>, 0};
-    default: return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE>, 0};
+    case PATH_INT: return {loco_reduce_adam_kernel<OUT, B2, MODE_FIXED, PATH_INT>, 0};
+    case PATH_MUL: return {loco_reduce_adam_kernel<OUT, B2, MODE_FIXED, PATH_MUL>, 0};
+    case PATH_NEWTON: return {loco_reduce_adam_kernel<OUT, B2, MODE_FIXED, PATH_NEWTON>, 0};
+    default: return {loco_reduce_adam_kernel<OUT, B2, MODE_FIXED, PATH_DIVIDE>, 0};
     }
 #else
     if (mode != MODE_FIXED) return {loco_reduce_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>, static_cast<int>(RecvRing<BITS, MODE_BLOCK>::kCtaBytes)};
     const int smem = static_cast<int>(RecvRing<BITS, MODE_FIXED>::kCtaBytes);
+    if (BITS == 1) return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, smem};
+    constexpr int B2 = BITS == 1 ? 2 : BITS;
     switch (path) {
-    case PATH_INT: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_INT>, smem};
-    case PATH_MUL: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, smem};
-    case PATH_NEWTON: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_NEWTON>, smem};
-    default: return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_DIVIDE>, smem};
+    case PATH_INT: return {loco_reduce_kernel<OUT, B2, MODE_FIXED, PATH_INT>, smem};
+    case PATH_MUL: return {loco_reduce_kernel<OUT, B2, MODE_FIXED, PATH_MUL>, smem};
+    case PATH_NEWTON: return {loco_reduce_kernel<OUT, B2, MODE_FIXED, PATH_NEWTON>, smem};
+    default: return {loco_reduce_kernel<OUT, B2, MODE_FIXED, PATH_DIVIDE>, smem};
     }
 #endif
 }
@@ -36,6 +43,7 @@ ReduceKernel pick_reduce_path(int mode, int path) {
 
 ReduceKernel LOCO_REDUCE_TU_NAME(LOCO_TU_OUT, LOCO_TU_ADAM)(int bits, int mode, int path) {
     switch (bits) {
+    case 1: return pick_reduce_path<LOCO_TU_OUT, 1>(mode, path);
     case 2: return pick_reduce_path<LOCO_TU_OUT, 2>(mode, path);
     case 4: return pick_reduce_path<LOCO_TU_OUT, 4>(mode, path);
     default: return pick_reduce_path<LOCO_TU_OUT, 8>(mode, path);

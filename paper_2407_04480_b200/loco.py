@@ -32,7 +32,7 @@ EXPORTS = ("loco_state_bytes", "loco_packed_bytes", "loco_partition_bytes", "loc
            "loco_compensate_quantize_pack_host", "loco_unpack_dequant_reduce_host",
            "loco_unpack_dequant_reduce_host_noalloc", "loco_selfcheck_block_division",
            "loco_unpack_dequant_reduce_adam", "loco_compensate_quantize_pack_scatter",
-           "loco_compensate_quantize_pack_multi", "loco_unpack_dequant_reduce_multi")
+           "loco_compensate_quantize_pack_multi", "loco_unpack_dequant_reduce_multi", "loco_status_counters")
 NOALLOC_SCRATCH_BYTES = 4 * 1024 * 1024
 
 
@@ -132,6 +132,8 @@ def lib() -> C.CDLL:
         L.loco_selfcheck_block_division.argtypes = [C.POINTER(u64)]
         L.loco_last_status.restype = C.c_int
         L.loco_last_status.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(u64), vp]
+        L.loco_status_counters.restype = C.c_int
+        L.loco_status_counters.argtypes = [vp, C.POINTER(C.c_uint32), C.POINTER(u64), C.POINTER(u64), vp]
         L.loco_status_string.restype = C.c_char_p
         L.loco_status_string.argtypes = [C.c_int]
         L.loco_launch_count.restype = u64
@@ -332,6 +334,14 @@ def loco_last_status(st: State, stream=None):
     flags, sat = C.c_uint32(0), C.c_uint64(0)
     _check(lib().loco_last_status(st.handle, C.byref(flags), C.byref(sat), _stream_ptr(stream)), "loco_last_status")
     return int(flags.value), int(sat.value)
+
+
+def loco_status_counters(st: State, stream=None):
+    """(flags, saturated gradient codes, saturated 8-bit error codes) accumulated since init/reset; synchronises the stream."""
+    flags, sat, ssat = C.c_uint32(0), C.c_uint64(0), C.c_uint64(0)
+    _check(lib().loco_status_counters(st.handle, C.byref(flags), C.byref(sat), C.byref(ssat), _stream_ptr(stream)),
+           "loco_status_counters")
+    return int(flags.value), int(sat.value), int(ssat.value)
 
 
 # ---- host-buffer variants --------------------------------------------------------------------

@@ -64,6 +64,7 @@ class Worker:
         self.ostate = orc.new_state(ocfg, n)
         self.ocomm = orc.new_comm(ocfg, n, fill=CANARY)
         self.osat = 0
+        self.ossat = 0
         self.oflags = 0
 
     def step(self, grad_np: np.ndarray, k: int):
@@ -72,9 +73,10 @@ class Worker:
         loco.loco_compensate_quantize_pack(self.gstate, g, self.gcomm, k)
         loco.loco_compensate_quantize_pack(self.tstate, g, self.tcomm, k)
         torch.cuda.synchronize()
-        flags, sat = orc.send_step(self.ocfg, grad_np, self.ostate, self.ocomm, k)
+        flags, sat, ssat = orc.send_step(self.ocfg, grad_np, self.ostate, self.ocomm, k, full_status=True)
         self.oflags |= flags
         self.osat += sat
+        self.ossat += ssat
 
     def compare(self, where=""):
         self._compare(self.gcfg, self.gstate, self.gcomm, self.state_whole, self.comm_whole, where)
@@ -108,12 +110,14 @@ class Worker:
             assert nbad == 0, "%s: %d fp32 state words are not bit-identical" % (where, nbad)
         check_guards(state_whole, max(self.state_bytes, 16))
         check_guards(comm_whole, max(self.packed_bytes, 16))
-        flags, sat = loco.loco_last_status(gstate_obj)
+        flags, sat, ssat = loco.loco_status_counters(gstate_obj)
+        assert (flags, sat) == loco.loco_last_status(gstate_obj)
         assert flags == self.oflags, "%s: flags %d vs %d" % (where, flags, self.oflags)
         if gcfg.collect_stats:
             assert sat == self.osat, "%s: saturated %d vs %d" % (where, sat, self.osat)
-        elif not gcfg.collect_stats:
-            assert sat == 0
+            assert ssat == self.ossat, "%s: saturated error codes %d vs %d" % (where, ssat, self.ossat)
+        else:
+            assert sat == 0 and ssat == 0
 
 
 def reduce_both(gcfg, ocfg, n, workers, first=0, count=None):

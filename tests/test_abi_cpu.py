@@ -44,7 +44,7 @@ def test_binding_has_the_same_names():
 
 def test_sizes_agree_with_the_oracle_layout():
     ns = [0, 1, 255, 256, 257, 1000, 4096, 65537, 25_000_000, 13_015_864_320]
-    for bits, mode, B, P, fmt in itertools.product((2, 4, 8), (0, 1), (32, 256, 4096), (1, 3, 8, 64), (0, 1, 2, 3)):
+    for bits, mode, B, P, fmt in itertools.product((1, 2, 4, 8), (0, 1), (32, 256, 4096), (1, 3, 8, 64), (0, 1, 2, 3)):
         if mode == 1 and fmt == 3:
             continue
         kw = dict(bits=bits, scale_mode=mode, block_size=B, s=2.0 ** 14, s_e=2.0 ** 16, beta=0.5, reset_period=512,
@@ -66,11 +66,16 @@ def test_bad_configurations_are_rejected():
     for bad in (dict(bits=3), dict(bits=16), dict(s=0.0), dict(s=float("inf")), dict(s_e=-1.0), dict(beta=1.5),
                 dict(beta=float("nan")), dict(reset_period=-1), dict(num_partitions=0), dict(state_fmt=7),
                 dict(grad_dtype=2), dict(scale_mode=1, block_size=48), dict(scale_mode=1, block_size=16),
-                dict(scale_mode=1, state_fmt=3)):
+                dict(scale_mode=1, state_fmt=3), dict(scale_mode=1, block_size=8192), dict(bits=1, rounding=1),
+                dict(bits=0)):
         cfg = loco.Config(**{**good, **bad})
         assert loco.loco_config_check(cfg) == loco.ERR_ARG, bad
         assert loco.loco_state_bytes(cfg, 1000) == 0 and loco.loco_packed_bytes(cfg, 1000) == 0
-    assert loco.loco_config_check(loco.Config(scale_mode=1, block_size=1024)) == loco.ERR_UNSUPPORTED
+    # every block size the layout defines is one the kernels run: powers of two from 32 to 4096; and every code width
+    for B in (32, 64, 128, 256, 512, 1024, 2048, 4096):
+        for bits in (1, 2, 4, 8):
+            assert loco.loco_config_check(loco.Config(bits=bits, scale_mode=1, block_size=B)) == loco.OK
+    assert loco.loco_config_check(loco.Config(bits=1, **{k: v for k, v in good.items() if k != "bits"})) == loco.OK
 
 
 def test_null_arguments_return_codes_without_a_device():
