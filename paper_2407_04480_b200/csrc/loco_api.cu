@@ -414,8 +414,8 @@ void fill_bucket(const loco_state_t *st, const void *d_grad, void *d_comm, SendB
     B.n = st->n;
     B.lp = st->layout.lp;
     B.stride = st->layout.stride;
-    B.unit_begin = 0;
-    B.units_per_part = 0;
+    B.grid_x = 0;
+    B.reserved = 0;
 }
 
 // The handle's kernels were prepared (shared-memory size, occupancy) on the device that was current at
@@ -457,43 +457,30 @@ int send_launch(loco_state_t *st, const void *d_grad, void *d_comm, void *const 
     return LOCO_OK;
 }
 
-// Elements of a work unit of the multi-bucket kernel, and units per partition.
-inline uint64_t unit_elems_of(const loco_config_t &c) {
-    return (c.scale_mode == LOCO_SCALE_BLOCK_ABSMAX && c.block_size > kWide) ? static_cast<uint64_t>(c.block_size) : static_cast<uint64_t>(kWide);
-}
-
 bool same_send_setup(const loco_state_t *a, const loco_state_t *b) {
     return std::memcmp(&a->cfg, &b->cfg, sizeof(loco_config_t)) == 0 && a->send_multi_fn == b->send_multi_fn &&
            a->device == b->device && a->fast == b->fast;
 }
 
-// Buckets [lo, hi) of a multi-bucket call, all of one configuration, in one launch of the table-driven kernel.
+// Buckets [lo, hi) of a multi-bucket call, all of one configuration, in one launch: grid.z = buckets.
 int send_multi_launch(loco_state_t *const *states, const void *const *d_grads, void *const *d_comms, int lo, int hi,
                       int64_t step_k, void *stream) {
-    static thread_local SendMultiParams P;             // 32 KB: not on the stack
+    static thread_local SendMultiParams P;             // 29 KB: not on the stack
     const loco_state_t *first = states[lo];
     fill_common(first, step_k, P.c);
-    const uint64_t ue = unit_elems_of(first->cfg);
-    P.parts = first->cfg.num_partitions;
-    P.unit_elems = static_cast<unsigned>(ue);
     P.count = 0;
-    uint64_t units = 0;
+    unsigned gx = 1;
     for (int i = lo; i < hi; ++i) {
         const loco_state_t *st = states[i];
         if (st->n == 0) continue;
         SendBucket &B = P.b[P.count++];
         fill_bucket(st, d_grads[i], d_comms[i], B);
-        const uint64_t upp = (st->layout.lp + ue - 1) / ue;
-        B.unit_begin = static_cast<unsigned>(units);
-        B.units_per_part = static_cast<unsigned>(upp);
-        units += upp * static_cast<uint64_t>(P.parts);
+        B.grid_x = grid_x_for(st->layout.lp / kRow, st->cfg.num_partitions, st->send_ctas_per_sm);
+        if (B.grid_x > gx) gx = B.grid_x;
     }
     if (P.count == 0) return LOCO_OK;
-    P.total_units = static_cast<unsigned>(units);
-    const uint64_t budget = static_cast<uint64_t>(num_sms()) * static_cast<uint64_t>(first->send_ctas_per_sm);
-    const uint64_t want = (units + kWarps - 1) / kWarps;
-    const unsigned gx = static_cast<unsigned>(want < budget ? want : budget);
-    first->send_multi_fn<<<gx, kThreads, static_cast<size_t>(first->send_smem_bytes), static_cast<cudaStream_t>(stream)>>>(P);
+    dim3 grid(gx, static_cast<unsigned>(first->cfg.num_partitions), static_cast<unsigned>(P.count));
+    first->send_multi_fn<<<grid, kThreads, static_cast<size_t>(first->send_smem_bytes), static_cast<cudaStream_t>(stream)>>>(P);
     if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;
     g_launches.fetch_add(1);
     return LOCO_OK;
@@ -763,25 +750,13 @@ int loco_compensate_quantize_pack_multi(loco_state_t *const *states, const void 
         const int rc = check_device(states[i]);
         if (rc != LOCO_OK) return rc;
     }
-    // consecutive buckets of one configuration share a launch: as many as the kernel's table holds, and no more work
-    // units than a 32-bit counter (with room for the grid's stride) can number
+    // consecutive buckets of one configuration share a launch, as many as the kernel's table holds
     int rc = LOCO_OK;
     int32_t lo = 0;
     while (lo < count) {
-        int32_t hi = lo;
-        uint64_t units = 0;
-        const uint64_t ue = unit_elems_of(states[lo]->cfg);
-        while (hi < count && hi - lo < kMaxMulti && same_send_setup(states[lo], states[hi])) {
-            const uint64_t u = ((states[hi]->layout.lp + ue - 1) / ue) * static_cast<uint64_t>(states[hi]->cfg.num_partitions);
-            if (hi > lo && units + u > 0xF0000000ull) break;
-            units += u;
-            ++hi;
-        }
-        int r;
-        if (units > 0xF0000000ull)       // a single bucket beyond the counter's range: the one-bucket kernel (64-bit indices)
-            r = send_launch(states[lo], d_grads[lo], d_comms[lo], nullptr, step_k, stream);
-        else
-            r = send_multi_launch(states, d_grads, d_comms, lo, hi, step_k, stream);
+        int32_t hi = lo + 1;
+        while (hi < count && hi - lo < kMaxMulti && same_send_setup(states[lo], states[hi])) ++hi;
+        const int r = send_multi_launch(states, d_grads, d_comms, lo, hi, step_k, stream);
         if (r != LOCO_OK && rc == LOCO_OK) rc = r;
         lo = hi;
     }

@@ -75,8 +75,8 @@ struct SendBucket {
     unsigned long long n;            // bucket elements
     unsigned long long lp;           // elements per partition (multiple of 256 and of B)
     unsigned long long stride;       // bytes per partition
-    unsigned unit_begin;             // multi-bucket launches: first work unit of this bucket in the launch
-    unsigned units_per_part;         // multi-bucket launches: work units per partition
+    unsigned grid_x;                 // multi-bucket launches: CTAs per partition that work on this bucket
+    unsigned reserved;
 };
 
 struct SendParams {
@@ -91,10 +91,7 @@ struct SendParams {
 constexpr int kMaxMulti = 448;
 struct SendMultiParams {
     SendCommon c;
-    int count;                       // buckets
-    int parts;                       // partitions per bucket
-    unsigned total_units;            // work units of all buckets
-    unsigned unit_elems;             // elements of a work unit: 512, or B when B > 512
+    int count;                       // buckets = gridDim.z
     SendBucket b[kMaxMulti];
 };
 static_assert(sizeof(SendMultiParams) <= 32764, "kernel parameter space");
@@ -1162,29 +1159,23 @@ __device__ __forceinline__ void flush_counts(unsigned long long *status, bool co
     nonfinite = 0u;
 }
 
-// One bucket per launch.  grid = (ctas per partition, partitions).  Each warp walks the partition's wide rows with the
-// stride of all warps working on that partition; the inputs of its next rows are on their way through the cp.async
-// ring.  What is left of the partition (a last half-wide row, partial and padding rows; every block when a block is
-// wider than a wide row) goes to the careful routine.
-// VAR_LEAN / VAR_LEAN_NR kernels are launched when the host proved the corresponding decompressor forms and neither
-// statistics nor clipping are wanted (VAR_LEAN also for every block-scaled configuration), VAR_LEAN_X / VAR_LEAN_NR_X
-// when they are; VAR_GENERAL chooses the decompressor forms at run time.
+// The work of one CTA on partition `part` of one bucket: CTA `cta` of the `ctas` that share the partition.  Each warp walks
+// the partition's wide rows with the stride of all warps working on that partition; the inputs of its next rows are on
+// their way through the cp.async ring.  What is left of the partition (a last half-wide row, partial and padding rows;
+// every block when a block is wider than a wide row) goes to the careful routine.
 template <int GRAD, int STATE, int BITS, int MODE, int VAR>
-__global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_constant__ SendParams P) {
+__device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucket &Bk, uint8_t *pbase, unsigned long long part,
+                                            unsigned cta, unsigned ctas) {
     using R = Ring<GRAD, STATE, MODE>;
     constexpr int D = R::kDepth;
     constexpr unsigned gbytes = (GRAD == GRAD_BF16 ? 2u : 4u) * kWide;       // gradient bytes of a wide row
     constexpr unsigned ebytes = (STATE == ST_INT8 ? 1u : 4u) * kWide;        // state bytes of a wide row
     extern __shared__ __align__(16) uint8_t ring[];
-    const SendCommon &C = P.c;
-    const SendBucket &Bk = P.b;
     const int lane = threadIdx.x & 31;
-    const unsigned long long part = blockIdx.y;
-    const unsigned warp = blockIdx.x * kWarps + (threadIdx.x >> 5);
-    const unsigned nwarps = gridDim.x * kWarps;
+    const unsigned warp = cta * kWarps + (threadIdx.x >> 5);
+    const unsigned nwarps = ctas * kWarps;
     const unsigned rows = static_cast<unsigned>(Bk.lp / kRow);               // 256-element rows of the partition
     const unsigned long long base = part * Bk.lp;
-    uint8_t *pbase = P.scatter ? P.part_dst[part] : Bk.comm + part * Bk.stride;
     // rows [0, full_rows) of this partition lie entirely below n
     unsigned full_rows = 0;
     if (Bk.n > base) {
@@ -1249,128 +1240,28 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_con
     flush_counts(Bk.status, C.collect_stats != 0, lane, saturated, state_saturated, nonfinite);
 }
 
-// Several buckets per launch.  The work units of all buckets -- per bucket and partition, ceil(Lp / unit) units of
-// 512 elements (of one block when a block is wider) -- form one sequence; warp w of the grid takes units w, w + W,
-// w + 2W, ... of it, so that the grid streams through the buckets like through one long buffer: no bucket boundary
-// drains the machine, and the launch costs of a bucket are paid once per call.  A unit that is a fully valid wide row
-// travels through the ring and takes the fast routine; every other unit (partial and padding rows, wide blocks) goes
-// to the careful routine.  Two cursors walk the sequence: the consumer's and, D - 1 units ahead, the producer's.
-struct UnitCursor {
-    int b;                  // bucket (== count: past the end)
-    unsigned part, r;       // partition, unit within it
-    unsigned upp;           // units per partition of bucket b
-    unsigned full_wide;     // units of (b, part) that are fully valid wide rows
-};
+// One bucket per launch: grid = (CTAs per partition, partitions).
+// VAR_LEAN / VAR_LEAN_NR kernels are launched when the host proved the corresponding decompressor forms and neither
+// statistics nor clipping are wanted (VAR_LEAN also for every block-scaled configuration), VAR_LEAN_X / VAR_LEAN_NR_X
+// when they are; VAR_GENERAL chooses the decompressor forms at run time.
+template <int GRAD, int STATE, int BITS, int MODE, int VAR>
+__global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_constant__ SendParams P) {
+    const unsigned long long part = blockIdx.y;
+    uint8_t *pbase = P.scatter ? P.part_dst[part] : P.b.comm + part * P.b.stride;
+    send_bucket<GRAD, STATE, BITS, MODE, VAR>(P.c, P.b, pbase, part, blockIdx.x, gridDim.x);
+}
 
+// Several buckets per launch: grid = (most CTAs per partition any bucket wants, partitions, buckets).  The CTAs of
+// bucket z do exactly what the one-bucket kernel's CTAs do; the hardware hands them to the SMs in order -- all of
+// bucket 0, then bucket 1, ... -- as places become free, so an SM that streams faster than another simply receives
+// more of them, no bucket boundary drains the machine, and the launch costs are paid once per call.  The table of
+// buckets travels in the kernel's parameters.
 template <int GRAD, int STATE, int BITS, int MODE, int VAR>
 __global__ void __launch_bounds__(kThreads, 3) loco_send_multi_kernel(const __grid_constant__ SendMultiParams P) {
-    using R = Ring<GRAD, STATE, MODE>;
-    constexpr int D = R::kDepth;
-    constexpr unsigned gsize = (GRAD == GRAD_BF16 ? 2u : 4u), esize = (STATE == ST_INT8 ? 1u : 4u);
-    extern __shared__ __align__(16) uint8_t ring[];
-    const SendCommon &C = P.c;
-    const int lane = threadIdx.x & 31;
-    const unsigned warp = blockIdx.x * kWarps + (threadIdx.x >> 5);
-    const unsigned nwarps = gridDim.x * kWarps;
-    if (warp >= P.total_units) return;
-    const unsigned cnt = (P.total_units - warp + nwarps - 1) / nwarps;       // this warp's units
-    const bool fast = C.fast != 0 && P.unit_elems == static_cast<unsigned>(kWide);
-    const unsigned unit_rows = P.unit_elems / kRow;
-
-    auto segment = [&](UnitCursor &c) {          // what depends on (b, part)
-        c.full_wide = 0u;
-        if (c.b >= P.count) return;
-        const SendBucket &Bk = P.b[c.b];
-        const unsigned long long base = static_cast<unsigned long long>(c.part) * Bk.lp;
-        if (Bk.n > base) {
-            const unsigned long long avail = Bk.n - base;
-            c.full_wide = static_cast<unsigned>((avail >= Bk.lp ? Bk.lp : avail) / kWide);
-        }
-    };
-    auto normalise = [&](UnitCursor &c) {        // carry r into (part, b)
-        while (c.b < P.count && c.r >= c.upp) {
-            c.r -= c.upp;
-            if (++c.part == static_cast<unsigned>(P.parts)) {
-                c.part = 0u;
-                ++c.b;
-                c.upp = c.b < P.count ? P.b[c.b].units_per_part : 0u;
-            }
-            segment(c);
-        }
-    };
-    UnitCursor cc;
-    {
-        int b = 0;
-        while (b + 1 < P.count && P.b[b + 1].unit_begin <= warp) ++b;
-        cc.b = b;
-        cc.upp = P.b[b].units_per_part;
-        const unsigned local = warp - P.b[b].unit_begin;
-        cc.part = local / cc.upp;
-        cc.r = local - cc.part * cc.upp;
-        segment(cc);
-    }
-    UnitCursor pc = cc;
-
-    SendConsts K;
-    load_consts(C, K);
-    const bool stats = C.collect_stats != 0;
-    RingAddr<GRAD, STATE> A;
-    ring_addresses<GRAD, STATE, MODE>(static_cast<unsigned>(__cvta_generic_to_shared(ring)), lane, threadIdx.x >> 5, A);
-
-    auto produce = [&](unsigned slot_off) {      // the copies of the producer's unit, if it takes the fast routine; then on
-        if (fast && pc.b < P.count && pc.r < pc.full_wide) {
-            const SendBucket &Bk = P.b[pc.b];
-            const unsigned long long e0 = static_cast<unsigned long long>(pc.part) * Bk.lp + static_cast<unsigned long long>(pc.r) * kWide;
-            const float *scales = reinterpret_cast<const float *>(static_cast<const uint8_t *>(Bk.state) + ((Bk.n + 255ull) & ~255ull));
-            stage_row<GRAD, STATE, MODE>(A, slot_off, static_cast<const uint8_t *>(Bk.grad) + e0 * gsize + lane * 16,
-                                         static_cast<const uint8_t *>(Bk.state) + e0 * esize + lane * 16,
-                                         scales + ((e0 + static_cast<unsigned long long>(lane) * kWideLane) >> K.block_log2));
-        }
-        cp_async_commit();                       // one group per unit, empty for units that are not staged
-        pc.r += nwarps;
-        normalise(pc);
-    };
-#pragma unroll 1
-    for (int i = 0; i < D - 1; ++i) produce(i * R::kSlotStride);
-
-    unsigned saturated = 0u, state_saturated = 0u, nonfinite = 0u;
-    unsigned slot_off = 0u, stage_off = (D - 1) * R::kSlotStride;
-#pragma unroll 1
-    for (unsigned i = 0; i < cnt; ++i) {
-        const SendBucket &Bk = P.b[cc.b];
-        uint8_t *pbase = Bk.comm + static_cast<unsigned long long>(cc.part) * Bk.stride;
-        cp_async_wait<D - 2>();                // every group but the newest D-2 has landed: this unit's inputs are there
-        __syncwarp();                          // ... for all lanes; and every lane is done reading the slot refilled next
-        bool done = false;
-        if (fast && cc.r < cc.full_wide) {
-            WideIn<GRAD, STATE> in;
-            fetch_row<GRAD, STATE, MODE>(A, slot_off, in);
-            produce(stage_off);
-            LanePtrs L;
-            lane_pointers<STATE, BITS>(Bk, pbase, cc.part, static_cast<unsigned long long>(cc.r) * kWide, lane, L);
-            done = send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, 0u, lane, stats, saturated, state_saturated);
-        } else {
-            produce(stage_off);
-        }
-        if (!done) {
-            const unsigned rows = static_cast<unsigned>(Bk.lp / kRow);
-            const unsigned r0 = cc.r * unit_rows;
-            const unsigned nr = rows - r0 < unit_rows ? rows - r0 : unit_rows;
-            const CarefulCounts N = send_careful<GRAD, STATE, BITS, MODE, var_is_sr(VAR)>(
-                C, Bk, pbase, cc.part, static_cast<unsigned long long>(r0) * kRow, static_cast<int>(nr), lane);
-            saturated += N.saturated;
-            state_saturated += N.state_saturated;
-            nonfinite |= N.nonfinite;
-        }
-        slot_off = slot_off + R::kSlotStride == R::kBytes ? 0u : slot_off + R::kSlotStride;
-        stage_off = stage_off + R::kSlotStride == R::kBytes ? 0u : stage_off + R::kSlotStride;
-        const int b_before = cc.b;
-        cc.r += nwarps;
-        normalise(cc);
-        if (cc.b != b_before || i + 1 == cnt)
-            flush_counts(P.b[b_before].status, stats, lane, saturated, state_saturated, nonfinite);
-    }
-    cp_async_wait<0>();
+    const SendBucket &Bk = P.b[blockIdx.z];
+    if (blockIdx.x >= Bk.grid_x) return;
+    const unsigned long long part = blockIdx.y;
+    send_bucket<GRAD, STATE, BITS, MODE, VAR>(P.c, Bk, Bk.comm + part * Bk.stride, part, blockIdx.x, Bk.grid_x);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -225,3 +225,48 @@ def test_multi_send_mixed_configurations_fall_into_runs():
         orc.send_step(o, inputs.as_numpy_bits(grads[i]), ostate, ocomm, 1)
         assert np.array_equal(comms[i].cpu().numpy()[:ocomm.size], ocomm)
         assert np.array_equal(states[i].buffer.cpu().numpy()[:n], ostate[:n])
+
+
+@pytest.mark.parametrize("kw", [
+    dict(bits=4, s=2.0 ** 14, s_e=2.0 ** 16, state_fmt=loco.STATE_INT8, num_partitions=8),
+    dict(bits=4, scale_mode=loco.SCALE_BLOCK_ABSMAX, block_size=256, state_fmt=loco.STATE_INT8, num_partitions=8),
+])
+def test_multi_send_large_buckets(kw):
+    """Seven buckets of about 25M elements in one launch (the size of the benchmark's buckets, ragged lengths among them).
+    Bit-identical to the single-bucket calls, whose results the other tests hold against the oracle; one bucket's head
+    and ragged tail also directly against the oracle."""
+    sizes = [25_000_000, 24_999_999, 25_000_000, 13_415_616, 25_000_001, 25_000_000, 20_000_123]
+    base = dict(beta=0.5, reset_period=0, grad_dtype=loco.BF16, out_dtype=loco.BF16)
+    base.update(kw)
+    gcfg, ocfg = both_configs(collect_stats=1, **base)
+    grads = [inputs.gaussian(n, 1e-4, seed=71, worker=i, dtype=torch.bfloat16, device="cuda") for i, n in enumerate(sizes)]
+    grads[3][777_777] = float("nan")
+    multi = [loco.State(gcfg, n) for n in sizes]
+    single = [loco.State(gcfg, n) for n in sizes]
+    c_multi = [torch.zeros(loco.loco_packed_bytes(gcfg, n), dtype=torch.uint8, device="cuda") for n in sizes]
+    c_single = [torch.zeros_like(c) for c in c_multi]
+    ms = loco.MultiSend(multi, grads, c_multi)
+    before = loco.loco_launch_count()
+    for k in (1, 2):
+        loco.loco_compensate_quantize_pack_multi(ms, k)
+    torch.cuda.synchronize()
+    assert loco.loco_launch_count() - before == 2
+    for k in (1, 2):
+        for st, g, c in zip(single, grads, c_single):
+            loco.loco_compensate_quantize_pack(st, g, c, k)
+    torch.cuda.synchronize()
+    for i in range(len(sizes)):
+        assert torch.equal(c_multi[i], c_single[i]), "bucket %d: codes differ" % i
+        assert torch.equal(multi[i].buffer, single[i].buffer), "bucket %d: state differs" % i
+        assert loco.loco_status_counters(multi[i]) == loco.loco_status_counters(single[i])
+    assert loco.loco_status_counters(multi[3])[0] & loco.FLAG_NONFINITE
+    # the head of the last bucket against the oracle (every element or block is computed independently of the rest)
+    i, n, ln = len(sizes) - 1, sizes[-1], 1 << 18
+    o1 = orc.OracleConfig(**{**base, "num_partitions": 1})
+    ostate, ocomm = orc.new_state(o1, ln), orc.new_comm(o1, ln)
+    for k in (1, 2):
+        orc.send_step(o1, inputs.as_numpy_bits(grads[i][:ln]), ostate, ocomm, k)
+    (oc, osc), = orc.comm_views(o1, ln, ocomm)
+    got = c_multi[i].cpu().numpy()
+    assert np.array_equal(got[:ln * 4 // 8], oc[:ln * 4 // 8])
+    assert np.array_equal(multi[i].buffer[:ln].cpu().numpy(), ostate[:ln])
