@@ -226,11 +226,17 @@ int loco_unpack_dequant_reduce_adam(const loco_config_t *cfg, const void *const 
  * (No counterpart in the paper: a convenience of the library.)  Algorithm 1 is applied bucket by bucket, and a
  * bucket of the usual size is a kernel of 15-30 microseconds, a third of which is start-up and tail when the
  * kernels of a stream run strictly one after the other.  These two calls do what `count` single-bucket calls on
- * `stream` would do -- same kernels, same results, everything ordered after the work `stream` already holds and
- * before whatever is enqueued on it next -- but issue the launches in turn on three streams that the library
- * owns, so that one bucket's tail overlaps the start-up of the next ones.
+ * `stream` would do -- same arithmetic, same results, ordered like any other work on `stream` -- in ONE kernel
+ * launch: the buckets are the third dimension of the grid and their table (pointers and sizes) travels in the
+ * kernel's parameters, so nothing is allocated, nothing is synchronised and a captured launch carries its own copy
+ * of the table.  The hardware hands the blocks of bucket 0, then bucket 1, ... to the SMs as places become free: no
+ * bucket boundary drains the machine and the launch costs are paid once per call.
  *   - The buckets of one call must be independent of each other (distinct states and buffers), as they run
  *     concurrently.  All of them belong to the current device.
+ *   - A launch holds up to 448 buckets on the send side (consecutive buckets of one configuration share a launch;
+ *     a change of configuration starts a new one) and min(280, 2304 / num_workers) on the receive side; longer lists
+ *     take several launches.
+ *   - Every argument is checked before anything is launched: on an argument error nothing has been enqueued.
  * count = 0 does nothing.  Errors: as for the single-bucket calls, ARG for null arrays or entries.
  */
 

@@ -144,15 +144,31 @@ DecChoice choose_dec(float scale, int lo, int hi, int bias) {
     return c;
 }
 
-// Does multiplying by fl(1/scale) reproduce the division by `scale` for every integer in [lo, hi]?
-bool reciprocal_exact(float scale, int lo, int hi) {
-    const volatile float inv = 1.0f / scale;
-    for (int q = lo; q <= hi; ++q) {
-        const volatile float a = static_cast<float>(q) * inv;
-        const volatile float b = static_cast<float>(q) / scale;
-        if (!same_bits(a, b)) return false;
+// A multiplier m with fl(q * m) == fl(q / scale) for every integer q in [lo, hi]: fl(1/scale) or one of its
+// neighbours (for a handful of small codes such an m very often exists even when 1/scale itself rounds badly).
+bool exact_multiplier(float scale, int lo, int hi, float *mul) {
+    const volatile float vinv = 1.0f / scale;
+    const float inv = vinv;
+    if (!std::isfinite(inv) || inv <= 0.0f) return false;
+    uint32_t bits;
+    std::memcpy(&bits, &inv, 4);
+    for (int step = 0; step <= 8; ++step) {
+        for (int sign = -1; sign <= 1; sign += 2) {
+            if (step == 0 && sign > 0) continue;
+            const uint32_t cand_bits = bits + static_cast<uint32_t>(sign * step);
+            float cand;
+            std::memcpy(&cand, &cand_bits, 4);
+            if (!std::isfinite(cand) || cand <= 0.0f) continue;
+            bool ok = true;
+            for (int q = lo; q <= hi && ok; ++q) {
+                const volatile float a = static_cast<float>(q) * cand;
+                const volatile float b = static_cast<float>(q) / scale;
+                ok = same_bits(a, b);
+            }
+            if (ok) { *mul = cand; return true; }
+        }
     }
-    return true;
+    return false;
 }
 
 bool is_pow2_float(float x) {
@@ -506,11 +522,135 @@ int loco_compensate_quantize_pack_scatter(loco_state_t *st, const void *d_grad, 
 
 namespace {
 
-// The receive pass; with `ad` the Adam-family step is applied to the averaged gradient in the same kernel and d_out
-// (the gradient itself) becomes optional.
-int reduce_launch(const loco_config_t *cfg, const void *const *d_packed, int32_t num_workers, uint64_t n,
-                  int32_t first_partition, int32_t partition_count, void *d_out, const loco_adam_t *ad, float *d_m,
-                  float *d_v, float *d_theta, void *stream) {
+// What Eq. 8 needs that does not depend on the bucket: the forms of dec(q; s) and of the division by N that the host
+// can prove equal to the IEEE divisions, and with them the kernel (`path`).  `max_code_bytes`: the largest code area of
+// a part among the call's buckets (the integer path keeps 32-bit byte offsets).
+int reduce_common(const loco_config_t *cfg, int32_t num_workers, int32_t first_partition, uint64_t max_code_bytes,
+                  const loco_adam_t *ad, float *d_m, float *d_v, float *d_theta, ReduceCommon &C, int &mode, int &path) {
+    std::memset(&C, 0, sizeof(C));
+    C.first = static_cast<unsigned long long>(first_partition);
+    C.num_workers = num_workers;
+    C.block_log2 = cfg->scale_mode == LOCO_SCALE_BLOCK_ABSMAX ? ilog2(static_cast<uint32_t>(cfg->block_size)) : 0;
+    C.s = cfg->s;
+    C.n_workers_f = static_cast<float>(num_workers);
+    {
+        const volatile float inv_n = 1.0f / static_cast<float>(num_workers);
+        C.inv_n = inv_n;
+    }
+    mode = kernel_mode(cfg);
+    const bool n_pow2 = is_pow2(static_cast<uint64_t>(num_workers));
+    C.div_mode = n_pow2 ? 0 : 2;          // a multiply by 1/N is the division only for powers of two
+    C.gen_mul = 0.0f;
+    C.gen_mode = 2;
+    C.inv_s = 0.0f;
+    C.int_path = 0;
+    if (mode == MODE_FIXED && cfg->bits == 1) {
+        // sign code: d = +-fl(1/s), which is (+-1) / s exactly as the division gives it
+        const volatile float vinv = 1.0f / cfg->s;
+        C.inv_s = vinv;
+        C.gen_mul = vinv;
+        C.gen_mode = 0;
+    } else if (mode == MODE_FIXED) {
+        const int half = 1 << (cfg->bits - 1);
+        {
+            const volatile float vinv = 1.0f / cfg->s;
+            const float inv = vinv;
+            C.inv_s = inv;
+            float mul = 0.0f;
+            if (exact_multiplier(cfg->s, -half, half - 1, &mul)) {
+                C.gen_mul = mul;
+                C.gen_mode = 0;
+            } else if (std::isfinite(inv) && inv != 0.0f) {
+                bool nr_ok = true;
+                for (int q = -half; q < half && nr_ok; ++q) {
+                    const float fq = static_cast<float>(q);
+                    const volatile float want = fq / cfg->s;
+                    const volatile float q0 = fq * inv;
+                    const float rem = std::fmaf(q0, -cfg->s, fq);
+                    nr_ok = same_bits(std::fmaf(rem, inv, q0), want);
+                }
+                if (nr_ok) C.gen_mode = 1;
+            }
+        }
+        // Integer path: with s a power of two every partial sum of Eq. 8 is exact in fp32, so the codes can be
+        // added as integers.  The lane sums are bounded by (2^p - 1) * N, which 8- and 16-bit lanes hold for N <= 16.
+        if (num_workers <= 16 && is_pow2_float(cfg->s) && max_code_bytes < (1ull << 32)) {
+            C.int_path = 1;
+            const float inv_s = 1.0f / cfg->s;                                    // exact
+            float ra = inv_s;
+            if (n_pow2) ra = inv_s * C.inv_n;                                     // exact: both powers of two
+            C.ra = ra;
+            C.rb = -(kMagic + static_cast<float>(half * num_workers)) * ra;       // exact: integer < 2^24 times 2^k
+            if (!n_pow2) {
+                // acc takes the values t / s, t in [-half N, (half-1) N]: check the short division on all of them
+                bool nr_ok = true;
+                for (int t = -half * num_workers; t <= (half - 1) * num_workers && nr_ok; ++t) {
+                    const float acc = static_cast<float>(t) * inv_s;
+                    const volatile float want = acc / C.n_workers_f;
+                    const volatile float q0 = acc * C.inv_n;
+                    const float rem = std::fmaf(-q0, C.n_workers_f, acc);
+                    nr_ok = same_bits(std::fmaf(rem, C.inv_n, q0), want);
+                }
+                C.div_mode = nr_ok ? 1 : 2;
+            }
+        }
+    }
+    path = mode == MODE_BLOCK ? PATH_MUL
+           : (cfg->bits == 1 ? PATH_MUL : (C.int_path ? PATH_INT : (C.gen_mode == 0 ? PATH_MUL : (C.gen_mode == 1 ? PATH_NEWTON : PATH_DIVIDE))));
+    if (ad) {
+        C.adam_m = d_m; C.adam_v = d_v; C.adam_theta = d_theta;
+        C.lr = ad->lr; C.beta1 = ad->beta1; C.beta2 = ad->beta2; C.delta = ad->delta;
+        const volatile float o1 = 1.0f - ad->beta1, o2 = 1.0f - ad->beta2;       // rounded once to fp32
+        C.omb1 = o1; C.omb2 = o2;
+    }
+    return LOCO_OK;
+}
+
+// Per device and kernel, once: the shared-memory attributes of the kernels and the CTAs of one that fit an SM.
+int reduce_occupancy(const loco_config_t *cfg, int mode, int path, bool adam, const ReduceKernel &rk, int &occ) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return LOCO_ERR_CUDA;
+    }
+    static int occ_cache[64][2][4][2][4][2] = {};
+    static std::mutex occ_mu;
+    std::lock_guard<std::mutex> lock(occ_mu);
+    int &slot = occ_cache[dev][cfg->out_dtype == LOCO_BF16][cfg->bits == 1 ? 0 : (cfg->bits == 2 ? 1 : (cfg->bits == 4 ? 2 : 3))][mode][path][adam];
+    if (slot == 0) {
+        int v = 0;
+        if (rk.smem_bytes > 0) {
+            for (const void *fn : {reinterpret_cast<const void *>(rk.fn), reinterpret_cast<const void *>(rk.multi_fn)}) {
+                if (!fn) continue;
+                if (cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, rk.smem_bytes) != cudaSuccess ||
+                    cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess) {
+                    cudaGetLastError();
+                    return LOCO_ERR_CUDA;
+                }
+            }
+        }
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, rk.fn, kThreads, rk.smem_bytes) != cudaSuccess || v < 1) {
+            cudaGetLastError();
+            return LOCO_ERR_CUDA;
+        }
+        slot = v;
+    }
+    occ = slot;
+    return LOCO_OK;
+}
+
+void fill_reduce_bucket(const Layout &L, uint64_t n, void *d_out, ReduceBucket &B) {
+    B.out = d_out;
+    B.n = n;
+    B.lp = L.lp;
+    B.stride = L.stride;
+    B.code_bytes = L.code_bytes;
+    B.grid_x = 0;
+    B.out_align32 = (reinterpret_cast<uintptr_t>(d_out) & 31u) == 0 ? 1 : 0;
+}
+
+int check_reduce_args(const loco_config_t *cfg, int32_t num_workers, int32_t first_partition, int32_t partition_count,
+                      const loco_adam_t *ad) {
     const int rc = check_config(cfg);
     if (rc != LOCO_OK) return rc;
     if (num_workers < 1 || first_partition < 0 || partition_count < 0 ||
@@ -518,6 +658,16 @@ int reduce_launch(const loco_config_t *cfg, const void *const *d_packed, int32_t
     if (num_workers > 64) return LOCO_ERR_UNSUPPORTED;
     if (ad && !(std::isfinite(ad->lr) && ad->beta1 >= 0.0f && ad->beta1 <= 1.0f && ad->beta2 >= 0.0f && ad->beta2 <= 1.0f &&
                 ad->delta >= 0.0f && std::isfinite(ad->delta))) return LOCO_ERR_ARG;
+    return LOCO_OK;
+}
+
+// The receive pass; with `ad` the Adam-family step is applied to the averaged gradient in the same kernel and d_out
+// (the gradient itself) becomes optional.
+int reduce_launch(const loco_config_t *cfg, const void *const *d_packed, int32_t num_workers, uint64_t n,
+                  int32_t first_partition, int32_t partition_count, void *d_out, const loco_adam_t *ad, float *d_m,
+                  float *d_v, float *d_theta, void *stream) {
+    const int rc = check_reduce_args(cfg, num_workers, first_partition, partition_count, ad);
+    if (rc != LOCO_OK) return rc;
     if (n == 0 || partition_count == 0) return LOCO_OK;
     const Layout L = make_layout(cfg, n);
     if (static_cast<uint64_t>(first_partition) * L.lp >= n) return LOCO_OK;      // nothing valid there
@@ -532,121 +682,16 @@ int reduce_launch(const loco_config_t *cfg, const void *const *d_packed, int32_t
         if (!aligned16(d_packed[w])) return LOCO_ERR_ALIGN;
         P.parts[w] = static_cast<const uint8_t *>(d_packed[w]);
     }
-    P.out = d_out;
-    P.n = n;
-    P.lp = L.lp;
-    P.stride = L.stride;
-    P.code_bytes = L.code_bytes;
-    P.first = static_cast<unsigned long long>(first_partition);
-    P.num_workers = num_workers;
-    P.block_log2 = cfg->scale_mode == LOCO_SCALE_BLOCK_ABSMAX ? ilog2(static_cast<uint32_t>(cfg->block_size)) : 0;
-    P.s = cfg->s;
-    P.n_workers_f = static_cast<float>(num_workers);
-    {
-        const volatile float inv_n = 1.0f / static_cast<float>(num_workers);
-        P.inv_n = inv_n;
-    }
-    const int mode = kernel_mode(cfg);
-    const bool n_pow2 = is_pow2(static_cast<uint64_t>(num_workers));
-    P.div_mode = n_pow2 ? 0 : 2;          // a multiply by 1/N is the division only for powers of two
-    P.gen_mul = 0.0f;
-    P.gen_mode = 2;
-    P.inv_s = 0.0f;
-    P.int_path = 0;
-    P.out_align32 = (reinterpret_cast<uintptr_t>(d_out) & 31u) == 0 ? 1 : 0;
-    if (mode == MODE_FIXED && cfg->bits == 1) {
-        // sign code: d = +-fl(1/s), which is (+-1) / s exactly as the division gives it
-        const volatile float vinv = 1.0f / cfg->s;
-        P.inv_s = vinv;
-        P.gen_mul = vinv;
-        P.gen_mode = 0;
-    } else if (mode == MODE_FIXED) {
-        const int half = 1 << (cfg->bits - 1);
-        {
-            const volatile float vinv = 1.0f / cfg->s;
-            const float inv = vinv;
-            P.inv_s = inv;
-            if (reciprocal_exact(cfg->s, -half, half - 1)) {
-                P.gen_mul = inv;
-                P.gen_mode = 0;
-            } else if (std::isfinite(inv) && inv != 0.0f) {
-                bool nr_ok = true;
-                for (int q = -half; q < half && nr_ok; ++q) {
-                    const float fq = static_cast<float>(q);
-                    const volatile float want = fq / cfg->s;
-                    const volatile float q0 = fq * inv;
-                    const float rem = std::fmaf(q0, -cfg->s, fq);
-                    nr_ok = same_bits(std::fmaf(rem, inv, q0), want);
-                }
-                if (nr_ok) P.gen_mode = 1;
-            }
-        }
-        // Integer path: with s a power of two every partial sum of Eq. 8 is exact in fp32, so the codes can be
-        // added as integers.  The lane sums are bounded by (2^p - 1) * N, which 8- and 16-bit lanes hold for N <= 16.
-        if (num_workers <= 16 && is_pow2_float(cfg->s) && L.code_bytes < (1ull << 32)) {
-            P.int_path = 1;
-            const float inv_s = 1.0f / cfg->s;                                    // exact
-            float ra = inv_s;
-            if (n_pow2) ra = inv_s * P.inv_n;                                     // exact: both powers of two
-            P.ra = ra;
-            P.rb = -(kMagic + static_cast<float>(half * num_workers)) * ra;       // exact: integer < 2^24 times 2^k
-            if (!n_pow2) {
-                // acc takes the values t / s, t in [-half N, (half-1) N]: check the short division on all of them
-                bool nr_ok = true;
-                for (int t = -half * num_workers; t <= (half - 1) * num_workers && nr_ok; ++t) {
-                    const float acc = static_cast<float>(t) * inv_s;
-                    const volatile float want = acc / P.n_workers_f;
-                    const volatile float q0 = acc * P.inv_n;
-                    const float rem = std::fmaf(-q0, P.n_workers_f, acc);
-                    nr_ok = same_bits(std::fmaf(rem, P.inv_n, q0), want);
-                }
-                P.div_mode = nr_ok ? 1 : 2;
-            }
-        }
-    }
-    const int path = mode == MODE_BLOCK ? PATH_MUL
-                     : (P.int_path ? PATH_INT : (P.gen_mode == 0 ? PATH_MUL : (P.gen_mode == 1 ? PATH_NEWTON : PATH_DIVIDE)));
-    if (ad) {
-        P.adam_m = d_m; P.adam_v = d_v; P.adam_theta = d_theta;
-        P.lr = ad->lr; P.beta1 = ad->beta1; P.beta2 = ad->beta2; P.delta = ad->delta;
-        const volatile float o1 = 1.0f - ad->beta1, o2 = 1.0f - ad->beta2;       // rounded once to fp32
-        P.omb1 = o1; P.omb2 = o2;
-    }
+    int mode = 0, path = 0;
+    reduce_common(cfg, num_workers, first_partition, L.code_bytes, ad, d_m, d_v, d_theta, P.c, mode, path);
+    fill_reduce_bucket(L, n, d_out, P.b);
     const ReduceKernel rk = pick_reduce(cfg, mode, path, ad != nullptr);
-    const ReduceFn fn = rk.fn;
-    const int smem = rk.smem_bytes;
-    // per device and kernel, once: the shared-memory attributes of the kernel and the CTAs of it that fit an SM
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
-        cudaGetLastError();
-        return LOCO_ERR_CUDA;
-    }
-    static int occ_cache[64][2][4][2][4][2] = {};
-    static std::mutex occ_mu;
     int occ = 0;
-    {
-        std::lock_guard<std::mutex> lock(occ_mu);
-        int &slot = occ_cache[dev][cfg->out_dtype == LOCO_BF16][cfg->bits == 1 ? 0 : (cfg->bits == 2 ? 1 : (cfg->bits == 4 ? 2 : 3))][mode][path][ad != nullptr];
-        if (slot == 0) {
-            int v = 0;
-            if (smem > 0) {
-                if (cudaFuncSetAttribute(reinterpret_cast<const void *>(fn), cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
-                    cudaFuncSetAttribute(reinterpret_cast<const void *>(fn), cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess) {
-                    cudaGetLastError();
-                    return LOCO_ERR_CUDA;
-                }
-            }
-            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, fn, kThreads, smem) != cudaSuccess || v < 1) {
-                cudaGetLastError();
-                return LOCO_ERR_CUDA;
-            }
-            slot = v;
-        }
-        occ = slot;
-    }
+    const int ro = reduce_occupancy(cfg, mode, path, ad != nullptr, rk, occ);
+    if (ro != LOCO_OK) return ro;
     const uint64_t rows = (L.lp + kWide - 1) / kWide;
     dim3 grid(grid_x_for(rows, partition_count, occ), static_cast<unsigned>(partition_count), 1);
-    fn<<<grid, kThreads, static_cast<size_t>(smem), static_cast<cudaStream_t>(stream)>>>(P);
+    rk.fn<<<grid, kThreads, static_cast<size_t>(rk.smem_bytes), static_cast<cudaStream_t>(stream)>>>(P);
     if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;
     g_launches.fetch_add(1);
     return LOCO_OK;
@@ -674,64 +719,6 @@ int loco_unpack_dequant_reduce_adam(const loco_config_t *cfg, const void *const 
 }  // extern "C"
 
 namespace {
-
-// kSide streams and kSide + 1 events per device, owned by the library, over which the multi-bucket calls spread their
-// launches: fork from the caller's stream, take the side streams in turn, join back.  Created on a device's first
-// multi-bucket call, kept until exit.  Three streams: with two a kernel's tail overlaps the next kernel's start-up; the
-// third lets the kernel after that begin while both are still draining (measured 5 % over two on the send pass, no
-// further gain from a fourth).
-constexpr int kSide = 3;
-struct SideStreams {
-    cudaStream_t s[kSide] = {};
-    cudaEvent_t fork = nullptr, join[kSide] = {};
-    bool ready = false;
-    std::mutex in_use;          // one fork / launch / join sequence at a time: the events are shared
-};
-
-int side_streams(SideStreams **out) {
-    static SideStreams per_device[64];
-    static std::mutex mu;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return LOCO_ERR_CUDA; }
-    std::lock_guard<std::mutex> lock(mu);
-    SideStreams &S = per_device[dev];
-    if (!S.ready) {
-        bool ok = cudaEventCreateWithFlags(&S.fork, cudaEventDisableTiming) == cudaSuccess;
-        for (int i = 0; i < kSide && ok; ++i)
-            ok = cudaStreamCreateWithFlags(&S.s[i], cudaStreamNonBlocking) == cudaSuccess &&
-                 cudaEventCreateWithFlags(&S.join[i], cudaEventDisableTiming) == cudaSuccess;
-        if (!ok) { cudaGetLastError(); return LOCO_ERR_CUDA; }
-        S.ready = true;
-    }
-    *out = &S;
-    return LOCO_OK;
-}
-
-// Run launch(i, stream_i) for i < count with the launches taking the side streams in turn, all of them after what
-// `stream` holds now and all of them before what is enqueued on `stream` next.
-template <typename Launch>
-int fan_out(int32_t count, void *stream, Launch launch) {
-    SideStreams *S = nullptr;
-    int rc = side_streams(&S);
-    if (rc != LOCO_OK) return rc;
-    cudaStream_t user = static_cast<cudaStream_t>(stream);
-    std::lock_guard<std::mutex> lock(S->in_use);
-    if (cudaEventRecord(S->fork, user) != cudaSuccess) { cudaGetLastError(); return LOCO_ERR_CUDA; }
-    const int used = count < kSide ? count : kSide;
-    for (int i = 0; i < used; ++i)
-        if (cudaStreamWaitEvent(S->s[i], S->fork, 0) != cudaSuccess) { cudaGetLastError(); return LOCO_ERR_CUDA; }
-    for (int32_t i = 0; i < count; ++i) {
-        const int r = launch(i, static_cast<void *>(S->s[i % kSide]));
-        if (r != LOCO_OK && rc == LOCO_OK) rc = r;            // the join below still happens
-    }
-    for (int i = 0; i < used; ++i) {
-        if (cudaEventRecord(S->join[i], S->s[i]) != cudaSuccess || cudaStreamWaitEvent(user, S->join[i], 0) != cudaSuccess) {
-            cudaGetLastError();
-            if (rc == LOCO_OK) rc = LOCO_ERR_CUDA;
-        }
-    }
-    return rc;
-}
 
 }  // namespace
 
@@ -767,11 +754,54 @@ int loco_unpack_dequant_reduce_multi(const loco_config_t *cfg, const void *const
                                      const uint64_t *n, void *const *d_outs, int32_t count, void *stream) {
     if (count < 0 || (count > 0 && (!cfg || !d_packed || !n || !d_outs))) return LOCO_ERR_ARG;
     if (count == 0) return LOCO_OK;
-    const int rc = check_config(cfg);
-    if (rc != LOCO_OK) return rc;
-    return fan_out(count, stream, [&](int32_t i, void *s) {
-        return loco_unpack_dequant_reduce(cfg, d_packed[i], num_workers, n[i], 0, cfg->num_partitions, d_outs[i], s);
-    });
+    const int rc0 = check_reduce_args(cfg, num_workers, 0, cfg ? cfg->num_partitions : 0, nullptr);
+    if (rc0 != LOCO_OK) return rc0;
+    // every argument is checked before anything is launched
+    uint64_t max_code_bytes = 0;
+    for (int32_t i = 0; i < count; ++i) {
+        if (n[i] == 0) continue;
+        if (!d_packed[i] || !d_outs[i]) return LOCO_ERR_ARG;
+        if (!aligned16(d_outs[i])) return LOCO_ERR_ALIGN;
+        for (int w = 0; w < num_workers; ++w) {
+            if (!d_packed[i][w]) return LOCO_ERR_ARG;
+            if (!aligned16(d_packed[i][w])) return LOCO_ERR_ALIGN;
+        }
+        const uint64_t cb = make_layout(cfg, n[i]).code_bytes;
+        if (cb > max_code_bytes) max_code_bytes = cb;
+    }
+    static thread_local ReduceMultiParams P;           // 32 KB: not on the stack
+    int mode = 0, path = 0;
+    reduce_common(cfg, num_workers, 0, max_code_bytes, nullptr, nullptr, nullptr, nullptr, P.c, mode, path);
+    const ReduceKernel rk = pick_reduce(cfg, mode, path, false);
+    int occ = 0;
+    const int ro = reduce_occupancy(cfg, mode, path, false, rk, occ);
+    if (ro != LOCO_OK) return ro;
+    // as many buckets per launch as the kernel's tables hold
+    const int per_launch_ptrs = kMaxReducePtrs / num_workers;
+    const int per_launch = per_launch_ptrs < kMaxReduceBuckets ? per_launch_ptrs : kMaxReduceBuckets;
+    int rc = LOCO_OK;
+    int32_t i = 0;
+    while (i < count) {
+        P.count = 0;
+        unsigned gx = 1;
+        for (; i < count && P.count < per_launch; ++i) {
+            if (n[i] == 0) continue;
+            const Layout L = make_layout(cfg, n[i]);
+            ReduceBucket &B = P.b[P.count];
+            fill_reduce_bucket(L, n[i], d_outs[i], B);
+            B.grid_x = grid_x_for((L.lp + kWide - 1) / kWide, cfg->num_partitions, occ);
+            if (B.grid_x > gx) gx = B.grid_x;
+            for (int w = 0; w < num_workers; ++w)
+                P.parts[P.count * num_workers + w] = static_cast<const uint8_t *>(d_packed[i][w]);
+            ++P.count;
+        }
+        if (P.count == 0) break;
+        dim3 grid(gx, static_cast<unsigned>(cfg->num_partitions), static_cast<unsigned>(P.count));
+        rk.multi_fn<<<grid, kThreads, static_cast<size_t>(rk.smem_bytes), static_cast<cudaStream_t>(stream)>>>(P);
+        if (cudaGetLastError() != cudaSuccess) { if (rc == LOCO_OK) rc = LOCO_ERR_CUDA; }
+        else g_launches.fetch_add(1);
+    }
+    return rc;
 }
 
 uint64_t loco_send_host_workspace_bytes(const loco_config_t *cfg, uint64_t n) {

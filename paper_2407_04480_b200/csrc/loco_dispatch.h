@@ -14,7 +14,8 @@ using SendMultiFn = void (*)(const SendMultiParams);
 struct SendKernel { SendFn fn; SendMultiFn multi_fn; int smem_bytes; };   // one bucket / several buckets per launch; smem_bytes: the cp.async ring
 
 using ReduceFn = void (*)(const ReduceParams);
-struct ReduceKernel { ReduceFn fn; int smem_bytes; };       // smem_bytes: the kernel's cp.async ring (0: none)
+using ReduceMultiFn = void (*)(const ReduceMultiParams);
+struct ReduceKernel { ReduceFn fn; ReduceMultiFn multi_fn; int smem_bytes; };   // multi_fn: several buckets per launch (none with the fused optimizer step); smem_bytes: the cp.async ring (0: none)
 
 #define LOCO_SEND_TU_NAME_(g, s) pick_send_g##g##_s##s
 #define LOCO_SEND_TU_NAME(g, s) LOCO_SEND_TU_NAME_(g, s)

@@ -96,10 +96,8 @@ struct SendMultiParams {
 };
 static_assert(sizeof(SendMultiParams) <= 32764, "kernel parameter space");
 
-struct ReduceParams {
-    const uint8_t *parts[64];        // partition `first` of each worker
-    void *out;
-    unsigned long long n, lp, stride, code_bytes;
+// What a receive pass needs that is the same for every bucket of a call.
+struct ReduceCommon {
     unsigned long long first;        // first partition
     int num_workers;
     int block_log2;
@@ -108,14 +106,38 @@ struct ReduceParams {
     int int_path;                    // codes may be summed as integers (power-of-two s, N <= 16)
     float ra, rb;                    // int path: sum/s (and /N when exact) = fma(kMagic + S, ra, rb)
     int div_mode;                    // division by N: 0 folded into ra/rb or a multiply, 1 Newton-Raphson, 2 IEEE
-    float gen_mul;                   // generic FIXED path, gen_mode 0: fl(1/s), which reproduces q/s for every code
+    float gen_mul;                   // generic FIXED path, gen_mode 0: a multiplier that reproduces q/s for every code; sign code: fl(1/s)
     float inv_s;                     // fl(1/s) for gen_mode 1
     int gen_mode;                    // generic FIXED path: 0 multiply, 1 Newton-Raphson division, 2 IEEE division
-    int out_align32;                 // the output pointer is 32-byte aligned: 256-bit stores may be used
     // fused Adam-family step (kernels instantiated with ADAM): moments and weights of the same elements as `out`
     float *adam_m, *adam_v, *adam_theta;
     float lr, beta1, beta2, omb1, omb2, delta;
 };
+
+// One bucket of a receive pass.
+struct ReduceBucket {
+    void *out;
+    unsigned long long n, lp, stride, code_bytes;
+    unsigned grid_x;                 // multi-bucket launches: CTAs per partition that work on this bucket
+    int out_align32;                 // the output pointer is 32-byte aligned: 256-bit stores may be used
+};
+
+struct ReduceParams {
+    ReduceCommon c;
+    ReduceBucket b;
+    const uint8_t *parts[64];        // partition `first` of each worker
+};
+
+// Several buckets in one launch (grid.z): bucket z's workers are parts[z * num_workers ...].
+constexpr int kMaxReduceBuckets = 280;
+constexpr int kMaxReducePtrs = 2304;
+struct ReduceMultiParams {
+    ReduceCommon c;
+    int count;
+    ReduceBucket b[kMaxReduceBuckets];
+    const uint8_t *parts[kMaxReducePtrs];
+};
+static_assert(sizeof(ReduceMultiParams) <= 32764, "kernel parameter space");
 
 // ------------------------------------------------------------------------------------------
 // small helpers
@@ -1368,14 +1390,14 @@ __device__ __forceinline__ void store_out16(void *out, unsigned long long oi, co
 }
 
 // acc / N as Eq. 8 writes it
-__device__ __forceinline__ float div_workers(const ReduceParams &P, float acc) {
-    if (P.div_mode == 0) return __fmul_rn(acc, P.inv_n);
-    if (P.div_mode == 1) {
-        const float q0 = __fmul_rn(acc, P.inv_n);
-        const float rem = __fmaf_rn(-q0, P.n_workers_f, acc);
-        return __fmaf_rn(rem, P.inv_n, q0);
+__device__ __forceinline__ float div_workers(const ReduceCommon &C, float acc) {
+    if (C.div_mode == 0) return __fmul_rn(acc, C.inv_n);
+    if (C.div_mode == 1) {
+        const float q0 = __fmul_rn(acc, C.inv_n);
+        const float rem = __fmaf_rn(-q0, C.n_workers_f, acc);
+        return __fmaf_rn(rem, C.inv_n, q0);
     }
-    return __fdiv_rn(acc, P.n_workers_f);
+    return __fdiv_rn(acc, C.n_workers_f);
 }
 
 // The paper's Adam-family step on the 16 averaged gradients of one lane (Algorithm 1 step 3: the update that
@@ -1386,8 +1408,8 @@ struct AdamRegs { float m[16], v[16], t[16]; };
 
 // Start the loads of a lane's 16 moments and weights (issued before the workers' codes are summed, so that they
 // are in flight meanwhile).  Only for lanes whose 16 elements all exist.
-__device__ __forceinline__ void adam_load16(const ReduceParams &P, unsigned long long oi, AdamRegs &R) {
-    const float *pm = P.adam_m + oi, *pv = P.adam_v + oi, *pt = P.adam_theta + oi;
+__device__ __forceinline__ void adam_load16(const ReduceCommon &C, unsigned long long oi, AdamRegs &R) {
+    const float *pm = C.adam_m + oi, *pv = C.adam_v + oi, *pt = C.adam_theta + oi;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const uint4 a = ld_stream16(pm + 4 * j), b = ld_stream16(pv + 4 * j), c = ld_stream16(pt + 4 * j);
@@ -1398,15 +1420,15 @@ __device__ __forceinline__ void adam_load16(const ReduceParams &P, unsigned long
 }
 
 template <int OUT>
-__device__ __forceinline__ void adam_finish16(const ReduceParams &P, unsigned long long oi, const float (&g)[16],
+__device__ __forceinline__ void adam_finish16(const ReduceCommon &C, void *out, unsigned long long oi, const float (&g)[16],
                                               unsigned long long left, bool wide32, AdamRegs &R) {
-    float *pm = P.adam_m + oi, *pv = P.adam_v + oi, *pt = P.adam_theta + oi;
+    float *pm = C.adam_m + oi, *pv = C.adam_v + oi, *pt = C.adam_theta + oi;
     if (left >= 16) {                                    // R was loaded by adam_load16
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-            R.m[j] = __fadd_rn(__fmul_rn(P.omb1, R.m[j]), __fmul_rn(P.beta1, g[j]));
-            R.v[j] = __fadd_rn(__fmul_rn(P.omb2, R.v[j]), __fmul_rn(P.beta2, __fmul_rn(g[j], g[j])));
-            const float eta_k = __fdiv_rn(P.lr, __fsqrt_rn(__fadd_rn(R.v[j], P.delta)));
+            R.m[j] = __fadd_rn(__fmul_rn(C.omb1, R.m[j]), __fmul_rn(C.beta1, g[j]));
+            R.v[j] = __fadd_rn(__fmul_rn(C.omb2, R.v[j]), __fmul_rn(C.beta2, __fmul_rn(g[j], g[j])));
+            const float eta_k = __fdiv_rn(C.lr, __fsqrt_rn(__fadd_rn(R.v[j], C.delta)));
             R.t[j] = __fsub_rn(R.t[j], __fmul_rn(eta_k, R.m[j]));
         }
 #pragma unroll
@@ -1420,16 +1442,16 @@ __device__ __forceinline__ void adam_finish16(const ReduceParams &P, unsigned lo
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
             if (j < cnt) {
-                const float mk = __fadd_rn(__fmul_rn(P.omb1, pm[j]), __fmul_rn(P.beta1, g[j]));
-                const float vk = __fadd_rn(__fmul_rn(P.omb2, pv[j]), __fmul_rn(P.beta2, __fmul_rn(g[j], g[j])));
-                const float eta_k = __fdiv_rn(P.lr, __fsqrt_rn(__fadd_rn(vk, P.delta)));
+                const float mk = __fadd_rn(__fmul_rn(C.omb1, pm[j]), __fmul_rn(C.beta1, g[j]));
+                const float vk = __fadd_rn(__fmul_rn(C.omb2, pv[j]), __fmul_rn(C.beta2, __fmul_rn(g[j], g[j])));
+                const float eta_k = __fdiv_rn(C.lr, __fsqrt_rn(__fadd_rn(vk, C.delta)));
                 pm[j] = mk;
                 pv[j] = vk;
                 pt[j] = __fsub_rn(pt[j], __fmul_rn(eta_k, mk));
             }
         }
     }
-    if (P.out) store_out16<OUT>(P.out, oi, g, left, wide32);
+    if (out) store_out16<OUT>(out, oi, g, left, wide32);
 }
 
 // Integer path (global power-of-two s, at most 16 workers): every dec(q; s) and every partial sum of Eq. 8
@@ -1481,23 +1503,26 @@ enum : int { PATH_INT = 0, PATH_MUL = 1, PATH_NEWTON = 2, PATH_DIVIDE = 3 };
 // the codes are read with plain loads (one wide row at a time on the integer path, groups of four workers with the
 // next group's loads in flight on the others).
 template <int OUT, int BITS, int MODE, int PATH>
-__global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const ReduceParams P) {
+__global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const __grid_constant__ ReduceParams P) {
+    const ReduceCommon &C = P.c;
+    const ReduceBucket &Bk = P.b;
+    const uint8_t *const *parts = P.parts;
     constexpr unsigned kRowBytes = kWide * BITS / 8;                  // code bytes of one wide row
     const int lane = threadIdx.x & 31;
-    const unsigned long long part = blockIdx.y;                       // relative to P.first
+    const unsigned long long part = blockIdx.y;                       // relative to C.first
     const unsigned warp = blockIdx.x * kWarps + (threadIdx.x >> 5);
     const unsigned nwarps = gridDim.x * kWarps;
-    const unsigned long long base = (P.first + part) * P.lp;          // first bucket element of the part
-    if (base >= P.n) return;
-    const unsigned long long avail = P.n - base;
-    const unsigned long long valid = avail >= P.lp ? P.lp : avail;
+    const unsigned long long base = (C.first + part) * Bk.lp;          // first bucket element of the part
+    if (base >= Bk.n) return;
+    const unsigned long long avail = Bk.n - base;
+    const unsigned long long valid = avail >= Bk.lp ? Bk.lp : avail;
     const unsigned rows = static_cast<unsigned>((valid + kWide - 1) / kWide);
-    const unsigned long long poff = part * P.stride;
-    const unsigned long long out0 = part * P.lp;                      // output index of the part's first element
+    const unsigned long long poff = part * Bk.stride;
+    const unsigned long long out0 = part * Bk.lp;                      // output index of the part's first element
     const unsigned lane_elem = static_cast<unsigned>(lane) * kWideLane;
     const unsigned lane_byte = lane_elem * BITS / 8;
-    const int N = P.num_workers;
-    const bool wide32 = P.out_align32 != 0;
+    const int N = C.num_workers;
+    const bool wide32 = Bk.out_align32 != 0;
 
     if (PATH == PATH_INT) {
         // code areas below 4 GiB (checked by the host): row offsets fit 32 bits
@@ -1509,7 +1534,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const Red
             AdamRegs AR;
             {
                 const unsigned long long o = static_cast<unsigned long long>(r) * kWide + lane_elem;
-                if (o + 16 <= valid) adam_load16(P, out0 + o, AR);
+                if (o + 16 <= valid) adam_load16(C, out0 + o, AR);
             }
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
@@ -1520,7 +1545,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const Red
             }
 #pragma unroll 4
             for (int w = 0; w < N; ++w) {
-                const uint8_t *src = P.parts[w] + poff;
+                const uint8_t *src = parts[w] + poff;
                 WideCodes<BITS> cw[kUnroll];
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
@@ -1538,10 +1563,10 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const Red
                 float res[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
-                    const float acc = __fmaf_rn(sums[u].get(j), P.ra, P.rb);
-                    res[j] = P.div_mode == 0 ? acc : div_workers(P, acc);
+                    const float acc = __fmaf_rn(sums[u].get(j), C.ra, C.rb);
+                    res[j] = C.div_mode == 0 ? acc : div_workers(C, acc);
                 }
-                adam_finish16<OUT>(P, out0 + o, res, valid - o, wide32, AR);
+                adam_finish16<OUT>(C, Bk.out, out0 + o, res, valid - o, wide32, AR);
             }
         }
         return;
@@ -1562,21 +1587,21 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const Red
         const unsigned long long o = static_cast<unsigned long long>(row) * kWide + lane_elem;
         const bool in = row < rows && o < valid;
         const unsigned off = row * kRowBytes + lane_byte;
-        const unsigned long long sidx = o >> P.block_log2;
+        const unsigned long long sidx = o >> C.block_log2;
 #pragma unroll
         for (int i = 0; i < kGroup; ++i) {
             const int w = g * kGroup + i;
 #pragma unroll
             for (int t = 0; t < WideCodes<BITS>::W; ++t) G.c[i].w[t] = 0u;
-            G.sc[i] = P.gen_mul;
+            G.sc[i] = C.gen_mul;
             if (in && w < N) {
-                const uint8_t *wbase = P.parts[w] + poff;
+                const uint8_t *wbase = parts[w] + poff;
                 load_codes<BITS>(wbase + off, G.c[i]);
-                if (MODE == MODE_BLOCK) G.sc[i] = __ldg(reinterpret_cast<const float *>(wbase + P.code_bytes) + sidx);
+                if (MODE == MODE_BLOCK) G.sc[i] = __ldg(reinterpret_cast<const float *>(wbase + Bk.code_bytes) + sidx);
             }
         }
     };
-    const f32x2 inv2 = dup2(P.inv_s), negs2 = dup2(-P.s);
+    const f32x2 inv2 = dup2(C.inv_s), negs2 = dup2(-C.s);
     Group cur;
     if (warp < rows) load_group(warp, 0, cur);
     for (unsigned r = warp; r < rows; r += nwarps) {
@@ -1585,7 +1610,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const Red
 #pragma unroll
         for (int i = 0; i < 8; ++i) acc2[i] = 0ull;
         AdamRegs AR;
-        if (o + 16 <= valid) adam_load16(P, out0 + o, AR);
+        if (o + 16 <= valid) adam_load16(C, out0 + o, AR);
         for (int g = 0; g < groups; ++g) {
             Group nxt;
             if (g + 1 < groups) load_group(r, g + 1, nxt);
@@ -1621,7 +1646,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const Red
                         float a, b, c, d;
                         unpk2(q2, a, b);
                         unpk2(acc2[k], c, d);
-                        acc2[k] = pk2(__fadd_rn(c, __fdiv_rn(a, P.s)), __fadd_rn(d, __fdiv_rn(b, P.s)));
+                        acc2[k] = pk2(__fadd_rn(c, __fdiv_rn(a, C.s)), __fadd_rn(d, __fdiv_rn(b, C.s)));
                     }
                 }
                 }
@@ -1634,10 +1659,10 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const Red
         for (int i = 0; i < 8; ++i) {
             float a, b;
             unpk2(acc2[i], a, b);
-            res[2 * i] = div_workers(P, a);                                          // the 1/N of Eq. 8
-            res[2 * i + 1] = div_workers(P, b);
+            res[2 * i] = div_workers(C, a);                                          // the 1/N of Eq. 8
+            res[2 * i + 1] = div_workers(C, b);
         }
-        adam_finish16<OUT>(P, out0 + o, res, valid - o, wide32, AR);
+        adam_finish16<OUT>(C, Bk.out, out0 + o, res, valid - o, wide32, AR);
     }
 }
 
@@ -1666,30 +1691,31 @@ template <int BITS, int MODE> struct RecvRing {
     static_assert(kGroups >= 3, "the ring must hold at least three groups");
 };
 
+// The work of one CTA on part `part` (relative to C.first) of one bucket: CTA `cta` of the `ctas` that share the part.
 template <int OUT, int BITS, int MODE, int PATH>
-__global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_constant__ ReduceParams P) {
+__device__ __forceinline__ void reduce_bucket(const ReduceCommon &C, const ReduceBucket &Bk, const uint8_t *const *parts,
+                                              unsigned long long part, unsigned cta, unsigned ctas) {
     using R = RecvRing<BITS, MODE>;
     constexpr int G = R::kGroups;
     constexpr unsigned kRowBytes = kWide * BITS / 8;                  // code bytes of one wide row
     extern __shared__ __align__(16) uint8_t ring[];
     const int lane = threadIdx.x & 31;
-    const unsigned long long part = blockIdx.y;                       // relative to P.first
-    const unsigned warp = blockIdx.x * kWarps + (threadIdx.x >> 5);
-    const unsigned nwarps = gridDim.x * kWarps;
-    const unsigned long long base = (P.first + part) * P.lp;          // first bucket element of the part
-    if (base >= P.n) return;
-    const unsigned long long avail = P.n - base;
-    const unsigned long long valid = avail >= P.lp ? P.lp : avail;
+    const unsigned warp = cta * kWarps + (threadIdx.x >> 5);
+    const unsigned nwarps = ctas * kWarps;
+    const unsigned long long base = (C.first + part) * Bk.lp;          // first bucket element of the part
+    if (base >= Bk.n) return;
+    const unsigned long long avail = Bk.n - base;
+    const unsigned long long valid = avail >= Bk.lp ? Bk.lp : avail;
     const unsigned rows = static_cast<unsigned>((valid + kWide - 1) / kWide);
-    const unsigned long long poff = part * P.stride;
-    const unsigned long long out0 = part * P.lp;                      // output index of the part's first element
+    const unsigned long long poff = part * Bk.stride;
+    const unsigned long long out0 = part * Bk.lp;                      // output index of the part's first element
     const unsigned lane_elem = static_cast<unsigned>(lane) * kWideLane;
     const unsigned lane_byte = static_cast<unsigned>(lane) * R::kLaneBytes;
-    const int N = P.num_workers;
-    const bool wide32 = P.out_align32 != 0;
-    const int C = N < 4 ? N : 4;                                      // workers per group
-    const int group_entries = (4 / C) * C;                            // 4, 4, 3, 4: (rows per group) x C
-    const unsigned row_step = static_cast<unsigned>(4 / C) * nwarps;  // a group's rows are r, r + nwarps, ...
+    const int N = C.num_workers;
+    const bool wide32 = Bk.out_align32 != 0;
+    const int WG = N < 4 ? N : 4;                                      // workers per group
+    const int group_entries = (4 / WG) * WG;                            // 4, 4, 3, 4: (rows per group) x C
+    const unsigned row_step = static_cast<unsigned>(4 / WG) * nwarps;  // a group's rows are r, r + nwarps, ...
     const unsigned my_ring = static_cast<unsigned>(__cvta_generic_to_shared(ring)) +
                              (threadIdx.x >> 5) * (G * R::kGroupBytes);
 
@@ -1707,10 +1733,10 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
     for (int i = 0; i < R::kCopies; ++i) {
         const int j = i * R::kEntriesPerCopy + lane / R::kLanesPerEntry;
         const unsigned chunk = static_cast<unsigned>(lane % R::kLanesPerEntry);
-        const int rr = C == 1 ? j : (C == 2 ? (j >> 1) : 0);
+        const int rr = WG == 1 ? j : (WG == 2 ? (j >> 1) : 0);
         const unsigned row_off = static_cast<unsigned>(rr) * nwarps;
         const unsigned lim_row = full_rows + (chunk * R::kChunkElems < tail ? 1u : 0u);
-        cp_w[i] = j - rr * C;
+        cp_w[i] = j - rr * WG;
         cp_lim[i] = j < group_entries ? N - cp_w[i] : 0;
         cp_rowlim[i] = lim_row > row_off ? lim_row - row_off : 0u;
         cp_dst[i] = static_cast<unsigned>(j) * R::kEntry + chunk * 16u;
@@ -1723,21 +1749,21 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
     unsigned sc_rowlim[2], sc_dst[2], sc_row[2];
     unsigned long long sc_base[2];
     if (MODE == MODE_BLOCK) {
-        const unsigned bpr = static_cast<unsigned>(kWide) >> P.block_log2;
+        const unsigned bpr = static_cast<unsigned>(kWide) >> C.block_log2;
         const unsigned blocks_per_row = bpr ? bpr : 1u;
         const unsigned idx = static_cast<unsigned>(lane & 15);
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int j = 2 * i + (lane >> 4);
-            const int rr = C == 1 ? j : (C == 2 ? (j >> 1) : 0);
+            const int rr = WG == 1 ? j : (WG == 2 ? (j >> 1) : 0);
             const unsigned row_off = static_cast<unsigned>(rr) * nwarps;
-            const unsigned lim_row = full_rows + ((idx << P.block_log2) < tail ? 1u : 0u);
-            sc_w[i] = j - rr * C;
+            const unsigned lim_row = full_rows + ((idx << C.block_log2) < tail ? 1u : 0u);
+            sc_w[i] = j - rr * WG;
             sc_lim[i] = (j < group_entries && idx < blocks_per_row) ? N - sc_w[i] : 0;
             sc_rowlim[i] = lim_row > row_off ? lim_row - row_off : 0u;
             sc_dst[i] = static_cast<unsigned>(j) * R::kEntry + R::kCodeBytes + 4u * idx;
             sc_row[i] = warp + row_off;
-            sc_base[i] = poff + P.code_bytes + 4ull * idx;
+            sc_base[i] = poff + Bk.code_bytes + 4ull * idx;
         }
     }
     const unsigned long long code_step = static_cast<unsigned long long>(row_step) * kRowBytes;             // per advance of p_row
@@ -1749,16 +1775,16 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
         const unsigned dst = my_ring + p_slot * R::kGroupBytes;
 #pragma unroll
         for (int i = 0; i < R::kCopies; ++i)
-            if (p_w0 < cp_lim[i] && p_row < cp_rowlim[i]) cp_async16(dst + cp_dst[i], P.parts[p_w0 + cp_w[i]] + cp_off[i]);
+            if (p_w0 < cp_lim[i] && p_row < cp_rowlim[i]) cp_async16(dst + cp_dst[i], parts[p_w0 + cp_w[i]] + cp_off[i]);
         if (MODE == MODE_BLOCK) {
 #pragma unroll
             for (int i = 0; i < 2; ++i)
                 if (p_w0 < sc_lim[i] && p_row < sc_rowlim[i])
-                    cp_async4(dst + sc_dst[i], P.parts[p_w0 + sc_w[i]] + sc_base[i] +
-                                                   4ull * ((static_cast<unsigned long long>(sc_row[i]) * kWide) >> P.block_log2));
+                    cp_async4(dst + sc_dst[i], parts[p_w0 + sc_w[i]] + sc_base[i] +
+                                                   4ull * ((static_cast<unsigned long long>(sc_row[i]) * kWide) >> C.block_log2));
         }
         cp_async_commit();
-        p_w0 += C;
+        p_w0 += WG;
         if (p_w0 >= N) {
             p_w0 = 0;
             p_row += row_step;
@@ -1774,8 +1800,8 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
 
     WideSums<BITS> sums;                                              // PATH_INT
     f32x2 acc2[8];                                                    // the other paths
-    const f32x2 inv2 = dup2(P.inv_s), negs2 = dup2(-P.s);
-    const unsigned scale_off = R::kCodeBytes + 4u * (lane_elem >> P.block_log2);      // this lane's scale within an entry
+    const f32x2 inv2 = dup2(C.inv_s), negs2 = dup2(-C.s);
+    const unsigned scale_off = R::kCodeBytes + 4u * (lane_elem >> C.block_log2);      // this lane's scale within an entry
 
     auto begin_row = [&]() {
         if (PATH == PATH_INT) sums.clear();
@@ -1789,7 +1815,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
         else if (BITS == 4) { const uint2 t = lds8(entry + lane_byte); cw.w[0] = t.x; cw.w[1 % WideCodes<BITS>::W] = t.y; }
         else if (BITS == 2) cw.w[0] = lds4(entry + lane_byte);
         else cw.w[0] = lds2(entry + lane_byte);
-        scale = (PATH != PATH_INT && MODE == MODE_BLOCK) ? __uint_as_float(lds4(entry + scale_off)) : P.gen_mul;
+        scale = (PATH != PATH_INT && MODE == MODE_BLOCK) ? __uint_as_float(lds4(entry + scale_off)) : C.gen_mul;
     };
     auto accumulate = [&](const WideCodes<BITS> &cw, float scale) {                   // one worker's codes into the row's sums
         if (PATH == PATH_INT) {
@@ -1823,7 +1849,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
                     float a, b, cc, d;
                     unpk2(q2, a, b);
                     unpk2(acc2[k], cc, d);
-                    acc2[k] = pk2(__fadd_rn(cc, __fdiv_rn(a, P.s)), __fadd_rn(d, __fdiv_rn(b, P.s)));
+                    acc2[k] = pk2(__fadd_rn(cc, __fdiv_rn(a, C.s)), __fadd_rn(d, __fdiv_rn(b, C.s)));
                 }
             }
         }
@@ -1833,27 +1859,27 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
         float res[16];
         if (PATH == PATH_INT) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) res[i] = __fmaf_rn(sums.get(i), P.ra, P.rb);
+            for (int i = 0; i < 16; ++i) res[i] = __fmaf_rn(sums.get(i), C.ra, C.rb);
         } else {
 #pragma unroll
             for (int i = 0; i < 8; ++i) unpk2(acc2[i], res[2 * i], res[2 * i + 1]);
         }
         // one branch per row, not per element: which form the division by N takes is the same for the whole launch
-        if (PATH != PATH_INT && P.div_mode == 0) {
+        if (PATH != PATH_INT && C.div_mode == 0) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) res[i] = __fmul_rn(res[i], P.inv_n);
-        } else if (P.div_mode == 1) {
+            for (int i = 0; i < 16; ++i) res[i] = __fmul_rn(res[i], C.inv_n);
+        } else if (C.div_mode == 1) {
 #pragma unroll
             for (int i = 0; i < 16; ++i) {
-                const float q0 = __fmul_rn(res[i], P.inv_n);
-                const float rem = __fmaf_rn(-q0, P.n_workers_f, res[i]);
-                res[i] = __fmaf_rn(rem, P.inv_n, q0);
+                const float q0 = __fmul_rn(res[i], C.inv_n);
+                const float rem = __fmaf_rn(-q0, C.n_workers_f, res[i]);
+                res[i] = __fmaf_rn(rem, C.inv_n, q0);
             }
-        } else if (P.div_mode == 2) {
+        } else if (C.div_mode == 2) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) res[i] = __fdiv_rn(res[i], P.n_workers_f);
+            for (int i = 0; i < 16; ++i) res[i] = __fdiv_rn(res[i], C.n_workers_f);
         }
-        store_out16<OUT>(P.out, out0 + o, res, valid - o, wide32);
+        store_out16<OUT>(Bk.out, out0 + o, res, valid - o, wide32);
     };
 
     auto next_group = [&]() -> unsigned {      // wait for the oldest group, refill the slot summed last, return the group's ring address
@@ -1917,6 +1943,20 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_c
         }
     }
     cp_async_wait<0>();
+}
+
+// One bucket per launch: grid = (CTAs per part, parts).
+template <int OUT, int BITS, int MODE, int PATH>
+__global__ void __launch_bounds__(kThreads, 3) loco_reduce_kernel(const __grid_constant__ ReduceParams P) {
+    reduce_bucket<OUT, BITS, MODE, PATH>(P.c, P.b, P.parts, blockIdx.y, blockIdx.x, gridDim.x);
+}
+
+// Several buckets per launch: grid = (most CTAs per part any bucket wants, parts, buckets); see loco_send_multi_kernel.
+template <int OUT, int BITS, int MODE, int PATH>
+__global__ void __launch_bounds__(kThreads, 3) loco_reduce_multi_kernel(const __grid_constant__ ReduceMultiParams P) {
+    const ReduceBucket &Bk = P.b[blockIdx.z];
+    if (blockIdx.x >= Bk.grid_x) return;
+    reduce_bucket<OUT, BITS, MODE, PATH>(P.c, Bk, P.parts + blockIdx.z * P.c.num_workers, blockIdx.y, blockIdx.x, Bk.grid_x);
 }
 
 }  // namespace loco

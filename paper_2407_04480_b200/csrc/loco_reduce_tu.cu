@@ -10,33 +10,28 @@ namespace loco {
 
 namespace {
 
+template <int OUT, int BITS, int MODE, int PATH>
+ReduceKernel both() {
+#if LOCO_TU_ADAM
+    return {loco_reduce_adam_kernel<OUT, BITS, MODE, PATH>, nullptr, 0};
+#else
+    return {loco_reduce_kernel<OUT, BITS, MODE, PATH>, loco_reduce_multi_kernel<OUT, BITS, MODE, PATH>,
+            static_cast<int>(RecvRing<BITS, MODE>::kCtaBytes)};
+#endif
+}
+
 template <int OUT, int BITS>
 ReduceKernel pick_reduce_path(int mode, int path) {
+    if (mode != MODE_FIXED) return both<OUT, BITS, MODE_BLOCK, PATH_MUL>();
     // the sign code has one form per scale rule: d = +-magnitude, summed in worker order
-    constexpr int kSignPath = PATH_MUL;
-    if (BITS == 1) path = kSignPath;
-#if LOCO_TU_ADAM
-    if (mode != MODE_FIXED) return {loco_reduce_adam_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>, 0};
-    if (BITS == 1) return {loco_reduce_adam_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, 0};
+    if (BITS == 1) return both<OUT, BITS, MODE_FIXED, PATH_MUL>();
     constexpr int B2 = BITS == 1 ? 2 : BITS;        // the other paths are not instantiated for the sign code
     switch (path) {
-    case PATH_INT: return {loco_reduce_adam_kernel<OUT, B2, MODE_FIXED, PATH_INT>, 0};
-    case PATH_MUL: return {loco_reduce_adam_kernel<OUT, B2, MODE_FIXED, PATH_MUL>, 0};
-    case PATH_NEWTON: return {loco_reduce_adam_kernel<OUT, B2, MODE_FIXED, PATH_NEWTON>, 0};
-    default: return {loco_reduce_adam_kernel<OUT, B2, MODE_FIXED, PATH_DIVIDE>, 0};
+    case PATH_INT: return both<OUT, B2, MODE_FIXED, PATH_INT>();
+    case PATH_MUL: return both<OUT, B2, MODE_FIXED, PATH_MUL>();
+    case PATH_NEWTON: return both<OUT, B2, MODE_FIXED, PATH_NEWTON>();
+    default: return both<OUT, B2, MODE_FIXED, PATH_DIVIDE>();
     }
-#else
-    if (mode != MODE_FIXED) return {loco_reduce_kernel<OUT, BITS, MODE_BLOCK, PATH_MUL>, static_cast<int>(RecvRing<BITS, MODE_BLOCK>::kCtaBytes)};
-    const int smem = static_cast<int>(RecvRing<BITS, MODE_FIXED>::kCtaBytes);
-    if (BITS == 1) return {loco_reduce_kernel<OUT, BITS, MODE_FIXED, PATH_MUL>, smem};
-    constexpr int B2 = BITS == 1 ? 2 : BITS;
-    switch (path) {
-    case PATH_INT: return {loco_reduce_kernel<OUT, B2, MODE_FIXED, PATH_INT>, smem};
-    case PATH_MUL: return {loco_reduce_kernel<OUT, B2, MODE_FIXED, PATH_MUL>, smem};
-    case PATH_NEWTON: return {loco_reduce_kernel<OUT, B2, MODE_FIXED, PATH_NEWTON>, smem};
-    default: return {loco_reduce_kernel<OUT, B2, MODE_FIXED, PATH_DIVIDE>, smem};
-    }
-#endif
 }
 
 }  // namespace
