@@ -43,13 +43,55 @@ L2_BYTES = 126 * 1024 * 1024
 # Paper-faithful settings (Eq. 1 global scale; Eq. 7 T_c; s_e = 4 s); beta is not printed in the paper.
 CFG = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 14, s_e=2.0 ** 16, beta=0.5, reset_period=512,
            state_fmt=0, grad_dtype=1, out_dtype=1, num_partitions=WORKERS)
-# Algorithmic HBM bytes per element (bf16 gradient read, int8 state read + written, 4-bit code written).
-SEND_BYTES_PER_ELEM = 2 + 1 + 1 + 0.5
-# dram__bytes_read.sum + dram__bytes_write.sum per launch (one 25M-element bucket) from the ncu captures summarised under
-# profiles/.  Reads equal the algorithmic reads; most written lines are still in the 126 MB L2 when a lone launch ends,
-# so the DRAM write counter of a single captured launch is far below the algorithmic 37.5 / 50 MB.
-SEND_DRAM_BYTES_PER_LAUNCH = 75.03e6 + 2.53e6
-REDUCE_DRAM_BYTES_PER_LAUNCH = 100.03e6 + 14.24e6
+TRAFFIC_JSON = os.path.join(ROOT, "profiles", "dram_traffic_llama2_7b_buckets.json")
+KERNEL_SOURCES = ("paper_2407_04480_b200/csrc/loco_kernels.cuh", "paper_2407_04480_b200/csrc/loco_api.cu",
+                  "paper_2407_04480_b200/csrc/loco_send_tu.cu", "paper_2407_04480_b200/csrc/loco_reduce_tu.cu",
+                  "paper_2407_04480_b200/csrc/loco_dispatch.h")
+
+
+def cfg_for(scale: str) -> dict:
+    """The bench configuration with the paper's global scale ("fixed") or one fp32 scale per 256 elements ("block")."""
+    c = dict(CFG)
+    if scale == "block":
+        c["scale_mode"] = 1
+    return c
+
+
+def send_bytes_per_elem(c: dict) -> float:
+    """Algorithmic HBM bytes per element of the send pass: gradient read, state read + written, code written (+ the
+    block's wire scale written and its state scale read and written)."""
+    g = 2 if c["grad_dtype"] == 1 else 4
+    st = {0: 2, 1: 8, 2: 0, 3: 8}[c["state_fmt"]]
+    sc = (4.0 / c["block_size"]) * (3 if c["state_fmt"] == 0 else 1) if c["scale_mode"] == 1 else 0.0
+    return g + st + c["bits"] / 8 + sc
+
+
+def reduce_bytes_per_elem(c: dict, workers: int) -> float:
+    """Algorithmic HBM bytes per output element of the receive pass: N workers' codes (+ block scales) read, output written."""
+    o = 2 if c["out_dtype"] == 1 else 4
+    return workers * (c["bits"] / 8 + (4.0 / c["block_size"] if c["scale_mode"] == 1 else 0.0)) + o
+
+
+def kernel_sources_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for rel in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def stored_traffic(kernel: str, scale: str):
+    """DRAM bytes (read + written) per 25M-element bucket from the stored profiler capture, or None if there is none
+    for this case or the kernel sources have changed since it was taken."""
+    try:
+        with open(TRAFFIC_JSON) as f:
+            rec = json.load(f)
+        if rec.get("kernel_sources_sha256_16") != kernel_sources_hash():
+            return None
+        return float(rec[scale][kernel]["dram_bytes_per_bucket"])
+    except Exception:
+        return None
 
 
 def measured_peak():
@@ -119,10 +161,11 @@ class ClockSampler:
 class RankWorkload:
     """Buffers of one rank: its gradient, error state, own packed buffers, the 7 received parts, the output."""
 
-    def __init__(self, rank: int, device: torch.device, max_buckets: int = 0):
+    def __init__(self, rank: int, device: torch.device, max_buckets: int = 0, scale: str = "fixed"):
         from paper_2407_04480_b200 import inputs, loco
         self.loco = loco
-        self.cfg = loco.Config(**CFG)
+        self.cfgd = cfg_for(scale)
+        self.cfg = loco.Config(**self.cfgd)
         self.part = rank % WORKERS
         layout = inputs.llama2_7b()
         scales = inputs.group_scales(1, layout.n_groups)
@@ -139,14 +182,7 @@ class RankWorkload:
         pb = [loco.loco_packed_bytes(cfg, hi - lo) for lo, hi in self.buckets]
         self.state_buf = torch.empty(sum(sb), dtype=torch.uint8, device=device)
         self.comm_buf = torch.empty(sum(pb), dtype=torch.uint8, device=device)
-        # packed buffers of the 7 other workers as they would sit after the exchange: any byte is two valid codes
-        gen = torch.Generator(device=device)
-        gen.manual_seed(1234 + rank)
         self.recv_buf = torch.empty(sum(pb) * (WORKERS - 1), dtype=torch.uint8, device=device)
-        chunk = 1 << 30
-        for off in range(0, self.recv_buf.numel(), chunk):
-            m = min(chunk, self.recv_buf.numel() - off)
-            self.recv_buf[off:off + m] = torch.randint(0, 256, (m,), dtype=torch.uint8, device=device, generator=gen)
         self.out_buf = torch.empty(self.total, dtype=torch.bfloat16, device=device)
         self.states, self.grads, self.comms, self.packed, self.outs = [], [], [], [], []
         so = co = ro = 0
@@ -167,8 +203,32 @@ class RankWorkload:
             self.outs.append(self.out_buf[lo:hi])
             so += sb[i]
             co += pb[i]
-        self.send_bytes = SEND_BYTES_PER_ELEM * self.total
-        self.recv_bytes = self.total * (WORKERS * 0.5 + 2)
+        # packed buffers of the 7 other workers as they would sit after the exchange
+        if scale == "fixed":
+            # with the global scale any byte is two valid codes
+            gen = torch.Generator(device=device)
+            gen.manual_seed(1234 + rank)
+            chunk = 1 << 30
+            for off in range(0, self.recv_buf.numel(), chunk):
+                m = min(chunk, self.recv_buf.numel() - off)
+                self.recv_buf[off:off + m] = torch.randint(0, 256, (m,), dtype=torch.uint8, device=device, generator=gen)
+        else:
+            # block scales must be numbers a send pass produces: compress this rank's buckets once more without error
+            # feedback and give every other worker a copy in memory of its own
+            gen_cfg = loco.Config(**{**self.cfgd, "state_fmt": 2})
+            tmp = torch.empty(max(pb), dtype=torch.uint8, device=device)
+            ro = 0
+            for i, (lo, hi) in enumerate(self.buckets):
+                st = loco.State(gen_cfg, hi - lo)
+                loco.loco_compensate_quantize_pack(st, self.grads[i], tmp, 1)
+                for w in range(WORKERS - 1):
+                    self.recv_buf[ro:ro + pb[i]].copy_(tmp[:pb[i]])
+                    ro += pb[i]
+            torch.cuda.synchronize()
+        self.send_bpe = send_bytes_per_elem(self.cfgd)
+        self.recv_bpe = reduce_bytes_per_elem(self.cfgd, WORKERS)
+        self.send_bytes = self.send_bpe * self.total
+        self.recv_bytes = self.recv_bpe * self.total
         self.grad_bytes = 2 * self.total
 
     def _fan_out(self, launch, n_items: int, streams):
@@ -253,16 +313,22 @@ def run_e2e(wl: RankWorkload, steps: int, warmup: int):
     return ms, h2d, d2h
 
 
-def oracle_sample(threads: int, buckets_per_thread: int):
-    """The oracle as it stands on `threads` host threads, each doing whole 25M-element buckets of the
-    workload (send pass, then the receive pass over the whole bucket with 8 workers)."""
+def oracle_sample(threads: int, buckets_per_thread: int, cfgd: dict = None, n: int = BUCKET, workers: int = WORKERS,
+                  sigma: float = 1e-4):
+    """The oracle as it stands on `threads` host threads, each doing whole buckets of n elements of the workload (send
+    pass, then the receive pass over the whole bucket with `workers` workers).  Returns (GB/s of gradient, seconds,
+    elements)."""
     import numpy as np
     from oracle import loco_oracle as orc
-    ocfg = orc.OracleConfig(**CFG)
-    n = BUCKET
+    cfgd = dict(cfgd or CFG)
+    ocfg = orc.OracleConfig(**cfgd)
     rng = np.random.default_rng(1)
-    g = (rng.normal(0, 1e-4, n).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
-    others = [rng.integers(0, 256, orc.packed_bytes(ocfg, n), dtype=np.uint8) for _ in range(2)]
+    g32 = rng.normal(0, sigma, n).astype(np.float32)
+    gsz = 2 if cfgd["grad_dtype"] == 1 else 4
+    g = (g32.view(np.uint32) >> 16).astype(np.uint16) if gsz == 2 else g32
+    block = cfgd["scale_mode"] == 1
+    # the other workers' buffers: random codes with the global scale; with block scales a buffer the oracle itself packed
+    others = [] if block else [rng.integers(0, 256, orc.packed_bytes(ocfg, n), dtype=np.uint8) for _ in range(2)]
     states = [orc.new_state(ocfg, n) for _ in range(threads)]
     comms = [orc.new_comm(ocfg, n) for _ in range(threads)]
     orc.lib()
@@ -270,14 +336,23 @@ def oracle_sample(threads: int, buckets_per_thread: int):
     def work(t):
         for b in range(buckets_per_thread):
             orc.send_step(ocfg, g, states[t], comms[t], 1 + b)
-            orc.reduce(ocfg, n, [comms[t]] + [others[w % 2] for w in range(WORKERS - 1)])
+            orc.reduce(ocfg, n, [comms[t]] + [comms[t] if block else others[w % 2] for w in range(workers - 1)])
 
     t0 = time.perf_counter()
     with ThreadPoolExecutor(max_workers=threads) as ex:
         list(ex.map(work, range(threads)))
     dt = time.perf_counter() - t0
     elems = threads * buckets_per_thread * n
-    return 2.0 * elems / dt / 1e9, dt, elems
+    return gsz * elems / dt / 1e9, dt, elems
+
+
+def cpu_baseline_record(cores: int, cfgd: dict, n: int, workers: int, what: str, per_thread: int = 2):
+    """The oracle on all host cores and on one thread, on a bounded sample of the workload's buckets."""
+    v, dt, _ = oracle_sample(cores, per_thread, cfgd, n, workers)
+    v1, dt1, _ = oracle_sample(1, 1, cfgd, n, workers)
+    return {"value": v, "unit": "GB/s", "cores": cores, "kind": "oracle",
+            "sample": "%d %s (%d per host thread), send + %d-worker reduce, %.1f s wall" % (per_thread * cores, what, per_thread, workers, dt),
+            "one_thread_value": v1, "one_thread_sample": "1 of the same, %.1f s" % dt1}
 
 
 # ------------------------------------------------------------------------------------------------ real exchange
@@ -293,7 +368,7 @@ def run_exchange(args, rank: int, world: int, device, config):
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         os.environ.setdefault("MASTER_PORT", "29531")
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=device)
-    cfg = loco.Config(**{**CFG, "num_partitions": world})
+    cfg = loco.Config(**{**cfg_for(args.scale), "num_partitions": world})
     layout = inputs.llama2_7b()
     scales = inputs.group_scales(1, layout.n_groups)
     buckets = inputs.bucket_ranges(layout.numel, BUCKET)
@@ -396,14 +471,21 @@ def sweep(args, device):
     # launches alternate between three streams, as the library's multi-bucket calls issue them (one stream with --streams 1)
     streams = [torch.cuda.Stream(device=device) for _ in range(3 if args.streams > 1 else 1)]
     rows = []
-    budget = 6 << 30                    # device bytes per case
+    budget = int(args.sweep_budget_gb * (1 << 30))      # device bytes per case
 
     def sets_for(bytes_per_set):
+        """Independent working sets of a case: enough that no launch finds its data in L2 (>= 1 GB in all), at least three
+        (concurrent launches must not share buffers), within the memory budget; a case too large for three sets gets one
+        and its launches are then issued on one stream."""
         want = max(3, -(-(1 << 30) // bytes_per_set))
-        return int(max(1, min(want, 256, budget // max(1, bytes_per_set))))
+        have = int(min(want, 256, budget // max(1, bytes_per_set)))
+        return have if have >= 3 else 1
+
+    def streams_for(nsets):
+        return streams if nsets >= 3 else streams[:1]
 
     def send_case(label, n, **kw):
-        if args.sweep_filter and args.sweep_filter not in "send: " + label:
+        if args.sweep_filter and args.sweep_filter not in "send: " + label + " |":
             return
         base = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=512, state_fmt=0,
                     grad_dtype=1, out_dtype=1, num_partitions=8)
@@ -427,7 +509,7 @@ def sweep(args, device):
         for i in range(nsets):                      # a first iteration, so that the timed ones meet a non-zero state
             send(i, 1)
         torch.cuda.synchronize()
-        us = _time_launches(lambda i, st: send(i, 2, st), nsets, max(12, min(200, 4 * nsets)), streams)
+        us = _time_launches(lambda i, st: send(i, 2, st), nsets, max(12, min(200, 4 * nsets)), streams_for(nsets))
         state_rw = {0: 2, 1: 8, 2: 0, 3: 8}[cfg.state_fmt]
         scale_b = (4.0 / cfg.block_size) * (3 if cfg.state_fmt == 0 else 1) if cfg.scale_mode == 1 else 0.0
         bpe = gsz + state_rw + cfg.bits / 8 + scale_b
@@ -438,7 +520,7 @@ def sweep(args, device):
         print(json.dumps(rows[-1]), flush=True)
 
     def reduce_case(label, n, workers, **kw):
-        if args.sweep_filter and args.sweep_filter not in "reduce: " + label:
+        if args.sweep_filter and args.sweep_filter not in "reduce: " + label + " | N=%d |" % workers:
             return
         base = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=512, state_fmt=2,
                     grad_dtype=1, out_dtype=1, num_partitions=8)
@@ -469,11 +551,11 @@ def sweep(args, device):
             slots = [[b[3 * stride:4 * stride] for b in bufs] for bufs in packed]
             us = _time_launches(lambda i, st: loco.loco_unpack_dequant_reduce(cfg, slots[i], n, outs[i], first_partition=3,
                                                                                 partition_count=1, stream=st),
-                                nsets, max(12, min(200, 4 * nsets)), streams)
+                                nsets, max(12, min(200, 4 * nsets)), streams_for(nsets))
             n = loco.loco_partition_elems(cfg, n, 3)        # elements this launch produces
         else:
             us = _time_launches(lambda i, st: loco.loco_unpack_dequant_reduce(cfg, packed[i], n, outs[i], stream=st),
-                                nsets, max(12, min(200, 4 * nsets)), streams)
+                                nsets, max(12, min(200, 4 * nsets)), streams_for(nsets))
         bpe = workers * cfg.bits / 8 + osz + (workers * 4.0 / cfg.block_size if cfg.scale_mode == 1 else 0.0)
         gbs = bpe * n / us / 1e3
         rows.append(dict(kernel="reduce", case=label, n=n, workers=workers, bytes_per_elem=round(bpe, 3), us=round(us, 2),
@@ -482,7 +564,7 @@ def sweep(args, device):
         print(json.dumps(rows[-1]), flush=True)
 
     def adam_case(label, n, workers, **kw):
-        if args.sweep_filter and args.sweep_filter not in "reduce+adam: " + label:
+        if args.sweep_filter and args.sweep_filter not in "reduce+adam: " + label + " | N=%d |" % workers:
             return
         base = dict(bits=4, scale_mode=0, block_size=256, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=512, state_fmt=2,
                     grad_dtype=1, out_dtype=1, num_partitions=8)
@@ -500,7 +582,7 @@ def sweep(args, device):
         torch.cuda.synchronize()
         us = _time_launches(lambda i, st: loco.loco_unpack_dequant_reduce_adam(cfg, packed[i], n, ms[i], vs[i], ths[i], lr=1e-3, beta1=0.1,
                                                                                  beta2=0.001, delta=1e-16, stream=st),
-                            nsets, max(12, min(200, 4 * nsets)), streams)
+                            nsets, max(12, min(200, 4 * nsets)), streams_for(nsets))
         bpe = workers * cfg.bits / 8 + 24
         gbs = bpe * n / us / 1e3
         rows.append(dict(kernel="reduce+adam", case=label, n=n, workers=workers, bytes_per_elem=round(bpe, 3), us=round(us, 2),
@@ -528,6 +610,10 @@ def sweep(args, device):
     for B in (256, 64, 32):
         send_case("bf16 g, int8 state, 4 bit, block-%d absmax" % B, M, scale_mode=1, block_size=B)
     send_case("fp32 g, int8 state, 4 bit, block-256 absmax", M, scale_mode=1, grad_dtype=0)
+    for B in (512, 1024, 4096):
+        send_case("bf16 g, int8 state, 4 bit, block-%d absmax%s" % (B, "" if B == 512 else " (block walked in several passes)"), M, scale_mode=1, block_size=B)
+    send_case("bf16 g, int8 state, 1 bit (sign code), fixed", M, bits=1)
+    send_case("bf16 g, int8 state, 1 bit (sign code), block-256 mean magnitude", M, bits=1, scale_mode=1)
     for log2n in (16, 20, 24, 27, 30):
         reduce_case("4 bit, bf16 out, fixed", 1 << log2n, 8)
     for bits in (2, 4, 8):
@@ -541,6 +627,9 @@ def sweep(args, device):
     reduce_case("4 bit, bf16 out, block-256 absmax", M, 8, scale_mode=1)
     reduce_case("4 bit, bf16 out, block-32 absmax", M, 8, scale_mode=1, block_size=32)
     reduce_case("8 bit, bf16 out, block-256 absmax, 1 worker (Zero++-style weight payload)", M, 1, bits=8, scale_mode=1)
+    reduce_case("4 bit, bf16 out, block-1024 absmax", M, 8, scale_mode=1, block_size=1024)
+    reduce_case("1 bit (sign code), bf16 out, fixed", M, 8, bits=1)
+    reduce_case("1 bit (sign code), bf16 out, block-256 mean magnitude", M, 8, bits=1, scale_mode=1)
     for N in (1, 8, 16):
         adam_case("4 bit, fixed, Adam-family step fused, no gradient output", M, N)
     adam_case("8 bit, fixed, Adam-family step fused, no gradient output", M, 8, bits=8)
@@ -552,6 +641,121 @@ def sweep(args, device):
                                                                       r["us"], r["hbm_gbs"], r["frac"], r["grad_gbs"], "yes" if r["l2_resident"] else ""))
 
 
+def run_other_config(args, device, cores):
+    """--config 1 | 3 | 4: the other workload configurations, one JSON line each with a row per pass and scale rule
+    (GB/s of gradient, HBM GB/s, fraction of the measured and of the nominal peak) next to the oracle on one thread and
+    on all host cores for the same shape."""
+    from paper_2407_04480_b200 import inputs, loco
+    peak, peak_kind = measured_peak()
+    rows = []
+
+    def timed(fn, reps, warm=3):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / reps          # microseconds
+
+    def row(kind, label, n_elems, bpe, esize, us, note=""):
+        gbs = bpe * n_elems / us / 1e3
+        r = dict(kernel=kind, case=label, n=n_elems, bytes_per_elem=round(bpe, 3), us=round(us, 2), hbm_gbs=round(gbs, 1),
+                 frac_of_measured=round(gbs / peak, 3), frac_of_nominal_8TBps=round(gbs / 8000.0, 3),
+                 gradient_gbs=round(esize * n_elems / us / 1e3, 1), note=note)
+        rows.append(r)
+        print(json.dumps(r), flush=True)
+
+    launches_before = loco.loco_launch_count()
+    if args.config == 1:
+        # one fp32 vector of 2^20 elements, 1 worker, 4 error-feedback steps: 6.5 MB per pass, resident in the 126 MB L2
+        n, workload = 1 << 20, "config 1: one fp32 vector of 1,048,576 elements, 1 worker, 4 error-feedback steps (L2-resident: 6.5 MB per pass)"
+        for scale in ("fixed", "block"):
+            c = dict(cfg_for(scale), s=2.0 ** 11, s_e=2.0 ** 13, grad_dtype=0, out_dtype=0, num_partitions=1)
+            cfg = loco.Config(**c)
+            grads = [inputs.gaussian(n, 1e-3, seed=0, step=k, dtype=torch.float32, device=device) for k in range(4)]
+            st = loco.State(cfg, n)
+            comm = torch.empty(loco.loco_packed_bytes(cfg, n), dtype=torch.uint8, device=device)
+            out = torch.empty(n, dtype=torch.float32, device=device)
+
+            def four_steps():
+                for k in range(4):
+                    loco.loco_compensate_quantize_pack(st, grads[k], comm, k + 1)
+
+            us = timed(four_steps, 50) / 4
+            row("send", "%s scale, fp32 g, int8 state, 4 bit" % scale, n, send_bytes_per_elem(c), 4, us, "L2-resident")
+            us = timed(lambda: loco.loco_unpack_dequant_reduce(cfg, [comm], n, out), 200)
+            row("reduce", "%s scale, 1 worker, fp32 out" % scale, n, reduce_bytes_per_elem(c, 1), 4, us, "L2-resident")
+        oc = dict(cfg_for("fixed"), s=2.0 ** 11, s_e=2.0 ** 13, grad_dtype=0, out_dtype=0, num_partitions=1)
+        cpu = cpu_baseline_record(cores, oc, n, 1, "vectors of 2^20 fp32 elements", per_thread=16)
+    elif args.config == 3:
+        # 13B dense transformer, one flat bf16 buffer in the reduce-scatter layout of 8 parts: one send launch over the whole
+        # buffer; a rank then averages its own part (1,626,983,040 elements) over 8 workers
+        layout = inputs.dense_13b()
+        n = layout.numel
+        workload = "config 3: 13B dense transformer, one flat bf16 buffer of 13,015,864,320 elements, 8 parts, T_c = 512; send = the whole buffer in one launch, reduce = one rank's part of 1,626,983,040 elements over 8 workers"
+        c = dict(cfg_for("fixed"))
+        cfg = loco.Config(**c)
+        grad = torch.empty(n, dtype=torch.bfloat16, device=device)
+        chunk = 1 << 28
+        for off in range(0, n, chunk):
+            m = min(chunk, n - off)
+            grad[off:off + m] = inputs.gaussian(m, 1e-4, seed=2, tag=off >> 8, dtype=torch.bfloat16, device=device)
+        st = loco.State(cfg, n)
+        comm = torch.empty(loco.loco_packed_bytes(cfg, n), dtype=torch.uint8, device=device)
+        loco.loco_compensate_quantize_pack(st, grad, comm, 1)
+        us = timed(lambda: loco.loco_compensate_quantize_pack(st, grad, comm, 5), 3, warm=1)
+        row("send", "fixed scale, bf16 g, int8 state, 4 bit, 8 parts, one launch", n, send_bytes_per_elem(c), 2, us)
+        us = timed(lambda: loco.loco_compensate_quantize_pack(st, grad, comm, 512), 3, warm=1)
+        row("send", "the same at k = 512 (the reset of Eq. 7 fires: the state is written as zeros)", n, send_bytes_per_elem(c), 2, us)
+        stride = loco.loco_partition_bytes(cfg, n)
+        r = 3
+        ln = loco.loco_partition_elems(cfg, n, r)
+        gen = torch.Generator(device=device)
+        gen.manual_seed(77)
+        others = [torch.randint(0, 256, (stride,), dtype=torch.uint8, device=device, generator=gen) for _ in range(WORKERS - 1)]
+        out = torch.empty(ln, dtype=torch.bfloat16, device=device)
+        packed = [comm[r * stride:(r + 1) * stride]] + others
+        us = timed(lambda: loco.loco_unpack_dequant_reduce(cfg, packed, n, out, first_partition=r, partition_count=1), 5, warm=2)
+        row("reduce", "fixed scale, part 3 of 8 (1,626,983,040 elements), 8 workers, bf16 out", ln, reduce_bytes_per_elem(c, WORKERS), 2, us)
+        cpu = cpu_baseline_record(cores, c, BUCKET, WORKERS, "windows of 25M elements of the flat buffer")
+    else:
+        # one Mixtral-8x7B decoder layer, Student-t(3) x 1e-4, 2 of 8 experts all-zero, 8 workers
+        layout = inputs.mixtral_layer()
+        n = layout.numel
+        workload = "config 4: one Mixtral-8x7B decoder layer of 1,451,270,144 bf16 elements, Student-t(nu=3) x 1e-4, 2 of 8 experts all-zero, 8 workers"
+        scales = inputs.zero_expert_scales(3, layer=0)
+        grad = torch.empty(n, dtype=torch.bfloat16, device=device)
+        chunk = 1 << 27
+        for off in range(0, n, chunk):
+            hi = min(off + chunk, n)
+            grad[off:hi] = inputs.layout_slice(layout, off, hi, scales, 1e-4, seed=3, worker=0, step=1, dist="student_t", device=device)
+        for scale in ("fixed", "block"):
+            c = dict(cfg_for(scale), reset_period=0)
+            cfg = loco.Config(**c)
+            st = loco.State(cfg, n)
+            comm = torch.empty(loco.loco_packed_bytes(cfg, n), dtype=torch.uint8, device=device)
+            loco.loco_compensate_quantize_pack(st, grad, comm, 1)
+            us = timed(lambda: loco.loco_compensate_quantize_pack(st, grad, comm, 2), 5, warm=2)
+            row("send", "%s scale, bf16 g, int8 state, 4 bit, 8 parts, the whole layer in one launch" % scale, n, send_bytes_per_elem(c), 2, us)
+            others = [comm.clone() for _ in range(WORKERS - 1)]       # the other workers' buffers: valid codes and scales
+            out = torch.empty(n, dtype=torch.bfloat16, device=device)
+            us = timed(lambda: loco.loco_unpack_dequant_reduce(cfg, [comm] + others, n, out), 5, warm=2)
+            row("reduce", "%s scale, 8 workers, bf16 out, all 8 parts in one launch" % scale, n, reduce_bytes_per_elem(c, WORKERS), 2, us)
+            del others, out, comm, st
+        cpu = cpu_baseline_record(cores, dict(cfg_for("fixed"), reset_period=0), BUCKET, WORKERS, "windows of 25M elements of the layer")
+    best = max(rows, key=lambda r: r["us"])
+    total_us = sum(r["us"] for r in rows)
+    print(json.dumps({"metric": METRIC, "value": None, "unit": "GB/s", "n_gpus": 1, "steps": None, "warmup": 3,
+                      "ms_per_step": total_us / 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                      "dtype": "f32", "data": "synthetic", "config": {"workload": workload}, "rows": rows,
+                      "slowest_row": best["case"], "peak": peak, "peak_kind": "%s HBM copy bandwidth" % peak_kind,
+                      "cpu_baseline": cpu, "gpu_launches": loco.loco_launch_count() - launches_before}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -561,12 +765,19 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--config", type=int, default=2, choices=(1, 2, 3, 4),
+                    help="2 (default): the bench workload, Llama-2-7B buckets; 1, 3, 4: the other workload configurations "
+                         "(a table of rows instead of the bench line); the size sweep of configuration 5 is --sweep")
+    ap.add_argument("--scale", default="fixed", choices=("fixed", "block"),
+                    help="fixed (default): the paper's global scale s (Eq. 1); block: one fp32 scale per 256 elements "
+                         "(the block-scaled twin of the bench workload)")
     ap.add_argument("--buckets", type=int, default=0,
                     help="profiling aid: only the first K buckets of the workload (0 = all 270); not a bench line")
     ap.add_argument("--no-graph", action="store_true", help="profiling aid: launch every kernel directly")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the bench line: the size / type / width / worker-count table (one JSON line per case, then markdown)")
-    ap.add_argument("--sweep-filter", default="", help="with --sweep: only the cases whose 'kernel: label' contains this text")
+    ap.add_argument("--sweep-filter", default="", help="with --sweep: only the cases whose 'kernel: label | N=workers |' contains this text")
+    ap.add_argument("--sweep-budget-gb", type=float, default=6.0, help="with --sweep: device memory per case (small for profiler captures)")
     ap.add_argument("--exchange", choices=("none", "collective", "peer_store", "reduce_scatter_bf16"), default="none",
                     help="none (default): every rank runs the two passes on its own buckets, no data-path collective; "
                          "collective / peer_store: the real exchange of Sec. 3.3 between the ranks (NCCL all-to-all, or the "
@@ -574,18 +785,21 @@ def main():
                          "reduce_scatter_bf16: what the method replaces -- NCCL reduce-scatter (average) of the uncompressed bf16 "
                          "buckets, none of this library's kernels, for comparison on the same buckets")
     ap.add_argument("--streams", type=int, default=2,
-                    help="2 or more (default): each phase is one multi-bucket call of the library on one stream (the library overlaps "
-                         "consecutive launches on streams of its own); 1: single-bucket calls strictly one after the other")
+                    help="2 or more (default): each phase is one multi-bucket call of the library, i.e. one kernel launch over all "
+                         "buckets; 1: single-bucket calls strictly one after the other")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     cores = os.cpu_count() or 1
+    multi = args.streams > 1 and not args.no_graph
+    cfgd = cfg_for(args.scale)
     config = {"workload": "llama2-7b: 270 bf16 buckets of 25M elements (6,738,415,616): one worker's send pass per bucket, then the 8-worker reduce of the bucket",
-              "bits": 4, "scale": "fixed s=2^14, s_e=4s (Eq. 1)", "beta": 0.5, "T_c": 512, "state": "int8",
-              "workers_on_reduce_side": WORKERS, "out": "bf16",
-              "streams": ("1 caller stream; loco_*_multi calls overlap consecutive buckets on the library's 3 streams"
-                          if args.streams > 1 and not args.no_graph else "1, single-bucket calls one after the other"),
+              "bits": 4,
+              "scale": "fixed s=2^14, s_e=4s (Eq. 1)" if args.scale == "fixed" else "one fp32 scale per block of 256 elements (extension, not in the paper)",
+              "beta": 0.5, "T_c": 512, "state": "int8", "workers_on_reduce_side": WORKERS, "out": "bf16",
+              "launches": ("one multi-bucket call per phase = one kernel launch over all buckets (the buckets are the grid's third "
+                           "dimension), on one stream" if multi else "single-bucket calls one after the other on one stream"),
               "l2": "inputs larger than L2: each step streams ~70 GB once, no reuse between launches"}
 
     if args.impl == "reference":
@@ -593,11 +807,11 @@ def main():
             return
         steps = max(1, args.steps)
         for _ in range(min(args.warmup, 1)):
-            oracle_sample(cores, 1)
+            oracle_sample(cores, 1, cfgd)
         t0 = time.perf_counter()
         elems = 0
         for _ in range(steps):
-            _, _, e = oracle_sample(cores, 1)
+            _, _, e = oracle_sample(cores, 1, cfgd)
             elems += e
         dt = time.perf_counter() - t0
         val = 2.0 * elems / dt / 1e9
@@ -631,15 +845,19 @@ def main():
         if rank == 0:
             sweep(args, device)
         return
+    if args.config != 2:
+        if rank == 0:
+            run_other_config(args, device, cores)
+        return
     if args.exchange != "none":
         run_exchange(args, rank, world, device, config)
         return
-    wl = RankWorkload(rank, device, args.buckets)
+    wl = RankWorkload(rank, device, args.buckets, args.scale)
     nb = len(wl.buckets)
     if args.buckets > 0:
         config["workload"] += " -- REDUCED to the first %d buckets (profiling aid, not the bench workload)" % nb
-    # The 540 launches of a step are captured once into two CUDA graphs (one per phase) and replayed,
-    # so that the host's launch cost does not sit between kernels of a few microseconds each.
+    # A step is captured once into two CUDA graphs (one per phase) and replayed, so that the host's launch cost does not sit
+    # between the kernels; the launches of a step are counted while the graphs are captured.
     wl.send_phase(1)
     wl.reduce_phase()
     torch.cuda.synchronize()
@@ -647,17 +865,14 @@ def main():
         class _Direct:
             def __init__(self, fn): self.replay = fn
         g_send, g_reduce = _Direct(lambda: wl.send_phase(100)), _Direct(wl.reduce_phase)
+        launches_per_step = 2 * nb
     else:
-        side = [torch.cuda.Stream(device=device) for _ in range(args.streams)] if args.streams > 1 else None
         g_send, g_reduce = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
-        if args.streams > 1:
-            # the library's multi-bucket calls, issued on this one stream: they take three streams of
-            # the library's own and join them back, so that a bucket's tail overlaps the next bucket's start-up
+        before = loco.loco_launch_count()
+        if multi:
+            # the library's multi-bucket calls: one kernel launch per phase, the buckets in the grid's third dimension
             ms = loco.MultiSend(wl.states, wl.grads, wl.comms)
             mr = loco.MultiReduce(wl.cfg, wl.packed, [hi - lo for lo, hi in wl.buckets], wl.outs)
-            loco.loco_compensate_quantize_pack_multi(ms, 100)       # first call outside capture: creates the library's streams
-            loco.loco_unpack_dequant_reduce_multi(mr)
-            torch.cuda.synchronize()
             with torch.cuda.graph(g_send):
                 loco.loco_compensate_quantize_pack_multi(ms, 100)
             with torch.cuda.graph(g_reduce):
@@ -667,6 +882,7 @@ def main():
                 wl.send_phase(100, None)
             with torch.cuda.graph(g_reduce):
                 wl.reduce_phase(None)
+        launches_per_step = loco.loco_launch_count() - before
     for k in range(max(3, args.warmup)):
         g_send.replay()
         g_reduce.replay()
@@ -686,12 +902,12 @@ def main():
         ev[k][2].record()
     end.record()
     barrier()
-    launches = 2 * nb * K          # one send and one receive kernel per bucket and step, replayed from the graphs
+    launches = launches_per_step * K
     clocks = sampler.stop()
-    # outside the timed region: the same two phases with every launch strictly after the previous one (one stream),
-    # which shows what a launch costs when nothing overlaps its start-up and its tail
+    # outside the timed region: the same two phases as single-bucket calls, every launch strictly after the previous one
+    # (one stream), which shows what a lone launch costs when nothing fills its start-up and its tail
     serial_us = None
-    if not args.no_graph and args.streams > 1:
+    if multi:
         s_send, s_reduce = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
         with torch.cuda.graph(s_send):
             wl.send_phase(100, None)
@@ -704,30 +920,24 @@ def main():
         torch.cuda.synchronize()
         serial_us = (sev[0].elapsed_time(sev[1]) * 1e3 / (2 * nb), sev[1].elapsed_time(sev[2]) * 1e3 / (2 * nb))
     # also outside the timed region, for scale: a plain device-to-device copy (the driver's cudaMemcpyAsync, issued by
-    # torch) that moves as many bytes per launch as the send kernel does, one launch per bucket over memory not in L2
+    # torch) that moves as many bytes per launch as the send kernel does per bucket, over memory not in L2
     copy_us = None
     if not args.no_graph:
-        half = int(SEND_BYTES_PER_ELEM * BUCKET / 2) // 256 * 256          # bytes copied = half of read + written
+        half = int(wl.send_bpe * BUCKET / 2) // 256 * 256                  # bytes copied = half of read + written
         src8, dst8 = wl.grad.view(torch.uint8), wl.out_buf.view(torch.uint8)
         span = min(src8.numel(), dst8.numel())
         count = max(1, min(nb, span // half))
-
-        def copies(streams):
-            wl._fan_out(lambda i, st: dst8[i * half:(i + 1) * half].copy_(src8[i * half:(i + 1) * half]), count, streams)
-
-        res = []
-        for strs in (None, side if args.streams > 1 else None):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g):
-                copies(strs)
-            g.replay()
-            ce = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
-            torch.cuda.synchronize()
-            ce[0].record(); g.replay(); g.replay(); ce[1].record()
-            torch.cuda.synchronize()
-            res.append(ce[0].elapsed_time(ce[1]) * 1e3 / (2 * count))
-        copy_us = {"bytes_moved_per_launch": 2 * half, "one_stream_launch_us": res[0], "one_stream_gbs": 2 * half / res[0] / 1e3,
-                   "two_stream_launch_us": res[1], "two_stream_gbs": 2 * half / res[1] / 1e3}
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for i in range(count):
+                dst8[i * half:(i + 1) * half].copy_(src8[i * half:(i + 1) * half])
+        g.replay()
+        ce = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        torch.cuda.synchronize()
+        ce[0].record(); g.replay(); g.replay(); ce[1].record()
+        torch.cuda.synchronize()
+        us = ce[0].elapsed_time(ce[1]) * 1e3 / (2 * count)
+        copy_us = {"bytes_moved_per_copy": 2 * half, "copy_us": us, "gbs": 2 * half / us / 1e3}
     total_ms = start.elapsed_time(end)
     send_ms = sum(e[0].elapsed_time(e[1]) for e in ev) / K
     recv_ms = sum(e[1].elapsed_time(e[2]) for e in ev) / K
@@ -749,8 +959,9 @@ def main():
             e_ms = float(t.item())
         e2e = {"value": world * wl.grad_bytes / (e_ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d * world,
                "d2h_bytes_per_step": d2h * world, "ms_per_step": e_ms, "steps": args.e2e_steps,
-               "how": "loco_*_host entry points, pinned host buffers, copies inside the timed region; send and receive passes "
-                      "on two streams so that host-to-device and device-to-host copies overlap"}
+               "how": "loco_*_host entry points, pinned host buffers, copies inside the timed region (this measures the host "
+                      "link: 57 GB cross it per step); send and receive passes on two streams so that host-to-device and "
+                      "device-to-host copies overlap"}
     if dist is not None:
         dist.barrier()
     if rank != 0:
@@ -761,40 +972,42 @@ def main():
     peak, peak_kind = measured_peak()
     send_gbs = wl.send_bytes / (send_ms * 1e-3) / 1e9
     recv_gbs = wl.recv_bytes / (recv_ms * 1e-3) / 1e9
-    how = ("CUDA events around this kernel's phase of every timed step / launches in it; " +
-           ("a phase is one multi-bucket call of the library on one stream, which spreads the launches over three streams of "
-            "its own, so a kernel's start-up and tail overlap its neighbour" if args.streams > 1 and not args.no_graph else
-            "every launch strictly after the previous one"))
-    roof_send = {"kernel": "loco_send_kernel<bf16 g, int8 state, 4 bit, fixed scale>", "bound": "hbm",
+    per_phase = max(1, launches_per_step // 2)
+    how = ("CUDA events around this kernel's phase of every timed step; " +
+           ("a phase is ONE launch that walks all %d buckets (grid.z = bucket), so the figures below are per bucket: "
+            "phase time / buckets" % nb if multi else "every bucket's launch strictly after the previous one"))
+    traffic_note = ("dram__bytes_read.sum + dram__bytes_write.sum of one captured multi-bucket launch / its buckets, read from "
+                    "profiles/dram_traffic_llama2_7b_buckets.json; null when there is no capture for this case or the kernel "
+                    "sources have changed since it was taken")
+    tag = "fixed scale" if args.scale == "fixed" else "block-256 scale"
+    roof_send = {"kernel": "loco_send%s_kernel<bf16 g, int8 state, 4 bit, %s>" % ("_multi" if multi else "", tag), "bound": "hbm",
                  "achieved": send_gbs, "peak": peak, "peak_kind": "%s HBM copy bandwidth" % peak_kind, "unit": "GB/s",
-                 "frac": send_gbs / peak, "frac_of_nominal_8TBps": send_gbs / 8000.0, "traffic": SEND_DRAM_BYTES_PER_LAUNCH,
-                 "algorithmic_bytes_per_launch": SEND_BYTES_PER_ELEM * BUCKET, "avg_launch_us": send_ms * 1e3 / nb,
-                 "launches_per_step": nb, "how": how}
-    roof_reduce = {"kernel": "loco_reduce_kernel<bf16 out, 4 bit, fixed scale>, 8 workers", "bound": "hbm",
+                 "frac": send_gbs / peak, "frac_of_nominal_8TBps": send_gbs / 8000.0, "traffic": stored_traffic("send", args.scale),
+                 "traffic_source": traffic_note, "algorithmic_bytes_per_bucket": wl.send_bpe * BUCKET,
+                 "avg_us_per_bucket": send_ms * 1e3 / nb, "launches_per_step": per_phase, "buckets_per_launch": nb // per_phase, "how": how}
+    roof_reduce = {"kernel": "loco_reduce%s_kernel<bf16 out, 4 bit, %s>, 8 workers" % ("_multi" if multi else "", tag), "bound": "hbm",
                    "achieved": recv_gbs, "peak": peak, "peak_kind": "%s HBM copy bandwidth" % peak_kind, "unit": "GB/s",
-                   "frac": recv_gbs / peak, "frac_of_nominal_8TBps": recv_gbs / 8000.0, "traffic": REDUCE_DRAM_BYTES_PER_LAUNCH,
-                   "algorithmic_bytes_per_launch": (WORKERS * 0.5 + 2) * BUCKET, "avg_launch_us": recv_ms * 1e3 / nb,
-                   "launches_per_step": nb, "how": how}
+                   "frac": recv_gbs / peak, "frac_of_nominal_8TBps": recv_gbs / 8000.0, "traffic": stored_traffic("reduce", args.scale),
+                   "traffic_source": traffic_note, "algorithmic_bytes_per_bucket": wl.recv_bpe * BUCKET,
+                   "avg_us_per_bucket": recv_ms * 1e3 / nb, "launches_per_step": per_phase, "buckets_per_launch": nb // per_phase, "how": how}
     # the roofline object describes the kernel that takes the larger share of the step; the other one rides along
     roofline, other = (roof_reduce, roof_send) if recv_ms >= send_ms else (roof_send, roof_reduce)
     roofline["other_kernel"] = other
     kernels = {"send": {"hbm_gbs": send_gbs, "frac_of_peak": send_gbs / peak, "gradient_gbs": wl.grad_bytes / (send_ms * 1e-3) / 1e9,
-                        "ms_per_step": send_ms, "avg_launch_us": send_ms * 1e3 / nb, "bytes_per_elem": SEND_BYTES_PER_ELEM},
+                        "ms_per_step": send_ms, "avg_us_per_bucket": send_ms * 1e3 / nb, "bytes_per_elem": wl.send_bpe},
                "reduce": {"hbm_gbs": recv_gbs, "frac_of_peak": recv_gbs / peak,
                           "gradient_gbs": wl.grad_bytes / (recv_ms * 1e-3) / 1e9, "ms_per_step": recv_ms,
-                          "avg_launch_us": recv_ms * 1e3 / nb, "bytes_per_out_elem": WORKERS * 0.5 + 2}}
+                          "avg_us_per_bucket": recv_ms * 1e3 / nb, "bytes_per_out_elem": wl.recv_bpe}}
     if serial_us is not None:
-        kernels["send"]["one_stream_launch_us"] = serial_us[0]
-        kernels["send"]["one_stream_hbm_gbs"] = wl.send_bytes / nb / (serial_us[0] * 1e-6) / 1e9
-        kernels["reduce"]["one_stream_launch_us"] = serial_us[1]
-        kernels["reduce"]["one_stream_hbm_gbs"] = wl.recv_bytes / nb / (serial_us[1] * 1e-6) / 1e9
+        kernels["send"]["single_bucket_calls_one_stream_us"] = serial_us[0]
+        kernels["send"]["single_bucket_calls_one_stream_hbm_gbs"] = wl.send_bytes / nb / (serial_us[0] * 1e-6) / 1e9
+        kernels["reduce"]["single_bucket_calls_one_stream_us"] = serial_us[1]
+        kernels["reduce"]["single_bucket_calls_one_stream_hbm_gbs"] = wl.recv_bytes / nb / (serial_us[1] * 1e-6) / 1e9
     if copy_us is not None:
-        kernels["device_copy_same_bytes_as_send"] = copy_us
+        kernels["device_copy_same_bytes_as_send_bucket"] = copy_us
     cpu = None
     if not args.no_cpu_baseline:
-        v, dt, elems = oracle_sample(cores, 2)
-        cpu = {"value": v, "unit": "GB/s", "cores": cores, "kind": "oracle",
-               "sample": "%d buckets of 25M elements (2 per host thread), send + 8-worker reduce, %.1f s wall" % (2 * cores, dt)}
+        cpu = cpu_baseline_record(cores, cfgd, BUCKET, WORKERS, "buckets of 25M elements")
     line = {"metric": METRIC, "value": world * wl.grad_bytes / (step_ms * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": world,
             "steps": K, "warmup": max(3, args.warmup), "ms_per_step": step_ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,

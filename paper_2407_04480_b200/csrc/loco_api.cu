@@ -208,14 +208,22 @@ ReduceKernel pick_reduce(const loco_config_t *c, int mode, int path, bool adam) 
     return adam ? pick_reduce_o0_a1(c->bits, mode, path) : pick_reduce_o0_a0(c->bits, mode, path);
 }
 
-unsigned grid_x_for(uint64_t rows_per_partition, int partitions, int ctas_per_sm) {
-    const uint64_t want = (rows_per_partition + kWarps - 1) / kWarps;             // one row per warp
+// CTAs per partition.  A bucket that fits one resident wave gets exactly that: every CTA resident at once, each warp a
+// handful of wide rows.  A larger bucket gets more CTAs than are resident, each with about kRowsPerWarp wide rows per
+// warp: the hardware then hands them out as SMs become free, which evens out the different speeds at which the SMs
+// stream under a saturated memory system (with one wave and a fixed split, the fast SMs would idle until the slowest
+// is done), at the price of one ring fill per CTA.
+constexpr uint64_t kRowsPerWarp = 16;
+unsigned grid_x_for(uint64_t wide_rows_per_partition, int partitions, int ctas_per_sm) {
+    const uint64_t want = (wide_rows_per_partition + kWarps - 1) / kWarps;        // one wide row per warp
     uint64_t budget = static_cast<uint64_t>(num_sms()) * static_cast<uint64_t>(ctas_per_sm);
-    // all CTAs of a launch must be resident together: a CTA that has to wait for a free slot would run alone
     uint64_t per_part = budget / static_cast<uint64_t>(partitions);
     if (per_part < 1) per_part = 1;
     uint64_t gx = want < per_part ? want : per_part;
+    const uint64_t many = (wide_rows_per_partition + kWarps * kRowsPerWarp - 1) / (kWarps * kRowsPerWarp);
+    if (many > gx) gx = many;
     if (gx < 1) gx = 1;
+    if (gx > 0x7fffffffull) gx = 0x7fffffffull;
     return static_cast<unsigned>(gx);
 }
 
@@ -465,7 +473,7 @@ int send_launch(loco_state_t *st, const void *d_grad, void *d_comm, void *const 
     }
     fill_common(st, step_k, P.c);
     fill_bucket(st, d_grad, d_comm, P.b);
-    const uint64_t rows = P.b.lp / kRow;
+    const uint64_t rows = (P.b.lp + kWide - 1) / kWide;
     dim3 grid(grid_x_for(rows, c.num_partitions, st->send_ctas_per_sm), static_cast<unsigned>(c.num_partitions), 1);
     st->send_fn<<<grid, kThreads, static_cast<size_t>(st->send_smem_bytes), static_cast<cudaStream_t>(stream)>>>(P);
     if (cudaGetLastError() != cudaSuccess) return LOCO_ERR_CUDA;
@@ -491,7 +499,7 @@ int send_multi_launch(loco_state_t *const *states, const void *const *d_grads, v
         if (st->n == 0) continue;
         SendBucket &B = P.b[P.count++];
         fill_bucket(st, d_grads[i], d_comms[i], B);
-        B.grid_x = grid_x_for(st->layout.lp / kRow, st->cfg.num_partitions, st->send_ctas_per_sm);
+        B.grid_x = grid_x_for((st->layout.lp + kWide - 1) / kWide, st->cfg.num_partitions, st->send_ctas_per_sm);
         if (B.grid_x > gx) gx = B.grid_x;
     }
     if (P.count == 0) return LOCO_OK;

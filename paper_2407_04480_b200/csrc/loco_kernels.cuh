@@ -617,7 +617,9 @@ struct LanePtrs {
     float *wire_scales;       // BLOCK: the partition's scale area
     float *state_scales;      // BLOCK + INT8: scale of the bucket's block 0
     unsigned long long elem0; // bucket index of this lane's first element of wide row 0
-    unsigned long long lane_elem;   // partition-local index of this lane's first element of wide row 0
+    unsigned lane_elem;       // partition-local index of this lane's first element of wide row 0
+    unsigned lane_block;      // BLOCK: index, within a wide row, of the block this lane's elements belong to
+    bool leader;              // BLOCK: this lane stores the scales of its block (the first lane of the block)
 };
 
 // ---- per-warp ring of asynchronous copies (cp.async) -------------------------------------------
@@ -759,22 +761,33 @@ __device__ __forceinline__ void fetch_row(const RingAddr<GRAD, STATE> &A, unsign
 struct SendConsts {
     float s, s_e, beta, omb, inv_s, inv_se, dq_a, dq_b, de_a, de_b, clip;
     int dq_mode, de_mode, block_log2, reset;
+    unsigned blocks_per_row;         // BLOCK, B <= 512: blocks in a wide row
     unsigned seed_lo, seed_hi, k_lo, k_hi;
 };
 
-// Field j of the packed codes sits in the low bits of mb[j] = bits(kMagic + 2^(p-1) + q_j):
-// sum_j mb[j] * R^j = kMagicBits * sum_j R^j + sum_j (q_j + 2^(p-1)) R^j  (mod 2^32), R = 2^p; removing the
-// constant and flipping each field's top bit turns the biased fields into two's complement.
-template <int BITS, int COUNT>
-__device__ __forceinline__ unsigned horner_codes(const unsigned *mb) {
-    unsigned acc = mb[COUNT - 1];
+// Field j of the packed codes sits in the low bits of mb_j = bits(kMagic + 2^(p-1) + q_j):
+// sum_j mb_j * R^j = kMagicBits * sum_j R^j + sum_j (q_j + 2^(p-1)) R^j  (mod 2^32), R = 2^p; removing the
+// constant and flipping each field's top bit turns the biased fields into two's complement.  The sum is taken one
+// multiply-add (fp32 pipe) per code as the codes are produced, so that no code has to wait in a register for the others.
+template <int BITS>
+struct CodePacker {
+    static constexpr int kPerWord = 32 / BITS;               // 16, 8 or 4 codes per word
+    static constexpr int kWords = 16 / kPerWord;             // words for a lane's 16 codes: 1, 2 or 4
+    unsigned w[kWords];
+    __device__ __forceinline__ void clear() {
 #pragma unroll
-    for (int j = COUNT - 2; j >= 0; --j) acc = acc * (1u << BITS) + mb[j];
-    unsigned ones = 0u, flip = 0u;
+        for (int i = 0; i < kWords; ++i) w[i] = 0u;
+    }
+    __device__ __forceinline__ void put(int j, unsigned mb) {        // code j of the lane's 16, j a compile-time constant
+        w[(j / kPerWord) % kWords] = mb * (1u << (BITS * (j % kPerWord))) + w[(j / kPerWord) % kWords];
+    }
+    __device__ __forceinline__ unsigned word(int i) const {
+        unsigned ones = 0u, flip = 0u;
 #pragma unroll
-    for (int j = 0; j < COUNT; ++j) { ones |= 1u << (BITS * j); flip |= (1u << (BITS - 1)) << (BITS * j); }
-    return (acc - kMagicBits * ones) ^ flip;
-}
+        for (int j = 0; j < kPerWord; ++j) { ones |= 1u << (BITS * j); flip |= (1u << (BITS - 1)) << (BITS * j); }
+        return (w[i % kWords] - kMagicBits * ones) ^ flip;
+    }
+};
 
 // ---- the two divisions of a block scale, without the general division routine --------------------------------
 // scale = amax / qmax and 1/scale = qmax / amax must carry the bits of the IEEE division (the oracle divides).
@@ -799,12 +812,12 @@ __device__ __forceinline__ float qmax_over(float c, float a) {
 }
 
 // sum over aligned groups of `lanes` lanes as a balanced tree in index order (fp32 addition commutes, so both lanes
-// of a pair form the same sum); every lane of a group ends with the group's sum
+// of a pair form the same sum); every lane of a group ends with the group's sum.  `lanes` is the same for the whole
+// launch, so the steps that a small group does not need are skipped by uniform predicates, not computed and dropped.
 __device__ __forceinline__ float group_sum32(float v, int lanes) {
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        const float w = __shfl_xor_sync(kFull, v, o);
-        v = o < lanes ? __fadd_rn(v, w) : v;
+        if (o < lanes) v = __fadd_rn(v, __shfl_xor_sync(kFull, v, o));
     }
     return v;
 }
@@ -819,13 +832,15 @@ __device__ __forceinline__ float qmax_over_midrange(float c, float a) {
 }
 __device__ __forceinline__ bool in_midrange(float a) { return __float_as_uint(a) - 0x0d800000u <= 0x71800000u - 0x0d800000u; }
 
-// max over aligned groups of `lanes` lanes (1 to 32) in a fixed number of steps, without a loop
+// max over aligned groups of `lanes` lanes (1 to 32): four steps without a branch, the fifth (a block of 512 elements
+// spans the whole warp) under a uniform one
 __device__ __forceinline__ float group_max32(float v, int lanes) {
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
+    for (int o = 1; o < 16; o <<= 1) {
         const float w = __shfl_xor_sync(kFull, v, o);
         v = o < lanes ? fmaxf(v, w) : v;
     }
+    if (lanes > 16) v = fmaxf(v, __shfl_xor_sync(kFull, v, 16));
     return v;
 }
 
@@ -1006,7 +1021,8 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     }
 
     // ---- Eq. 1 / Eq. 3: q = round_p-bit(h x s);  step 2: d, Eq. 5 ---------------------------------------------
-    unsigned mb[16];
+    CodePacker<BITS == 1 ? 2 : BITS> pack;
+    pack.clear();
     f32x2 en2[8];
     const f32x2 mult2 = dup2(mult), qmagic2 = dup2(qmagic), omb2 = dup2(K.omb), beta2 = dup2(K.beta);
     uint4 rnd = make_uint4(0u, 0u, 0u, 0u);                // the lane's 16 elements are one block of the Philox stream
@@ -1046,16 +1062,17 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             }
             m2 = fadd2(pk2(fminf(fmaxf(t0, lo), hi), fminf(fmaxf(t1, lo), hi)), qmagic2);
         }
-        mb[2 * k] = static_cast<unsigned>(m2);
-        mb[2 * k + 1] = static_cast<unsigned>(m2 >> 32);
+        const unsigned mb0 = static_cast<unsigned>(m2), mb1 = static_cast<unsigned>(m2 >> 32);
+        pack.put(2 * k, mb0);
+        pack.put(2 * k + 1, mb1);
         f32x2 d2;
         if (MODE == MODE_BLOCK) {
             d2 = fmul2_pz(fadd2(m2, dup2(-qmagic)), dup2(scale));          // q is never -0 and a non-zero q times a block scale never underflows
         } else if (LEAN) {
             d2 = ffma2(m2, dup2(K.dq_a), dup2(K.dq_b));
         } else {
-            d2 = pk2(dec_fast(__uint_as_float(mb[2 * k]), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s),
-                     dec_fast(__uint_as_float(mb[2 * k + 1]), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s));
+            d2 = pk2(dec_fast(__uint_as_float(mb0), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s),
+                     dec_fast(__uint_as_float(mb1), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s));
         }
         if (MODE != MODE_BLOCK && EXTRAS && stats) {
             if (var_is_sr(VAR)) {
@@ -1072,18 +1089,17 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     }
     uint8_t *cdst = L.codes + static_cast<size_t>(wrow) * (kWide * BITS / 8);
     if (BITS == 4) {
-        st_stream8(cdst, make_uint2(horner_codes<4, 8>(mb), horner_codes<4, 8>(mb + 8)));
+        st_stream8(cdst, make_uint2(pack.word(0), pack.word(1)));
     } else if (BITS == 8) {
-        st_stream16(cdst, make_uint4(horner_codes<8, 4>(mb), horner_codes<8, 4>(mb + 4), horner_codes<8, 4>(mb + 8), horner_codes<8, 4>(mb + 12)));
+        st_stream16(cdst, make_uint4(pack.word(0), pack.word(1), pack.word(2), pack.word(3)));
     } else if (BITS == 2) {
-        st_stream4(cdst, horner_codes<2, 16>(mb));
+        st_stream4(cdst, pack.word(0));
     } else {
         st_stream2(cdst, static_cast<uint16_t>(signs));
     }
+    // the scales of wide row w: L.wire_scales / L.state_scales point at this lane's block of row 0; a row holds 512 / B blocks
     if (MODE == MODE_BLOCK) {
-        const unsigned long long ol = L.lane_elem + static_cast<unsigned long long>(wrow) * kWide;     // partition-local element index
-        if ((lane & (lanes_per_block - 1)) == 0 && ((ol & ((1ull << K.block_log2) - 1)) == 0))
-            L.wire_scales[ol >> K.block_log2] = scale;
+        if (L.leader) L.wire_scales[static_cast<size_t>(wrow) * K.blocks_per_row] = scale;
     }
 
     // ---- Eq. 7 ---------------------------------------------------------------------------------------------------
@@ -1124,9 +1140,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         }
         st_stream16(L.state + static_cast<size_t>(wrow) * kWide, v);
         if (MODE == MODE_BLOCK) {
-            const unsigned long long i0 = L.elem0 + static_cast<unsigned long long>(wrow) * kWide;
-            if ((lane & (lanes_per_block - 1)) == 0 && (i0 & ((1ull << K.block_log2) - 1)) == 0)
-                L.state_scales[i0 >> K.block_log2] = escale;
+            if (L.leader) L.state_scales[static_cast<size_t>(wrow) * K.blocks_per_row] = escale;
         }
     } else if (kStateF32) {
         unsigned w[16];
@@ -1142,14 +1156,15 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     return true;
 }
 
-// The lane's pointers for the wide rows of partition `part` of one bucket, row 0 at partition-local element `o0`.
+// The lane's pointers for the wide rows of partition `part` of one bucket.
 template <int STATE, int BITS>
-__device__ __forceinline__ void lane_pointers(const SendBucket &Bk, uint8_t *pbase, unsigned long long part,
-                                              unsigned long long o0, int lane, LanePtrs &L) {
-    L.lane_elem = o0 + static_cast<unsigned long long>(lane) * kWideLane;
+__device__ __forceinline__ void lane_pointers(const SendBucket &Bk, uint8_t *pbase, unsigned long long part, int lane, LanePtrs &L) {
+    L.lane_elem = static_cast<unsigned>(lane) * kWideLane;
+    L.lane_block = 0u;
+    L.leader = false;
     L.elem0 = part * Bk.lp + L.lane_elem;
     L.state = static_cast<uint8_t *>(Bk.state) + L.elem0 * (STATE == ST_INT8 ? 1u : 4u);
-    L.codes = pbase + L.lane_elem * BITS / 8;
+    L.codes = pbase + static_cast<size_t>(L.lane_elem) * BITS / 8;
     L.wire_scales = reinterpret_cast<float *>(pbase + Bk.lp * BITS / 8);
     L.state_scales = reinterpret_cast<float *>(static_cast<uint8_t *>(Bk.state) + ((Bk.n + 255ull) & ~255ull));
 }
@@ -1158,6 +1173,7 @@ __device__ __forceinline__ void load_consts(const SendCommon &C, SendConsts &K) 
     K.s = C.s; K.s_e = C.s_e; K.beta = C.beta; K.omb = C.omb; K.inv_s = C.inv_s; K.inv_se = C.inv_se;
     K.dq_a = C.dq_a; K.dq_b = C.dq_b; K.de_a = C.de_a; K.de_b = C.de_b;
     K.dq_mode = C.dq_mode; K.de_mode = C.de_mode; K.block_log2 = C.block_log2; K.reset = C.reset; K.clip = C.clip;
+    K.blocks_per_row = static_cast<unsigned>(kWide) >> (C.block_log2 > 9 ? 9 : C.block_log2);
     K.seed_lo = C.seed_lo; K.seed_hi = C.seed_hi; K.k_lo = C.k_lo; K.k_hi = C.k_hi;
 }
 
@@ -1185,8 +1201,10 @@ __device__ __forceinline__ void flush_counts(unsigned long long *status, bool co
 // the partition's wide rows with the stride of all warps working on that partition; the inputs of its next rows are on
 // their way through the cp.async ring.  What is left of the partition (a last half-wide row, partial and padding rows;
 // every block when a block is wider than a wide row) goes to the careful routine.
-template <int GRAD, int STATE, int BITS, int MODE, int VAR>
-__device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucket &Bk, uint8_t *pbase, unsigned long long part,
+// `part_base()` gives where the partition's codes and scales go; it is asked again wherever the address is needed, so
+// that the address does not occupy registers across the streaming loop.
+template <int GRAD, int STATE, int BITS, int MODE, int VAR, typename PartBase>
+__device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucket &Bk, PartBase part_base, unsigned long long part,
                                             unsigned cta, unsigned ctas) {
     using R = Ring<GRAD, STATE, MODE>;
     constexpr int D = R::kDepth;
@@ -1206,7 +1224,7 @@ __device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucke
     }
     unsigned saturated = 0u, state_saturated = 0u, nonfinite = 0u;
     auto careful = [&](unsigned long long o, int nrows) {
-        const CarefulCounts N = send_careful<GRAD, STATE, BITS, MODE, var_is_sr(VAR)>(C, Bk, pbase, part, o, nrows, lane);
+        const CarefulCounts N = send_careful<GRAD, STATE, BITS, MODE, var_is_sr(VAR)>(C, Bk, part_base(), part, o, nrows, lane);
         saturated += N.saturated;
         state_saturated += N.state_saturated;
         nonfinite |= N.nonfinite;
@@ -1216,7 +1234,16 @@ __device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucke
         const unsigned full_wide = full_rows / 2;
         first_careful = 2 * full_wide;
         LanePtrs L;
-        lane_pointers<STATE, BITS>(Bk, pbase, part, 0ull, lane, L);
+        lane_pointers<STATE, BITS>(Bk, part_base(), part, lane, L);
+        if (MODE == MODE_BLOCK) {
+            // blocks of at most 512 elements here: a wide row and a partition start on a block boundary, so which lane
+            // leads a block, and which block of its row a lane is in, never changes
+            const unsigned lanes_per_block = C.block_log2 >= 9 ? 32u : (1u << (C.block_log2 - 4));
+            L.leader = (static_cast<unsigned>(lane) & (lanes_per_block - 1u)) == 0u;
+            L.lane_block = L.lane_elem >> C.block_log2;
+            L.wire_scales += L.lane_block;
+            L.state_scales += (L.elem0 >> C.block_log2);
+        }
         // staging reads: chunk `lane` of each 512-byte piece of the row
         const uint8_t *g_stage = static_cast<const uint8_t *>(Bk.grad) + base * (GRAD == GRAD_BF16 ? 2u : 4u) + lane * 16;
         const uint8_t *e_stage = static_cast<const uint8_t *>(Bk.state) + base * (STATE == ST_INT8 ? 1u : 4u) + lane * 16;
@@ -1228,7 +1255,7 @@ __device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucke
         // this warp's wide rows are warp + i * nwarps, i < cnt
         const unsigned cnt = full_wide > warp ? (full_wide - warp + nwarps - 1) / nwarps : 0u;
         auto stage = [&](unsigned slot_off, unsigned wrow) {
-            const float *sp = L.state_scales + ((L.elem0 + static_cast<unsigned long long>(wrow) * kWide) >> K.block_log2);
+            const float *sp = L.state_scales + static_cast<size_t>(wrow) * K.blocks_per_row;      // MODE_BLOCK only
             stage_row<GRAD, STATE, MODE>(A, slot_off, g_stage + static_cast<size_t>(wrow) * gbytes,
                                          e_stage + static_cast<size_t>(wrow) * ebytes, sp);
         };
@@ -1239,20 +1266,34 @@ __device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucke
         }
         unsigned slot_off = 0u, stage_off = (D - 1) * R::kSlotStride;
         unsigned wrow = warp, stage_wrow = warp + (D - 1) * nwarps;
+        // Rows the fast routine hands back (a NaN, an Inf, a block maximum out of range: rare) are noted in a mask and
+        // redone by the careful routine after every 32 rows, outside the streaming loop: a call inside it would make
+        // the compiler keep part of the loop's registers in local memory on every iteration.
 #pragma unroll 1
-        for (unsigned i = 0; i < cnt; ++i) {
-            cp_async_wait<D - 2>();            // every group but the newest D-2 has landed: this row is there
-            __syncwarp();                      // ... for all lanes; and every lane is done reading the slot refilled next
-            WideIn<GRAD, STATE> in;
-            fetch_row<GRAD, STATE, MODE>(A, slot_off, in);
-            if (stage_wrow < full_wide) stage(stage_off, stage_wrow);
-            cp_async_commit();                 // one group per iteration, empty near the end
-            if (!send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, wrow, lane, stats, saturated, state_saturated))
-                careful(static_cast<unsigned long long>(wrow) * kWide, 2);
-            slot_off = slot_off + R::kSlotStride == R::kBytes ? 0u : slot_off + R::kSlotStride;
-            stage_off = stage_off + R::kSlotStride == R::kBytes ? 0u : stage_off + R::kSlotStride;
-            wrow += nwarps;
-            stage_wrow += nwarps;
+        for (unsigned i0 = 0; i0 < cnt; i0 += 32u) {
+            const unsigned i1 = cnt - i0 < 32u ? cnt : i0 + 32u;
+            const unsigned wrow0 = wrow;
+            unsigned failed = 0u;
+#pragma unroll 1
+            for (unsigned i = i0; i < i1; ++i) {
+                cp_async_wait<D - 2>();        // every group but the newest D-2 has landed: this row is there
+                __syncwarp();                  // ... for all lanes; and every lane is done reading the slot refilled next
+                WideIn<GRAD, STATE> in;
+                fetch_row<GRAD, STATE, MODE>(A, slot_off, in);
+                if (stage_wrow < full_wide) stage(stage_off, stage_wrow);
+                cp_async_commit();             // one group per iteration, empty near the end
+                if (!send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, wrow, lane, stats, saturated, state_saturated))
+                    failed |= 1u << (i - i0);
+                slot_off = slot_off + R::kSlotStride == R::kBytes ? 0u : slot_off + R::kSlotStride;
+                stage_off = stage_off + R::kSlotStride == R::kBytes ? 0u : stage_off + R::kSlotStride;
+                wrow += nwarps;
+                stage_wrow += nwarps;
+            }
+            while (failed) {
+                const unsigned j = static_cast<unsigned>(__ffs(static_cast<int>(failed))) - 1u;
+                failed &= failed - 1u;
+                careful(static_cast<unsigned long long>(wrow0 + j * nwarps) * kWide, 2);
+            }
         }
     }
     // the careful routine's unit: a row, or the rows of a block wider than a row
@@ -1269,8 +1310,8 @@ __device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucke
 template <int GRAD, int STATE, int BITS, int MODE, int VAR>
 __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_constant__ SendParams P) {
     const unsigned long long part = blockIdx.y;
-    uint8_t *pbase = P.scatter ? P.part_dst[part] : P.b.comm + part * P.b.stride;
-    send_bucket<GRAD, STATE, BITS, MODE, VAR>(P.c, P.b, pbase, part, blockIdx.x, gridDim.x);
+    send_bucket<GRAD, STATE, BITS, MODE, VAR>(
+        P.c, P.b, [&]() -> uint8_t * { return P.scatter ? P.part_dst[part] : P.b.comm + part * P.b.stride; }, part, blockIdx.x, gridDim.x);
 }
 
 // Several buckets per launch: grid = (most CTAs per partition any bucket wants, partitions, buckets).  The CTAs of
@@ -1283,7 +1324,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_multi_kernel(const __gr
     const SendBucket &Bk = P.b[blockIdx.z];
     if (blockIdx.x >= Bk.grid_x) return;
     const unsigned long long part = blockIdx.y;
-    send_bucket<GRAD, STATE, BITS, MODE, VAR>(P.c, Bk, Bk.comm + part * Bk.stride, part, blockIdx.x, Bk.grid_x);
+    send_bucket<GRAD, STATE, BITS, MODE, VAR>(P.c, Bk, [&]() -> uint8_t * { return Bk.comm + part * Bk.stride; }, part, blockIdx.x, Bk.grid_x);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1586,7 +1627,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const __g
     auto load_group = [&](unsigned row, int g, Group &G) {
         const unsigned long long o = static_cast<unsigned long long>(row) * kWide + lane_elem;
         const bool in = row < rows && o < valid;
-        const unsigned off = row * kRowBytes + lane_byte;
+        const unsigned long long off = static_cast<unsigned long long>(row) * kRowBytes + lane_byte;    // a part's code area may exceed 4 GiB
         const unsigned long long sidx = o >> C.block_log2;
 #pragma unroll
         for (int i = 0; i < kGroup; ++i) {

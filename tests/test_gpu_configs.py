@@ -155,7 +155,8 @@ def _random_codes(nbytes: int, seed: int) -> torch.Tensor:
 
 def test_config3_dense_13b_flat_buffer():
     """One flat bf16 buffer of 13,015,864,320 elements (more than 2^32: 64-bit indexing), reduce-scatter layout of 8
-    parts, 4-bit codes, T_c = 512: iterations 511, 512 (reset fires), 513; then the 8-worker reduce of all parts."""
+    parts, 4-bit codes, T_c = 512: eight ordinary iterations, then iterations 510 ... 515 and 1022 ... 1026 (the reset
+    fires at 512 and 1024); then the 8-worker reduce of all parts."""
     if _free_gb() < 110:
         pytest.skip("needs ~105 GB of free device memory")
     layout = inputs.dense_13b()
@@ -167,13 +168,15 @@ def test_config3_dense_13b_flat_buffer():
     assert lp * 8 >= n and loco.loco_partition_elems(gcfg, n, 7) == n - 7 * lp
     wb = WindowedBucket(gcfg, n, _windows(n, lp, 8, 1 << 18, 10, seed=3))
     grad = torch.empty(n, dtype=torch.bfloat16, device="cuda")
-    for k in (511, 512, 513):
+    ks = list(range(1, 9)) + list(range(510, 516)) + list(range(1022, 1027))
+    for k in ks:
         _fill_gaussian_bf16(grad, 1e-4, seed=2, worker=0, step=k)
         wb.step(grad, k)
         wb.compare("k=%d" % k)
-        if k == 512:
+        if k in (512, 1024):
             assert not bool(wb.state.buffer[:1 << 20].any()), "reset must zero the state"
-    assert len(wb.windows) >= 20 and wb.compared >= 3 * 20 * (1 << 17)
+            assert not bool(wb.state.buffer[n - (1 << 20):n].any()), "reset must zero the state"
+    assert len(wb.windows) >= 20 and wb.compared >= len(ks) * 20 * (1 << 17)
     assert bool(wb.comm[:1 << 20].any()) and bool(wb.state.buffer[:1 << 20].any())
     del grad
     pb = loco.loco_packed_bytes(gcfg, n)
@@ -197,7 +200,7 @@ def test_config3_dense_13b_flat_buffer():
 @pytest.mark.parametrize("mode", [loco.SCALE_FIXED, loco.SCALE_BLOCK_ABSMAX])
 def test_config4_mixtral_layer(mode):
     """One decoder layer (1,451,270,144 elements incl. 8 experts of 176,160,768), Student-t(3) x 1e-4 values, 2 of 8 experts
-    all-zero; 8 workers each compress their own gradient for 3 iterations; then the 8-worker reduce."""
+    all-zero; 8 workers each compress their own gradient for 8 iterations; then the 8-worker reduce."""
     if _free_gb() < 40:
         pytest.skip("needs ~35 GB of free device memory")
     layout = inputs.mixtral_layer()
@@ -220,7 +223,7 @@ def test_config4_mixtral_layer(mode):
     workers = [WindowedBucket(gcfg, n, wins if w in (0, 7) else []) for w in range(8)]
     grad = torch.empty(n, dtype=torch.bfloat16, device="cuda")
     chunk = 1 << 27
-    for k in (1, 2, 3):
+    for k in range(1, 9):
         for w, wb in enumerate(workers):
             for off in range(0, n, chunk):
                 hi = min(off + chunk, n)
@@ -241,8 +244,8 @@ def test_config4_mixtral_layer(mode):
 @pytest.mark.parametrize("bits", [2, 4, 8])
 @pytest.mark.parametrize("gd", [loco.F32, loco.BF16])
 def test_config5_sweep_small_sizes_full(bits, gd):
-    """n = 2^16 .. 2^22: every byte against the oracle, 2 iterations, then reduces over 1..16 workers."""
-    for log2n in (16, 18, 20, 22):
+    """n = 2^16 .. 2^24: every byte against the oracle, 2 iterations, then reduces over 1..16 workers."""
+    for log2n in (16, 18, 20, 22, 24):
         n = 1 << log2n
         gcfg = loco.Config(bits=bits, s=2.0 ** 11, s_e=2.0 ** 13, beta=0.5, reset_period=0, state_fmt=loco.STATE_INT8,
                            grad_dtype=gd, out_dtype=gd, num_partitions=1)
@@ -255,7 +258,7 @@ def test_config5_sweep_small_sizes_full(bits, gd):
             wb.compare("n=2^%d" % log2n)
         pb = loco.loco_packed_bytes(gcfg, n)
         comms = [wb.comm for wb in workers] + [_random_codes(pb, 200 + w) for w in range(14)]
-        for N in (1, 2, 4, 8, 16):
+        for N in ((1, 2, 4, 8, 16) if log2n < 24 else (1, 8, 16)):
             out = torch.empty(n, dtype=dt, device="cuda")
             loco.loco_unpack_dequant_reduce(gcfg, comms[:N], n, out)
             torch.cuda.synchronize()
@@ -289,3 +292,154 @@ def test_config5_sweep_large_sizes_windows(bits, gd, log2n):
     loco.loco_unpack_dequant_reduce(gcfg, comms, n, out)
     torch.cuda.synchronize()
     wb.compare_reduce(comms, out, "N=16")
+
+
+# ---------------------------------------------------------------- config 4, the view of one rank under expert parallelism 8
+
+def test_config4_mixtral_per_rank_view():
+    """Expert parallelism 8: a rank holds one expert of each of the 32 layers (32 x 176,160,768 elements) and the shared
+    parameters (1,605,636,096): one flat bf16 buffer of 7,242,780,672 elements, heavy-tailed values, every fourth
+    expert all-zero (an expert no token was routed to), 8 parts, fixed and block scales, 2 iterations."""
+    if _free_gb() < 60:
+        pytest.skip("needs ~45 GB of free device memory")
+    expert, shared = 3 * 4096 * 14336, 1_605_636_096
+    n = 32 * expert + shared
+    assert n == 7_242_780_672
+    grad = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    for mode in (loco.SCALE_FIXED, loco.SCALE_BLOCK_ABSMAX):
+        gcfg = loco.Config(bits=4, scale_mode=mode, block_size=256, s=2.0 ** 14, s_e=2.0 ** 16, beta=0.5, reset_period=0,
+                           state_fmt=loco.STATE_INT8, grad_dtype=loco.BF16, out_dtype=loco.BF16, num_partitions=8)
+        lp = loco.loco_partition_capacity(gcfg, n)
+        wins = _windows(n, lp, 8, 1 << 17, 6, seed=6)
+        for e in (3, 4, 31):                       # the start of a dead expert, of a live one, of the last one
+            s0 = (e * expert + 255) // 256 * 256
+            wins.append((s0, min(1 << 16, (s0 // lp + 1) * lp - s0)))
+        wb = WindowedBucket(gcfg, n, wins)
+        chunk = 1 << 27
+        for k in (1, 2):
+            for off in range(0, n, chunk):
+                m = min(chunk, n - off)
+                grad[off:off + m] = inputs.student_t(m, 3.0, 1e-4, seed=3, worker=0, step=k, tag=off >> 8, dtype=torch.bfloat16, device="cuda")
+            for e in range(3, 32, 4):
+                grad[e * expert:(e + 1) * expert] = 0
+            wb.step(grad, k)
+            wb.compare("mode %d k=%d" % (mode, k))
+        del wb
+    del grad
+
+
+# ---------------------------------------------------------------- config 2: Llama-2-7B buckets over 100 iterations
+
+def test_config2_llama_buckets_100_iterations():
+    """Twelve 25M-element buckets of the Llama-2-7B layout -- the first, the partial last one, buckets that straddle
+    tensors, the buckets of the layer groups with the largest and the smallest gradient scale -- each with 8 workers over
+    100 iterations with T_c = 32 (three resets); the oracle follows windows of every bucket and worker (head, ragged tail,
+    a part boundary, a random place); the 8-worker average is compared at iterations around a reset and at the end."""
+    if _free_gb() < 12:
+        pytest.skip("needs ~8 GB of free device memory")
+    layout = inputs.llama2_7b()
+    scales = inputs.group_scales(1, layout.n_groups)
+    buckets = inputs.bucket_ranges(layout.numel, 25_000_000)
+    assert len(buckets) == 270 and buckets[-1][1] - buckets[-1][0] == 13_415_616
+    # first element of every layer group, to find the buckets of the extreme scales
+    starts, pos = {}, 0
+    for numel, grp in layout.segments:
+        starts.setdefault(grp, pos)
+        pos += numel
+    big = max(range(1, 33), key=lambda g: scales[g])
+    small = min(range(1, 33), key=lambda g: scales[g])
+    picked = {0, 269, 5, starts[big] // 25_000_000 + 1, starts[small] // 25_000_000 + 1}
+    rng = np.random.default_rng(12)
+    while len(picked) < 12:
+        picked.add(int(rng.integers(1, 269)))
+    gcfg = loco.Config(bits=4, s=2.0 ** 14, s_e=2.0 ** 16, beta=0.5, reset_period=32, state_fmt=loco.STATE_INT8,
+                       grad_dtype=loco.BF16, out_dtype=loco.BF16, num_partitions=8)
+    workers = 8
+    cells = []
+    for b in sorted(picked):
+        lo, hi = buckets[b]
+        n = hi - lo
+        lp = loco.loco_partition_capacity(gcfg, n)
+        tail = max(0, (n - 1) // 256 * 256 - 4096)
+        wins = [(0, 8192), (tail, n - tail), (3 * lp - 4096, 4096), (3 * lp, 4096)]
+        s0 = int(rng.integers(0, n // 256 - 64)) * 256
+        wins.append((s0, min(8192, (s0 // lp + 1) * lp - s0)))
+        cells.append((b, lo, hi, [WindowedBucket(gcfg, n, wins) for _ in range(workers)]))
+    check_reduce_at = {0, 31, 32, 33, 64, 99}
+    for k in range(100):
+        for b, lo, hi, wbs in cells:
+            for w, wb in enumerate(wbs):
+                g = inputs.layout_slice(layout, lo, hi, scales, 1e-4, seed=1, worker=w, step=k, device="cuda")
+                wb.step(g, k)
+            if k in check_reduce_at or k % 10 == 0:
+                for wb in wbs:
+                    wb.compare("bucket %d k=%d" % (b, k))
+            if k in check_reduce_at:
+                n = hi - lo
+                out = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+                comms = [wb.comm for wb in wbs]
+                loco.loco_unpack_dequant_reduce(gcfg, comms, n, out)
+                torch.cuda.synchronize()
+                wbs[0].compare_reduce(comms, out, "bucket %d k=%d" % (b, k))
+    for b, lo, hi, wbs in cells:
+        for wb in wbs:
+            wb.compare("bucket %d end" % b)
+
+
+# ---------------------------------------------------------------- more than 2^32 elements in ONE part
+
+def test_block_scales_with_more_than_2_to_32_elements_in_one_part():
+    """4,400,000,512 bf16 elements in a single part (num_partitions = 1), one scale per 256 elements: partition-local
+    element indices and scale indices beyond 2^32.  Windows on both sides of the 2^32-nd element and at the ragged end;
+    then the 2-worker average of the whole part."""
+    if _free_gb() < 40:
+        pytest.skip("needs ~30 GB of free device memory")
+    n = 4_400_000_512 + 77
+    gcfg = loco.Config(bits=4, scale_mode=loco.SCALE_BLOCK_ABSMAX, block_size=256, beta=0.5, reset_period=0,
+                       state_fmt=loco.STATE_INT8, grad_dtype=loco.BF16, out_dtype=loco.BF16, num_partitions=1)
+    lp = loco.loco_partition_capacity(gcfg, n)
+    assert lp >= n > 1 << 32
+    wins = _windows(n, lp, 1, 1 << 17, 4, seed=7) + [((1 << 32) - (1 << 16), 1 << 17), ((1 << 32) + 512 * 7, 1 << 16)]
+    wb = WindowedBucket(gcfg, n, wins)
+    grad = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    for k in (1, 2):
+        _fill_gaussian_bf16(grad, 1e-3, seed=8, worker=0, step=k)
+        wb.step(grad, k)
+        wb.compare("k=%d" % k)
+    del grad
+    out = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    other = wb.comm.clone()
+    loco.loco_unpack_dequant_reduce(gcfg, [wb.comm, other], n, out)
+    torch.cuda.synchronize()
+    wb.compare_reduce([wb.comm, other], out, "reduce")
+
+
+def test_adam_fused_part_with_more_than_4_gib_of_codes():
+    """The receive pass fused with the Adam-family step on one part whose 8-bit codes fill more than 4 GiB (4,300,000,256
+    elements, 1 worker, non-power-of-two s so that the generic path runs): moments and weights of windows on both sides of
+    the 4-GiB offset against the oracle."""
+    if _free_gb() < 70:
+        pytest.skip("needs ~60 GB of free device memory")
+    n = 4_300_000_256 + 33
+    kw = dict(bits=8, s=3000.0, s_e=12000.0, beta=0.5, reset_period=0, state_fmt=loco.STATE_NONE, grad_dtype=loco.BF16,
+              out_dtype=loco.F32, num_partitions=1)
+    gcfg = loco.Config(**kw)
+    pb = loco.loco_packed_bytes(gcfg, n)
+    assert pb > 1 << 32
+    comm = _random_codes(pb, 900)
+    m = torch.zeros(n, dtype=torch.float32, device="cuda")
+    v = torch.zeros(n, dtype=torch.float32, device="cuda")
+    theta = torch.ones(n, dtype=torch.float32, device="cuda")
+    ad = dict(lr=1e-3, beta1=0.1, beta2=0.001, delta=1e-16)
+    loco.loco_unpack_dequant_reduce_adam(gcfg, [comm], n, m, v, theta, **ad)
+    torch.cuda.synchronize()
+    ocfg = orc.OracleConfig(**kw)
+    for s0 in (0, (1 << 32) - (1 << 15), (1 << 32) + 4096, n - 5000):
+        ln = min(1 << 16, n - s0)
+        mini = orc.new_comm(ocfg, ln)
+        mini[:ln] = comm[s0:s0 + ln].cpu().numpy()
+        om, ov, ot = np.zeros(ln, np.float32), np.zeros(ln, np.float32), np.ones(ln, np.float32)
+        orc.reduce_adam(ocfg, ln, [mini], om, ov, ot, **ad)
+        for got, want, name in ((m, om, "m"), (v, ov, "v"), (theta, ot, "theta")):
+            g = got[s0:s0 + ln].cpu().numpy()
+            assert np.array_equal(g.view(np.uint32), want.view(np.uint32)), "%s differs in window at %d" % (name, s0)

@@ -4,13 +4,15 @@ Some users of the library cannot give it device memory: their framework's alloca
 taken the whole GPU, or they call from a place where cudaMalloc is not allowed.  For them the
 library stages host buffers through a fixed array inside its own image.  This test calls that
 entry point through the C ABI twice in a row and requires the bytes the workspace-taking entry
-point produces, then checks that a request beyond the array's size is refused.  The file name
+point produces -- and the bytes the CPU oracle computes from the same parts (Eq. 8) -- then
+checks that a request beyond the array's size is refused.  The file name
 sorts last so that a run stopping at the first failure has already run everything else.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import loco_oracle as orc
 from paper_2407_04480_b200 import loco
 
 pytestmark = pytest.mark.gpu
@@ -54,6 +56,18 @@ def test_noalloc_reduce_matches_the_workspace_variant_twice():
         assert want.abs().max() > 0
         # same kernel on the same bytes: the outputs are identical, which is inside every tolerance in use
         assert np.array_equal(got.view(torch.int16).numpy(), want.view(torch.int16).numpy())
+        # and they are what the oracle averages from these parts: each worker's host buffer holds parts first..first+count-1,
+        # which the oracle addresses inside a whole communication buffer
+        ocfg = orc.OracleConfig(bits=4, s=2.0 ** 12, s_e=2.0 ** 14, beta=0.5, reset_period=0, state_fmt=orc.STATE_NONE,
+                                grad_dtype=orc.BF16, out_dtype=orc.BF16, num_partitions=4)
+        stride = orc.partition_bytes(ocfg, n)
+        comms = []
+        for p in parts:
+            whole = np.zeros(orc.packed_bytes(ocfg, n), dtype=np.uint8)
+            whole[first * stride:(first + count) * stride] = p.numpy()
+            comms.append(whole)
+        oracle = orc.reduce(ocfg, n, comms, first=first, count=count)
+        assert np.array_equal(got.view(torch.int16).numpy().view(np.uint16), oracle)
 
 
 def test_noalloc_reduce_refuses_requests_beyond_its_array():
