@@ -558,6 +558,27 @@ int reduce_common(const loco_config_t *cfg, int32_t num_workers, int32_t first_p
         C.inv_s = vinv;
         C.gen_mul = vinv;
         C.gen_mode = 0;
+        // Integer path: with s a power of two every partial sum of the +-1/s is exact, so the negative workers of an
+        // element can be counted; the kernel's byte lanes hold 2c <= 32 and the sum is (N - 2c) / s (/ N)
+        if (num_workers <= 16 && is_pow2_float(cfg->s) && max_code_bytes < (1ull << 32)) {
+            C.int_path = 1;
+            const float inv_s = 1.0f / cfg->s;                                    // exact
+            float r = inv_s;
+            if (n_pow2) r = inv_s * C.inv_n;                                      // exact: both powers of two
+            C.ra = -r;
+            C.rb = (kMagic + static_cast<float>(num_workers)) * r;                // exact: integer < 2^24 times 2^k
+            if (!n_pow2) {
+                bool nr_ok = true;
+                for (int c2 = 0; c2 <= num_workers && nr_ok; ++c2) {
+                    const float acc = static_cast<float>(num_workers - 2 * c2) * inv_s;
+                    const volatile float want = acc / C.n_workers_f;
+                    const volatile float q0 = acc * C.inv_n;
+                    const float rem = std::fmaf(-q0, C.n_workers_f, acc);
+                    nr_ok = same_bits(std::fmaf(rem, C.inv_n, q0), want);
+                }
+                C.div_mode = nr_ok ? 1 : 2;
+            }
+        }
     } else if (mode == MODE_FIXED) {
         const int half = 1 << (cfg->bits - 1);
         {
@@ -604,7 +625,7 @@ int reduce_common(const loco_config_t *cfg, int32_t num_workers, int32_t first_p
         }
     }
     path = mode == MODE_BLOCK ? PATH_MUL
-           : (cfg->bits == 1 ? PATH_MUL : (C.int_path ? PATH_INT : (C.gen_mode == 0 ? PATH_MUL : (C.gen_mode == 1 ? PATH_NEWTON : PATH_DIVIDE))));
+           : (C.int_path ? PATH_INT : (cfg->bits == 1 || C.gen_mode == 0 ? PATH_MUL : (C.gen_mode == 1 ? PATH_NEWTON : PATH_DIVIDE)));
     if (ad) {
         C.adam_m = d_m; C.adam_v = d_v; C.adam_theta = d_theta;
         C.lr = ad->lr; C.beta1 = ad->beta1; C.beta2 = ad->beta2; C.delta = ad->delta;

@@ -767,8 +767,9 @@ struct SendConsts {
 
 // Field j of the packed codes sits in the low bits of mb_j = bits(kMagic + 2^(p-1) + q_j):
 // sum_j mb_j * R^j = kMagicBits * sum_j R^j + sum_j (q_j + 2^(p-1)) R^j  (mod 2^32), R = 2^p; removing the
-// constant and flipping each field's top bit turns the biased fields into two's complement.  The sum is taken one
-// multiply-add (fp32 pipe) per code as the codes are produced, so that no code has to wait in a register for the others.
+// constant and flipping each field's top bit turns the biased fields into two's complement.  The sum is a Horner
+// chain of integer multiply-adds (fp32 pipe), fed with the codes from the last one down as they are produced, so that
+// no code has to wait in a register for the others.
 template <int BITS>
 struct CodePacker {
     static constexpr int kPerWord = 32 / BITS;               // 16, 8 or 4 codes per word
@@ -778,8 +779,9 @@ struct CodePacker {
 #pragma unroll
         for (int i = 0; i < kWords; ++i) w[i] = 0u;
     }
-    __device__ __forceinline__ void put(int j, unsigned mb) {        // code j of the lane's 16, j a compile-time constant
-        w[(j / kPerWord) % kWords] = mb * (1u << (BITS * (j % kPerWord))) + w[(j / kPerWord) % kWords];
+    // code j of the lane's 16; the codes of a word must arrive in descending order of j
+    __device__ __forceinline__ void push(int j, unsigned mb) {
+        w[(j / kPerWord) % kWords] = w[(j / kPerWord) % kWords] * (1u << BITS) + mb;
     }
     __device__ __forceinline__ unsigned word(int i) const {
         unsigned ones = 0u, flip = 0u;
@@ -1043,7 +1045,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         }
     }
 #pragma unroll
-    for (int k = 0; k < (BITS == 1 ? 0 : 8); ++k) {
+    for (int k = (BITS == 1 ? -1 : 7); k >= 0; --k) {      // from the last pair down: the order the code packer wants
         float y0 = 0.0f, y1 = 0.0f, t0 = 0.0f, t1 = 0.0f;
         f32x2 m2;                                                                                    // kMagic + 2^(p-1) + q
         if (MODE == MODE_BLOCK && !var_is_sr(VAR)) {
@@ -1063,8 +1065,8 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             m2 = fadd2(pk2(fminf(fmaxf(t0, lo), hi), fminf(fmaxf(t1, lo), hi)), qmagic2);
         }
         const unsigned mb0 = static_cast<unsigned>(m2), mb1 = static_cast<unsigned>(m2 >> 32);
-        pack.put(2 * k, mb0);
-        pack.put(2 * k + 1, mb1);
+        pack.push(2 * k + 1, mb1);
+        pack.push(2 * k, mb0);
         f32x2 d2;
         if (MODE == MODE_BLOCK) {
             d2 = fmul2_pz(fadd2(m2, dup2(-qmagic)), dup2(scale));          // q is never -0 and a non-zero q times a block scale never underflows
@@ -1303,12 +1305,16 @@ __device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucke
     flush_counts(Bk.status, C.collect_stats != 0, lane, saturated, state_saturated, nonfinite);
 }
 
+// CTAs per SM the send kernels are compiled for: three with the global scale (80 registers per thread); the block-scaled
+// form keeps a whole row's h and error in registers while the block maxima are formed and gets 120 registers (two CTAs).
+template <int MODE> constexpr int kSendCtasPerSm = (MODE == MODE_BLOCK) ? 2 : 3;
+
 // One bucket per launch: grid = (CTAs per partition, partitions).
 // VAR_LEAN / VAR_LEAN_NR kernels are launched when the host proved the corresponding decompressor forms and neither
 // statistics nor clipping are wanted (VAR_LEAN also for every block-scaled configuration), VAR_LEAN_X / VAR_LEAN_NR_X
 // when they are; VAR_GENERAL chooses the decompressor forms at run time.
 template <int GRAD, int STATE, int BITS, int MODE, int VAR>
-__global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_constant__ SendParams P) {
+__global__ void __launch_bounds__(kThreads, kSendCtasPerSm<MODE>) loco_send_kernel(const __grid_constant__ SendParams P) {
     const unsigned long long part = blockIdx.y;
     send_bucket<GRAD, STATE, BITS, MODE, VAR>(
         P.c, P.b, [&]() -> uint8_t * { return P.scatter ? P.part_dst[part] : P.b.comm + part * P.b.stride; }, part, blockIdx.x, gridDim.x);
@@ -1320,7 +1326,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_send_kernel(const __grid_con
 // more of them, no bucket boundary drains the machine, and the launch costs are paid once per call.  The table of
 // buckets travels in the kernel's parameters.
 template <int GRAD, int STATE, int BITS, int MODE, int VAR>
-__global__ void __launch_bounds__(kThreads, 3) loco_send_multi_kernel(const __grid_constant__ SendMultiParams P) {
+__global__ void __launch_bounds__(kThreads, kSendCtasPerSm<MODE>) loco_send_multi_kernel(const __grid_constant__ SendMultiParams P) {
     const SendBucket &Bk = P.b[blockIdx.z];
     if (blockIdx.x >= Bk.grid_x) return;
     const unsigned long long part = blockIdx.y;
@@ -1500,6 +1506,9 @@ __device__ __forceinline__ void adam_finish16(const ReduceCommon &C, void *out, 
 // order or the format it is taken in.  The codes, biased to be non-negative, are added side by side inside
 // 32-bit words (8-bit lanes for 2- and 4-bit codes, 16-bit lanes for 8-bit codes); the lane sums S reach
 // fp32 through the mantissa of kMagic and one fused multiply-add gives (S - bias N) / s (/ N).
+// Sign code: a byte lane counts twice the negative workers of its element, 2c (a multiply spreads four wire bits to
+// four bytes: bit i of a nibble times 0x00408102 lands, among others, on bit 8 i + 1, and no two bits meet), and the
+// sum of the +-1 is N - 2c.
 template <int BITS>
 struct WideSums {
     static constexpr int S = (BITS == 8) ? 8 : 4;
@@ -1521,15 +1530,19 @@ struct WideSums {
                 s[(2 * h) % S] += xor_and(c.w[h % WideCodes<BITS>::W], 0x00800080u, 0x00FF00FFu);
                 s[(2 * h + 1) % S] += xor_and(c.w[h % WideCodes<BITS>::W] >> 8, 0x00800080u, 0x00FF00FFu);
             }
-        } else {                    // byte b of s[k] holds element 4b + k
+        } else if (BITS == 2) {     // byte b of s[k] holds element 4b + k
 #pragma unroll
             for (int k = 0; k < 4; ++k) s[k % S] += xor_and(c.w[0] >> (2 * k), 0x02020202u, 0x03030303u);
+        } else {                    // sign code: byte b of s[g] holds 2 x (negative workers of element 4g + b)
+#pragma unroll
+            for (int g = 0; g < 4; ++g) s[g % S] += (((c.w[0] >> (4 * g)) & 0xFu) * 0x00408102u) & 0x02020202u;
         }
     }
     // kMagic + S_j as a float
     __device__ __forceinline__ float get(int j) const {
         if (BITS == 4) return __uint_as_float(__byte_perm(s[(2 * (j >> 3) + (j & 1)) % S], kMagicBits, 0x7650 + ((j & 7) >> 1)));
         if (BITS == 8) return __uint_as_float(__byte_perm(s[(2 * (j >> 2) + (j & 1)) % S], kMagicBits, ((j & 3) >> 1) ? 0x7632 : 0x7610));
+        if (BITS == 1) return __uint_as_float(__byte_perm(s[(j >> 2) % S], kMagicBits, 0x7650 + (j & 3)));
         return __uint_as_float(__byte_perm(s[(j & 3) % S], kMagicBits, 0x7650 + (j >> 2)));
     }
 };

@@ -23,9 +23,9 @@ ReduceKernel both() {
 template <int OUT, int BITS>
 ReduceKernel pick_reduce_path(int mode, int path) {
     if (mode != MODE_FIXED) return both<OUT, BITS, MODE_BLOCK, PATH_MUL>();
-    // the sign code has one form per scale rule: d = +-magnitude, summed in worker order
-    if (BITS == 1) return both<OUT, BITS, MODE_FIXED, PATH_MUL>();
-    constexpr int B2 = BITS == 1 ? 2 : BITS;        // the other paths are not instantiated for the sign code
+    // the sign code has two forms with the global scale: the integer sum (power-of-two s) and d = +-fl(1/s) summed in worker order
+    if (BITS == 1) return path == PATH_INT ? both<OUT, BITS, MODE_FIXED, PATH_INT>() : both<OUT, BITS, MODE_FIXED, PATH_MUL>();
+    constexpr int B2 = BITS == 1 ? 2 : BITS;        // the division paths are not instantiated for the sign code
     switch (path) {
     case PATH_INT: return both<OUT, B2, MODE_FIXED, PATH_INT>();
     case PATH_MUL: return both<OUT, B2, MODE_FIXED, PATH_MUL>();

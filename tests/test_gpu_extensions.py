@@ -63,16 +63,29 @@ def test_sign_code_ragged_and_special_values(mode):
             assert_reduced_equal(got, want, gd == loco.BF16, "n=%d" % n)
 
 
-@pytest.mark.parametrize("N", [1, 2, 3, 5, 8, 16])
-def test_sign_code_reduce_workers(N):
+@pytest.mark.parametrize("N", [1, 2, 3, 5, 8, 13, 16, 17])
+@pytest.mark.parametrize("s", [3000.0, 2.0 ** 10])
+def test_sign_code_reduce_workers(N, s):
+    """Non-power-of-two s: +-fl(1/s) summed in worker order; power-of-two s and at most 16 workers: the negative
+    workers of every element are counted and the sum is exact."""
     n = 300_003
-    gcfg, ocfg = both_configs(bits=1, s=3000.0, s_e=12000.0, beta=0.5, reset_period=0, state_fmt=loco.STATE_NONE,
+    gcfg, ocfg = both_configs(bits=1, s=s, s_e=4 * s, beta=0.5, reset_period=0, state_fmt=loco.STATE_NONE,
                               grad_dtype=loco.BF16, out_dtype=loco.BF16, num_partitions=4)
     ws = [run_steps(gcfg, ocfg, n, 1, 1e-3, seed=24, worker=w) for w in range(N)]
     got, want = reduce_both(gcfg, ocfg, n, ws)
     assert_reduced_equal(got, want, True)
     got, want = reduce_both(gcfg, ocfg, n, ws, first=1, count=2)
     assert_reduced_equal(got, want, True)
+
+
+@pytest.mark.parametrize("s", [3000.0, 2.0 ** 10])
+@pytest.mark.parametrize("mode", [loco.SCALE_FIXED, loco.SCALE_BLOCK_ABSMAX])
+def test_sign_code_receive_fused_with_the_adam_family_step(s, mode):
+    from tests.test_gpu_adam import _check
+    gcfg, _ = both_configs(bits=1, scale_mode=mode, block_size=128, s=s, s_e=4 * s, beta=0.5, reset_period=0,
+                           state_fmt=loco.STATE_INT8, grad_dtype=loco.BF16, out_dtype=loco.F32, num_partitions=2)
+    for workers in (3, 8):
+        _check(gcfg, 200_003, workers, seed=25)
 
 
 def test_sign_code_rejects_stochastic_rounding():
