@@ -346,13 +346,13 @@ def oracle_sample(threads: int, buckets_per_thread: int, cfgd: dict = None, n: i
     return gsz * elems / dt / 1e9, dt, elems
 
 
-def cpu_baseline_record(cores: int, cfgd: dict, n: int, workers: int, what: str, per_thread: int = 2):
+def cpu_baseline_record(cores: int, cfgd: dict, n: int, workers: int, what: str, per_thread: int = 4):
     """The oracle on all host cores and on one thread, on a bounded sample of the workload's buckets."""
     v, dt, _ = oracle_sample(cores, per_thread, cfgd, n, workers)
-    v1, dt1, _ = oracle_sample(1, 1, cfgd, n, workers)
+    v1, dt1, _ = oracle_sample(1, max(1, per_thread // 2), cfgd, n, workers)
     return {"value": v, "unit": "GB/s", "cores": cores, "kind": "oracle",
             "sample": "%d %s (%d per host thread), send + %d-worker reduce, %.1f s wall" % (per_thread * cores, what, per_thread, workers, dt),
-            "one_thread_value": v1, "one_thread_sample": "1 of the same, %.1f s" % dt1}
+            "one_thread_value": v1, "one_thread_sample": "%d of the same on one thread, %.1f s" % (max(1, per_thread // 2), dt1)}
 
 
 # ------------------------------------------------------------------------------------------------ real exchange
@@ -650,13 +650,20 @@ def run_other_config(args, device, cores):
     rows = []
 
     def timed(fn, reps, warm=3):
+        """Average device time of fn() in microseconds; the launches are replayed from a CUDA graph so that the host's
+        launch cost (several microseconds per call from Python) is not what is timed."""
         for _ in range(warm):
             fn()
         torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for _ in range(reps):
+                fn()
+        graph.replay()
+        torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for _ in range(reps):
-            fn()
+        graph.replay()
         e1.record()
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) * 1e3 / reps          # microseconds
@@ -690,7 +697,7 @@ def run_other_config(args, device, cores):
             us = timed(lambda: loco.loco_unpack_dequant_reduce(cfg, [comm], n, out), 200)
             row("reduce", "%s scale, 1 worker, fp32 out" % scale, n, reduce_bytes_per_elem(c, 1), 4, us, "L2-resident")
         oc = dict(cfg_for("fixed"), s=2.0 ** 11, s_e=2.0 ** 13, grad_dtype=0, out_dtype=0, num_partitions=1)
-        cpu = cpu_baseline_record(cores, oc, n, 1, "vectors of 2^20 fp32 elements", per_thread=16)
+        cpu = cpu_baseline_record(cores, oc, n, 1, "vectors of 2^20 fp32 elements", per_thread=128)
     elif args.config == 3:
         # 13B dense transformer, one flat bf16 buffer in the reduce-scatter layout of 8 parts: one send launch over the whole
         # buffer; a rank then averages its own part (1,626,983,040 elements) over 8 workers

@@ -164,9 +164,10 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, unsigned k0, unsigned k1
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
         if (r > 0) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
-        const unsigned hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
-        const unsigned hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
-        c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+        const unsigned long long p0 = static_cast<unsigned long long>(0xD2511F53u) * c.x;      // one wide multiply: both halves
+        const unsigned long long p1 = static_cast<unsigned long long>(0xCD9E8D57u) * c.z;
+        c = make_uint4(static_cast<unsigned>(p1 >> 32) ^ c.y ^ k0, static_cast<unsigned>(p1),
+                       static_cast<unsigned>(p0 >> 32) ^ c.w ^ k1, static_cast<unsigned>(p0));
     }
     return c;
 }
@@ -585,6 +586,8 @@ __device__ __forceinline__ f32x2 fadd2(f32x2 a, f32x2 b) { f32x2 d; asm("add.rn.
 __device__ __forceinline__ f32x2 fsub2(f32x2 a, f32x2 b) { f32x2 d; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 __device__ __forceinline__ f32x2 fmul2(f32x2 a, f32x2 b) { f32x2 d; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 __device__ __forceinline__ f32x2 ffma2(f32x2 a, f32x2 b, f32x2 c) { f32x2 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d; }
+// a + b rounded toward minus infinity: with b = kMagic (+ bias) the sum's mantissa holds floor(a) (+ bias)
+__device__ __forceinline__ f32x2 fadd2_down(f32x2 a, f32x2 b) { f32x2 d; asm("add.rm.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d; }
 // The assembler contracts a packed multiply that feeds a packed add or subtract into one packed FMA even
 // though both carry an explicit rounding mode (seen as single-rounded results on sm_100a, CUDA 12.9; the same
 // happens when the product is written fma(a, b, -0)).  Where Algorithm 1 rounds the product and the sum
@@ -1054,15 +1057,21 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             // magic constant cannot be contracted with it (the sign of a zero product does not reach the sum).
             m2 = fadd2(fmul2_pz(h2[k], mult2), qmagic2);
         } else {
-            unpk2(fmul2(h2[k], mult2), y0, y1);
-            t0 = y0;
-            t1 = y1;
-            if (var_is_sr(VAR)) {                   // floor(y + u): up with probability frac(y)
+            if (var_is_sr(VAR)) {
+                // floor(y + u): up with probability frac(y).  y + u is one rounded add; clamping it to [lo, hi + 1/2]
+                // clamps its floor to [lo, hi]; adding the magic constant rounding DOWN leaves that floor in the mantissa
                 const unsigned word = (k >> 1) == 0 ? rnd.x : ((k >> 1) == 1 ? rnd.y : ((k >> 1) == 2 ? rnd.z : rnd.w));
-                t0 = floorf(__fadd_rn(y0, sr_dither(word, 2 * (k & 1))));
-                t1 = floorf(__fadd_rn(y1, sr_dither(word, 2 * (k & 1) + 1)));
+                const f32x2 mu2 = pk2(__uint_as_float(__byte_perm(word, 0x4B000000u, 0x7540 + 2 * (k & 1))),
+                                      __uint_as_float(__byte_perm(word, 0x4B000000u, 0x7540 + 2 * (k & 1) + 1)));     // 2^23 + byte
+                const f32x2 u2 = ffma2(mu2, dup2(0.00390625f), dup2(-32767.998046875f));               // byte / 256 + 1 / 512, exact
+                unpk2(fadd2(fmul2_pz(h2[k], mult2), u2), t0, t1);             // the product as fma(h, s, +0): not contracted with the add
+                m2 = fadd2_down(pk2(fminf(fmaxf(t0, lo), hi + 0.5f), fminf(fmaxf(t1, lo), hi + 0.5f)), qmagic2);
+            } else {
+                unpk2(fmul2(h2[k], mult2), y0, y1);
+                t0 = y0;
+                t1 = y1;
+                m2 = fadd2(pk2(fminf(fmaxf(t0, lo), hi), fminf(fmaxf(t1, lo), hi)), qmagic2);
             }
-            m2 = fadd2(pk2(fminf(fmaxf(t0, lo), hi), fminf(fmaxf(t1, lo), hi)), qmagic2);
         }
         const unsigned mb0 = static_cast<unsigned>(m2), mb1 = static_cast<unsigned>(m2 >> 32);
         pack.push(2 * k + 1, mb1);
@@ -1077,8 +1086,8 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
                      dec_fast(__uint_as_float(mb1), qmagic, dq_mode, K.dq_a, K.dq_b, K.s, K.inv_s));
         }
         if (MODE != MODE_BLOCK && EXTRAS && stats) {
-            if (var_is_sr(VAR)) {
-                saturated += ((t0 < lo || t0 > hi) ? 1u : 0u) + ((t1 < lo || t1 > hi) ? 1u : 0u);
+            if (var_is_sr(VAR)) {               // t = y + u before the floor: its floor leaves [lo, hi] iff t < lo or t >= hi + 1
+                saturated += ((t0 < lo || t0 >= hi + 1.0f) ? 1u : 0u) + ((t1 < lo || t1 >= hi + 1.0f) ? 1u : 0u);
             } else {
                 if (y0 >= hi + 0.5f || y0 < lo - 0.5f) saturated += 1u;
                 if (y1 >= hi + 0.5f || y1 < lo - 0.5f) saturated += 1u;
