@@ -611,7 +611,7 @@ def sweep(args, device):
         send_case("bf16 g, int8 state, 4 bit, block-%d absmax" % B, M, scale_mode=1, block_size=B)
     send_case("fp32 g, int8 state, 4 bit, block-256 absmax", M, scale_mode=1, grad_dtype=0)
     for B in (512, 1024, 4096):
-        send_case("bf16 g, int8 state, 4 bit, block-%d absmax%s" % (B, "" if B == 512 else " (block walked in several passes)"), M, scale_mode=1, block_size=B)
+        send_case("bf16 g, int8 state, 4 bit, block-%d absmax%s" % (B, "" if B == 512 else " (rows of a block on neighbouring warps)"), M, scale_mode=1, block_size=B)
     send_case("bf16 g, int8 state, 1 bit (sign code), fixed", M, bits=1)
     send_case("bf16 g, int8 state, 1 bit (sign code), block-256 mean magnitude", M, bits=1, scale_mode=1)
     for log2n in (16, 20, 24, 27, 30):

@@ -324,8 +324,6 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
         // the fast routine tests only g for NaN / Inf when the state is 8-bit: dec(e) must be too small to push a
         // finite g to infinity (|e / s_e| <= 128 / s_e < 2^100)
         if (cfg->state_fmt == LOCO_STATE_INT8 && !(cfg->s_e > 1e-28f)) st->fast = 0;
-    } else if (cfg->block_size > kWide) {
-        st->fast = 0;           // a block wider than a wide row: the careful routine walks it
     }
     {
         int var = VAR_GENERAL;
@@ -335,6 +333,7 @@ int loco_state_init(loco_state_t **out, const loco_config_t *cfg, uint64_t n, vo
             else if (st->dq.mode == DEC_FMA && st->de.mode == DEC_FMA) var = VAR_LEAN_SR;
         } else if (st->mode == MODE_BLOCK) {
             var = cfg->clip > 0.0f ? VAR_GENERAL : VAR_LEAN;      // the plain lean variants carry no clipping
+            if (cfg->block_size > kWide) var |= VAR_WIDE_BLOCKS;   // the rows of a block on neighbouring warps
         } else {
             const bool extras = cfg->collect_stats || cfg->clip > 0.0f;
             if (st->dq.mode == DEC_FMA && st->de.mode == DEC_FMA) var = extras ? VAR_LEAN_X : VAR_LEAN;

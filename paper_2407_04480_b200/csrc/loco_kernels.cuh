@@ -764,7 +764,14 @@ __device__ __forceinline__ void fetch_row(const RingAddr<GRAD, STATE> &A, unsign
 struct SendConsts {
     float s, s_e, beta, omb, inv_s, inv_se, dq_a, dq_b, de_a, de_b, clip;
     int dq_mode, de_mode, block_log2, reset;
-    unsigned blocks_per_row;         // BLOCK, B <= 512: blocks in a wide row
+    // BLOCK: the scales of wide row w start at index (w << row_shl) >> row_shr of the partition's scales: 512 / B
+    // blocks per row when B <= 512, one block per B / 512 rows otherwise
+    unsigned row_shl, row_shr;
+    // BLOCK, B > 512: a block spans `group_warps` (2, 4 or 8) wide rows, which neighbouring warps of the CTA hold at the
+    // same time; they exchange their rows' maxima (sums) through shared memory
+    unsigned group_warps;            // 1 when B <= 512
+    unsigned xslot, xgroup;          // shared-memory addresses: this warp's slot; the slot this lane reads back
+    unsigned bar_id, bar_threads;    // the named barrier of the warp's group
     unsigned seed_lo, seed_hi, k_lo, k_hi;
 };
 
@@ -837,6 +844,11 @@ __device__ __forceinline__ float qmax_over_midrange(float c, float a) {
 }
 __device__ __forceinline__ bool in_midrange(float a) { return __float_as_uint(a) - 0x0d800000u <= 0x71800000u - 0x0d800000u; }
 
+template <bool WIDE>
+__device__ __forceinline__ size_t scale_index(const SendConsts &K, unsigned wrow) {
+    return WIDE ? static_cast<size_t>(wrow >> K.row_shr) : static_cast<size_t>(wrow) << K.row_shl;
+}
+
 // max over aligned groups of `lanes` lanes (1 to 32): four steps without a branch, the fifth (a block of 512 elements
 // spans the whole warp) under a uniform one
 __device__ __forceinline__ float group_max32(float v, int lanes) {
@@ -847,6 +859,20 @@ __device__ __forceinline__ float group_max32(float v, int lanes) {
     }
     if (lanes > 16) v = fmaxf(v, __shfl_xor_sync(kFull, v, 16));
     return v;
+}
+
+// A block wider than a wide row: the warps that hold its rows combine their (warp-uniform) row values -- the maximum, or
+// for the sign code the sum as a balanced tree in row order.  Every warp of the group calls this the same number of
+// times; successive calls alternate between two sets of slots, so that a warp that runs ahead to its next exchange
+// writes where the others have long since read (it had to pass the barrier of the exchange in between, which they
+// reach only after reading).  The barrier is the hardware's named barrier for the group's threads, not a spin.
+template <bool SUM>
+__device__ __forceinline__ float wide_exchange(const SendConsts &K, unsigned &xphase, float v, int lane) {
+    if (lane == 0) asm volatile("st.shared.f32 [%0], %1;" :: "r"(K.xslot + xphase), "f"(v) : "memory");
+    asm volatile("bar.sync %0, %1;" :: "r"(K.bar_id), "r"(K.bar_threads) : "memory");
+    const float x = __uint_as_float(lds4(K.xgroup + xphase));
+    xphase ^= 4u * kWarps;
+    return SUM ? group_sum32(x, static_cast<int>(K.group_warps)) : group_max32(x, static_cast<int>(K.group_warps));
 }
 
 // One wide row.  Returns false if some lane of the warp met a value that the fast arithmetic does not cover (NaN,
@@ -861,9 +887,14 @@ __device__ __forceinline__ float group_max32(float v, int lanes) {
 // VAR_LEAN_X / VAR_LEAN_NR_X: the lean forms plus what a call may ask for on top (statistics, clipping of g).
 // VAR_LEAN_SR: VAR_LEAN_X with stochastic rounding.
 enum : int { VAR_LEAN = 0, VAR_LEAN_NR = 1, VAR_GENERAL = 2, VAR_STOCHASTIC = 3, VAR_LEAN_X = 4, VAR_LEAN_NR_X = 5, VAR_LEAN_SR = 6 };
-__host__ __device__ constexpr bool var_is_lean(int var) { return var == VAR_LEAN || var == VAR_LEAN_NR || var == VAR_LEAN_X || var == VAR_LEAN_NR_X || var == VAR_LEAN_SR; }
-__host__ __device__ constexpr bool var_has_extras(int var) { return var != VAR_LEAN && var != VAR_LEAN_NR; }
-__host__ __device__ constexpr bool var_is_sr(int var) { return var == VAR_STOCHASTIC || var == VAR_LEAN_SR; }
+// added to VAR_LEAN or VAR_GENERAL of a block-scaled kernel: a block is wider than a wide row (B > 512) and its rows sit
+// on neighbouring warps, which exchange their maxima (see wide_exchange)
+enum : int { VAR_WIDE_BLOCKS = 16 };
+__host__ __device__ constexpr int var_base(int var) { return var & 15; }
+__host__ __device__ constexpr bool var_is_wide(int var) { return (var & VAR_WIDE_BLOCKS) != 0; }
+__host__ __device__ constexpr bool var_is_lean(int var) { return var_base(var) == VAR_LEAN || var_base(var) == VAR_LEAN_NR || var_base(var) == VAR_LEAN_X || var_base(var) == VAR_LEAN_NR_X || var_base(var) == VAR_LEAN_SR; }
+__host__ __device__ constexpr bool var_has_extras(int var) { return var_base(var) != VAR_LEAN && var_base(var) != VAR_LEAN_NR; }
+__host__ __device__ constexpr bool var_is_sr(int var) { return var_base(var) == VAR_STOCHASTIC || var_base(var) == VAR_LEAN_SR; }
 
 // dec(e; s_e) of a pair from the magic floats m2 = kMagic + 128 + e
 template <int VAR>
@@ -884,7 +915,8 @@ __device__ __forceinline__ f32x2 dec_state2(const SendConsts &K, f32x2 m2, float
 
 template <int GRAD, int STATE, int BITS, int MODE, int VAR>
 __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtrs &L, const WideIn<GRAD, STATE> &in,
-                                              unsigned wrow, int lane, bool stats, unsigned &saturated, unsigned &state_saturated) {
+                                              unsigned wrow, int lane, bool stats, unsigned &saturated, unsigned &state_saturated,
+                                              unsigned &xphase) {
     constexpr float lo = QRange<BITS>::lo, hi = QRange<BITS>::hi, qmagic = kMagic + QRange<BITS>::off;
     constexpr float emagic = kMagic + 128.0f;
     constexpr bool kStateF32 = (STATE == ST_FP32 || STATE == ST_Q8COMP);
@@ -893,7 +925,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     // a packed add; with an fp32 state the sign of a zero is stored, so there the sum stays scalar (see fadd2_after_mul).
     constexpr bool kSignFree = !kStateF32;
     constexpr int GW = WideIn<GRAD, STATE>::GW, EW = WideIn<GRAD, STATE>::EW;
-    constexpr bool LEAN = var_is_lean(VAR), EXTRAS = var_has_extras(VAR);
+    constexpr bool LEAN = var_is_lean(VAR), EXTRAS = var_has_extras(VAR), WIDE = var_is_wide(VAR);
     const int dq_mode = LEAN ? DEC_FMA : K.dq_mode, de_mode = K.de_mode;
     const int lanes_per_block = (MODE == MODE_BLOCK) ? (K.block_log2 >= 9 ? 32 : (1 << (K.block_log2 - 4))) : 1;    // B <= 512 here
     const f32x2 zero2 = 0ull;
@@ -1004,7 +1036,11 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
 #pragma unroll
             for (int j = 0; j < 16; j += 2 * w) a[j] = __fadd_rn(a[j], a[j + w]);
         }
-        const float sum = group_sum32(a[0], lanes_per_block);
+        float sum = group_sum32(a[0], lanes_per_block);
+        if (WIDE) {                           // a NaN in place of the sum makes every warp of the block give up
+            if (__any_sync(kFull, bad_bits != 0u)) sum = __uint_as_float(0x7fc00000u);
+            sum = wide_exchange<true>(K, xphase, sum, lane);
+        }
         // an overflowing h or sum leaves the row to the careful routine (which forms the same infinities the plain way)
         if (__any_sync(kFull, bad_bits != 0u || !(sum <= kFltMax))) return false;
         scale = __fmul_rn(sum, __uint_as_float(static_cast<unsigned>(127 - K.block_log2) << 23));     // sum / B, exact scaling
@@ -1018,6 +1054,10 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
             amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
         }
         amax = group_max32(amax, lanes_per_block);
+        if (WIDE) {                           // +Inf in place of the maximum makes every warp of the block give up
+            if (__any_sync(kFull, bad_bits != 0u)) amax = __uint_as_float(0x7f800000u);
+            amax = wide_exchange<false>(K, xphase, amax, lane);
+        }
         // g is finite here, so h can only be +-Inf (an overflowing sum), never NaN, and the maximum shows it.  A block
         // maximum outside [2^-100, 2^100] (other than 0) also leaves the row to the careful routine, which divides.
         if (__any_sync(kFull, bad_bits != 0u || !(amax == 0.0f || in_midrange(amax)))) return false;
@@ -1108,9 +1148,9 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     } else {
         st_stream2(cdst, static_cast<uint16_t>(signs));
     }
-    // the scales of wide row w: L.wire_scales / L.state_scales point at this lane's block of row 0; a row holds 512 / B blocks
+    // the scales of wide row w: L.wire_scales / L.state_scales point at this lane's block of row 0
     if (MODE == MODE_BLOCK) {
-        if (L.leader) L.wire_scales[static_cast<size_t>(wrow) * K.blocks_per_row] = scale;
+        if (L.leader) L.wire_scales[scale_index<WIDE>(K, wrow)] = scale;
     }
 
     // ---- Eq. 7 ---------------------------------------------------------------------------------------------------
@@ -1128,6 +1168,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
                     amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
                 }
                 amax = group_max32(amax, lanes_per_block);
+                if (WIDE) amax = wide_exchange<false>(K, xphase, amax, lane);
                 // nothing of the state has been written yet, and the codes stored above are what the careful routine stores
                 if (__any_sync(kFull, !(amax == 0.0f || in_midrange(amax)))) return false;
                 escale = amax > 0.0f ? div_by_qmax(amax, 127.0f, 1.0f / 127.0f) : 0.0f;
@@ -1151,7 +1192,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
         }
         st_stream16(L.state + static_cast<size_t>(wrow) * kWide, v);
         if (MODE == MODE_BLOCK) {
-            if (L.leader) L.state_scales[static_cast<size_t>(wrow) * K.blocks_per_row] = escale;
+            if (L.leader) L.state_scales[scale_index<WIDE>(K, wrow)] = escale;
         }
     } else if (kStateF32) {
         unsigned w[16];
@@ -1184,7 +1225,12 @@ __device__ __forceinline__ void load_consts(const SendCommon &C, SendConsts &K) 
     K.s = C.s; K.s_e = C.s_e; K.beta = C.beta; K.omb = C.omb; K.inv_s = C.inv_s; K.inv_se = C.inv_se;
     K.dq_a = C.dq_a; K.dq_b = C.dq_b; K.de_a = C.de_a; K.de_b = C.de_b;
     K.dq_mode = C.dq_mode; K.de_mode = C.de_mode; K.block_log2 = C.block_log2; K.reset = C.reset; K.clip = C.clip;
-    K.blocks_per_row = static_cast<unsigned>(kWide) >> (C.block_log2 > 9 ? 9 : C.block_log2);
+    K.row_shl = C.block_log2 < 9 ? static_cast<unsigned>(9 - C.block_log2) : 0u;
+    K.row_shr = C.block_log2 > 9 ? static_cast<unsigned>(C.block_log2 - 9) : 0u;
+    K.group_warps = 1u;
+    K.xslot = K.xgroup = 0u;
+    K.bar_id = 0u;
+    K.bar_threads = 32u;
     K.seed_lo = C.seed_lo; K.seed_hi = C.seed_hi; K.k_lo = C.k_lo; K.k_hi = C.k_hi;
 }
 
@@ -1241,32 +1287,48 @@ __device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucke
         nonfinite |= N.nonfinite;
     };
     unsigned first_careful = 0u;             // first 256-element row left to the careful routine
+    // a block of more than 512 elements spans G = B / 512 wide rows; the warps of a CTA hold 8 consecutive wide rows
+    // at a time (warp w of every CTA takes the rows = w mod 8), so the G warps w, w + 1, ... with w a multiple of G hold
+    // one block.  Only whole blocks go through the fast routine, so these warps do the same number of rows.
+    constexpr bool WIDE = var_is_wide(VAR);
+    const unsigned G = WIDE ? (1u << (C.block_log2 - 9)) : 1u;
+    const unsigned warp_in_cta = threadIdx.x >> 5;
+    __shared__ float wide_slots[WIDE ? 2 * kWarps : 1];
     if (C.fast) {
-        const unsigned full_wide = full_rows / 2;
+        const unsigned full_wide = (full_rows / 2) & ~(G - 1u);
         first_careful = 2 * full_wide;
         LanePtrs L;
         lane_pointers<STATE, BITS>(Bk, part_base(), part, lane, L);
+        SendConsts K;
+        load_consts(C, K);
         if (MODE == MODE_BLOCK) {
-            // blocks of at most 512 elements here: a wide row and a partition start on a block boundary, so which lane
-            // leads a block, and which block of its row a lane is in, never changes
+            // a wide row and a partition start on a block boundary (or inside the same block as the row's first element),
+            // so which lane leads a block, and which block of its row a lane is in, never changes
             const unsigned lanes_per_block = C.block_log2 >= 9 ? 32u : (1u << (C.block_log2 - 4));
-            L.leader = (static_cast<unsigned>(lane) & (lanes_per_block - 1u)) == 0u;
+            L.leader = (static_cast<unsigned>(lane) & (lanes_per_block - 1u)) == 0u && (warp_in_cta & (G - 1u)) == 0u;
             L.lane_block = L.lane_elem >> C.block_log2;
             L.wire_scales += L.lane_block;
             L.state_scales += (L.elem0 >> C.block_log2);
+            if (WIDE) {
+                const unsigned slots = static_cast<unsigned>(__cvta_generic_to_shared(wide_slots));
+                K.group_warps = G;
+                K.xslot = slots + 4u * warp_in_cta;
+                K.xgroup = slots + 4u * ((warp_in_cta & ~(G - 1u)) + (static_cast<unsigned>(lane) & (G - 1u)));
+                K.bar_id = 1u + warp_in_cta / G;
+                K.bar_threads = 32u * G;
+            }
         }
+        unsigned xphase = 0u;
         // staging reads: chunk `lane` of each 512-byte piece of the row
         const uint8_t *g_stage = static_cast<const uint8_t *>(Bk.grad) + base * (GRAD == GRAD_BF16 ? 2u : 4u) + lane * 16;
         const uint8_t *e_stage = static_cast<const uint8_t *>(Bk.state) + base * (STATE == ST_INT8 ? 1u : 4u) + lane * 16;
-        SendConsts K;
-        load_consts(C, K);
         const bool stats = C.collect_stats != 0;
         RingAddr<GRAD, STATE> A;
         ring_addresses<GRAD, STATE, MODE>(static_cast<unsigned>(__cvta_generic_to_shared(ring)), lane, threadIdx.x >> 5, A);
         // this warp's wide rows are warp + i * nwarps, i < cnt
         const unsigned cnt = full_wide > warp ? (full_wide - warp + nwarps - 1) / nwarps : 0u;
         auto stage = [&](unsigned slot_off, unsigned wrow) {
-            const float *sp = L.state_scales + static_cast<size_t>(wrow) * K.blocks_per_row;      // MODE_BLOCK only
+            const float *sp = L.state_scales + scale_index<WIDE>(K, wrow);                              // MODE_BLOCK only
             stage_row<GRAD, STATE, MODE>(A, slot_off, g_stage + static_cast<size_t>(wrow) * gbytes,
                                          e_stage + static_cast<size_t>(wrow) * ebytes, sp);
         };
@@ -1293,7 +1355,7 @@ __device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucke
                 fetch_row<GRAD, STATE, MODE>(A, slot_off, in);
                 if (stage_wrow < full_wide) stage(stage_off, stage_wrow);
                 cp_async_commit();             // one group per iteration, empty near the end
-                if (!send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, wrow, lane, stats, saturated, state_saturated))
+                if (!send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, wrow, lane, stats, saturated, state_saturated, xphase))
                     failed |= 1u << (i - i0);
                 slot_off = slot_off + R::kSlotStride == R::kBytes ? 0u : slot_off + R::kSlotStride;
                 stage_off = stage_off + R::kSlotStride == R::kBytes ? 0u : stage_off + R::kSlotStride;
@@ -1303,7 +1365,9 @@ __device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucke
             while (failed) {
                 const unsigned j = static_cast<unsigned>(__ffs(static_cast<int>(failed))) - 1u;
                 failed &= failed - 1u;
-                careful(static_cast<unsigned long long>(wrow0 + j * nwarps) * kWide, 2);
+                // every warp of a wide block noted the failure; the one that holds the block's first row redoes the block
+                if ((warp_in_cta & (G - 1u)) == 0u)
+                    careful(static_cast<unsigned long long>(wrow0 + j * nwarps) * kWide, static_cast<int>(2u * G));
             }
         }
     }

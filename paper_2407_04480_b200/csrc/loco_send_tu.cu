@@ -33,6 +33,8 @@ SendKernel pick_send_mode(int mode, int var) {
     }
     if (STATE == ST_Q8COMP) return {nullptr, nullptr, 0};        // Q8COMP exists for the global scales only
     constexpr int ST = (STATE == ST_Q8COMP ? ST_FP32 : STATE);
+    if (var == (VAR_LEAN | VAR_WIDE_BLOCKS)) return both<GRAD, ST, BITS, MODE_BLOCK, VAR_LEAN | VAR_WIDE_BLOCKS>();
+    if (var == (VAR_GENERAL | VAR_WIDE_BLOCKS)) return both<GRAD, ST, BITS, MODE_BLOCK, VAR_GENERAL | VAR_WIDE_BLOCKS>();
     if (var == VAR_GENERAL) return both<GRAD, ST, BITS, MODE_BLOCK, VAR_GENERAL>();
     if (var == VAR_STOCHASTIC) return both<GRAD, ST, B2, MODE_BLOCK, VAR_STOCHASTIC>();
     return both<GRAD, ST, BITS, MODE_BLOCK, VAR_LEAN>();
