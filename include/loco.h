@@ -85,10 +85,10 @@ typedef struct {
                                 (1 = negative), d = q / s, or q x (mean |h| of the block) with block
                                 scales, that mean summed pairwise in fp32 over the block's positions */
     int32_t scale_mode;      /* loco_scale_mode_t                                                 */
-    int32_t block_size;      /* B, BLOCK_ABSMAX only: power of two in [32, 4096].  Blocks of up to 512
-                                elements run in the fused streaming routine; wider ones are walked block
-                                by block (several passes over the block, served by the caches): same
-                                results, lower speed                                              */
+    int32_t block_size;      /* B, BLOCK_ABSMAX only: power of two in [32, 4096].  A block of up to 512
+                                elements lives in one warp of the streaming routine; a wider one is
+                                spread over 2, 4 or 8 neighbouring warps that exchange their maxima
+                                (with stochastic rounding: walked block by block instead, slower)  */
     float   s;               /* Eq. 1 / Eq. 3 scale, FIXED only (> 0, finite)                     */
     float   s_e;             /* Eq. 2 / Eq. 7 scale of the 8-bit error, FIXED only                */
     float   beta;            /* Eq. 5, in [0, 1]: weight of the NEW compression error             */

@@ -1326,7 +1326,8 @@ __device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucke
         RingAddr<GRAD, STATE> A;
         ring_addresses<GRAD, STATE, MODE>(static_cast<unsigned>(__cvta_generic_to_shared(ring)), lane, threadIdx.x >> 5, A);
         // this warp's wide rows are warp + i * nwarps, i < cnt
-        const unsigned cnt = full_wide > warp ? (full_wide - warp + nwarps - 1) / nwarps : 0u;
+        const unsigned cnt_all = full_wide > warp ? (full_wide - warp + nwarps - 1) / nwarps : 0u;
+        const unsigned cnt = cnt_all < 32u ? cnt_all : 32u;        // the rows that stream through the fast routine
         auto stage = [&](unsigned slot_off, unsigned wrow) {
             const float *sp = L.state_scales + scale_index<WIDE>(K, wrow);                              // MODE_BLOCK only
             stage_row<GRAD, STATE, MODE>(A, slot_off, g_stage + static_cast<size_t>(wrow) * gbytes,
@@ -1340,35 +1341,34 @@ __device__ __forceinline__ void send_bucket(const SendCommon &C, const SendBucke
         unsigned slot_off = 0u, stage_off = (D - 1) * R::kSlotStride;
         unsigned wrow = warp, stage_wrow = warp + (D - 1) * nwarps;
         // Rows the fast routine hands back (a NaN, an Inf, a block maximum out of range: rare) are noted in a mask and
-        // redone by the careful routine after every 32 rows, outside the streaming loop: a call inside it would make
-        // the compiler keep part of the loop's registers in local memory on every iteration.
+        // redone by the careful routine after the streaming loop: a call inside it, or between two runs of it, would
+        // make the compiler keep part of the loop's registers in local memory.
+        unsigned failed = 0u;
 #pragma unroll 1
-        for (unsigned i0 = 0; i0 < cnt; i0 += 32u) {
-            const unsigned i1 = cnt - i0 < 32u ? cnt : i0 + 32u;
-            const unsigned wrow0 = wrow;
-            unsigned failed = 0u;
-#pragma unroll 1
-            for (unsigned i = i0; i < i1; ++i) {
-                cp_async_wait<D - 2>();        // every group but the newest D-2 has landed: this row is there
-                __syncwarp();                  // ... for all lanes; and every lane is done reading the slot refilled next
-                WideIn<GRAD, STATE> in;
-                fetch_row<GRAD, STATE, MODE>(A, slot_off, in);
-                if (stage_wrow < full_wide) stage(stage_off, stage_wrow);
-                cp_async_commit();             // one group per iteration, empty near the end
-                if (!send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, wrow, lane, stats, saturated, state_saturated, xphase))
-                    failed |= 1u << (i - i0);
-                slot_off = slot_off + R::kSlotStride == R::kBytes ? 0u : slot_off + R::kSlotStride;
-                stage_off = stage_off + R::kSlotStride == R::kBytes ? 0u : stage_off + R::kSlotStride;
-                wrow += nwarps;
-                stage_wrow += nwarps;
-            }
+        for (unsigned i = 0; i < cnt; ++i) {
+            cp_async_wait<D - 2>();            // every group but the newest D-2 has landed: this row is there
+            __syncwarp();                      // ... for all lanes; and every lane is done reading the slot refilled next
+            WideIn<GRAD, STATE> in;
+            fetch_row<GRAD, STATE, MODE>(A, slot_off, in);
+            if (i + (D - 1) < cnt) stage(stage_off, stage_wrow);
+            cp_async_commit();                 // one group per iteration, empty near the end
+            if (!send_wide_row<GRAD, STATE, BITS, MODE, VAR>(K, L, in, wrow, lane, stats, saturated, state_saturated, xphase))
+                failed |= 1u << i;
+            slot_off = slot_off + R::kSlotStride == R::kBytes ? 0u : slot_off + R::kSlotStride;
+            stage_off = stage_off + R::kSlotStride == R::kBytes ? 0u : stage_off + R::kSlotStride;
+            wrow += nwarps;
+            stage_wrow += nwarps;
+        }
+        // every warp of a wide block noted the failure; the one that holds the block's first row redoes the block
+        if ((warp_in_cta & (G - 1u)) == 0u) {
             while (failed) {
                 const unsigned j = static_cast<unsigned>(__ffs(static_cast<int>(failed))) - 1u;
                 failed &= failed - 1u;
-                // every warp of a wide block noted the failure; the one that holds the block's first row redoes the block
-                if ((warp_in_cta & (G - 1u)) == 0u)
-                    careful(static_cast<unsigned long long>(wrow0 + j * nwarps) * kWide, static_cast<int>(2u * G));
+                careful(static_cast<unsigned long long>(warp + j * nwarps) * kWide, static_cast<int>(2u * G));
             }
+            // rows beyond what the mask can note: the host's grid leaves a warp about kRowsPerWarp rows, so there are none
+            for (unsigned i = cnt; i < cnt_all; ++i)
+                careful(static_cast<unsigned long long>(warp + i * nwarps) * kWide, static_cast<int>(2u * G));
         }
     }
     // the careful routine's unit: a row, or the rows of a block wider than a row
