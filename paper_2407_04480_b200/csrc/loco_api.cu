@@ -425,6 +425,10 @@ void fill_common(const loco_state_t *st, int64_t step_k, SendCommon &C) {
     C.clip = c.clip;
     C.stochastic = c.rounding == LOCO_ROUND_STOCHASTIC ? 1 : 0;
     C.seed_lo = c.seed_lo; C.seed_hi = c.seed_hi;
+    for (uint32_t r = 0; r < 10; ++r) {                  // Philox round keys: the Weyl sequence of the key
+        C.sr_keys[2 * r] = c.seed_lo + r * 0x9E3779B9u;
+        C.sr_keys[2 * r + 1] = c.seed_hi + r * 0xBB67AE85u;
+    }
     C.k_lo = static_cast<unsigned>(static_cast<uint64_t>(step_k));
     C.k_hi = static_cast<unsigned>(static_cast<uint64_t>(step_k) >> 32);
 }

@@ -62,6 +62,7 @@ struct SendCommon {
     float clip;                      // > 0: element-wise clipping of g to [-clip, clip] before step 1
     int stochastic;                  // stochastic rounding of the gradient codes (extension)
     unsigned seed_lo, seed_hi;       // key of its Philox stream
+    unsigned sr_keys[20];            // the ten round keys (seed + r x the Weyl constants), low and high word interleaved
     unsigned k_lo, k_hi;             // the iteration counter, part of the Philox counter
 };
 
@@ -160,10 +161,12 @@ __device__ __forceinline__ float round_clamp(float y, float lo, float hi, unsign
 
 // Philox4x32-10 (Salmon et al., SC'11), from its published definition: ten rounds of two 32x32->64 multiplications by
 // fixed constants, xors with the key, a Weyl bump of the key between rounds.
-__device__ __forceinline__ uint4 philox4x32_10(uint4 c, unsigned k0, unsigned k1) {
+// `keys`: the round keys (k0 + r 0x9E3779B9, k1 + r 0xBB67AE85), r = 0..9, formed once per call on the host and read
+// here as operands from the kernel's parameters, so that the bumps cost no instructions.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, const unsigned *keys) {
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        if (r > 0) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+        const unsigned k0 = keys[2 * r], k1 = keys[2 * r + 1];
         const unsigned long long p0 = static_cast<unsigned long long>(0xD2511F53u) * c.x;      // one wide multiply: both halves
         const unsigned long long p1 = static_cast<unsigned long long>(0xCD9E8D57u) * c.z;
         c = make_uint4(static_cast<unsigned>(p1 >> 32) ^ c.y ^ k0, static_cast<unsigned>(p1),
@@ -174,8 +177,8 @@ __device__ __forceinline__ uint4 philox4x32_10(uint4 c, unsigned k0, unsigned k1
 // Stochastic rounding adds (b + 1/2) / 256 to h x s, b = one byte of the Philox block of the element's group of 16:
 // element i of the bucket takes byte (i mod 4) of word ((i mod 16) / 4) of
 // philox(counter = (i/16 low, i/16 high, k low, k high), key = seed).
-__device__ __forceinline__ uint4 sr_block(unsigned long long blk, unsigned k_lo, unsigned k_hi, unsigned seed_lo, unsigned seed_hi) {
-    return philox4x32_10(make_uint4(static_cast<unsigned>(blk), static_cast<unsigned>(blk >> 32), k_lo, k_hi), seed_lo, seed_hi);
+__device__ __forceinline__ uint4 sr_block(unsigned long long blk, unsigned k_lo, unsigned k_hi, const unsigned *keys) {
+    return philox4x32_10(make_uint4(static_cast<unsigned>(blk), static_cast<unsigned>(blk >> 32), k_lo, k_hi), keys);
 }
 __device__ __forceinline__ float sr_dither(unsigned word, int byte) {
     const float m = __uint_as_float(__byte_perm(word, 0x4B000000u, 0x7540 + byte));      // 2^23 + b
@@ -378,7 +381,7 @@ __device__ __forceinline__ void careful_quantise(const SendCommon &C, const Care
                                                  unsigned (&code)[8], float (&e_new)[8], CarefulCounts &N) {
     float u8[8];
     if (STOCH) {                                            // i0 is a multiple of 8: one half of a block of 16
-        const uint4 r = sr_block(V.i0 >> 4, C.k_lo, C.k_hi, C.seed_lo, C.seed_hi);
+        const uint4 r = sr_block(V.i0 >> 4, C.k_lo, C.k_hi, C.sr_keys);
         const bool upper = ((V.i0 >> 3) & 1ull) != 0ull;
         const unsigned w0 = upper ? r.z : r.x, w1 = upper ? r.w : r.y;
 #pragma unroll
@@ -772,7 +775,8 @@ struct SendConsts {
     unsigned group_warps;            // 1 when B <= 512
     unsigned xslot, xgroup;          // shared-memory addresses: this warp's slot; the slot this lane reads back
     unsigned bar_id, bar_threads;    // the named barrier of the warp's group
-    unsigned seed_lo, seed_hi, k_lo, k_hi;
+    unsigned k_lo, k_hi;
+    const unsigned *sr_keys;         // the Philox round keys, in the kernel's parameters
 };
 
 // Field j of the packed codes sits in the low bits of mb_j = bits(kMagic + 2^(p-1) + q_j):
@@ -1072,7 +1076,7 @@ __device__ __forceinline__ bool send_wide_row(const SendConsts &K, const LanePtr
     const f32x2 mult2 = dup2(mult), qmagic2 = dup2(qmagic), omb2 = dup2(K.omb), beta2 = dup2(K.beta);
     uint4 rnd = make_uint4(0u, 0u, 0u, 0u);                // the lane's 16 elements are one block of the Philox stream
     if (var_is_sr(VAR))
-        rnd = sr_block((L.elem0 + static_cast<unsigned long long>(wrow) * kWide) >> 4, K.k_lo, K.k_hi, K.seed_lo, K.seed_hi);
+        rnd = sr_block((L.elem0 + static_cast<unsigned long long>(wrow) * kWide) >> 4, K.k_lo, K.k_hi, K.sr_keys);
     unsigned signs = 0u;                                   // sign code: bit j = 1 when element j is negative
     if (BITS == 1) {
         const unsigned mag = __float_as_uint(MODE == MODE_BLOCK ? scale : K.inv_s);     // d = q x mean|h|, or q / s = +-fl(1/s)
@@ -1231,7 +1235,7 @@ __device__ __forceinline__ void load_consts(const SendCommon &C, SendConsts &K) 
     K.xslot = K.xgroup = 0u;
     K.bar_id = 0u;
     K.bar_threads = 32u;
-    K.seed_lo = C.seed_lo; K.seed_hi = C.seed_hi; K.k_lo = C.k_lo; K.k_hi = C.k_hi;
+    K.k_lo = C.k_lo; K.k_hi = C.k_hi; K.sr_keys = C.sr_keys;
 }
 
 // What a warp has counted goes to the bucket's status words: [0] flags, [1] saturated gradient codes, [2] saturated
