@@ -125,6 +125,34 @@ def test_wide_blocks_small_and_ragged(B):
         assert_reduced_equal(got, want, False, "n=%d" % n)
 
 
+@pytest.mark.parametrize("B", [64, 256, 512, 1024, 4096])
+def test_block_whose_error_maximum_is_below_the_fast_range(B):
+    """The fast routine gives a row up at two points: the block maximum of h outside [2^-100, 2^100], and the block maximum of
+    the new error outside it.  Here the second one alone fires: |h| <= 2^-90, every h one ulp beside a multiple of the block's
+    scale, so the error is ~2^-115 everywhere in the block.  With blocks wider than a row all warps of the block must give up
+    together, and the block is redone by one of them."""
+    n = 40 * 4096 + 1234
+    gcfg, ocfg = both_configs(bits=4, scale_mode=loco.SCALE_BLOCK_ABSMAX, block_size=B, beta=0.5, reset_period=0,
+                              state_fmt=loco.STATE_INT8, grad_dtype=loco.F32, out_dtype=loco.F32, num_partitions=2)
+    rng = np.random.default_rng(77)
+    amax = np.float32(2.0 ** -90)
+    scale = np.float32(amax / np.float32(7.0))
+
+    def plant(g, i):
+        if i != 0:
+            return
+        for blk in (3, 17):                                      # two blocks of the first partition
+            kq = rng.integers(-6, 7, B).astype(np.float32)
+            h = (kq * scale).astype(np.float32)
+            h = np.nextafter(h, np.float32(np.inf)).astype(np.float32)     # one ulp off the code's value (0 becomes the smallest denormal)
+            h[0] = amax
+            g[blk * B:(blk + 1) * B] = torch.from_numpy(h).to(g.device)
+
+    ws = [run_steps(gcfg, ocfg, n, 3, 1e-3, seed=41, worker=w, plant=plant) for w in range(2)]
+    got, want = reduce_both(gcfg, ocfg, n, ws)
+    assert_reduced_equal(got, want, False)
+
+
 # ---------------------------------------------------------------- clamped 8-bit error codes are counted
 
 @pytest.mark.parametrize("fmt", [loco.STATE_INT8, loco.STATE_FP32_Q8COMP])
