@@ -104,7 +104,7 @@ def measured_peak():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle samples taken every 200 ms while the timed region runs."""
+    """SM clock and throttle-reason samples taken while the timed region runs: NVML polled every 5 ms, else nvidia-smi every 200 ms."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -115,6 +115,8 @@ class ClockSampler:
         self.path = None
 
     def start(self):
+        if self._start_nvml():
+            return
         try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
@@ -124,8 +126,51 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def _start_nvml(self) -> bool:
+        """Poll NVML from a thread every 5 ms (read-only queries): a timed region of a tenth of a second still gets
+        a couple of dozen samples, where a 200 ms nvidia-smi loop gets one."""
+        try:
+            import threading
+            import pynvml
+            pynvml.nvmlInit()
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(self.dev).uuid)
+                h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                h = pynvml.nvmlDeviceGetHandleByIndex(self.dev)
+            names = (("hw_slowdown", pynvml.nvmlClocksEventReasonHwSlowdown), ("hw_thermal_slowdown", pynvml.nvmlClocksEventReasonHwThermalSlowdown),
+                     ("sw_thermal_slowdown", pynvml.nvmlClocksEventReasonSwThermalSlowdown), ("sw_power_cap", pynvml.nvmlClocksEventReasonSwPowerCap))
+            self.nvml_max = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            self.nvml_sm, self.nvml_reasons, self.nvml_stop = [], set(), threading.Event()
+
+            def poll():
+                while not self.nvml_stop.is_set():
+                    try:
+                        self.nvml_sm.append(float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM)))
+                        mask = pynvml.nvmlDeviceGetCurrentClocksEventReasons(h)
+                        for name, bit in names:
+                            if mask & bit:
+                                self.nvml_reasons.add(name)
+                    except Exception:
+                        pass
+                    self.nvml_stop.wait(0.005)
+
+            self.nvml_thread = threading.Thread(target=poll, daemon=True)
+            self.nvml_thread.start()
+            return True
+        except Exception:
+            self.nvml_thread = None
+            return False
+
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if getattr(self, "nvml_thread", None) is not None:
+            self.nvml_stop.set()
+            self.nvml_thread.join(timeout=2)
+            if self.nvml_sm:
+                out.update(sm_mhz=statistics.median(self.nvml_sm), sm_max_mhz=self.nvml_max, reasons=sorted(self.nvml_reasons),
+                           samples=len(self.nvml_sm), source="nvml, 5 ms period")
+            return out
         if self.proc is None:
             return out
         time.sleep(0.25)
