@@ -1586,13 +1586,29 @@ __device__ __forceinline__ void adam_finish16(const ReduceCommon &C, void *out, 
 // Sign code: a byte lane counts twice the negative workers of its element, 2c (a multiply spreads four wire bits to
 // four bytes: bit i of a nibble times 0x00408102 lands, among others, on bit 8 i + 1, and no two bits meet), and the
 // sum of the +-1 is N - 2c.
+// three-input bit operations in one instruction each: a ^ b ^ c and the majority of a, b, c (a full adder on 32 positions at once)
+__device__ __forceinline__ unsigned xor3(unsigned a, unsigned b, unsigned c) {
+    unsigned d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned maj3(unsigned a, unsigned b, unsigned c) {
+    unsigned d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xE8;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 template <int BITS>
 struct WideSums {
     static constexpr int S = (BITS == 8) ? 8 : 4;
+    static constexpr int P = (BITS == 1) ? 5 : 1;           // sign code: bit planes of the per-element count (at most 16 workers)
     unsigned s[S];
+    unsigned p[P];
     __device__ __forceinline__ void clear() {
 #pragma unroll
         for (int i = 0; i < S; ++i) s[i] = 0u;
+#pragma unroll
+        for (int i = 0; i < P; ++i) p[i] = 0u;
     }
     __device__ __forceinline__ void add(const WideCodes<BITS> &c) {
         if (BITS == 4) {            // s[2h] holds elements 8h + {0,2,4,6}, s[2h+1] elements 8h + {1,3,5,7}
@@ -1610,9 +1626,52 @@ struct WideSums {
         } else if (BITS == 2) {     // byte b of s[k] holds element 4b + k
 #pragma unroll
             for (int k = 0; k < 4; ++k) s[k % S] += xor_and(c.w[0] >> (2 * k), 0x02020202u, 0x03030303u);
-        } else {                    // sign code: byte b of s[g] holds 2 x (negative workers of element 4g + b)
+        } else {
+            // sign code: the lane's word has one bit per element (1 = negative).  The number of negative workers of every
+            // element is kept bit-sliced -- plane k holds bit k of all 16 counts -- so one worker costs a ripple of half
+            // adders over the planes, eight logic instructions for 16 elements
+            unsigned carry = c.w[0];
 #pragma unroll
-            for (int g = 0; g < 4; ++g) s[g % S] += (((c.w[0] >> (4 * g)) & 0xFu) * 0x00408102u) & 0x02020202u;
+            for (int k = 0; k < P; ++k) {
+                const unsigned t = p[k % P] & carry;
+                p[k % P] ^= carry;
+                carry = t;
+            }
+        }
+    }
+    // Sign code, four workers at once: two full adders fold them and plane 0 into a new plane 0 and two carries of weight 2,
+    // a third folds those and plane 1, the rest ripples: eleven logic instructions for 64 wire bits.
+    __device__ __forceinline__ void add4(const WideCodes<BITS> &a, const WideCodes<BITS> &b, const WideCodes<BITS> &c, const WideCodes<BITS> &d) {
+        if (BITS != 1) {
+            add(a); add(b); add(c); add(d);
+        } else {
+            const unsigned s1 = xor3(a.w[0], b.w[0], c.w[0]), c1 = maj3(a.w[0], b.w[0], c.w[0]);
+            const unsigned c2 = maj3(s1, d.w[0], p[0]);
+            p[0] = xor3(s1, d.w[0], p[0]);
+            const unsigned c3 = maj3(c1, c2, p[1 % P]);
+            p[1 % P] = xor3(c1, c2, p[1 % P]);
+            const unsigned c4 = p[2 % P] & c3;
+            p[2 % P] ^= c3;
+            const unsigned c5 = p[3 % P] & c4;
+            p[3 % P] ^= c4;
+            p[4 % P] ^= c5;
+        }
+    }
+    // Sign code: the planes become byte lanes once per row -- byte b of s[g] = 2 x (negative workers of element 4g + b).
+    // A multiply spreads the four bits of a nibble to four bytes (bit i times 0x00408102 lands, among others, on bit
+    // 8i + 1, and no two bits meet); plane k adds its spread nibble shifted by k.  `planes` = how many planes can be
+    // non-zero (bit length of the worker count), the same for the whole launch.
+    __device__ __forceinline__ void finalize(int planes) {
+        if (BITS == 1) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+                unsigned acc = 0u;
+#pragma unroll
+                for (int k = 0; k < P; ++k) {
+                    if (k < planes) acc += ((((p[k % P] >> (4 * g)) & 0xFu) * 0x00408102u) & 0x02020202u) << k;
+                }
+                s[g % S] = acc;
+            }
         }
     }
     // kMagic + S_j as a float
@@ -1653,6 +1712,7 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const __g
     const unsigned lane_elem = static_cast<unsigned>(lane) * kWideLane;
     const unsigned lane_byte = lane_elem * BITS / 8;
     const int N = C.num_workers;
+    const int count_planes = 32 - __clz(N);                            // sign code, integer path: bit length of a count of workers
     const bool wide32 = Bk.out_align32 != 0;
 
     if (PATH == PATH_INT) {
@@ -1687,6 +1747,8 @@ __global__ void __launch_bounds__(kThreads, 3) loco_reduce_adam_kernel(const __g
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) sums[u].add(cw[u]);
             }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) sums[u].finalize(count_planes);
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
                 if (!ok[u]) continue;
@@ -1843,6 +1905,7 @@ __device__ __forceinline__ void reduce_bucket(const ReduceCommon &C, const Reduc
     const unsigned lane_elem = static_cast<unsigned>(lane) * kWideLane;
     const unsigned lane_byte = static_cast<unsigned>(lane) * R::kLaneBytes;
     const int N = C.num_workers;
+    const int count_planes = 32 - __clz(N);                            // sign code, integer path: bit length of a count of workers
     const bool wide32 = Bk.out_align32 != 0;
     const int WG = N < 4 ? N : 4;                                      // workers per group
     const int group_entries = (4 / WG) * WG;                            // 4, 4, 3, 4: (rows per group) x C
@@ -1989,6 +2052,7 @@ __device__ __forceinline__ void reduce_bucket(const ReduceCommon &C, const Reduc
         if (o >= valid) return;
         float res[16];
         if (PATH == PATH_INT) {
+            sums.finalize(count_planes);
 #pragma unroll
             for (int i = 0; i < 16; ++i) res[i] = __fmaf_rn(sums.get(i), C.ra, C.rb);
         } else {
@@ -2038,8 +2102,12 @@ __device__ __forceinline__ void reduce_bucket(const ReduceCommon &C, const Reduc
                     float sc[4];
 #pragma unroll
                     for (int e = 0; e < 4; ++e) fetch(src + e * R::kEntry, cw[e], sc[e]);
+                    if (PATH == PATH_INT && BITS == 1) {
+                        sums.add4(cw[0], cw[1], cw[2], cw[3]);
+                    } else {
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) accumulate(cw[e], sc[e]);
+                        for (int e = 0; e < 4; ++e) accumulate(cw[e], sc[e]);
+                    }
                 } else {
 #pragma unroll 1
                     for (int e = 0; e < left; ++e) {
